@@ -1,0 +1,41 @@
+"""CPU oracle for the NetSenseML adaptive-compression hot path.
+
+TEST INFRASTRUCTURE ONLY.  This package is a plain, slow, obviously-correct
+restatement of what the path computes (Alg. 1, Alg. 2 Steps 2-3, Eq. 1-3 of
+the paper, plus the int8 / fp16 value codecs and the multi-worker sum).  It
+shares no code with the CUDA library and never imports it.  Only the tests,
+the smoke check and the CPU-baseline leg of the benchmark may import it; the
+product path must never route through it.
+
+Pins (what each function is checked against, independently of itself):
+  select_topk        brute force over all k-subsets, partial-sort special
+                     case, worked examples, invariants
+  quantize_int8      worked half-way examples, invariants, fractions.Fraction
+                     exact arithmetic on small blocks
+  f32_to_f16_bits    NumPy's float16 cast on finite in-range inputs, worked
+                     bit patterns
+  decompress_sum     closed forms (identical payloads, disjoint payloads),
+                     dense brute-force loop
+  Controller (NetSense phase)  hand trace from Eq. 1-3, closed forms for the
+                     multiplicative-decrease / additive-increase recurrences
+  Controller (start-up phase)  parity unpinned: the paper gives neither the
+                     increment beta_1, the phase length nor the exit test, so
+                     the start-up recurrence is checked only against the
+                     reading stated in this package.
+"""
+from .compress import (  # noqa: F401
+    QBLOCK,
+    NonFiniteGradient,
+    k_of,
+    widen_bf16,
+    keys_of,
+    select_topk,
+    quantize_int8,
+    dequantize_int8,
+    f32_to_f16_bits,
+    f16_bits_to_f32,
+    compress,
+    decompress_sum,
+    Payload,
+)
+from .controller import Controller, ControllerParams  # noqa: F401

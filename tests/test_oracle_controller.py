@@ -1,0 +1,137 @@
+"""Pins for the oracle's ratio controller (Alg. 1, Eq. 1-3)."""
+import math
+
+import pytest
+
+from oracle import Controller, ControllerParams
+from conftest import read_golden
+
+
+def test_golden_h4_trace():
+    gold = read_golden("h4_controller.txt")
+    kv = dict(item.split("=") for item in gold["params"][0])
+    p = ControllerParams(ratio_init=float(kv["ratio_init"]), startup_max_steps=int(kv["startup_max_steps"]),
+                         btlbw_window=int(kv["btlbw_window"]), rtprop_window=int(kv["rtprop_window"]))
+    dense = float(kv["next_dense_bytes"])
+    c = Controller(p)
+    assert c.select_ratio(0, 0, dense) == float(kv["ratio_init"])
+    for row in gold["step"]:
+        nbytes, secs, ebb, btlbw, rtprop, bdp, ratio = (float(x) for x in row)
+        got = c.select_ratio(nbytes, secs, dense)
+        assert c.last_ebb == ebb and c.btlbw == btlbw and c.rtprop == rtprop and c.bdp == bdp
+        assert got == ratio
+
+
+def test_paper_defaults():
+    p = ControllerParams()
+    assert (p.ratio_init, p.ratio_min, p.ratio_max) == (0.01, 0.005, 1.0)  # Alg. 1 / Eq. 3
+    assert (p.alpha, p.beta2, p.bdp_frac) == (0.5, 0.01, 0.9)  # Section 4.1
+    assert Controller().select_ratio(0, 0, 1e8) == 0.01  # start-up begins at 0.01
+
+
+def _netsense(ratio_init, **kw):
+    return Controller(ControllerParams(ratio_init=ratio_init, startup_max_steps=0, **kw))
+
+
+def test_multiplicative_decrease_closed_form_and_floor():
+    c = _netsense(0.64, btlbw_window=0, rtprop_window=0)
+    dense = 1e9
+    r = c.select_ratio(0, 0, dense)
+    # a fixed-capacity link that is always over-filled: every sample has the
+    # same EBB and RTT, so BDP is constant and far below the data size
+    for t in range(1, 12):
+        r = c.select_ratio(1e6, 1.0, dense)
+        assert r == max(0.005, 0.64 * 0.5 ** t)  # powers of two: exact
+    assert r == 0.005
+
+
+def test_additive_increase_closed_form_and_cap():
+    c = _netsense(0.9, btlbw_window=0, rtprop_window=0)
+    r = c.select_ratio(0, 0, 1.0)
+    want = 0.9
+    for _ in range(15):
+        r = c.select_ratio(1e9, 1.0, 1.0)  # BDP 1e9 >> data size 1
+        want = min(1.0, want + 0.01)
+        assert r == want
+    assert r == 1.0
+    # 0.995 + 0.01 is capped
+    c = _netsense(0.995)
+    c.select_ratio(0, 0, 1.0)
+    assert c.select_ratio(1e9, 1.0, 1.0) == 1.0
+
+
+def test_threshold_is_strict_and_uses_upcoming_size():
+    # BDP = 1e6 B/s * 1 s; 0.9*BDP = 9e5.  ratio 0.5: dense 1.8e6 -> data = 9e5 (not >) -> +beta2
+    c = _netsense(0.5, btlbw_window=0, rtprop_window=0)
+    c.select_ratio(0, 0, 1.8e6)
+    assert c.select_ratio(1e6, 1.0, 1.8e6) == 0.51
+    c = _netsense(0.5, btlbw_window=0, rtprop_window=0)
+    c.select_ratio(0, 0, 1.8e6)
+    assert c.select_ratio(1e6, 1.0, 1.8e6 + 1.0) == 0.25
+
+
+def test_windows_forget_old_extremes():
+    lit = _netsense(0.5, btlbw_window=0, rtprop_window=0)
+    win = _netsense(0.5, btlbw_window=3, rtprop_window=3)
+    for c in (lit, win):
+        c.select_ratio(0, 0, 1e6)
+        c.select_ratio(1e9, 0.01, 1e6)  # one fast sample: EBB 1e11
+        for _ in range(4):
+            c.select_ratio(1e6, 1.0, 1e6)  # slow link afterwards: EBB 1e6
+    assert lit.btlbw == 1e11 and lit.rtprop == 0.01
+    assert win.btlbw == 1e6 and win.rtprop == 1.0
+
+
+def test_startup_ramp_under_stated_reading():
+    # parity unpinned against the paper (beta1 / exit rule not given); this
+    # checks the recurrence of the stated reading only
+    c = Controller(ControllerParams(beta1=0.1, startup_max_steps=4, rtt_excess=1.25))
+    dense = 1e8
+    seq = [c.select_ratio(0, 0, dense)]
+    for _ in range(3):
+        seq.append(c.select_ratio(seq[-1] * dense, 0.1, dense))  # flat transfer time: no congestion
+    assert seq == [0.01, 0.11, 0.21000000000000002, 0.31000000000000005]
+    assert c.phase == Controller.STARTUP
+    # excessive transfer time ends start-up and halves at once
+    r = c.select_ratio(seq[-1] * dense, 0.2, dense)
+    assert c.phase == Controller.NETSENSE and r == 0.31000000000000005 * 0.5
+
+
+def test_startup_ends_after_max_steps():
+    c = Controller(ControllerParams(beta1=0.05, startup_max_steps=2))
+    c.select_ratio(0, 0, 1.0)
+    c.select_ratio(1e9, 1.0, 1.0)
+    c.select_ratio(1e9, 1.0, 1.0)
+    assert c.phase == Controller.STARTUP and c.startup_steps == 2
+    r = c.select_ratio(1e9, 1.0, 1.0)
+    assert c.phase == Controller.NETSENSE and r == pytest.approx(0.12)
+
+
+def test_bad_measurements_leave_state_untouched():
+    c = _netsense(0.3)
+    c.select_ratio(0, 0, 1e6)
+    c.select_ratio(1e6, 1.0, 1e6)
+    snap = (c.ratio, c.btlbw, c.rtprop, c.calls)
+    for args in ((1e6, 0.0, 1e6), (1e6, -1.0, 1e6), (1e6, math.nan, 1e6), (-1.0, 1.0, 1e6),
+                 (math.inf, 1.0, 1e6), (1e6, 1.0, math.nan)):
+        with pytest.raises(ValueError):
+            c.select_ratio(*args)
+    assert (c.ratio, c.btlbw, c.rtprop, c.calls) == snap
+
+
+def test_converges_to_link_capacity():
+    # link model: transfer time = rtprop0 + bytes / bandwidth.  The controller
+    # should hover where ratio*dense is about 0.9*BDP, i.e. ratio stays within
+    # [0.45, 1.0] * (0.9 * BDP_true / dense) up to the probing increments.
+    bw, rt0, dense = 1.25e9, 1e-3, 1e8  # 10 Gbps
+    c = Controller()
+    r = c.select_ratio(0, 0, dense)
+    hist = []
+    for _ in range(400):
+        nbytes = r * dense
+        r = c.select_ratio(nbytes, rt0 + nbytes / bw, dense)
+        hist.append(r)
+        assert 0.005 <= r <= 1.0
+    tail = hist[200:]
+    # estimated BDP can never exceed bandwidth * (largest transfer time seen)
+    assert max(tail) < 0.2 and min(tail) >= 0.005
