@@ -1,0 +1,275 @@
+/*
+ * nsml.h -- C ABI of libnsml: the data-parallel hot path of NetSenseML's
+ * adaptive compression phase on one NVIDIA B200 (sm_100a).
+ *
+ * Three operations, named after the paper's statement of the problem:
+ *
+ *   nsml_select_ratio            host   Alg. 1 (network status sensing and
+ *                                       adaptive compression-ratio adjustment)
+ *   nsml_compress                device Alg. 2 Steps 2-3 (apply the pruning
+ *                                       mask, top-k sparsification at `ratio`)
+ *                                       plus the value codec of Alg. 2 Step 1
+ *   nsml_decompress_accumulate   device aggregation of the W gathered sparse
+ *                                       payloads into one dense gradient
+ *                                       (Section 4.2 Step 3; AllGather pattern
+ *                                       of Section 5.3)
+ *
+ * `ratio` is the KEPT fraction, as in the paper (1 = send everything).
+ *
+ * Conventions
+ *   - Every function returns NSML_OK (0) or a negative NSML_ERR_* code.  Nothing
+ *     throws, aborts or traps.
+ *   - "device pointer" = CUDA global memory of the current device, owned by the
+ *     caller before and after the call.  "host pointer" = ordinary memory.
+ *   - Device work is enqueued on `stream` (a cudaStream_t passed as void*, NULL
+ *     = the default stream) and the call returns without synchronising.
+ *   - Argument errors are returned at once and enqueue nothing.  Errors that only
+ *     the device can see (non-finite input, corrupt payload, a bounded wait that
+ *     ran out) are written to a status word at the start of `workspace`; read it
+ *     with nsml_last_status().
+ *   - The library allocates no device memory: scratch comes in as `workspace`.
+ *     Two calls that share a workspace must not overlap on the GPU.
+ */
+#ifndef NSML_H
+#define NSML_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+  NSML_OK = 0,
+  NSML_ERR_ARG = -1,       /* NULL / misaligned pointer, size or enum out of range */
+  NSML_ERR_CAPACITY = -2,  /* payload buffer or workspace too small */
+  NSML_ERR_CUDA = -3,      /* a CUDA runtime call failed (no device, launch error) */
+  NSML_ERR_NONFINITE = -4, /* device: the bucket holds NaN or Inf */
+  NSML_ERR_TIMEOUT = -5,   /* device: a bounded wait between thread blocks ran out */
+  NSML_ERR_PAYLOAD = -6,   /* device: payload header or index out of range */
+  NSML_ERR_INTERNAL = -7   /* device: an internal invariant failed (survivor count != k) */
+};
+
+enum { NSML_F32 = 0, NSML_BF16 = 1 };              /* gradient element type */
+enum { NSML_BITS_INT8 = 8, NSML_BITS_FP16 = 16 };  /* value codec ("bits") */
+
+#define NSML_QBLOCK 1024         /* survivors per int8 scale block */
+#define NSML_MAX_WORKERS 64      /* largest W of nsml_decompress_accumulate */
+#define NSML_MAX_N 2147483647LL  /* largest bucket, elements */
+#define NSML_PAYLOAD_MAGIC 0x4C4D534Eu /* "NSML" */
+#define NSML_PAYLOAD_VERSION 1u
+
+/* ------------------------------------------------------------------------
+ * Payload: one worker's compressed bucket, one contiguous buffer, every
+ * section 16-byte aligned:
+ *   header (64 B) | idx: u32[k] strictly ascending | val: i8[k] or f16[k]
+ *   | scale: f32[nblocks] (int8 only; block b covers payload entries
+ *   [b*1024, (b+1)*1024))
+ * The paper leaves the layout of Com_grads open (Alg. 2 names only
+ * top_k(grads, ratio)); this one is defined here.
+ * ---------------------------------------------------------------------- */
+typedef struct nsml_payload_header {
+  uint32_t magic;     /* NSML_PAYLOAD_MAGIC */
+  uint32_t version;   /* NSML_PAYLOAD_VERSION */
+  uint64_t n;         /* elements in the dense bucket */
+  uint64_t k;         /* survivors = ceil(ratio*n) */
+  uint32_t bits;      /* NSML_BITS_INT8 or NSML_BITS_FP16 */
+  uint32_t qblock;    /* NSML_QBLOCK */
+  uint64_t nblocks;   /* ceil(k/qblock) for int8, 0 for fp16 */
+  uint64_t idx_off;   /* byte offsets from the start of the payload */
+  uint64_t val_off;
+  uint64_t scale_off; /* 0 for fp16 */
+} nsml_payload_header;
+
+/* ------------------------------------------------------------------------
+ * Host controller -- Alg. 1, Eq. 1-3.
+ * ---------------------------------------------------------------------- */
+typedef struct nsml_ctrl nsml_ctrl; /* opaque, host memory, owned by the library */
+
+typedef struct nsml_ctrl_params {
+  double ratio_init;     /* 0.01  Alg. 1 Step 1 */
+  double ratio_min;      /* 0.005 Eq. 3 */
+  double ratio_max;      /* 1.0   Eq. 3 */
+  double alpha;          /* 0.5   Section 4.1 */
+  double beta1;          /* start-up increment; not given in the paper: 0.1 */
+  double beta2;          /* 0.01  Section 4.1 */
+  double bdp_frac;       /* 0.9   Eq. 3 */
+  double rtt_excess;     /* start-up ends when a transfer time exceeds
+                            rtt_excess*RTprop; not given in the paper: 1.25 */
+  int32_t startup_max_steps; /* not given ("first few steps"): 10; 0 = no start-up */
+  int32_t btlbw_window;  /* samples the BtlBw maximum runs over: 10; 0 = all-time
+                            (the literal reading of Alg. 1) */
+  int32_t rtprop_window; /* samples the RTprop minimum runs over: 100; 0 = all-time */
+  int32_t reserved;
+} nsml_ctrl_params;
+
+typedef struct nsml_ctrl_state {
+  double ratio;   /* ratio the last call returned */
+  double ebb;     /* Eq. 1 of the last sample, bytes/s */
+  double btlbw;   /* bytes/s */
+  double rtprop;  /* seconds (+inf before the first sample) */
+  double bdp;     /* Eq. 2, bytes */
+  int32_t phase;  /* 0 = start-up, 1 = NetSense */
+  int32_t startup_steps;
+  int64_t calls;
+} nsml_ctrl_state;
+
+/* Fills *p with the defaults listed above.  Returns NSML_ERR_ARG if p is NULL. */
+int nsml_ctrl_default_params(nsml_ctrl_params* p);
+
+/* Creates a controller.  p == NULL takes the defaults.  Parameters are checked
+ * (0 < ratio_min <= ratio_init <= ratio_max <= 1, 0 < alpha < 1, beta1, beta2 > 0,
+ * bdp_frac > 0, rtt_excess >= 1, windows and steps >= 0; windows <= 4096):
+ * NSML_ERR_ARG otherwise.  *out is written only on success; free it with
+ * nsml_ctrl_destroy (NULL is allowed there). */
+int nsml_ctrl_create(const nsml_ctrl_params* p, nsml_ctrl** out);
+void nsml_ctrl_destroy(nsml_ctrl* c);
+
+/* Alg. 1, one call per gradient-transmission interval i.
+ *   last_bytes, last_seconds  size and measured transfer time of interval i-1
+ *                             (ignored on the first call: nothing was sent yet)
+ *   next_dense_bytes          size the upcoming transfer would have at ratio 1;
+ *                             Eq. 3 compares ratio*next_dense_bytes with
+ *                             bdp_frac*BDP
+ *   ratio_out                 host pointer, receives the ratio for interval i
+ * First call: returns ratio_init.  Start-up calls add beta1 until a transfer
+ * time exceeds rtt_excess*RTprop, startup_max_steps increments were made or the
+ * ratio reached ratio_max; the call that ends start-up, and every later call,
+ * applies Eq. 1-3: EBB = last_bytes/last_seconds, BtlBw = max EBB, RTprop = min
+ * transfer time, BDP = BtlBw*RTprop, then ratio = max(ratio_min, ratio*alpha) if
+ * ratio*next_dense_bytes > bdp_frac*BDP else min(ratio_max, ratio+beta2).
+ * All arithmetic is IEEE double in the operand order written here.
+ * Errors: NSML_ERR_ARG for NULL pointers, last_seconds <= 0 or non-finite,
+ * negative or non-finite sizes; the state is then unchanged. */
+int nsml_select_ratio(nsml_ctrl* c, double last_bytes, double last_seconds,
+                      double next_dense_bytes, double* ratio_out);
+
+/* Copies the controller's current estimates to *out (host pointer). */
+int nsml_ctrl_get_state(const nsml_ctrl* c, nsml_ctrl_state* out);
+
+/* Checkpointing: the state is a flat blob of nsml_ctrl_save_bytes() bytes.
+ * nsml_ctrl_save writes it to buf (capacity cap, NSML_ERR_CAPACITY if too
+ * small); nsml_ctrl_load replaces c's parameters and state from such a blob
+ * (NSML_ERR_ARG if the blob's size or tag is wrong; c is then unchanged). */
+size_t nsml_ctrl_save_bytes(const nsml_ctrl* c);
+int nsml_ctrl_save(const nsml_ctrl* c, void* buf, size_t cap);
+int nsml_ctrl_load(nsml_ctrl* c, const void* buf, size_t bytes);
+
+/* ------------------------------------------------------------------------
+ * Sizes (pure host arithmetic; 0 is returned for arguments out of range).
+ * ---------------------------------------------------------------------- */
+/* k = ceil(ratio*n) evaluated in IEEE double, clamped to [1, n] (Alg. 2 Step 3
+ * gives only top_k(grads, ratio); ceil is the reading used). */
+int64_t nsml_k_of(int64_t n, double ratio);
+/* Exact size in bytes of the payload nsml_compress writes for (n, ratio, bits). */
+size_t nsml_payload_bytes(int64_t n, double ratio, int bits);
+/* Scratch needed by nsml_compress for a bucket of n elements (any ratio, bits). */
+size_t nsml_workspace_bytes(int64_t n, int grad_dtype);
+/* Scratch needed by nsml_decompress_accumulate for (n, W). */
+size_t nsml_accumulate_workspace_bytes(int64_t n, int W);
+
+/* ------------------------------------------------------------------------
+ * nsml_compress -- Alg. 2 Steps 2-3 and the value codec, one flat bucket.
+ *
+ *   grad        device pointer, 16-byte aligned: n elements, float32
+ *               (NSML_F32) or bfloat16 (NSML_BF16, widened exactly to float32).
+ *               Values must be finite.
+ *   n           1 .. NSML_MAX_N
+ *   ratio       kept fraction in (0, 1]; k = nsml_k_of(n, ratio)
+ *   bits        NSML_BITS_INT8: per block of 1024 consecutive survivors
+ *               scale = maxabs/127, code = clamp(rint(v/scale), +-127), both
+ *               IEEE float32 divisions, round half to even, denormals kept;
+ *               scale 0 gives codes 0.  (Not in the paper.)
+ *               NSML_BITS_FP16: float32 -> binary16, round to nearest even
+ *               (Alg. 2 Step 1 "quantize"); |v| >= 65520 saturates to +-65504.
+ *   prune_mask  device pointer (4-byte aligned) to ceil(n/32) words, bit (i&31)
+ *               of word i>>5 set = parameter i is pruned: its gradient counts as
+ *               +0.0 (Alg. 2 Step 2).  NULL = nothing pruned.
+ *   payload     device pointer, 16-byte aligned, capacity payload_capacity >=
+ *               nsml_payload_bytes(n, ratio, bits) (else NSML_ERR_CAPACITY)
+ *   workspace   device pointer, 256-byte aligned, workspace_bytes >=
+ *               nsml_workspace_bytes(n, grad_dtype)
+ *
+ * Result: the k entries of largest magnitude (compared on the float32 bit
+ * pattern with the sign cleared; ties: larger magnitude first, then lower
+ * index), in ascending index order; exactly k entries even if fewer than k
+ * gradients are non-zero.  The result is unique, so the payload is
+ * bit-reproducible.  Device-detected: NSML_ERR_NONFINITE (payload contents
+ * then unspecified), NSML_ERR_TIMEOUT.
+ * ---------------------------------------------------------------------- */
+int nsml_compress(const void* grad, int64_t n, int grad_dtype, double ratio, int bits,
+                  const uint32_t* prune_mask, void* payload, size_t payload_capacity,
+                  void* workspace, size_t workspace_bytes, void* stream);
+
+/* ------------------------------------------------------------------------
+ * nsml_decompress_accumulate -- dense += sum over W payloads (plain sum, no
+ * averaging), after optionally zeroing dense.
+ *
+ *   payloads    HOST array of W device pointers (16-byte aligned), each a payload
+ *               written by nsml_compress (or laid out the same way) for this n;
+ *               int8 and fp16 payloads may be mixed; 1 <= W <= NSML_MAX_WORKERS
+ *   dense       device pointer, 16-byte aligned, n float32; read unless
+ *               zero_first, always written
+ *   zero_first  non-zero: dense is overwritten by the sum; zero: the sum is
+ *               added to what dense holds
+ *   workspace   device pointer, 256-byte aligned, >=
+ *               nsml_accumulate_workspace_bytes(n, W)
+ *
+ * Values are dequantised as float(code)*scale (one float32 multiply) or
+ * float(half), and added in float32 in worker order w = 0..W-1, each dense
+ * element by one thread: the result is deterministic.  Device-detected:
+ * NSML_ERR_PAYLOAD if a header does not match (magic, version, n, bits, k) or
+ * an index is >= n; nothing is written out of range.
+ * ---------------------------------------------------------------------- */
+int nsml_decompress_accumulate(const void* const* payloads, int W, float* dense, int64_t n,
+                               int zero_first, void* workspace, size_t workspace_bytes,
+                               void* stream);
+
+/* Host-buffer variants: the same operations for callers whose gradients and
+ * payloads live in host memory (pinned memory gives asynchronous copies).
+ * `device_scratch` (device pointer, 256-byte aligned) must hold
+ * nsml_compress_host_scratch_bytes(n, grad_dtype, ratio, bits), respectively
+ * nsml_accumulate_host_scratch_bytes(n, W, total_payload_bytes); the call copies
+ * the inputs to the device, runs the operation and copies the result back, all
+ * on `stream`, and returns without synchronising.  payload_host / dense_host
+ * are valid once the stream has been synchronised. */
+size_t nsml_compress_host_scratch_bytes(int64_t n, int grad_dtype, double ratio, int bits);
+int nsml_compress_host(const void* grad_host, int64_t n, int grad_dtype, double ratio, int bits,
+                       const uint32_t* prune_mask_host, void* payload_host,
+                       size_t payload_capacity, void* device_scratch, size_t scratch_bytes,
+                       void* stream);
+size_t nsml_accumulate_host_scratch_bytes(int64_t n, int W, size_t total_payload_bytes);
+int nsml_decompress_accumulate_host(const void* const* payloads_host, const size_t* payload_bytes,
+                                    int W, float* dense_host, int64_t n, int zero_first,
+                                    void* device_scratch, size_t scratch_bytes, void* stream);
+
+/* Synchronises `stream`, then copies the status word of `workspace` (or of a
+ * host-variant `device_scratch`) to *status_out (host pointer): NSML_OK or the
+ * first device-detected error of the last call that used it. */
+int nsml_last_status(const void* workspace, void* stream, int* status_out);
+
+/* Static, NUL-terminated description of a status code. */
+const char* nsml_strerror(int status);
+
+/* ------------------------------------------------------------------------
+ * Instrumentation (optional; off by default).
+ * ---------------------------------------------------------------------- */
+/* Number of distinct kernels the library launches, and their names. */
+int nsml_kernel_count(void);
+const char* nsml_kernel_name(int kernel_id);
+/* Total kernel launches made by this process through the library so far. */
+int64_t nsml_launch_count(void);
+/* on != 0: bracket every kernel launch with CUDA events on its stream, so that
+ * per-kernel device time can be read back; slows the host side slightly.
+ * Turning it off drops recorded samples. */
+int nsml_prof_enable(int on);
+/* Synchronises the recorded events and returns, for kernel_id, the summed
+ * device time in milliseconds and the number of launches since the last reset. */
+int nsml_prof_read(int kernel_id, double* total_ms, int64_t* launches);
+int nsml_prof_reset(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* NSML_H */

@@ -1,0 +1,155 @@
+// Decompress and sum the W gathered payloads into one dense float32 gradient
+// (Section 4.2 Step 3 "further aggregation"; with top-k payloads every worker
+// receives all payloads, the AllGather pattern of Section 5.3, and sums them).
+//
+// Payload indices are ascending, so the work is split by dense range instead
+// of by payload entry: a block owns a tile of the dense buffer, finds each
+// worker's entries for that tile from a precomputed offset table, adds them in
+// worker order in shared memory and writes the tile once, coalesced.  No
+// atomics, fixed summation order, and in overwrite mode the zero fill costs
+// nothing extra.
+#pragma once
+
+#include "nsml_common.cuh"
+#include "nsml_codec.cuh"
+
+namespace nsml {
+
+constexpr int kDenseTile = 8192;  // dense elements per block iteration (32 KB of shared memory)
+
+struct PayloadTable {
+  const unsigned char* p[NSML_MAX_WORKERS];
+};
+
+struct AccumulateLayout {
+  size_t offsets;  // u32[W][tiles + 1]
+  size_t total;
+};
+
+inline AccumulateLayout accumulate_layout(int64_t n, int W) {
+  AccumulateLayout L;
+  size_t tiles = (size_t)((n + kDenseTile - 1) / kDenseTile);
+  L.offsets = 256;
+  L.total = L.offsets + align_up((size_t)W * (tiles + 1) * 4, 256);
+  return L;
+}
+
+__device__ inline bool header_ok(const nsml_payload_header* h, unsigned long long n) {
+  if (h->magic != NSML_PAYLOAD_MAGIC || h->version != NSML_PAYLOAD_VERSION) return false;
+  if (h->n != n || h->k < 1 || h->k > n || h->qblock != NSML_QBLOCK) return false;
+  if (h->bits != NSML_BITS_INT8 && h->bits != NSML_BITS_FP16) return false;
+  const unsigned long long k = h->k;
+  const unsigned long long val_off = 64 + (k * 4 + 15) / 16 * 16;
+  if (h->idx_off != 64 || h->val_off != val_off) return false;
+  if (h->bits == NSML_BITS_INT8) {
+    if (h->nblocks != (k + NSML_QBLOCK - 1) / NSML_QBLOCK) return false;
+    if (h->scale_off != val_off + (k + 15) / 16 * 16) return false;
+  }
+  return true;
+}
+
+// offsets[w][b] = first payload entry of worker w whose index is >= b*kDenseTile.
+__global__ void __launch_bounds__(kCta)
+k_partition(PayloadTable table, int W, unsigned long long n, unsigned int tiles, unsigned int* offsets, int* status) {
+  const unsigned long long g = (unsigned long long)blockIdx.x * kCta + threadIdx.x;
+  const unsigned long long per = (unsigned long long)tiles + 1;
+  if (g >= per * W) return;
+  const int w = (int)(g / per);
+  const unsigned long long b = g % per;
+  const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(table.p[w]);
+  if (!header_ok(h, n)) {
+    if (b == 0) set_status(status, NSML_ERR_PAYLOAD);
+    offsets[g] = 0;
+    return;
+  }
+  const uint32_t* idx = reinterpret_cast<const uint32_t*>(table.p[w] + h->idx_off);
+  const unsigned long long target = b * kDenseTile;
+  unsigned long long lo = 0, hi = h->k;  // lower bound
+  while (lo < hi) {
+    const unsigned long long mid = (lo + hi) >> 1;
+    if (idx[mid] < target) lo = mid + 1; else hi = mid;
+  }
+  offsets[g] = (unsigned int)lo;
+}
+
+__global__ void __launch_bounds__(kCta)
+k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long n, int zero_first,
+        unsigned int tiles, const unsigned int* __restrict__ offsets, int* status) {
+  __shared__ __align__(16) float s_acc[kDenseTile];
+  __shared__ unsigned int s_from[NSML_MAX_WORKERS], s_to[NSML_MAX_WORKERS];
+  __shared__ unsigned int s_total;
+  const unsigned long long per = (unsigned long long)tiles + 1;
+  bool bad = false;
+
+  for (unsigned int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    const unsigned long long lo = (unsigned long long)tile * kDenseTile;
+    const unsigned int len = (unsigned int)min((unsigned long long)kDenseTile, n - lo);
+    __syncthreads();  // the previous tile is fully written out
+    if (threadIdx.x == 0) s_total = 0;
+    __syncthreads();
+    if (threadIdx.x < W) {
+      unsigned int a = offsets[threadIdx.x * per + tile];
+      unsigned int b = offsets[threadIdx.x * per + tile + 1];
+      if (b < a) b = a;  // only a corrupt (unsorted) payload gets here
+      s_from[threadIdx.x] = a;
+      s_to[threadIdx.x] = b;
+      if (b > a) atomicAdd(&s_total, b - a);
+    }
+    __syncthreads();
+    const unsigned int total = s_total;
+    if (total == 0 && !zero_first) continue;
+    // Accumulate mode with few entries: touch only their elements.  Otherwise
+    // stage the whole tile in shared memory and write it back in one sweep.
+    const bool staged = zero_first || (unsigned long long)total * 16 > len;
+
+    if (staged) {
+      float* dtile = dense + lo;
+      for (unsigned int i = threadIdx.x * 4; i < len; i += kCta * 4) {
+        if (i + 4 <= len) {
+          float4 v = zero_first ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(dtile + i);
+          *reinterpret_cast<float4*>(s_acc + i) = v;
+        } else {
+          for (unsigned int e = i; e < len; ++e) s_acc[e] = zero_first ? 0.f : dtile[e];
+        }
+      }
+      __syncthreads();
+    }
+
+    for (int w = 0; w < W; ++w) {
+      const unsigned int from = s_from[w], to = s_to[w];
+      if (to > from) {
+        const unsigned char* base = table.p[w];
+        const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(base);
+        const uint32_t* idx = reinterpret_cast<const uint32_t*>(base + h->idx_off);
+        const bool int8 = (h->bits == NSML_BITS_INT8);
+        const signed char* codes = reinterpret_cast<const signed char*>(base + h->val_off);
+        const uint16_t* halves = reinterpret_cast<const uint16_t*>(base + h->val_off);
+        const float* scales = reinterpret_cast<const float*>(base + h->scale_off);
+        for (unsigned int j = from + threadIdx.x; j < to; j += kCta) {
+          const unsigned long long off = (unsigned long long)idx[j] - lo;  // wraps if idx < lo
+          const float v = int8 ? decode_i8(codes[j], scales[j >> 10]) : decode_f16(halves[j]);
+          if (off < len) {
+            if (staged) s_acc[off] += v; else dense[lo + off] += v;
+          } else {
+            bad = true;
+          }
+        }
+      }
+      __syncthreads();  // worker w is done before worker w+1 adds to the same elements
+    }
+
+    if (staged) {
+      float* dtile = dense + lo;
+      for (unsigned int i = threadIdx.x * 4; i < len; i += kCta * 4) {
+        if (i + 4 <= len) {
+          *reinterpret_cast<float4*>(dtile + i) = *reinterpret_cast<const float4*>(s_acc + i);
+        } else {
+          for (unsigned int e = i; e < len; ++e) dtile[e] = s_acc[e];
+        }
+      }
+    }
+  }
+  if (bad) set_status(status, NSML_ERR_PAYLOAD);
+}
+
+}  // namespace nsml

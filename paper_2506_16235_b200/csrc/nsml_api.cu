@@ -1,0 +1,427 @@
+// libnsml C ABI: argument checks, workspace carving and kernel launches.
+// See include/nsml.h for the contract of every entry point.
+#include <atomic>
+#include <cmath>
+#include <cstring>
+#include <mutex>
+#include <vector>
+
+#include "nsml_accumulate.cuh"
+#include "nsml_codec.cuh"
+#include "nsml_common.cuh"
+#include "nsml_compact.cuh"
+#include "nsml_select.cuh"
+
+namespace nsml {
+
+enum KernelId {
+  K_HIST_BUCKET = 0,
+  K_COMPACT_BUCKET,
+  K_HIST_LIST_1,
+  K_HIST_LIST_2,
+  K_COMPACT_LIST,
+  K_QUANTIZE,
+  K_PARTITION,
+  K_MERGE,
+  K_COUNT
+};
+
+static const char* const kKernelNames[K_COUNT] = {
+    "k_histogram<0,bucket>", "k_compact_bucket", "k_histogram<1,list>", "k_histogram<2,list>",
+    "k_compact_list",        "k_quantize",       "k_partition",         "k_merge"};
+
+static std::atomic<int64_t> g_launches{0};
+
+// ---- optional per-kernel timing with CUDA events --------------------------
+struct ProfRecord {
+  int id;
+  cudaEvent_t start, stop;
+};
+static std::mutex g_prof_mutex;
+static bool g_prof_on = false;
+static std::vector<ProfRecord> g_prof_records;
+static double g_prof_ms[K_COUNT];
+static int64_t g_prof_launches[K_COUNT];
+
+static void prof_drain_locked() {
+  for (ProfRecord& r : g_prof_records) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(r.stop) == cudaSuccess && cudaEventElapsedTime(&ms, r.start, r.stop) == cudaSuccess) {
+      g_prof_ms[r.id] += ms;
+      g_prof_launches[r.id] += 1;
+    }
+    cudaEventDestroy(r.start);
+    cudaEventDestroy(r.stop);
+  }
+  g_prof_records.clear();
+}
+
+struct LaunchScope {  // brackets one kernel launch
+  int id;
+  cudaStream_t stream;
+  cudaEvent_t start = nullptr, stop = nullptr;
+  LaunchScope(int id_, cudaStream_t s) : id(id_), stream(s) {
+    if (g_prof_on) {
+      cudaEventCreate(&start);
+      cudaEventCreate(&stop);
+      cudaEventRecord(start, stream);
+    }
+  }
+  ~LaunchScope() {
+    g_launches.fetch_add(1, std::memory_order_relaxed);
+    if (start) {
+      cudaEventRecord(stop, stream);
+      std::lock_guard<std::mutex> lock(g_prof_mutex);
+      g_prof_records.push_back({id, start, stop});
+    }
+  }
+};
+
+// ---- per-device launch geometry -------------------------------------------
+struct DeviceInfo {
+  bool ready = false;
+  int sms = 0;
+  int compact_f32 = 0, compact_bf16 = 0, compact_list = 0, merge = 0;  // resident blocks per SM
+};
+static DeviceInfo g_dev[64];
+static std::mutex g_dev_mutex;
+
+static int device_info(const DeviceInfo** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NSML_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_dev_mutex);
+  DeviceInfo& d = g_dev[dev];
+  if (!d.ready) {
+    if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return NSML_ERR_CUDA;
+    cudaError_t e = cudaSuccess;
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_f32, k_compact_bucket<NSML_F32>, kCta, 0);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_bf16, k_compact_bucket<NSML_BF16>, kCta, 0);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_list, k_compact_list, kCta, 0);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.merge, k_merge, kCta, 0);
+    if (e != cudaSuccess || d.compact_f32 < 1 || d.compact_bf16 < 1 || d.compact_list < 1 || d.merge < 1) {
+      cudaGetLastError();
+      return NSML_ERR_CUDA;
+    }
+    d.ready = true;
+  }
+  *out = &d;
+  return NSML_OK;
+}
+
+static inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+static inline unsigned int grid_for(unsigned long long work_items, unsigned long long per_block, int cap) {
+  unsigned long long blocks = (work_items + per_block - 1) / per_block;
+  if (blocks < 1) blocks = 1;
+  if (blocks > (unsigned long long)cap) blocks = cap;
+  return (unsigned int)blocks;
+}
+
+static int64_t k_of(int64_t n, double ratio) {
+  if (n < 1 || n > NSML_MAX_N || !(ratio > 0.0) || !(ratio <= 1.0)) return 0;
+  double kd = std::ceil(ratio * (double)n);
+  int64_t k = (int64_t)kd;
+  if (k < 1) k = 1;
+  if (k > n) k = n;
+  return k;
+}
+
+template <int DTYPE>
+static void launch_bucket_stage(const void* grad, const uint32_t* mask, int64_t n, int64_t k, unsigned char* ws,
+                                const CompressLayout& L, const DeviceInfo& dev, cudaStream_t st) {
+  Ctl* ctl = reinterpret_cast<Ctl*>(ws);
+  unsigned int* hist = reinterpret_cast<unsigned int*>(ws + L.hist);
+  BucketSrc<DTYPE> src{grad, mask};
+  {
+    LaunchScope scope(K_HIST_BUCKET, st);
+    unsigned int grid = grid_for((unsigned long long)n, kCta * 4 * 4, dev.sms * 4);
+    k_histogram<0, BucketSrc<DTYPE>><<<grid, kCta, 0, st>>>(src, (unsigned long long)n, (unsigned long long)k, ctl, hist);
+  }
+  {
+    LaunchScope scope(K_COMPACT_BUCKET, st);
+    int occ = (DTYPE == NSML_F32) ? dev.compact_f32 : dev.compact_bf16;
+    unsigned int grid = grid_for((unsigned long long)n, kTile, dev.sms * occ);
+    k_compact_bucket<DTYPE><<<grid, kCta, 0, st>>>(src, (unsigned long long)n, ctl,
+                                                   reinterpret_cast<unsigned long long*>(ws + L.state_bucket),
+                                                   reinterpret_cast<uint32_t*>(ws + L.list_idx),
+                                                   reinterpret_cast<uint32_t*>(ws + L.list_val));
+  }
+}
+
+static int compress_impl(const void* grad, int64_t n, int grad_dtype, double ratio, int bits,
+                         const uint32_t* prune_mask, void* payload, size_t payload_capacity, void* workspace,
+                         size_t workspace_bytes, cudaStream_t st) {
+  if (grad == nullptr || payload == nullptr || workspace == nullptr) return NSML_ERR_ARG;
+  if (grad_dtype != NSML_F32 && grad_dtype != NSML_BF16) return NSML_ERR_ARG;
+  if (bits != NSML_BITS_INT8 && bits != NSML_BITS_FP16) return NSML_ERR_ARG;
+  const int64_t k = k_of(n, ratio);
+  if (k == 0) return NSML_ERR_ARG;
+  if (!aligned(grad, 16) || !aligned(payload, 16) || !aligned(workspace, 256)) return NSML_ERR_ARG;
+  if (prune_mask != nullptr && !aligned(prune_mask, 4)) return NSML_ERR_ARG;
+  const PayloadLayout P = payload_layout(k, bits);
+  const CompressLayout L = compress_layout(n);
+  if (payload_capacity < P.total || workspace_bytes < L.total) return NSML_ERR_CAPACITY;
+  const DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != NSML_OK) return rc;
+
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  unsigned char* pl = static_cast<unsigned char*>(payload);
+  Ctl* ctl = reinterpret_cast<Ctl*>(ws);
+  unsigned int* hist = reinterpret_cast<unsigned int*>(ws + L.hist);
+  if (cudaMemsetAsync(ws, 0, L.zero_bytes, st) != cudaSuccess) return NSML_ERR_CUDA;
+
+  if (grad_dtype == NSML_F32) launch_bucket_stage<NSML_F32>(grad, prune_mask, n, k, ws, L, *dev, st);
+  else launch_bucket_stage<NSML_BF16>(grad, prune_mask, n, k, ws, L, *dev, st);
+
+  ListSrc list{reinterpret_cast<const uint32_t*>(ws + L.list_idx), reinterpret_cast<const uint32_t*>(ws + L.list_val)};
+  const unsigned int list_grid = (unsigned int)(dev->sms * 2);
+  {
+    LaunchScope scope(K_HIST_LIST_1, st);
+    k_histogram<1, ListSrc><<<list_grid, kCta, 0, st>>>(list, 0ull, (unsigned long long)k, ctl, hist);
+  }
+  {
+    LaunchScope scope(K_HIST_LIST_2, st);
+    k_histogram<2, ListSrc><<<list_grid, kCta, 0, st>>>(list, 0ull, (unsigned long long)k, ctl, hist);
+  }
+  {
+    LaunchScope scope(K_COMPACT_LIST, st);
+    unsigned int grid = (unsigned int)(dev->sms * dev->compact_list);
+    k_compact_list<<<grid, kCta, 0, st>>>(list, ctl, reinterpret_cast<unsigned long long*>(ws + L.state_list),
+                                          reinterpret_cast<uint32_t*>(pl + P.idx_off),
+                                          reinterpret_cast<uint32_t*>(ws + L.raw_val));
+  }
+  {
+    LaunchScope scope(K_QUANTIZE, st);
+    unsigned int grid = (unsigned int)((k + NSML_QBLOCK - 1) / NSML_QBLOCK);
+    const float* raw = reinterpret_cast<const float*>(ws + L.raw_val);
+    if (bits == NSML_BITS_INT8)
+      k_quantize<NSML_BITS_INT8><<<grid, kCta, 0, st>>>(raw, (unsigned long long)k, (unsigned long long)n, ctl, pl, P);
+    else
+      k_quantize<NSML_BITS_FP16><<<grid, kCta, 0, st>>>(raw, (unsigned long long)k, (unsigned long long)n, ctl, pl, P);
+  }
+  if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
+  return NSML_OK;
+}
+
+static int accumulate_impl(const void* const* payloads, int W, float* dense, int64_t n, int zero_first,
+                           void* workspace, size_t workspace_bytes, cudaStream_t st) {
+  if (payloads == nullptr || dense == nullptr || workspace == nullptr) return NSML_ERR_ARG;
+  if (W < 1 || W > NSML_MAX_WORKERS || n < 1 || n > NSML_MAX_N) return NSML_ERR_ARG;
+  if (!aligned(dense, 16) || !aligned(workspace, 256)) return NSML_ERR_ARG;
+  PayloadTable table;
+  std::memset(&table, 0, sizeof(table));
+  for (int w = 0; w < W; ++w) {
+    if (payloads[w] == nullptr || !aligned(payloads[w], 16)) return NSML_ERR_ARG;
+    table.p[w] = static_cast<const unsigned char*>(payloads[w]);
+  }
+  const AccumulateLayout L = accumulate_layout(n, W);
+  if (workspace_bytes < L.total) return NSML_ERR_CAPACITY;
+  const DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != NSML_OK) return rc;
+
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  int* status = reinterpret_cast<int*>(ws);
+  unsigned int* offsets = reinterpret_cast<unsigned int*>(ws + L.offsets);
+  const unsigned int tiles = (unsigned int)((n + kDenseTile - 1) / kDenseTile);
+  if (cudaMemsetAsync(ws, 0, 256, st) != cudaSuccess) return NSML_ERR_CUDA;
+  {
+    LaunchScope scope(K_PARTITION, st);
+    unsigned long long threads = (unsigned long long)W * (tiles + 1ull);
+    unsigned int grid = (unsigned int)((threads + kCta - 1) / kCta);
+    k_partition<<<grid, kCta, 0, st>>>(table, W, (unsigned long long)n, tiles, offsets, status);
+  }
+  {
+    LaunchScope scope(K_MERGE, st);
+    unsigned int grid = grid_for(tiles, 1, dev->sms * dev->merge);
+    k_merge<<<grid, kCta, 0, st>>>(table, W, dense, (unsigned long long)n, zero_first, tiles, offsets, status);
+  }
+  if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
+  return NSML_OK;
+}
+
+}  // namespace nsml
+
+using namespace nsml;
+
+extern "C" {
+
+int64_t nsml_k_of(int64_t n, double ratio) { return k_of(n, ratio); }
+
+size_t nsml_payload_bytes(int64_t n, double ratio, int bits) {
+  if (bits != NSML_BITS_INT8 && bits != NSML_BITS_FP16) return 0;
+  const int64_t k = k_of(n, ratio);
+  if (k == 0) return 0;
+  return payload_layout(k, bits).total;
+}
+
+size_t nsml_workspace_bytes(int64_t n, int grad_dtype) {
+  if (n < 1 || n > NSML_MAX_N || (grad_dtype != NSML_F32 && grad_dtype != NSML_BF16)) return 0;
+  return compress_layout(n).total;
+}
+
+size_t nsml_accumulate_workspace_bytes(int64_t n, int W) {
+  if (n < 1 || n > NSML_MAX_N || W < 1 || W > NSML_MAX_WORKERS) return 0;
+  return accumulate_layout(n, W).total;
+}
+
+int nsml_compress(const void* grad, int64_t n, int grad_dtype, double ratio, int bits, const uint32_t* prune_mask,
+                  void* payload, size_t payload_capacity, void* workspace, size_t workspace_bytes, void* stream) {
+  return compress_impl(grad, n, grad_dtype, ratio, bits, prune_mask, payload, payload_capacity, workspace,
+                       workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int nsml_decompress_accumulate(const void* const* payloads, int W, float* dense, int64_t n, int zero_first,
+                               void* workspace, size_t workspace_bytes, void* stream) {
+  return accumulate_impl(payloads, W, dense, n, zero_first, workspace, workspace_bytes,
+                         static_cast<cudaStream_t>(stream));
+}
+
+// ---- host-buffer variants --------------------------------------------------
+static size_t elem_size(int grad_dtype) { return grad_dtype == NSML_F32 ? 4 : 2; }
+
+size_t nsml_compress_host_scratch_bytes(int64_t n, int grad_dtype, double ratio, int bits) {
+  const size_t ws = nsml_workspace_bytes(n, grad_dtype);
+  const size_t pb = nsml_payload_bytes(n, ratio, bits);
+  if (ws == 0 || pb == 0) return 0;
+  return align_up(ws, 256) + align_up((size_t)n * elem_size(grad_dtype), 256) +
+         align_up((size_t)((n + 31) / 32) * 4, 256) + align_up(pb, 256);
+}
+
+int nsml_compress_host(const void* grad_host, int64_t n, int grad_dtype, double ratio, int bits,
+                       const uint32_t* prune_mask_host, void* payload_host, size_t payload_capacity,
+                       void* device_scratch, size_t scratch_bytes, void* stream) {
+  if (grad_host == nullptr || payload_host == nullptr || device_scratch == nullptr) return NSML_ERR_ARG;
+  const size_t need = nsml_compress_host_scratch_bytes(n, grad_dtype, ratio, bits);
+  if (need == 0 || !aligned(device_scratch, 256)) return NSML_ERR_ARG;
+  const size_t pb = nsml_payload_bytes(n, ratio, bits);
+  if (scratch_bytes < need || payload_capacity < pb) return NSML_ERR_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned char* base = static_cast<unsigned char*>(device_scratch);
+  const size_t ws = align_up(nsml_workspace_bytes(n, grad_dtype), 256);
+  const size_t gbytes = (size_t)n * elem_size(grad_dtype);
+  const size_t mbytes = (size_t)((n + 31) / 32) * 4;
+  unsigned char* d_grad = base + ws;
+  unsigned char* d_mask = d_grad + align_up(gbytes, 256);
+  unsigned char* d_payload = d_mask + align_up(mbytes, 256);
+  if (cudaMemcpyAsync(d_grad, grad_host, gbytes, cudaMemcpyHostToDevice, st) != cudaSuccess) return NSML_ERR_CUDA;
+  if (prune_mask_host != nullptr &&
+      cudaMemcpyAsync(d_mask, prune_mask_host, mbytes, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return NSML_ERR_CUDA;
+  int rc = compress_impl(d_grad, n, grad_dtype, ratio, bits,
+                         prune_mask_host ? reinterpret_cast<const uint32_t*>(d_mask) : nullptr, d_payload, pb, base, ws,
+                         st);
+  if (rc != NSML_OK) return rc;
+  if (cudaMemcpyAsync(payload_host, d_payload, pb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return NSML_ERR_CUDA;
+  return NSML_OK;
+}
+
+size_t nsml_accumulate_host_scratch_bytes(int64_t n, int W, size_t total_payload_bytes) {
+  const size_t ws = nsml_accumulate_workspace_bytes(n, W);
+  if (ws == 0) return 0;
+  return align_up(ws, 256) + align_up((size_t)n * 4, 256) + total_payload_bytes + (size_t)W * 256;
+}
+
+int nsml_decompress_accumulate_host(const void* const* payloads_host, const size_t* payload_bytes, int W,
+                                    float* dense_host, int64_t n, int zero_first, void* device_scratch,
+                                    size_t scratch_bytes, void* stream) {
+  if (payloads_host == nullptr || payload_bytes == nullptr || dense_host == nullptr || device_scratch == nullptr)
+    return NSML_ERR_ARG;
+  if (W < 1 || W > NSML_MAX_WORKERS || !aligned(device_scratch, 256)) return NSML_ERR_ARG;
+  size_t total = 0;
+  for (int w = 0; w < W; ++w) {
+    if (payloads_host[w] == nullptr || payload_bytes[w] < sizeof(nsml_payload_header)) return NSML_ERR_ARG;
+    total += payload_bytes[w];
+  }
+  const size_t need = nsml_accumulate_host_scratch_bytes(n, W, total);
+  if (need == 0) return NSML_ERR_ARG;
+  if (scratch_bytes < need) return NSML_ERR_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  unsigned char* base = static_cast<unsigned char*>(device_scratch);
+  const size_t ws = align_up(nsml_accumulate_workspace_bytes(n, W), 256);
+  float* d_dense = reinterpret_cast<float*>(base + ws);
+  unsigned char* cursor = base + ws + align_up((size_t)n * 4, 256);
+  const void* d_payloads[NSML_MAX_WORKERS];
+  for (int w = 0; w < W; ++w) {
+    if (cudaMemcpyAsync(cursor, payloads_host[w], payload_bytes[w], cudaMemcpyHostToDevice, st) != cudaSuccess)
+      return NSML_ERR_CUDA;
+    d_payloads[w] = cursor;
+    cursor += align_up(payload_bytes[w], 256);
+  }
+  if (!zero_first &&
+      cudaMemcpyAsync(d_dense, dense_host, (size_t)n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+    return NSML_ERR_CUDA;
+  int rc = accumulate_impl(d_payloads, W, d_dense, n, zero_first, base, ws, st);
+  if (rc != NSML_OK) return rc;
+  if (cudaMemcpyAsync(dense_host, d_dense, (size_t)n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+    return NSML_ERR_CUDA;
+  return NSML_OK;
+}
+
+int nsml_last_status(const void* workspace, void* stream, int* status_out) {
+  if (workspace == nullptr || status_out == nullptr) return NSML_ERR_ARG;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int value = 0;
+  if (cudaMemcpyAsync(&value, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return NSML_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return NSML_ERR_CUDA;
+  *status_out = value;
+  return NSML_OK;
+}
+
+const char* nsml_strerror(int status) {
+  switch (status) {
+    case NSML_OK: return "ok";
+    case NSML_ERR_ARG: return "bad argument (null or misaligned pointer, size or enum out of range)";
+    case NSML_ERR_CAPACITY: return "payload buffer or workspace too small";
+    case NSML_ERR_CUDA: return "a CUDA runtime call failed";
+    case NSML_ERR_NONFINITE: return "the gradient bucket holds NaN or Inf";
+    case NSML_ERR_TIMEOUT: return "a bounded wait between thread blocks ran out";
+    case NSML_ERR_PAYLOAD: return "payload header or index out of range";
+    case NSML_ERR_INTERNAL: return "internal invariant failed: survivor count differs from k";
+    default: return "unknown status";
+  }
+}
+
+// ---- instrumentation -------------------------------------------------------
+int nsml_kernel_count(void) { return K_COUNT; }
+
+const char* nsml_kernel_name(int kernel_id) {
+  return (kernel_id >= 0 && kernel_id < K_COUNT) ? kKernelNames[kernel_id] : "";
+}
+
+int64_t nsml_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+int nsml_prof_enable(int on) {
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  if (!on) {
+    for (ProfRecord& r : g_prof_records) {
+      cudaEventDestroy(r.start);
+      cudaEventDestroy(r.stop);
+    }
+    g_prof_records.clear();
+  }
+  g_prof_on = (on != 0);
+  return NSML_OK;
+}
+
+int nsml_prof_read(int kernel_id, double* total_ms, int64_t* launches) {
+  if (kernel_id < 0 || kernel_id >= K_COUNT || total_ms == nullptr || launches == nullptr) return NSML_ERR_ARG;
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  prof_drain_locked();
+  *total_ms = g_prof_ms[kernel_id];
+  *launches = g_prof_launches[kernel_id];
+  return NSML_OK;
+}
+
+int nsml_prof_reset(void) {
+  std::lock_guard<std::mutex> lock(g_prof_mutex);
+  prof_drain_locked();
+  for (int i = 0; i < K_COUNT; ++i) {
+    g_prof_ms[i] = 0.0;
+    g_prof_launches[i] = 0;
+  }
+  return NSML_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,152 @@
+"""GPU parity: nsml_compress against the oracle, bit-exact (index sets, int8
+codes, scales, fp16 bit patterns), on small and adversarial buckets."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2506_16235_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+if torch.cuda.is_available():
+    import paper_2506_16235_b200 as nsml
+    from gpu_util import (assert_payload_equal, check_compress, gpu_compress, oracle_compress, to_device_grad)
+
+SIZES = [1, 2, 3, 4, 5, 7, 31, 32, 33, 127, 128, 129, 511, 512, 513, 4095, 4096, 4097, 8191, 12289, 100003]
+
+
+def make(kind, n, rng):
+    if kind == "normal":
+        return (rng.standard_normal(n) * 10.0 ** rng.uniform(-4, -1, n)).astype(np.float32)
+    if kind == "equal":
+        return np.full(n, -0.375, dtype=np.float32)
+    if kind == "zero":
+        g = np.zeros(n, dtype=np.float32)
+        g[rng.random(n) < 0.5] = -0.0
+        return g
+    if kind == "ties":
+        return (rng.integers(-3, 4, n) * 0.5).astype(np.float32)
+    if kind == "sparse":
+        g = rng.standard_normal(n).astype(np.float32)
+        g[rng.random(n) < 0.9] = 0.0
+        return g
+    if kind == "denormal":
+        bits = rng.integers(0, 1 << 12, n).astype(np.uint32)  # keys far below 2**19
+        bits |= (rng.integers(0, 2, n).astype(np.uint32) << 31)
+        return bits.view(np.float32)
+    if kind == "wide":
+        return (rng.standard_normal(n) * 10.0 ** rng.uniform(-38, 38, n)).astype(np.float32)
+    raise ValueError(kind)
+
+
+@pytest.mark.parametrize("kind", ["normal", "equal", "zero", "ties", "sparse", "denormal"])
+@pytest.mark.parametrize("n", SIZES)
+def test_small_buckets(kind, n):
+    rng = np.random.default_rng(n * 7 + len(kind))
+    g = make(kind, n, rng)
+    for ratio in (1e-9, 0.01, 0.3, 0.5, 1.0):
+        for bits in (8, 16):
+            check_compress(g, ratio, bits)
+
+
+def test_wide_range_saturates_fp16_and_keeps_int8_exact():
+    rng = np.random.default_rng(1)
+    g = make("wide", 50000, rng)
+    for ratio in (0.02, 0.7):
+        for bits in (8, 16):
+            check_compress(g, ratio, bits)
+
+
+def test_config1_full():
+    g = synth.config1_bucket()
+    payload, want = check_compress(g, 0.01, 8)
+    assert want.k == 10486 and want.scales.size == 11
+    check_compress(g, 0.01, 16)
+
+
+@pytest.mark.parametrize("ratio", [0.001, 0.05, 0.25, 0.8, 0.81, 1.0])
+def test_zero_heavy_bucket_all_ratios(ratio):
+    # 20 % zeros: ratios above 0.8 must fill up with zeros, lowest index first
+    g = synth.config1_bucket(n=300001, seed=3)
+    check_compress(g, ratio, 8)
+
+
+def test_threshold_ties_span_many_tiles():
+    rng = np.random.default_rng(5)
+    n = 40 * 4096 + 77
+    g = np.full(n, 0.25, dtype=np.float32)
+    g[rng.random(n) < 0.001] = 3.0
+    g[rng.random(n) < 0.3] *= -1.0
+    for ratio in (0.0005, 0.01, 0.5, 0.9999):
+        check_compress(g, ratio, 16)
+
+
+def test_prune_mask():
+    rng = np.random.default_rng(8)
+    for n in (37, 4096, 50001):
+        g = (rng.standard_normal(n)).astype(np.float32)
+        for ratio in (0.05, 0.5, 0.9):
+            # the paper's pruning rate for this ratio: 0.5 * (1 - ratio)
+            mask = rng.random(n) < 0.5 * (1.0 - ratio)
+            check_compress(g, ratio, 8, mask_bool=mask)
+            check_compress(g, ratio, 16, mask_bool=mask)
+    # everything pruned: k zeros, lowest indices
+    g = rng.standard_normal(1000).astype(np.float32)
+    payload, want = check_compress(g, 0.1, 16, mask_bool=np.ones(1000, bool))
+    assert want.idx.tolist() == list(range(100)) and not want.half.any()
+
+
+@pytest.mark.parametrize("n", [5, 4096, 70001])
+def test_bf16_buckets(n):
+    rng = np.random.default_rng(n)
+    g = synth.f32_to_bf16_bits((rng.standard_normal(n) * 10.0 ** rng.uniform(-6, -2, n)).astype(np.float32))
+    for ratio in (0.001, 0.1, 0.6):
+        for bits in (8, 16):
+            check_compress(g, ratio, bits)
+
+
+def test_nonfinite_is_reported_not_trapped():
+    rng = np.random.default_rng(2)
+    for bad in (np.inf, -np.inf, np.nan):
+        g = rng.standard_normal(9000).astype(np.float32)
+        g[4321] = bad
+        _, status = gpu_compress(g, 0.1, 8)
+        assert status == nsml.NSML_ERR_NONFINITE
+        with pytest.raises(oracle.NonFiniteGradient):
+            oracle_compress(g, 0.1, 8)
+    # the same workspace is usable afterwards
+    check_compress(rng.standard_normal(9000).astype(np.float32), 0.1, 8)
+
+
+def test_payload_is_bit_reproducible():
+    g = synth.config1_bucket(n=777777, seed=4)
+    a, _ = gpu_compress(g, 0.03, 8)
+    b, _ = gpu_compress(g, 0.03, 8)
+    assert torch.equal(a, b)
+
+
+def test_workspace_reuse_across_calls_and_sizes():
+    rng = np.random.default_rng(12)
+    ws = nsml.alloc_bytes(nsml.nsml_workspace_bytes(200000), "cuda")
+    for n, ratio, bits in ((200000, 0.01, 8), (1234, 0.5, 16), (199999, 0.2, 8), (4096, 1.0, 16)):
+        g = rng.standard_normal(n).astype(np.float32)
+        grad = to_device_grad(g)
+        payload = nsml.nsml_compress(grad, ratio, bits, workspace=ws)
+        assert nsml.nsml_last_status(ws) == 0
+        assert_payload_equal(payload, oracle_compress(g, ratio, bits))
+
+
+def test_runtime_argument_errors():
+    grad = torch.zeros(1000, device="cuda")
+    with pytest.raises(nsml.NsmlError) as e:
+        nsml.nsml_compress(grad, 0.5, 8, payload=torch.zeros(64, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == nsml.NSML_ERR_CAPACITY
+    with pytest.raises(nsml.NsmlError) as e:
+        nsml.nsml_compress(grad, 0.5, 8, workspace=torch.zeros(1024, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == nsml.NSML_ERR_CAPACITY
+    with pytest.raises(nsml.NsmlError):
+        nsml.nsml_compress(grad, 0.0, 8)
+    with pytest.raises(nsml.NsmlError) as e:
+        nsml.nsml_compress(grad[1:], 0.5, 8)  # 4-byte offset: not 16-byte aligned
+    assert e.value.status == nsml.NSML_ERR_ARG
