@@ -48,9 +48,10 @@ def test_identical_payloads_sum_exactly():
     n = 50000
     g = worker_grads(n, 1, 3)[0]
     payload, want = check_compress(g, 0.2, 8)
-    got, _ = check_accumulate([payload] * 8, [want] * 8, n, zero_first=True)
+    check_accumulate([payload] * 8, [want] * 8, n, zero_first=True)  # sequential float32 adds: within tolerance
+    got, _ = check_accumulate([payload] * 2, [want] * 2, n, zero_first=True)
     one, _ = check_accumulate([payload], [want], n, zero_first=True)
-    assert np.array_equal(got, 8 * one)
+    assert np.array_equal(got, 2 * one)  # v + v is exact
     twice, _ = check_accumulate([payload], [want], n, zero_first=False, dense_init=one)
     assert np.array_equal(twice, 2 * one)
 
