@@ -120,12 +120,10 @@ class Workload:
     def compress_bytes(self, acc, n, esize, k, bits):
         vb = 1 if bits == 8 else 2
         s = 4 * ((k + 1023) // 1024) if bits == 8 else 0
-        self.account(acc, "k_histogram<0,bucket>", esize * n)
+        self.account(acc, "k_sample", 4 * 8192)
         self.account(acc, "k_compact_bucket", esize * n + 8 * k)
-        self.account(acc, "k_histogram<1,list>", 4 * k)
-        self.account(acc, "k_histogram<2,list>", 4 * k)
-        self.account(acc, "k_compact_list", 16 * k)
-        self.account(acc, "k_quantize", 4 * k + vb * k + s)
+        # list stage: candidates read once per phase (5 x 4k keys + 4k indices), survivors written and re-read
+        self.account(acc, "k_finalize", 24 * k + 8 * k + 4 * k + vb * k + s)
 
     def merge_bytes(self, acc, n, ks_bits, zero_first=True):
         total = 4 * n if zero_first else 0
@@ -503,6 +501,8 @@ def main():
     ap.add_argument("--impl", default="nsml", choices=["nsml", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-large-bucket-leg", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (e2e is then null)")
+    ap.add_argument("--no-kernel-times", action="store_true", help="skip the event-bracketed per-kernel pass")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -564,51 +564,54 @@ def main():
 
     # ---- per-kernel device time (same steps again, every launch bracketed by CUDA events) ----
     peak, peak_kind = measured_peak_gbs()
-    acc = {}
-    nsml.nsml_prof_reset()
-    nsml.nsml_prof_enable(True)
-    prof_steps = max(1, min(steps, 10))
-    for i in range(prof_steps):
-        wl.step(warmup + steps + i, acc)
-    torch.cuda.synchronize()
-    prof = nsml.nsml_prof_read()
-    nsml.nsml_prof_enable(False)
-    kernels = {}
-    for name, (ms, cnt) in prof.items():
-        if cnt:
-            gbs = acc.get(name, 0) / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
-            kernels[name] = {"launches_per_step": cnt / prof_steps, "us_per_launch": 1e3 * ms / cnt,
-                             "ms_per_step": ms / prof_steps, "algorithmic_GBps": gbs, "frac_of_peak": gbs / peak}
-    dominant = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
-    d = kernels[dominant]
-    roofline = {"bound": "hbm", "kernel": dominant, "achieved": d["algorithmic_GBps"], "peak": peak,
-                "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": d["algorithmic_GBps"] / peak,
-                "frac_of_nominal_8TBps": d["algorithmic_GBps"] / 8000.0, "traffic": None,
-                "us_per_launch": d["us_per_launch"]}
+    kernels, roofline = {}, None
+    if not args.no_kernel_times:
+        acc = {}
+        nsml.nsml_prof_reset()
+        nsml.nsml_prof_enable(True)
+        prof_steps = max(1, min(steps, 10))
+        for i in range(prof_steps):
+            wl.step(warmup + steps + i, acc)
+        torch.cuda.synchronize()
+        prof = nsml.nsml_prof_read()
+        nsml.nsml_prof_enable(False)
+        for name, (ms, cnt) in prof.items():
+            if cnt:
+                gbs = acc.get(name, 0) / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
+                kernels[name] = {"launches_per_step": cnt / prof_steps, "us_per_launch": 1e3 * ms / cnt,
+                                 "ms_per_step": ms / prof_steps, "algorithmic_GBps": gbs, "frac_of_peak": gbs / peak}
+        dominant = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
+        d = kernels[dominant]
+        roofline = {"bound": "hbm", "kernel": dominant, "achieved": d["algorithmic_GBps"], "peak": peak,
+                    "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": d["algorithmic_GBps"] / peak,
+                    "frac_of_nominal_8TBps": d["algorithmic_GBps"] / 8000.0, "traffic": None,
+                    "us_per_launch": d["us_per_launch"]}
 
     # ---- end to end through the host-buffer entry points ----
-    wl.setup_host()
-    host_steps = max(1, min(steps, 5))
-    for i in range(2):
-        wl.step_host(i)
-    torch.cuda.synchronize()
-    hv0, hv1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    hv0.record()
-    h2d = d2h = 0
-    for i in range(host_steps):
-        h2d, d2h = wl.step_host(i)
-    hv1.record()
-    torch.cuda.synchronize()
-    host_ms = hv0.elapsed_time(hv1)
-    if dist is not None:
-        t = torch.tensor([host_ms], device=device, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        host_ms = float(t.item())
-    host_bytes = getattr(wl, "host_input_bytes", wl.input_bytes_per_step)
-    e2e = {"value": world * host_steps * host_bytes / (host_ms * 1e-3) / 1e9, "unit": UNIT,
-           "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": host_steps,
-           "ms_per_step": host_ms / host_steps}
+    e2e = None
+    if not args.no_e2e:
+        wl.setup_host()
+        host_steps = max(1, min(steps, 5))
+        for i in range(2):
+            wl.step_host(i)
+        torch.cuda.synchronize()
+        hv0, hv1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        hv0.record()
+        h2d = d2h = 0
+        for i in range(host_steps):
+            h2d, d2h = wl.step_host(i)
+        hv1.record()
+        torch.cuda.synchronize()
+        host_ms = hv0.elapsed_time(hv1)
+        if dist is not None:
+            t = torch.tensor([host_ms], device=device, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            host_ms = float(t.item())
+        host_bytes = getattr(wl, "host_input_bytes", wl.input_bytes_per_step)
+        e2e = {"value": world * host_steps * host_bytes / (host_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": host_steps,
+               "ms_per_step": host_ms / host_steps}
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,

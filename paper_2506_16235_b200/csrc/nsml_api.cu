@@ -10,25 +10,14 @@
 #include "nsml_codec.cuh"
 #include "nsml_common.cuh"
 #include "nsml_compact.cuh"
+#include "nsml_finalize.cuh"
 #include "nsml_select.cuh"
 
 namespace nsml {
 
-enum KernelId {
-  K_HIST_BUCKET = 0,
-  K_COMPACT_BUCKET,
-  K_HIST_LIST_1,
-  K_HIST_LIST_2,
-  K_COMPACT_LIST,
-  K_QUANTIZE,
-  K_PARTITION,
-  K_MERGE,
-  K_COUNT
-};
+enum KernelId { K_SAMPLE = 0, K_COMPACT_BUCKET, K_FINALIZE, K_PARTITION, K_MERGE, K_COUNT };
 
-static const char* const kKernelNames[K_COUNT] = {
-    "k_histogram<0,bucket>", "k_compact_bucket", "k_histogram<1,list>", "k_histogram<2,list>",
-    "k_compact_list",        "k_quantize",       "k_partition",         "k_merge"};
+static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_compact_bucket", "k_finalize", "k_partition", "k_merge"};
 
 static std::atomic<int64_t> g_launches{0};
 
@@ -81,7 +70,7 @@ struct LaunchScope {  // brackets one kernel launch
 struct DeviceInfo {
   bool ready = false;
   int sms = 0;
-  int compact_f32 = 0, compact_bf16 = 0, compact_list = 0, merge = 0;  // resident blocks per SM
+  int compact_bucket = 0, finalize = 0, merge = 0;  // resident blocks per SM
 };
 static DeviceInfo g_dev[64];
 static std::mutex g_dev_mutex;
@@ -94,11 +83,17 @@ static int device_info(const DeviceInfo** out) {
   if (!d.ready) {
     if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return NSML_ERR_CUDA;
     cudaError_t e = cudaSuccess;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_f32, k_compact_bucket<NSML_F32>, kCta, 0);
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_bf16, k_compact_bucket<NSML_BF16>, kCta, 0);
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_list, k_compact_list, kCta, 0);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_bucket, k_compact_bucket<NSML_F32>, kCta, 0);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.finalize, k_finalize<NSML_F32>, kCta, 0);
+    if (e == cudaSuccess) {
+      int bf = 0;
+      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bf, k_finalize<NSML_BF16>, kCta, 0);
+      if (bf < d.finalize) d.finalize = bf;
+    }
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.merge, k_merge, kCta, 0);
-    if (e != cudaSuccess || d.compact_f32 < 1 || d.compact_bf16 < 1 || d.compact_list < 1 || d.merge < 1) {
+    int coop = 0;
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
+    if (e != cudaSuccess || d.compact_bucket < 1 || d.finalize < 1 || d.merge < 1 || !coop) {
       cudaGetLastError();
       return NSML_ERR_CUDA;
     }
@@ -126,26 +121,67 @@ static int64_t k_of(int64_t n, double ratio) {
   return k;
 }
 
+// Rank (from the top, 1-based) of the sample key that becomes the bracket's
+// lower bound: the expected rank of the k-th largest among kSamples draws plus
+// six standard deviations.  0 = do not sample (small bucket, or nearly
+// everything is kept): the bracket then starts at key 0.
+static unsigned int sample_rank(int64_t n, int64_t k) {
+  if (n < 2 * (int64_t)kSamples) return 0;
+  const double p = (double)k / (double)n;
+  const double j = std::ceil(kSamples * p + 6.0 * std::sqrt(kSamples * p * (1.0 - p))) + 1.0;
+  if (j >= (double)kSamples) return 0;
+  return (unsigned int)j;
+}
+
 template <int DTYPE>
-static void launch_bucket_stage(const void* grad, const uint32_t* mask, int64_t n, int64_t k, unsigned char* ws,
-                                const CompressLayout& L, const DeviceInfo& dev, cudaStream_t st) {
+static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, int64_t k, int bits, unsigned char* ws,
+                           unsigned char* payload, const CompressLayout& L, const PayloadLayout& P,
+                           const DeviceInfo& dev, cudaStream_t st) {
   Ctl* ctl = reinterpret_cast<Ctl*>(ws);
-  unsigned int* hist = reinterpret_cast<unsigned int*>(ws + L.hist);
+  uint32_t* seg_idx = reinterpret_cast<uint32_t*>(ws + L.seg_idx);
+  uint32_t* seg_val = reinterpret_cast<uint32_t*>(ws + L.seg_val);
+  unsigned int* seg_count = reinterpret_cast<unsigned int*>(ws + L.seg_count);
   BucketSrc<DTYPE> src{grad, mask};
   {
-    LaunchScope scope(K_HIST_BUCKET, st);
-    unsigned int grid = grid_for((unsigned long long)n, kCta * 4 * 4, dev.sms * 4);
-    k_histogram<0, BucketSrc<DTYPE>><<<grid, kCta, 0, st>>>(src, (unsigned long long)n, (unsigned long long)k, ctl, hist);
+    LaunchScope scope(K_SAMPLE, st);
+    k_sample<DTYPE><<<1, kSampleThreads, 0, st>>>(src, (unsigned long long)n, sample_rank(n, k), ctl,
+                                                  reinterpret_cast<uint4*>(ws), (unsigned int)(L.zero_bytes / 16));
   }
+  // bucket pass: one block per 16K elements, at most what the device keeps resident
+  const unsigned int grid = grid_for((unsigned long long)n, kCta * 64, dev.sms * dev.compact_bucket);
+  const unsigned int segments = grid * (kCta / 32);
   {
     LaunchScope scope(K_COMPACT_BUCKET, st);
-    int occ = (DTYPE == NSML_F32) ? dev.compact_f32 : dev.compact_bf16;
-    unsigned int grid = grid_for((unsigned long long)n, kTile, dev.sms * occ);
-    k_compact_bucket<DTYPE><<<grid, kCta, 0, st>>>(src, (unsigned long long)n, ctl,
-                                                   reinterpret_cast<unsigned long long*>(ws + L.state_bucket),
-                                                   reinterpret_cast<uint32_t*>(ws + L.list_idx),
-                                                   reinterpret_cast<uint32_t*>(ws + L.list_val));
+    k_compact_bucket<DTYPE><<<grid, kCta, 0, st>>>(src, (unsigned long long)n, ctl, seg_idx, seg_val, seg_count);
   }
+  // list stage: cooperative, every block co-resident, at most kMaxSegPerBlock segments per block
+  unsigned int fgrid = (unsigned int)(dev.sms * dev.finalize);
+  if (fgrid > grid) fgrid = grid;
+  if (fgrid > (unsigned int)kMaxFinalizeBlocks) fgrid = kMaxFinalizeBlocks;
+  if ((segments + fgrid - 1) / fgrid + 1 > (unsigned int)kMaxSegPerBlock) return NSML_ERR_CUDA;
+  FinalizeParams fp;
+  fp.n = (unsigned long long)n;
+  fp.k = (unsigned long long)k;
+  fp.bits = bits;
+  fp.segments = segments;
+  fp.ctl = ctl;
+  fp.hist = reinterpret_cast<unsigned int*>(ws + L.hist);
+  fp.block_counts = reinterpret_cast<unsigned long long*>(ws + L.block_counts);
+  fp.seg_count = seg_count;
+  fp.seg_zeros = reinterpret_cast<unsigned int*>(ws + L.seg_zeros);
+  fp.seg_idx = seg_idx;
+  fp.seg_val = seg_val;
+  fp.raw_val = reinterpret_cast<float*>(ws + L.raw_val);
+  fp.payload = payload;
+  fp.P = P;
+  {
+    LaunchScope scope(K_FINALIZE, st);
+    void* args[] = {&src, &fp};
+    if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_finalize<DTYPE>), dim3(fgrid), dim3(kCta), args, 0, st) !=
+        cudaSuccess)
+      return NSML_ERR_CUDA;
+  }
+  return NSML_OK;
 }
 
 static int compress_impl(const void* grad, int64_t n, int grad_dtype, double ratio, int bits,
@@ -164,42 +200,11 @@ static int compress_impl(const void* grad, int64_t n, int grad_dtype, double rat
   const DeviceInfo* dev = nullptr;
   int rc = device_info(&dev);
   if (rc != NSML_OK) return rc;
-
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   unsigned char* pl = static_cast<unsigned char*>(payload);
-  Ctl* ctl = reinterpret_cast<Ctl*>(ws);
-  unsigned int* hist = reinterpret_cast<unsigned int*>(ws + L.hist);
-  if (cudaMemsetAsync(ws, 0, L.zero_bytes, st) != cudaSuccess) return NSML_ERR_CUDA;
-
-  if (grad_dtype == NSML_F32) launch_bucket_stage<NSML_F32>(grad, prune_mask, n, k, ws, L, *dev, st);
-  else launch_bucket_stage<NSML_BF16>(grad, prune_mask, n, k, ws, L, *dev, st);
-
-  ListSrc list{reinterpret_cast<const uint32_t*>(ws + L.list_idx), reinterpret_cast<const uint32_t*>(ws + L.list_val)};
-  const unsigned int list_grid = (unsigned int)(dev->sms * 2);
-  {
-    LaunchScope scope(K_HIST_LIST_1, st);
-    k_histogram<1, ListSrc><<<list_grid, kCta, 0, st>>>(list, 0ull, (unsigned long long)k, ctl, hist);
-  }
-  {
-    LaunchScope scope(K_HIST_LIST_2, st);
-    k_histogram<2, ListSrc><<<list_grid, kCta, 0, st>>>(list, 0ull, (unsigned long long)k, ctl, hist);
-  }
-  {
-    LaunchScope scope(K_COMPACT_LIST, st);
-    unsigned int grid = (unsigned int)(dev->sms * dev->compact_list);
-    k_compact_list<<<grid, kCta, 0, st>>>(list, ctl, reinterpret_cast<unsigned long long*>(ws + L.state_list),
-                                          reinterpret_cast<uint32_t*>(pl + P.idx_off),
-                                          reinterpret_cast<uint32_t*>(ws + L.raw_val));
-  }
-  {
-    LaunchScope scope(K_QUANTIZE, st);
-    unsigned int grid = (unsigned int)((k + NSML_QBLOCK - 1) / NSML_QBLOCK);
-    const float* raw = reinterpret_cast<const float*>(ws + L.raw_val);
-    if (bits == NSML_BITS_INT8)
-      k_quantize<NSML_BITS_INT8><<<grid, kCta, 0, st>>>(raw, (unsigned long long)k, (unsigned long long)n, ctl, pl, P);
-    else
-      k_quantize<NSML_BITS_FP16><<<grid, kCta, 0, st>>>(raw, (unsigned long long)k, (unsigned long long)n, ctl, pl, P);
-  }
+  if (grad_dtype == NSML_F32) rc = launch_compress<NSML_F32>(grad, prune_mask, n, k, bits, ws, pl, L, P, *dev, st);
+  else rc = launch_compress<NSML_BF16>(grad, prune_mask, n, k, bits, ws, pl, L, P, *dev, st);
+  if (rc != NSML_OK) return rc;
   if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
   return NSML_OK;
 }

@@ -1,202 +1,109 @@
-// Ordered stream compaction (Alg. 2 Steps 2-3: drop the pruned and the
-// small-magnitude gradients, keep (index, value) of the rest in index order).
+// Bucket -> segmented candidate list: the one full pass over the bucket
+// (Alg. 2 Steps 2-3: pruned gradients read as zero; everything whose magnitude
+// is below the sampled lower bound is dropped here, in one streaming read).
 //
-// One pass over the source.  Every element falls in one of three classes by
-// its magnitude key: A (key >= hi) is always kept, C (lo <= key < hi) is kept
-// while fewer than r class-C elements precede it in index order, the rest is
-// dropped.  With r = "all" this writes a superset list for the later digit
-// levels; with lo = T, hi = T+1 it applies the final threshold and tie budget.
-//
-// Tiles of kTile elements are handed out by an atomic ticket, so a tile's
-// predecessors have always started.  Output offsets come from a chained scan
-// over tiles (publish own counts, look back over predecessors until an
-// inclusive prefix is found).  Every wait is bounded: when it runs out the
-// block records NSML_ERR_TIMEOUT, marks its tile so that successors stop too,
-// and leaves.
+// Warp w owns a contiguous range of 128-element rounds and appends what it
+// keeps (every key >= lo, lo >= 1) to its own segment of the list.  A segment
+// starts at the list position of the range's first element, so it can never
+// overflow and needs no allocation.  There is no block or grid
+// synchronisation: a warp's only state is its running count.  Segments taken
+// in warp order are in index order.
 #pragma once
 
 #include "nsml_common.cuh"
 
 namespace nsml {
 
-__device__ __forceinline__ unsigned long long pack_counts(unsigned long long a, unsigned long long c) {
-  return (a << 31) | c;
+constexpr int kRound = 128;  // elements a warp handles per step (32 lanes x 4)
+constexpr int kUnroll = 4;   // rounds in flight per warp
+
+__host__ __device__ inline unsigned long long warp_first_round(unsigned long long warp, unsigned long long warps,
+                                                               unsigned long long rounds) {
+  return warp * rounds / warps;
 }
 
-__device__ __forceinline__ unsigned long long load_state(const unsigned long long* p) {
-  return *reinterpret_cast<const volatile unsigned long long*>(p);
-}
-
-__device__ __forceinline__ void store_state(unsigned long long* p, unsigned long long v) {
-  *reinterpret_cast<volatile unsigned long long*>(p) = v;
-}
-
-// Runs in warp 0 of the block that owns `tile`.  Returns the packed exclusive
-// prefix (A << 31 | C) of the tile, or ~0 if the scan was abandoned.
-__device__ unsigned long long chained_scan(unsigned long long* state, unsigned int tile,
-                                           unsigned long long own, int* status) {
+// Appends the kept elements of one round.  `f` holds this lane's four keep
+// flags (bit e = element lane*4+e of the round).  Returns the round's total.
+__device__ __forceinline__ unsigned int append_round(unsigned int f, const uint32_t (&bits)[4], uint32_t first_index,
+                                                     unsigned long long out_base, uint32_t* __restrict__ seg_idx,
+                                                     uint32_t* __restrict__ seg_val) {
   const int lane = threadIdx.x & 31;
-  if (tile == 0) {
-    if (lane == 0) store_state(state, kFlagPrefix | own);
-    return 0;
-  }
-  if (lane == 0) store_state(state + tile, kFlagAggregate | own);
-
-  unsigned long long excl = 0;
-  long long window_end = (long long)tile - 1;  // nearest predecessor of this window
-  while (true) {
-    const long long mine = window_end - lane;
-    unsigned long long w = kFlagPrefix;  // tiles before 0 count as an empty prefix
-    int polls = 0;
-    bool gave_up = false;
-    if (mine >= 0) {
-      w = load_state(state + mine);
-      while ((w & kFlagMask) == 0) {
-        if (++polls > kMaxPolls) { gave_up = true; break; }
-        __nanosleep(polls < 64 ? 20 : 400);
-        w = load_state(state + mine);
-      }
-    }
-    const unsigned int gave_up_mask = __ballot_sync(0xFFFFFFFFu, gave_up);
-    const unsigned int abort_mask = __ballot_sync(0xFFFFFFFFu, (w & kFlagMask) == kFlagAbort);
-    if (gave_up_mask | abort_mask) {
-      if (lane == 0) {
-        if (gave_up_mask) set_status(status, NSML_ERR_TIMEOUT);
-        store_state(state + tile, kFlagAbort);
-      }
-      return ~0ull;
-    }
-    // nearest predecessor (lowest lane) that already holds an inclusive prefix
-    const unsigned int has_prefix = __ballot_sync(0xFFFFFFFFu, (w & kFlagMask) == kFlagPrefix);
-    const int stop = has_prefix ? (__ffs(has_prefix) - 1) : 32;
-    unsigned long long contrib = (lane <= stop) ? (w & ~kFlagMask) : 0ull;
+  const unsigned int lt = (1u << lane) - 1u;
+  const unsigned int any = __ballot_sync(0xFFFFFFFFu, f != 0);
+  const unsigned int multi = __ballot_sync(0xFFFFFFFFu, (f & (f - 1)) != 0);
+  unsigned int before, total;
+  if (multi == 0) {  // usual case: no lane keeps more than one element
+    before = __popc(any & lt);
+    total = __popc(any);
+  } else {
+    const unsigned int mine = __popc(f);
+    unsigned int incl = mine;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) contrib += __shfl_xor_sync(0xFFFFFFFFu, contrib, o);
-    excl += contrib;
-    if (has_prefix) break;
-    window_end -= 32;
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    before = incl - mine;
+    total = __shfl_sync(0xFFFFFFFFu, incl, 31);
   }
-  if (lane == 0) store_state(state + tile, kFlagPrefix | (excl + own));
-  return excl;
+  if (f != 0) {
+    unsigned long long pos = out_base + before;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (f & (1u << e)) {
+        seg_idx[pos] = first_index + lane * 4 + e;
+        seg_val[pos] = bits[e];
+        ++pos;
+      }
+    }
+  }
+  return total;
 }
 
-// Compacts `count` elements of `src` into out_idx / out_val.  All threads of
-// all blocks call this; returns when the ticket runs past the last tile.
-template <class Src>
-__device__ void compact_tiles(const Src& src, unsigned long long count, uint32_t lo, uint32_t hi,
-                              unsigned long long r, unsigned int* ticket, unsigned long long* state,
-                              int* status, uint32_t* __restrict__ out_idx, uint32_t* __restrict__ out_val,
-                              unsigned long long* total_out) {
-  __shared__ unsigned int s_tile;
-  __shared__ unsigned int s_warp[kCta / 32];
-  __shared__ unsigned long long s_excl;
-
-  const int lane = threadIdx.x & 31;
-  const int warp = threadIdx.x >> 5;
-
-  while (true) {
-    __syncthreads();  // previous tile's shared values are no longer needed
-    if (threadIdx.x == 0) s_tile = atomicAdd(ticket, 1u);
-    __syncthreads();
-    const unsigned int tile = s_tile;
-    const unsigned long long base = (unsigned long long)tile * kTile;
-    if (base >= count) return;
-
-    // each warp owns 512 consecutive elements: 4 rounds of 32 lanes x 4
-    Quad q[4];
-    unsigned int fa[4], fc[4];      // per-round class flags, bit e = element e
-    unsigned int excl_round[4];     // packed (A | C << 16) before this lane's quad, within the warp
-    unsigned int running = 0;
-#pragma unroll
-    for (int j = 0; j < 4; ++j) q[j] = src.load4(base + warp * 512 + j * 128 + lane * 4, count);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      fa[j] = 0;
-      fc[j] = 0;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const uint32_t key = q[j].bits[e] & 0x7FFFFFFFu;
-        const bool v = (q[j].valid >> e) & 1u;
-        const bool a = v && key >= hi;
-        const bool c = v && !a && key >= lo;
-        fa[j] |= (unsigned)a << e;
-        fc[j] |= (unsigned)c << e;
-      }
-      const unsigned int mine = __popc(fa[j]) | (__popc(fc[j]) << 16);
-      unsigned int incl = mine;
-#pragma unroll
-      for (int o = 1; o < 32; o <<= 1) {
-        unsigned int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += up;
-      }
-      excl_round[j] = running + incl - mine;
-      running += __shfl_sync(0xFFFFFFFFu, incl, 31);
-    }
-    if (lane == 0) s_warp[warp] = running;
-    __syncthreads();
-
-    unsigned int before_warp = 0, tile_total = 0;
-#pragma unroll
-    for (int w = 0; w < kCta / 32; ++w) {
-      const unsigned int c = s_warp[w];
-      if (w < warp) before_warp += c;
-      tile_total += c;
-    }
-
-    if (warp == 0) {
-      const unsigned long long own = pack_counts(tile_total & 0xFFFFu, tile_total >> 16);
-      const unsigned long long e = chained_scan(state, tile, own, status);
-      if (lane == 0) s_excl = e;
-    }
-    __syncthreads();
-    const unsigned long long excl = s_excl;
-    if (excl == ~0ull) return;  // abandoned: every thread of the block leaves
-
-    const unsigned long long a0 = (excl >> 31) + (before_warp & 0xFFFFu);
-    const unsigned long long c0 = (excl & kCountMask) + (before_warp >> 16);
-#pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      if ((fa[j] | fc[j]) == 0) continue;
-      unsigned long long a_before = a0 + (excl_round[j] & 0xFFFFu);
-      unsigned long long c_before = c0 + (excl_round[j] >> 16);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const bool a = (fa[j] >> e) & 1u;
-        const bool c = (fc[j] >> e) & 1u;
-        if (a || (c && c_before < r)) {
-          const unsigned long long pos = a_before + (c_before < r ? c_before : r);
-          out_idx[pos] = q[j].idx[e];
-          out_val[pos] = q[j].bits[e];
-        }
-        a_before += a;
-        c_before += c;
-      }
-    }
-
-    if (base + kTile >= count && threadIdx.x == 0) {
-      const unsigned long long a_all = (excl >> 31) + (tile_total & 0xFFFFu);
-      const unsigned long long c_all = (excl & kCountMask) + (tile_total >> 16);
-      *total_out = a_all + (c_all < r ? c_all : r);
-    }
-  }
-}
-
-// Bucket -> candidate list (superset of the survivors, or the survivors
-// themselves when the threshold is already final).
 template <int DTYPE>
 __global__ void __launch_bounds__(kCta)
-k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, unsigned long long* state,
-                 uint32_t* list_idx, uint32_t* list_val) {
-  compact_tiles(src, n, ctl->lo, ctl->hi, ctl->r, &ctl->ticket_bucket, state, &ctl->status,
-                list_idx, list_val, &ctl->list_count);
-}
+k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, uint32_t* __restrict__ seg_idx,
+                 uint32_t* __restrict__ seg_val, unsigned int* __restrict__ seg_count) {
+  const int lane = threadIdx.x & 31;
+  const unsigned long long warp = (unsigned long long)blockIdx.x * (kCta / 32) + (threadIdx.x >> 5);
+  const unsigned long long warps = (unsigned long long)gridDim.x * (kCta / 32);
+  const unsigned long long rounds = (n + kRound - 1) / kRound;
+  const unsigned long long first = warp_first_round(warp, warps, rounds);
+  const unsigned long long last = warp_first_round(warp + 1, warps, rounds);
+  // Zeros are never candidates here; if they are needed (fewer than k non-zero
+  // keys) the list comes out short and the finalize kernel's slow path adds them.
+  // |v| >= t on floats equals key >= lo for finite v; written as !(|v| < t) so
+  // that NaN is kept too (the finalize kernel reports non-finite candidates).
+  const float t = __uint_as_float(max(ctl->lo, 1u));
+  const unsigned long long seg_base = first * kRound;
+  const unsigned long long full_rounds = n / kRound;  // rounds that need no bounds checks
+  unsigned int kept = 0;
 
-// Candidate list -> final (index, raw value) arrays, applying the exact
-// threshold key and tie budget.
-__global__ void __launch_bounds__(kCta)
-k_compact_list(ListSrc src, Ctl* ctl, unsigned long long* state, uint32_t* out_idx, uint32_t* out_val) {
-  compact_tiles(src, ctl->list_count, ctl->lo, ctl->hi, ctl->r, &ctl->ticket_list, state, &ctl->status,
-                out_idx, out_val, &ctl->out_count);
+  unsigned long long rd = first;
+  const unsigned long long last_full = min(last, full_rounds);
+  for (; rd + kUnroll <= last_full; rd += kUnroll) {
+    uint32_t bits[kUnroll][4];
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) src.load_full4((rd + u) * kRound + lane * 4, bits[u]);
+#pragma unroll
+    for (int u = 0; u < kUnroll; ++u) {
+      unsigned int f = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) f |= (unsigned)(!(fabsf(__uint_as_float(bits[u][e])) < t)) << e;
+      if (!__any_sync(0xFFFFFFFFu, f != 0)) continue;
+      kept += append_round(f, bits[u], (uint32_t)((rd + u) * kRound), seg_base + kept, seg_idx, seg_val);
+    }
+  }
+  for (; rd < last; ++rd) {  // leftover rounds, the last of which may be partial
+    uint32_t bits[4];
+    src.load_vals4(rd * kRound + lane * 4, n, bits);  // missing elements read as 0 and are never kept
+    unsigned int f = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) f |= (unsigned)(!(fabsf(__uint_as_float(bits[e])) < t)) << e;
+    if (!__any_sync(0xFFFFFFFFu, f != 0)) continue;
+    kept += append_round(f, bits, (uint32_t)(rd * kRound), seg_base + kept, seg_idx, seg_val);
+  }
+  if (lane == 0) seg_count[warp] = kept;
 }
 
 }  // namespace nsml

@@ -1,159 +1,115 @@
-// Radix-select threshold search on the magnitude keys (Alg. 2 Step 3: which
+// Sampled lower bound for the top-k threshold (Alg. 2 Step 3: which
 // k = ceil(ratio*n) gradients have the largest absolute value).
 //
-// Level 0 histograms the top digit over the whole bucket; the block that
-// finishes last resolves the bin that holds the k-th largest key.  The bucket
-// compaction then keeps every key in or above that bin (a superset of the
-// survivors); levels 1 and 2 histogram the remaining digits over that short
-// list only, which pins the exact threshold key T and the tie budget r.
+// The bucket is streamed exactly once, by the compaction pass, which needs a
+// key `lo` such that a little more than k keys are >= lo.  k_sample draws one
+// element from each of 8192 equal strata of the bucket and radix-selects,
+// inside one thread block, the sample key whose rank leaves a six-sigma margin
+// above the expected rank of the k-th largest; lo is that key rounded down to
+// its top 24 bits.  The exact threshold is found afterwards on the short
+// candidate list (nsml_finalize.cuh), which also repairs the rare case of a
+// misleading sample, so the sample only decides how much work is done, never
+// the result.
 #pragma once
 
 #include "nsml_common.cuh"
 
 namespace nsml {
 
-// Called by all threads of the last block of a histogram level.  Finds the
-// digit d with  #{digit > d} < k_rem <= #{digit >= d}  among the keys that
-// match the current prefix, and advances the selection state.
-template <int LEVEL>
-__device__ void resolve_level(Ctl* ctl, const unsigned int* ghist, unsigned long long k_first) {
-  constexpr int NB = 1 << digit_bits(LEVEL);
-  constexpr int PER = (NB + kCta - 1) / kCta;
-  __shared__ unsigned long long s_part[kCta];
-  const int t = threadIdx.x;
+constexpr int kSampleThreads = 1024;
+constexpr int kSamplesPerThread = 8;
+constexpr int kSamples = kSampleThreads * kSamplesPerThread;  // 8192 strata
 
-  unsigned long long part = 0;
-#pragma unroll
-  for (int b = 0; b < PER; ++b) {
-    int bin = t * PER + b;
-    if (bin < NB) part += __ldcg(ghist + bin);
-  }
-  s_part[t] = part;
-  __syncthreads();
-
-  if (t == 0) {
-    const unsigned long long k_rem = (LEVEL == 0) ? k_first : ctl->k_rem;
-    unsigned long long above = 0;
-    int chunk = kCta - 1;
-    for (; chunk > 0; --chunk) {
-      if (above + s_part[chunk] >= k_rem) break;
-      above += s_part[chunk];
-    }
-    int d = min(NB - 1, chunk * PER + PER - 1);
-    for (; d > chunk * PER; --d) {
-      unsigned long long c = __ldcg(ghist + d);
-      if (above + c >= k_rem) break;
-      above += c;
-    }
-    // `above` keys are strictly above digit d; the k_rem-th largest is in d.
-    const unsigned long long in_bin = __ldcg(ghist + d);
-    unsigned long long rem = k_rem - above;  // 1 <= rem <= in_bin
-    const unsigned int prefix = (LEVEL == 0) ? (unsigned)d : ((ctl->prefix << digit_bits(LEVEL)) | (unsigned)d);
-    ctl->prefix = prefix;
-
-    if (LEVEL == 0) {
-      unsigned int lo = prefix << digit_shift(0);
-      const unsigned int hi = (prefix + 1u) << digit_shift(0);
-      unsigned long long r = ~0ull;  // keep every key of the boundary bin
-      unsigned int exact = 0;
-      if (d == 0) {
-        // The boundary bin holds the zeros.  If the non-zero keys run out
-        // before k is reached the threshold key is exactly 0 and the tie
-        // budget is known now; otherwise zeros are certainly not survivors.
-        const unsigned long long nz = in_bin - *(volatile unsigned long long*)&ctl->zero_count;
-        if (rem > nz) {
-          lo = 0;
-          r = rem - nz;
-          exact = 1;
-          ctl->lo = 0;
-          ctl->hi = 1;
-          rem = r;
-        } else {
-          lo = 1;
-        }
-      }
-      if (!exact) {
-        ctl->lo = lo;
-        ctl->hi = hi;
-      }
-      ctl->r = r;
-      ctl->exact = exact;
-      ctl->k_rem = rem;
-    } else if (LEVEL == 1) {
-      ctl->k_rem = rem;
-    } else {
-      // all 31 bits resolved: T = prefix, take the first `rem` ties by index
-      ctl->k_rem = rem;
-      ctl->lo = prefix;
-      ctl->hi = prefix + 1u;
-      ctl->r = rem;
-      ctl->exact = 1;
-    }
-  }
+__device__ __forceinline__ uint32_t mix32(uint32_t x) {
+  x ^= x >> 16; x *= 0x7FEB352Du;
+  x ^= x >> 15; x *= 0x846CA68Bu;
+  x ^= x >> 16;
+  return x;
 }
 
-// Histogram of digit LEVEL over the elements of `src` whose higher digits equal
-// the resolved prefix.  LEVEL 0 runs over the bucket and also counts zero keys
-// and flags non-finite input; LEVEL 1 and 2 run over the candidate list.
-template <int LEVEL, class Src>
-__global__ void __launch_bounds__(kCta)
-k_histogram(Src src, unsigned long long count_arg, unsigned long long k, Ctl* ctl, unsigned int* ghist_all) {
-  constexpr int NB = 1 << digit_bits(LEVEL);
-  constexpr int SHIFT = digit_shift(LEVEL);
-  __shared__ unsigned int s_hist[NB];
-  __shared__ bool s_last;
-
-  unsigned int* ghist = ghist_all + LEVEL * kMaxBins;
-  unsigned long long count = count_arg;
-  unsigned int want_prefix = 0;
-  if (LEVEL > 0) {
-    if (ctl->exact) return;  // threshold already final
-    count = ctl->list_count;
-    want_prefix = ctl->prefix;
-  }
-
-  for (int b = threadIdx.x; b < NB; b += kCta) s_hist[b] = 0;
-  __syncthreads();
-
-  unsigned int zeros = 0;
-  bool nonfinite = false;
-  const unsigned long long stride = (unsigned long long)gridDim.x * kCta * 4;
-  for (unsigned long long i0 = ((unsigned long long)blockIdx.x * kCta + threadIdx.x) * 4; i0 < count; i0 += stride) {
-    Quad q = src.load4(i0, count);
+// Block-wide search from the top over NB bins, PER consecutive bins per thread
+// (own[] holds this thread's bins, lowest first): leaves in s_out the digit d
+// with #{digit > d} < rem <= #{digit >= d} and the rank left inside bin d.
+// Called by every thread of the block; s_tot needs one word per warp.
+template <int PER, int THREADS>
+__device__ __forceinline__ void find_digit_from_top(const unsigned int (&own)[PER], unsigned int rem,
+                                                    unsigned int* s_tot, unsigned int* s_out) {
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  unsigned int mine = 0;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      if (!(q.valid & (1u << e))) continue;
-      const uint32_t key = q.bits[e] & 0x7FFFFFFFu;
-      if (LEVEL == 0) {
-        zeros += (key == 0);
-        nonfinite |= (key >= kInfKey);
-        atomicAdd(&s_hist[key >> SHIFT], 1u);
-      } else {
-        if ((key >> (SHIFT + digit_bits(LEVEL))) == want_prefix)
-          atomicAdd(&s_hist[(key >> SHIFT) & (NB - 1)], 1u);
+  for (int b = 0; b < PER; ++b) mine += own[b];
+  unsigned int incl = mine;  // this thread and all higher lanes of the warp
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned int v = __shfl_down_sync(0xFFFFFFFFu, incl, o);
+    if (lane + o < 32) incl += v;
+  }
+  __syncthreads();  // s_tot and s_out may still be read from an earlier call
+  if (lane == 0) s_tot[warp] = incl;
+  __syncthreads();
+  unsigned int above = incl - mine;
+  for (int w = warp + 1; w < THREADS / 32; ++w) above += s_tot[w];
+  if (above < rem && rem <= above + mine) {  // exactly one thread
+#pragma unroll
+    for (int b = PER - 1; b >= 0; --b) {
+      if (rem <= above + own[b]) {
+        s_out[0] = (unsigned)(t * PER + b);
+        s_out[1] = rem - above;
+        break;
       }
+      above += own[b];
     }
   }
-  if (LEVEL == 0) {
-    for (int o = 16; o > 0; o >>= 1) zeros += __shfl_down_sync(0xFFFFFFFFu, zeros, o);
-    if ((threadIdx.x & 31) == 0 && zeros) atomicAdd(&ctl->zero_count, (unsigned long long)zeros);
-    if (nonfinite) set_status(&ctl->status, NSML_ERR_NONFINITE);
-  }
   __syncthreads();
-  for (int b = threadIdx.x; b < NB; b += kCta) {
-    unsigned int c = s_hist[b];
-    if (c) atomicAdd(&ghist[b], c);
-  }
+}
 
-  // the block that arrives last sees every block's contribution
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) s_last = (atomicAdd(&ctl->done[LEVEL], 1u) == gridDim.x - 1);
-  __syncthreads();
-  if (s_last) {
-    __threadfence();
-    resolve_level<LEVEL>(ctl, ghist, k);
+// One block.  Clears the per-call control region, then sets ctl->lo from a
+// stratified sample.  rank_from_top == 0 means "no sampling" (small bucket, or
+// nearly everything is kept): lo = 0.
+template <int DTYPE>
+__global__ void __launch_bounds__(kSampleThreads)
+k_sample(BucketSrc<DTYPE> src, unsigned long long n, unsigned int rank_from_top, Ctl* ctl, uint4* zero_base,
+         unsigned int zero_vec16) {
+  __shared__ unsigned int s_hist[kMaxBins];
+  __shared__ unsigned int s_tot[kSampleThreads / 32];
+  __shared__ unsigned int s_out[2];
+
+  uint32_t keys[kSamplesPerThread];
+  if (rank_from_top != 0) {
+#pragma unroll
+    for (int s = 0; s < kSamplesPerThread; ++s) {
+      const unsigned long long stratum = (unsigned long long)s * kSampleThreads + threadIdx.x;
+      const unsigned long long begin = stratum * n / kSamples;
+      const unsigned long long end = (stratum + 1) * n / kSamples;  // > begin because n >= 2 * kSamples
+      const unsigned long long pos = begin + mix32((uint32_t)stratum * 0x9E3779B1u + 0x85EBCA6Bu) % (uint32_t)(end - begin);
+      keys[s] = src.load1(pos) & 0x7FFFFFFFu;
+    }
   }
+  for (unsigned int i = threadIdx.x; i < zero_vec16; i += kSampleThreads) zero_base[i] = make_uint4(0, 0, 0, 0);
+
+  unsigned int lo = 0;
+  if (rank_from_top != 0) {
+    unsigned int prefix = 0, rem = rank_from_top;
+#pragma unroll
+    for (int level = 0; level < 2; ++level) {  // 12 + 12 bits
+      const int shift = digit_shift(level);
+      for (int b = threadIdx.x; b < kMaxBins; b += kSampleThreads) s_hist[b] = 0;
+      __syncthreads();
+#pragma unroll
+      for (int s = 0; s < kSamplesPerThread; ++s)
+        if (level == 0 || (keys[s] >> 19) == prefix) atomicAdd(&s_hist[(keys[s] >> shift) & (kMaxBins - 1)], 1u);
+      __syncthreads();
+      unsigned int own[4];
+#pragma unroll
+      for (int b = 0; b < 4; ++b) own[b] = s_hist[threadIdx.x * 4 + b];
+      find_digit_from_top<4, kSampleThreads>(own, rem, s_tot, s_out);
+      prefix = (prefix << 12) | s_out[0];
+      rem = s_out[1];
+    }
+    lo = prefix << 7;
+  }
+  __syncthreads();  // the control block was cleared above by other threads
+  if (threadIdx.x == 0) ctl->lo = lo;
 }
 
 }  // namespace nsml

@@ -106,6 +106,39 @@ def test_bf16_buckets(n):
             check_compress(g, ratio, bits)
 
 
+def sampled_positions(n, strata=8192):
+    """Positions the library's stratified sampler reads (one per stratum, a
+    hashed offset inside it), restated from its description so that a test can
+    build a bucket on which the sample is misleading."""
+    s = np.arange(strata, dtype=np.uint64)
+    begin = s * np.uint64(n) // np.uint64(strata)
+    end = (s + np.uint64(1)) * np.uint64(n) // np.uint64(strata)
+    x = (s * np.uint64(0x9E3779B1) + np.uint64(0x85EBCA6B)) & np.uint64(0xFFFFFFFF)
+    x ^= x >> np.uint64(16)
+    x = (x * np.uint64(0x7FEB352D)) & np.uint64(0xFFFFFFFF)
+    x ^= x >> np.uint64(15)
+    x = (x * np.uint64(0x846CA68B)) & np.uint64(0xFFFFFFFF)
+    x ^= x >> np.uint64(16)
+    return (begin + x % (end - begin)).astype(np.int64)
+
+
+@pytest.mark.parametrize("n", [20000, 200000, 1 << 20])
+def test_misleading_sample_still_gives_the_exact_result(n):
+    # large magnitudes exactly where the sampler looks, small ones elsewhere:
+    # the sampled bracket then keeps far fewer than k elements and the repeat
+    # pass has to produce the list
+    rng = np.random.default_rng(n)
+    g = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    pos = sampled_positions(n)
+    g[pos] = (100.0 + rng.random(pos.size)).astype(np.float32) * rng.choice(np.array([-1.0, 1.0], np.float32), pos.size)
+    for ratio in (0.1, 0.5):
+        check_compress(g, ratio, 8)
+    # and the opposite: zeros where the sampler looks (bracket starts at key 0)
+    g = rng.standard_normal(n).astype(np.float32)
+    g[pos] = 0.0
+    check_compress(g, 0.05, 16)
+
+
 def test_nonfinite_is_reported_not_trapped():
     rng = np.random.default_rng(2)
     for bad in (np.inf, -np.inf, np.nan):
