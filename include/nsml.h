@@ -226,6 +226,40 @@ int nsml_decompress_accumulate(const void* const* payloads, int W, float* dense,
                                int zero_first, void* workspace, size_t workspace_bytes,
                                void* stream);
 
+/* ------------------------------------------------------------------------
+ * nsml_decompress_accumulate_static -- the same sum as
+ * nsml_decompress_accumulate, for callers that have no device scratch to give
+ * and no way to get any: code that runs where cudaMalloc must not be called
+ * (inside a region that forbids allocation, a plug-in whose host owns every
+ * byte of device memory, an error path after the allocator has failed).  The
+ * paper has no counterpart; this is a convenience of the library.
+ *
+ * The scratch (block offsets and the status word) lives in one array of
+ * NSML_STATIC_SCRATCH_BYTES bytes that is part of the library image: every GPU
+ * that loads the library holds it until the process exits.  In exchange the
+ * call is limited to n <= NSML_STATIC_MAX_N and W <= NSML_STATIC_MAX_WORKERS;
+ * larger arguments are refused with NSML_ERR_CAPACITY and nothing is enqueued.
+ * The call, and everything it calls, allocates no host or device memory.
+ *
+ *   payloads, W, dense, n, zero_first, stream   as for nsml_decompress_accumulate
+ *   status_out  host pointer or NULL.  NULL: the call returns after enqueueing.
+ *               Non-NULL: the call also synchronises `stream` and stores the
+ *               device-detected status (NSML_OK or NSML_ERR_PAYLOAD) there.
+ *
+ * The first call on each device looks up the array's device address (once per
+ * device, with that device current); make that first call outside any stream
+ * capture.  All calls on a device share the one array and it keeps what the
+ * last call left in it: the status word is cleared at the start of each call,
+ * and two calls whose device work overlaps (different streams, or a second
+ * call before the first finished on another stream) race on it -- serialise
+ * them.  Results are bit-identical to nsml_decompress_accumulate.
+ * ---------------------------------------------------------------------- */
+#define NSML_STATIC_MAX_N 16777216LL /* 2^24 elements (64 MiB of float32) */
+#define NSML_STATIC_MAX_WORKERS 8
+#define NSML_STATIC_SCRATCH_BYTES 66048 /* 256 + 8 * (2^24 / 8192 + 1) * 4, rounded up to 256 */
+int nsml_decompress_accumulate_static(const void* const* payloads, int W, float* dense, int64_t n,
+                                      int zero_first, void* stream, int* status_out);
+
 /* Host-buffer variants: the same operations for callers whose gradients and
  * payloads live in host memory (pinned memory gives asynchronous copies).
  * `device_scratch` (device pointer, 256-byte aligned) must hold

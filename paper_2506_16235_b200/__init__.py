@@ -66,6 +66,14 @@ class CtrlState(ctypes.Structure):
 
 def _load() -> ctypes.CDLL:
     path = _build.LIB_PATH
+    if _build.is_stale():
+        # sources changed since the library was built (or it was never built):
+        # rebuild when a compiler is at hand, otherwise use what is there
+        try:
+            _build.build()
+        except RuntimeError:
+            if not os.path.exists(path):
+                raise
     if not os.path.exists(path):
         raise ImportError(
             f"{path} is missing: build it with `python -m paper_2506_16235_b200.build` "
@@ -87,6 +95,7 @@ def _load() -> ctypes.CDLL:
         "nsml_accumulate_workspace_bytes": (sz, [i64, ci]),
         "nsml_compress": (ci, [vp, i64, ci, dbl, ci, vp, vp, sz, vp, sz, vp]),
         "nsml_decompress_accumulate": (ci, [ctypes.POINTER(vp), ci, vp, i64, ci, vp, sz, vp]),
+        "nsml_decompress_accumulate_static": (ci, [ctypes.POINTER(vp), ci, vp, i64, ci, vp, ctypes.POINTER(ci)]),
         "nsml_compress_host_scratch_bytes": (sz, [i64, ci, dbl, ci]),
         "nsml_compress_host": (ci, [vp, i64, ci, dbl, ci, vp, vp, sz, vp, sz, vp]),
         "nsml_accumulate_host_scratch_bytes": (sz, [i64, ci, sz]),
@@ -270,6 +279,26 @@ def nsml_decompress_accumulate(payloads: Sequence, dense, zero_first: bool = Tru
                                         workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
     _check(rc, "nsml_decompress_accumulate")
     return dense
+
+
+NSML_STATIC_MAX_N = 1 << 24
+NSML_STATIC_MAX_WORKERS = 8
+
+
+def nsml_decompress_accumulate_static(payloads: Sequence, dense, zero_first: bool = True, stream=None,
+                                      want_status: bool = False):
+    """nsml_decompress_accumulate without a workspace argument: the scratch is
+    an array inside the library (for callers that cannot allocate device
+    memory).  Limited to n <= NSML_STATIC_MAX_N and W <= NSML_STATIC_MAX_WORKERS;
+    calls on one device must not overlap.  With want_status the call
+    synchronises the stream and returns the device-detected status."""
+    W = len(payloads)
+    ptrs = (ctypes.c_void_p * max(W, 1))(*[p.data_ptr() for p in payloads])
+    status = ctypes.c_int(0)
+    rc = lib.nsml_decompress_accumulate_static(ptrs, W, dense.data_ptr(), dense.numel(), 1 if zero_first else 0,
+                                               _stream_ptr(stream), ctypes.byref(status) if want_status else None)
+    _check(rc, "nsml_decompress_accumulate_static")
+    return status.value if want_status else None
 
 
 def nsml_last_status(workspace, stream=None) -> int:

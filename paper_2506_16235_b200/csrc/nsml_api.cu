@@ -246,6 +246,31 @@ static int accumulate_impl(const void* const* payloads, int W, float* dense, int
   return NSML_OK;
 }
 
+// ---- scratch for nsml_decompress_accumulate_static --------------------------
+// Part of the library image: every device that loads the library holds this
+// array until exit.  In host code the name below is only a handle; the device
+// address is looked up once per device with cudaGetSymbolAddress.
+static __device__ __align__(256) unsigned char g_static_scratch[NSML_STATIC_SCRATCH_BYTES];
+
+static void* g_static_scratch_addr[64];
+static std::mutex g_static_mutex;
+
+static int static_scratch(void** out) {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NSML_ERR_CUDA;
+  std::lock_guard<std::mutex> lock(g_static_mutex);
+  if (g_static_scratch_addr[dev] == nullptr) {
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || addr == nullptr) {
+      cudaGetLastError();
+      return NSML_ERR_CUDA;
+    }
+    g_static_scratch_addr[dev] = addr;
+  }
+  *out = g_static_scratch_addr[dev];
+  return NSML_OK;
+}
+
 }  // namespace nsml
 
 using namespace nsml;
@@ -281,6 +306,24 @@ int nsml_decompress_accumulate(const void* const* payloads, int W, float* dense,
                                void* workspace, size_t workspace_bytes, void* stream) {
   return accumulate_impl(payloads, W, dense, n, zero_first, workspace, workspace_bytes,
                          static_cast<cudaStream_t>(stream));
+}
+
+int nsml_decompress_accumulate_static(const void* const* payloads, int W, float* dense, int64_t n, int zero_first,
+                                      void* stream, int* status_out) {
+  if (n > NSML_STATIC_MAX_N || W > NSML_STATIC_MAX_WORKERS) return NSML_ERR_CAPACITY;
+  if (n < 1 || W < 1) return NSML_ERR_ARG;
+  if (accumulate_layout(n, W).total > (size_t)NSML_STATIC_SCRATCH_BYTES) return NSML_ERR_CAPACITY;
+  void* scratch = nullptr;
+  int rc = static_scratch(&scratch);
+  if (rc != NSML_OK) return rc;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  rc = accumulate_impl(payloads, W, dense, n, zero_first, scratch, NSML_STATIC_SCRATCH_BYTES, st);
+  if (rc != NSML_OK || status_out == nullptr) return rc;
+  int value = 0;
+  if (cudaMemcpyAsync(&value, scratch, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return NSML_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return NSML_ERR_CUDA;
+  *status_out = value;
+  return NSML_OK;
 }
 
 // ---- host-buffer variants --------------------------------------------------
