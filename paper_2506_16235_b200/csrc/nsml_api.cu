@@ -84,12 +84,9 @@ static int device_info(const DeviceInfo** out) {
     if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return NSML_ERR_CUDA;
     cudaError_t e = cudaSuccess;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_bucket, k_compact_bucket<NSML_F32>, kCta, 0);
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.finalize, k_finalize<NSML_F32>, kCta, 0);
-    if (e == cudaSuccess) {
-      int bf = 0;
-      e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&bf, k_finalize<NSML_BF16>, kCta, 0);
-      if (bf < d.finalize) d.finalize = bf;
-    }
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finalize<NSML_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFinalizeDynSmem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finalize<NSML_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFinalizeDynSmem);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.finalize, k_finalize<NSML_F32>, kFinThreads, kFinalizeDynSmem);
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.merge, k_merge, kCta, 0);
     int coop = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
@@ -140,45 +137,50 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
   Ctl* ctl = reinterpret_cast<Ctl*>(ws);
   uint32_t* seg_idx = reinterpret_cast<uint32_t*>(ws + L.seg_idx);
   uint32_t* seg_val = reinterpret_cast<uint32_t*>(ws + L.seg_val);
-  unsigned int* seg_count = reinterpret_cast<unsigned int*>(ws + L.seg_count);
+  unsigned short* seg_count = reinterpret_cast<unsigned short*>(ws + L.seg_count);
+  const unsigned long long nseg = ((unsigned long long)n + kSegElems - 1) / kSegElems;
   BucketSrc<DTYPE> src{grad, mask};
   {
-    LaunchScope scope(K_SAMPLE, st);
-    k_sample<DTYPE><<<1, kSampleThreads, 0, st>>>(src, (unsigned long long)n, sample_rank(n, k), ctl,
-                                                  reinterpret_cast<uint4*>(ws), (unsigned int)(L.zero_bytes / 16));
+    LaunchScope scope(K_SAMPLE, st);  // one cluster of kSampleBlocks blocks
+    k_sample<DTYPE><<<kSampleBlocks, kSampleThreads, 0, st>>>(src, (unsigned long long)n, sample_rank(n, k), ctl,
+                                                              reinterpret_cast<uint4*>(ws),
+                                                              (unsigned int)(L.zero_bytes / 16));
   }
-  // bucket pass: one block per 16K elements, at most what the device keeps resident
-  const unsigned int grid = grid_for((unsigned long long)n, kCta * 64, dev.sms * dev.compact_bucket);
-  const unsigned int segments = grid * (kCta / 32);
   {
+    // bucket pass: a block takes 8 segments per step; at most 4 resident blocks per SM
     LaunchScope scope(K_COMPACT_BUCKET, st);
-    k_compact_bucket<DTYPE><<<grid, kCta, 0, st>>>(src, (unsigned long long)n, ctl, seg_idx, seg_val, seg_count);
+    const int per_sm = dev.compact_bucket < 4 ? dev.compact_bucket : 4;
+    const unsigned int grid = grid_for(nseg, kCta / 32, dev.sms * per_sm);
+    k_compact_bucket<DTYPE><<<grid, kCta, 0, st>>>(src, (unsigned long long)n, ctl, seg_idx, seg_val, seg_count,
+                                                   reinterpret_cast<unsigned int*>(ws + L.group_count));
   }
-  // list stage: cooperative, every block co-resident, at most kMaxSegPerBlock segments per block
+  // list stage: cooperative, one block per SM, every block co-resident
   unsigned int fgrid = (unsigned int)(dev.sms * dev.finalize);
-  if (fgrid > grid) fgrid = grid;
+  if (fgrid > (unsigned int)dev.sms) fgrid = dev.sms;
+  if ((unsigned long long)fgrid > nseg) fgrid = (unsigned int)nseg;
   if (fgrid > (unsigned int)kMaxFinalizeBlocks) fgrid = kMaxFinalizeBlocks;
-  if ((segments + fgrid - 1) / fgrid + 1 > (unsigned int)kMaxSegPerBlock) return NSML_ERR_CUDA;
   FinalizeParams fp;
   fp.n = (unsigned long long)n;
   fp.k = (unsigned long long)k;
   fp.bits = bits;
-  fp.segments = segments;
+  fp.nseg = nseg;
   fp.ctl = ctl;
   fp.hist = reinterpret_cast<unsigned int*>(ws + L.hist);
   fp.block_counts = reinterpret_cast<unsigned long long*>(ws + L.block_counts);
   fp.seg_count = seg_count;
-  fp.seg_zeros = reinterpret_cast<unsigned int*>(ws + L.seg_zeros);
+  fp.group_count = reinterpret_cast<const unsigned int*>(ws + L.group_count);
   fp.seg_idx = seg_idx;
   fp.seg_val = seg_val;
+  fp.list_idx = reinterpret_cast<uint32_t*>(ws + L.list_idx);
+  fp.list_val = reinterpret_cast<uint32_t*>(ws + L.list_val);
   fp.raw_val = reinterpret_cast<float*>(ws + L.raw_val);
   fp.payload = payload;
   fp.P = P;
   {
     LaunchScope scope(K_FINALIZE, st);
     void* args[] = {&src, &fp};
-    if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_finalize<DTYPE>), dim3(fgrid), dim3(kCta), args, 0, st) !=
-        cudaSuccess)
+    if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_finalize<DTYPE>), dim3(fgrid), dim3(kFinThreads), args,
+                                    kFinalizeDynSmem, st) != cudaSuccess)
       return NSML_ERR_CUDA;
   }
   return NSML_OK;

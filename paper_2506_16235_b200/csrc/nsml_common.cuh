@@ -32,17 +32,20 @@ struct Ctl {
 };
 static_assert(sizeof(Ctl) <= 256, "control block must fit its 256-byte slot");
 
-constexpr int kMaxSegments = 1 << 14;    // upper bound on warps of the bucket pass
-constexpr int kMaxFinalizeBlocks = 2048;  // upper bound on blocks of the finalize kernel
+constexpr int kSegElems = 512;            // bucket elements per candidate-list segment (4 rounds of 128)
+constexpr int kGroupSegs = 64;            // segments per group; the bucket pass keeps a candidate count per group
+constexpr int kMaxFinalizeBlocks = 1024;  // upper bound on blocks of the finalize kernel
 
 struct CompressLayout {  // byte offsets inside a compress workspace
   size_t hist;          // u32[4][kMaxBins]: digit histograms (levels 0..2, level 0 again after a rebuild)
+  size_t group_count;   // u32[ceil(segments / kGroupSegs)]: candidates per group of segments
   size_t zero_bytes;    // everything before this offset is cleared per call
   size_t block_counts;  // u64[4][kMaxFinalizeBlocks]: per-block counts exchanged at barriers
-  size_t seg_count;     // u32[kMaxSegments]: entries per segment
-  size_t seg_zeros;     // u32[kMaxSegments]: slow path, zeros per segment
-  size_t seg_idx;       // u32[n]: segmented candidate list (bucket pass output)
+  size_t seg_count;     // u16[ceil(n / kSegElems)]: entries per segment
+  size_t seg_idx;       // u32[n]: segmented candidate list (bucket pass output); segment s starts at s * kSegElems
   size_t seg_val;       // u32[n] (float32 bit patterns)
+  size_t list_idx;      // u32[n]: the same candidates, contiguous per finalize block
+  size_t list_val;      // u32[n]
   size_t raw_val;       // f32[n]: survivor values before quantisation
   size_t total;
 };
@@ -51,15 +54,18 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 
 inline CompressLayout compress_layout(int64_t n) {
   CompressLayout L;
-  size_t npad = align_up((size_t)n, 64);
+  const size_t npad = align_up((size_t)n, kSegElems);
+  const size_t segs = npad / kSegElems;
   L.hist = 256;
-  L.zero_bytes = L.hist + 4 * kMaxBins * sizeof(unsigned int);
+  L.group_count = L.hist + 4 * kMaxBins * sizeof(unsigned int);
+  L.zero_bytes = L.group_count + align_up(((segs + kGroupSegs - 1) / kGroupSegs) * 4, 256);
   L.block_counts = L.zero_bytes;
   L.seg_count = L.block_counts + 4 * kMaxFinalizeBlocks * 8;
-  L.seg_zeros = L.seg_count + kMaxSegments * 4;
-  L.seg_idx = L.seg_zeros + kMaxSegments * 4;
+  L.seg_idx = L.seg_count + align_up(segs * 2, 256);
   L.seg_val = L.seg_idx + npad * 4;
-  L.raw_val = L.seg_val + npad * 4;
+  L.list_idx = L.seg_val + npad * 4;
+  L.list_val = L.list_idx + npad * 4;
+  L.raw_val = L.list_val + npad * 4;
   L.total = L.raw_val + npad * 4;
   return L;
 }

@@ -2,25 +2,27 @@
 // (Alg. 2 Steps 2-3: pruned gradients read as zero; everything whose magnitude
 // is below the sampled lower bound is dropped here, in one streaming read).
 //
-// Warp w owns a contiguous range of 128-element rounds and appends what it
-// keeps (every key >= lo, lo >= 1) to its own segment of the list.  A segment
-// starts at the list position of the range's first element, so it can never
-// overflow and needs no allocation.  There is no block or grid
-// synchronisation: a warp's only state is its running count.  Segments taken
-// in warp order are in index order.
+// The bucket is cut into segments of kSegElems elements.  A warp takes one
+// segment at a time and appends what it keeps (every key >= lo, lo >= 1) to
+// the segment's own slots of the list, [s * kSegElems, s * kSegElems + count),
+// so nothing can overflow, nothing is allocated and no warp ever waits for
+// another: there is no block or grid synchronisation in this kernel.
+// Segments in increasing order are in index order.
+//
+// Blocks walk the bucket block-cyclically (block b takes segments 8b..8b+7,
+// then 8(b+G).., ...), so at any moment the whole grid reads one compact
+// window of the bucket, which is what DRAM row buffers like.  Every lane
+// keeps its part of the warp's next segment in flight with asynchronous
+// copies into a private shared-memory slot: a lane reads back only what it
+// copied itself, so the double buffer needs no synchronisation either.
 #pragma once
 
 #include "nsml_common.cuh"
 
 namespace nsml {
 
-constexpr int kRound = 128;  // elements a warp handles per step (32 lanes x 4)
-constexpr int kUnroll = 4;   // rounds in flight per warp
-
-__host__ __device__ inline unsigned long long warp_first_round(unsigned long long warp, unsigned long long warps,
-                                                               unsigned long long rounds) {
-  return warp * rounds / warps;
-}
+constexpr int kRound = 128;                       // elements a warp handles per step (32 lanes x 4)
+constexpr int kSegRounds = kSegElems / kRound;    // 4
 
 // Appends the kept elements of one round.  `f` holds this lane's four keep
 // flags (bit e = element lane*4+e of the round).  Returns the round's total.
@@ -60,50 +62,104 @@ __device__ __forceinline__ unsigned int append_round(unsigned int f, const uint3
   return total;
 }
 
+// ---- per-lane asynchronous copies (global -> shared) ----
+template <int BYTES>
+__device__ __forceinline__ void cp_async_lane(void* smem_dst, const void* gsrc) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  if (BYTES == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+  else asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
+
+// |v| >= t on floats equals key >= lo for finite v; written as !(|v| < t) so
+// that NaN is kept too (the finalize kernel reports non-finite candidates).
+__device__ __forceinline__ unsigned int keep_flags(const uint32_t (&bits)[4], float t) {
+  unsigned int f = 0;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) f |= (unsigned)(!(fabsf(__uint_as_float(bits[e])) < t)) << e;
+  return f;
+}
+
 template <int DTYPE>
 __global__ void __launch_bounds__(kCta)
 k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, uint32_t* __restrict__ seg_idx,
-                 uint32_t* __restrict__ seg_val, unsigned int* __restrict__ seg_count) {
-  const int lane = threadIdx.x & 31;
-  const unsigned long long warp = (unsigned long long)blockIdx.x * (kCta / 32) + (threadIdx.x >> 5);
-  const unsigned long long warps = (unsigned long long)gridDim.x * (kCta / 32);
-  const unsigned long long rounds = (n + kRound - 1) / kRound;
-  const unsigned long long first = warp_first_round(warp, warps, rounds);
-  const unsigned long long last = warp_first_round(warp + 1, warps, rounds);
+                 uint32_t* __restrict__ seg_val, unsigned short* __restrict__ seg_count,
+                 unsigned int* __restrict__ group_count) {
+  constexpr int ESIZE = (DTYPE == NSML_F32) ? 4 : 2;
+  constexpr int LANE_BYTES = 4 * ESIZE;
+  constexpr int BUF_BYTES = kSegRounds * 32 * LANE_BYTES;  // one segment of one warp
+  __shared__ __align__(16) unsigned char s_fifo[(kCta / 32) * 2 * BUF_BYTES];
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  unsigned char* fifo = s_fifo + (size_t)w * 2 * BUF_BYTES + lane * LANE_BYTES;  // round r of buffer b at + (b*kSegRounds + r)*32*LANE_BYTES
+
+  const unsigned long long nseg = (n + kSegElems - 1) / kSegElems;
+  const unsigned long long nseg_full = n / kSegElems;  // segments that need no bounds checks
+  const unsigned long long step = (unsigned long long)gridDim.x * (kCta / 32);
+  const unsigned char* g = static_cast<const unsigned char*>(src.grad) + (size_t)lane * 4 * ESIZE;
+
+  unsigned long long seg = (unsigned long long)blockIdx.x * (kCta / 32) + w;
+  if (seg < nseg_full) {
+#pragma unroll
+    for (int r = 0; r < kSegRounds; ++r)
+      cp_async_lane<LANE_BYTES>(fifo + r * 32 * LANE_BYTES, g + (seg * kSegElems + r * kRound) * ESIZE);
+  }
+  cp_async_commit();
   // Zeros are never candidates here; if they are needed (fewer than k non-zero
   // keys) the list comes out short and the finalize kernel's slow path adds them.
-  // |v| >= t on floats equals key >= lo for finite v; written as !(|v| < t) so
-  // that NaN is kept too (the finalize kernel reports non-finite candidates).
   const float t = __uint_as_float(max(ctl->lo, 1u));
-  const unsigned long long seg_base = first * kRound;
-  const unsigned long long full_rounds = n / kRound;  // rounds that need no bounds checks
-  unsigned int kept = 0;
+  int buf = 0;
 
-  unsigned long long rd = first;
-  const unsigned long long last_full = min(last, full_rounds);
-  for (; rd + kUnroll <= last_full; rd += kUnroll) {
-    uint32_t bits[kUnroll][4];
+  while (seg < nseg) {
+    const unsigned long long next = seg + step;
+    if (next < nseg_full) {
 #pragma unroll
-    for (int u = 0; u < kUnroll; ++u) src.load_full4((rd + u) * kRound + lane * 4, bits[u]);
-#pragma unroll
-    for (int u = 0; u < kUnroll; ++u) {
-      unsigned int f = 0;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) f |= (unsigned)(!(fabsf(__uint_as_float(bits[u][e])) < t)) << e;
-      if (!__any_sync(0xFFFFFFFFu, f != 0)) continue;
-      kept += append_round(f, bits[u], (uint32_t)((rd + u) * kRound), seg_base + kept, seg_idx, seg_val);
+      for (int r = 0; r < kSegRounds; ++r)
+        cp_async_lane<LANE_BYTES>(fifo + ((buf ^ 1) * kSegRounds + r) * 32 * LANE_BYTES,
+                                  g + (next * kSegElems + r * kRound) * ESIZE);
     }
-  }
-  for (; rd < last; ++rd) {  // leftover rounds, the last of which may be partial
-    uint32_t bits[4];
-    src.load_vals4(rd * kRound + lane * 4, n, bits);  // missing elements read as 0 and are never kept
-    unsigned int f = 0;
+    cp_async_commit();
+    cp_async_wait<1>();  // this segment's copies have landed; the next segment's stay in flight
+
+    const unsigned long long seg_base = seg * kSegElems;
+    unsigned int kept = 0;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) f |= (unsigned)(!(fabsf(__uint_as_float(bits[e])) < t)) << e;
-    if (!__any_sync(0xFFFFFFFFu, f != 0)) continue;
-    kept += append_round(f, bits, (uint32_t)(rd * kRound), seg_base + kept, seg_idx, seg_val);
+    for (int r = 0; r < kSegRounds; ++r) {
+      uint32_t bits[4];
+      if (seg < nseg_full) {
+        const unsigned char* slot = fifo + (buf * kSegRounds + r) * 32 * LANE_BYTES;
+        if (DTYPE == NSML_F32) {
+          const uint4 v = *reinterpret_cast<const uint4*>(slot);
+          bits[0] = v.x; bits[1] = v.y; bits[2] = v.z; bits[3] = v.w;
+        } else {
+          const uint2 v = *reinterpret_cast<const uint2*>(slot);
+          bits[0] = v.x << 16; bits[1] = v.x & 0xFFFF0000u;
+          bits[2] = v.y << 16; bits[3] = v.y & 0xFFFF0000u;
+        }
+        if (src.mask != nullptr) {
+          const unsigned long long i0 = seg_base + r * kRound + lane * 4;
+          const uint32_t m = (src.mask[i0 >> 5] >> (unsigned)(i0 & 31)) & 0xFu;
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            if (m & (1u << e)) bits[e] = 0;
+        }
+      } else {
+        // the bucket's ragged last segment: plain loads, missing elements read as 0 and are never kept
+        src.load_vals4(seg_base + r * kRound + lane * 4, n, bits);
+      }
+      const unsigned int f = keep_flags(bits, t);
+      if (!__any_sync(0xFFFFFFFFu, f != 0)) continue;
+      kept += append_round(f, bits, (uint32_t)(seg_base + r * kRound), seg_base + kept, seg_idx, seg_val);
+    }
+    if (lane == 0) {
+      seg_count[seg] = (unsigned short)kept;
+      if (kept) atomicAdd(group_count + seg / kGroupSegs, kept);  // result unused: a fire-and-forget reduction
+    }
+    seg = next;
+    buf ^= 1;
   }
-  if (lane == 0) seg_count[warp] = kept;
+  cp_async_wait<0>();
 }
 
 }  // namespace nsml

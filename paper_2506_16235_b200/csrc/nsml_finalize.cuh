@@ -2,24 +2,28 @@
 //
 // The bucket pass leaves a segmented list of candidates (every key >= lo).
 // This kernel finds the exact threshold key T and the tie budget r by radix
-// select on the candidates' magnitude keys (12 + 12 + 7 bits, Alg. 2 Step 3
+// select on the candidates' magnitude keys (12 + 12 + 7 bits; Alg. 2 Step 3
 // read as: keep the k largest |g|, ties by lower index), writes the k
 // survivors in index order and quantises them (Alg. 2 Step 1 "quantize" for
 // fp16; int8 per block of 1024 survivors).
 //
-// All blocks are co-resident (cooperative launch); block b owns a contiguous
-// run of segments, i.e. a contiguous index range, for the whole kernel, so
-// "index order" is block order.  Phases are separated by grid barriers:
-//   1  count own candidates, histogram of key digit 0        | barrier
-//   2  every block resolves digit 0; histogram of digit 1    | barrier
-//   3  resolve digit 1; histogram of digit 2                 | barrier
-//   4  resolve digit 2 -> T, r; count own (> T, == T)        | barrier
-//   5  prefix over blocks; write survivors (index, value)    | barrier
-//   6  quantise blocks of 1024 survivors, write the header
+// One block per SM, all co-resident (cooperative launch).  The bucket pass
+// also leaves a candidate count per group of 64 segments; every block scans
+// those, which gives it the list position of every group without a barrier,
+// and takes an equal share of the candidates in list order (so "index order"
+// is block order, and the blocks' work is balanced however the candidates
+// crowd).  Phases, separated by grid barriers:
+//   0  gather the share into one contiguous array (global, plus a copy in
+//      shared memory when it fits), histogram of key digit 0               | barrier
+//   1  every block resolves digit 0; histogram of digit 1                  | barrier
+//   2  resolve digit 1; histogram of digit 2                               | barrier
+//   3  resolve digit 2 -> T, r; count own keys > T and == T                | barrier
+//   4  prefix over blocks; write survivors (index, raw value) in order     | barrier
+//   5  quantise blocks of 1024 survivors, write the header
 // If the list holds fewer than k candidates (fewer than k non-zero keys, or a
-// misleading sample) phase 1 is followed by a slow path that rebuilds the
-// segments from the bucket: every non-zero key plus the first k - nnz zeros in
-// index order; then phase 1 runs again.
+// misleading sample) phase 0 is replaced by a slow path in which block b owns
+// an index range and rebuilds its array from the bucket: every non-zero key
+// plus the first k - nnz zeros in index order (one more barrier).
 //
 // Every barrier wait is bounded: when it runs out the block records
 // NSML_ERR_TIMEOUT and leaves; the others then time out as well.
@@ -32,19 +36,25 @@
 
 namespace nsml {
 
-constexpr int kMaxSegPerBlock = 64;
+constexpr int kFinThreads = 1024;
+constexpr int kFinWarps = kFinThreads / 32;
+constexpr int kCacheEntries = 20480;  // candidates a block keeps in shared memory (index + value: 160 KB)
+constexpr size_t kFinalizeDynSmem = (size_t)kCacheEntries * 8;
+constexpr int kGatherChunk = kFinThreads * 8;  // segments per gather step
 
 struct FinalizeParams {
   unsigned long long n, k;
   int bits;
-  unsigned int segments;             // warps of the bucket pass
+  unsigned long long nseg;           // ceil(n / kSegElems)
   Ctl* ctl;
   unsigned int* hist;                // [4][kMaxBins]
   unsigned long long* block_counts;  // [4][kMaxFinalizeBlocks]
-  unsigned int* seg_count;
-  unsigned int* seg_zeros;
-  uint32_t* seg_idx;
-  uint32_t* seg_val;
+  const unsigned short* seg_count;
+  const unsigned int* group_count;   // [ceil(nseg / kGroupSegs)]
+  const uint32_t* seg_idx;
+  const uint32_t* seg_val;
+  uint32_t* list_idx;
+  uint32_t* list_val;
   float* raw_val;
   unsigned char* payload;
   PayloadLayout P;
@@ -52,30 +62,51 @@ struct FinalizeParams {
 
 struct FinalizeShared {
   unsigned int hist[kMaxBins];
-  unsigned long long red[kCta / 32];
-  unsigned int tot[kCta / 32];
+  unsigned int off[kFinThreads];  // gather: exclusive offset of each thread's 8 segments within the chunk
+  uint4 cnt8[kFinThreads];        // gather: the 8 segment counts of each thread (16 bits each)
+  unsigned long long red[kFinWarps];
+  unsigned int scan[kFinWarps];
+  unsigned int tot[kFinWarps];
   unsigned int out[2];
-  unsigned int seg_a[kMaxSegPerBlock];
-  unsigned int seg_c[kMaxSegPerBlock];
-  float qmax[kCta / 32];
+  unsigned long long start[2];  // gather: first group of this block's share, list position where that group starts
+  float qmax[kFinWarps];
   int ok;
 };
-
-__device__ __forceinline__ unsigned long long ld_cg_u64(const unsigned long long* p) {
-  return __ldcg(p);
-}
 
 // Sum over the block; every thread gets the result.
 __device__ __forceinline__ unsigned long long block_sum(unsigned long long v, FinalizeShared& sh) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-  __syncthreads();
+  __syncthreads();  // sh.red may still be read from an earlier call
   if ((threadIdx.x & 31) == 0) sh.red[threadIdx.x >> 5] = v;
   __syncthreads();
   unsigned long long s = 0;
 #pragma unroll
-  for (int w = 0; w < kCta / 32; ++w) s += sh.red[w];
+  for (int w = 0; w < kFinWarps; ++w) s += sh.red[w];
   return s;
+}
+
+// Exclusive prefix over the block in thread order; `total` = sum over the block.
+__device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned int& total, FinalizeShared& sh) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += up;
+  }
+  __syncthreads();  // sh.scan may still be read from an earlier call
+  if (lane == 31) sh.scan[warp] = incl;
+  __syncthreads();
+  unsigned int before = 0, all = 0;
+#pragma unroll
+  for (int w = 0; w < kFinWarps; ++w) {
+    const unsigned int c = sh.scan[w];
+    if (w < warp) before += c;
+    all += c;
+  }
+  total = all;
+  return before + incl - v;
 }
 
 // All blocks arrive, then all leave.  `target` = barrier ordinal * gridDim.x.
@@ -87,7 +118,7 @@ __device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, Fina
     int ok = 1, polls = 0;
     while (*reinterpret_cast<volatile unsigned int*>(&ctl->barrier) < target) {
       if (++polls > kMaxPolls) { ok = 0; break; }
-      if (polls > 64) __nanosleep(100);
+      if (polls > 256) __nanosleep(64);
     }
     __threadfence();
     if (!ok) set_status(&ctl->status, NSML_ERR_TIMEOUT);
@@ -101,98 +132,182 @@ __device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, Fina
 template <int NB>
 __device__ __forceinline__ void flush_hist(FinalizeShared& sh, unsigned int* ghist) {
   __syncthreads();
-  for (int b = threadIdx.x; b < NB; b += kCta) {
+  for (int b = threadIdx.x; b < NB; b += kFinThreads) {
     const unsigned int c = sh.hist[b];
     if (c) atomicAdd(&ghist[b], c);
   }
 }
 
 // Every block reads the global histogram of a level and finds the digit that
-// holds the rem-th largest key; returns it and the rank left inside (sh.out).
+// holds the rem-th largest key; digit and the rank left inside land in sh.out.
 template <int NB>
 __device__ __forceinline__ void resolve_digit(const unsigned int* ghist, unsigned int rem, FinalizeShared& sh) {
-  constexpr int PER = (NB + kCta - 1) / kCta;
+  constexpr int PER = (NB + kFinThreads - 1) / kFinThreads;
   unsigned int own[PER];
 #pragma unroll
   for (int b = 0; b < PER; ++b) {
     const int bin = threadIdx.x * PER + b;
     own[b] = (bin < NB) ? __ldcg(ghist + bin) : 0u;
   }
-  find_digit_from_top<PER, kCta>(own, rem, sh.tot, sh.out);
+  find_digit_from_top<PER, kFinThreads>(own, rem, sh.tot, sh.out);
 }
 
 template <int DTYPE>
-__global__ void __launch_bounds__(kCta, 4)
+__global__ void __launch_bounds__(kFinThreads, 1)
 k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   __shared__ FinalizeShared sh;
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  extern __shared__ __align__(16) uint32_t s_cache[];  // values [kCacheEntries], then indices [kCacheEntries]
+  uint32_t* cache_val = s_cache;
+  uint32_t* cache_idx = s_cache + kCacheEntries;
+  const int lane = threadIdx.x & 31;
   const unsigned int G = gridDim.x, blk = blockIdx.x;
-  const unsigned int s0 = (unsigned int)((unsigned long long)blk * p.segments / G);
-  const unsigned int s1 = (unsigned int)((unsigned long long)(blk + 1) * p.segments / G);
-  const unsigned long long rounds = (p.n + kRound - 1) / kRound;
+  // Index-range ownership (used by the slow path only) and the block's array.
+  const unsigned long long seg_first = (unsigned long long)blk * p.nseg / G;
+  const unsigned long long seg_last = (unsigned long long)(blk + 1) * p.nseg / G;
+  uint32_t* my_idx = p.list_idx;  // set below
+  uint32_t* my_val = p.list_val;
   unsigned int barriers = 0;
-  unsigned long long list_total = 0;
-  int used_attempt = 0;  // which level-0 histogram belongs to the list in use
+  unsigned int E = 0;  // candidates this block owns
 
-  // ---------------- phase 1 (twice if the slow path runs) ----------------
-  for (int attempt = 0; attempt < 2; ++attempt) {
-    unsigned int* ghist0 = p.hist + (attempt == 0 ? 0 : 3) * kMaxBins;
-    unsigned long long* totals = p.block_counts + (attempt == 0 ? 0 : 3) * kMaxFinalizeBlocks;
-    for (int b = threadIdx.x; b < kMaxBins; b += kCta) sh.hist[b] = 0;
+  auto entry_val = [&](unsigned int j) -> uint32_t { return j < (unsigned)kCacheEntries ? cache_val[j] : __ldcg(my_val + j); };
+  auto entry_idx = [&](unsigned int j) -> uint32_t { return j < (unsigned)kCacheEntries ? cache_idx[j] : __ldcg(my_idx + j); };
+  auto put_entry = [&](unsigned int j, uint32_t idx, uint32_t val) {
+    my_idx[j] = idx;
+    my_val[j] = val;
+    if (j < (unsigned)kCacheEntries) {
+      cache_idx[j] = idx;
+      cache_val[j] = val;
+    }
+  };
+
+  // ---------------- phase 0: take an equal share of the candidates, histogram of digit 0 ----------------
+  // Every block reads the per-group candidate counts the bucket pass left and
+  // scans them, which gives the list position of every group and the total.
+  const unsigned long long ngroups = (p.nseg + kGroupSegs - 1) / kGroupSegs;
+  const unsigned long long per_thread = (ngroups + kFinThreads - 1) / kFinThreads;
+  const unsigned long long g_begin = min(ngroups, threadIdx.x * per_thread);
+  const unsigned long long g_end = min(ngroups, g_begin + per_thread);
+  unsigned long long thread_sum = 0;
+  for (unsigned long long gi = g_begin; gi < g_end; ++gi) thread_sum += p.group_count[gi];
+  unsigned long long list_total;
+  unsigned long long thread_pos;  // list position where this thread's first group starts
+  {
+    // 64-bit exclusive scan over the block
+    const int warp = threadIdx.x >> 5;
+    unsigned long long incl = thread_sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    if (lane == 31) sh.red[warp] = incl;
     __syncthreads();
-    unsigned long long mine = 0;
-    bool nonfinite = false;
-    for (unsigned int seg = s0 + warp; seg < s1; seg += kCta / 32) {
-      const unsigned int cnt = __ldcg(p.seg_count + seg);
-      const unsigned long long base = warp_first_round(seg, p.segments, rounds) * kRound;
-      for (unsigned int i = lane; i < cnt; i += 32) {
-        const uint32_t key = __ldcg(p.seg_val + base + i) & 0x7FFFFFFFu;
+    unsigned long long before = 0, all = 0;
+#pragma unroll
+    for (int w = 0; w < kFinWarps; ++w) {
+      const unsigned long long c = sh.red[w];
+      if (w < warp) before += c;
+      all += c;
+    }
+    list_total = all;
+    thread_pos = before + incl - thread_sum;
+  }
+  const unsigned long long share_lo = (unsigned long long)blk * list_total / G;
+  const unsigned long long share_hi = (unsigned long long)(blk + 1) * list_total / G;
+  for (int b = threadIdx.x; b < kMaxBins; b += kFinThreads) sh.hist[b] = 0;
+  bool nonfinite = false;
+  if (list_total >= p.k) {
+    my_idx = p.list_idx + share_lo;
+    my_val = p.list_val + share_lo;
+    E = (unsigned int)(share_hi - share_lo);
+    if (E > 0 && thread_pos <= share_lo && share_lo < thread_pos + thread_sum) {  // exactly one thread
+      unsigned long long pos = thread_pos, gi = g_begin;
+      for (; gi < g_end; ++gi) {
+        const unsigned long long c = p.group_count[gi];
+        if (share_lo < pos + c) break;
+        pos += c;
+      }
+      sh.start[0] = gi;
+      sh.start[1] = pos;
+    }
+    __syncthreads();
+    unsigned long long seg_cursor = (E > 0) ? sh.start[0] * kGroupSegs : p.nseg;
+    unsigned long long pos_cursor = (E > 0) ? sh.start[1] : 0;
+    // A chunk is 8 segments per thread.  Thin stretches of the bucket make a
+    // share span many chunks, so the next chunk's counts are fetched before
+    // the current chunk's entries are copied.
+    auto load_counts = [&](unsigned long long first_seg) -> uint4 {
+      const unsigned long long s = first_seg + threadIdx.x * 8ull;  // a multiple of 8: the 16-byte load is aligned
+      if (s + 8 <= p.nseg) return *reinterpret_cast<const uint4*>(p.seg_count + s);
+      unsigned short c[8];
+#pragma unroll
+      for (int e = 0; e < 8; ++e) c[e] = (s + e < p.nseg) ? p.seg_count[s + e] : (unsigned short)0;
+      uint4 v;
+      v.x = c[0] | ((uint32_t)c[1] << 16); v.y = c[2] | ((uint32_t)c[3] << 16);
+      v.z = c[4] | ((uint32_t)c[5] << 16); v.w = c[6] | ((uint32_t)c[7] << 16);
+      return v;
+    };
+    uint4 counts = load_counts(seg_cursor);
+    while (pos_cursor < share_hi && seg_cursor < p.nseg) {
+      const uint4 next_counts = load_counts(seg_cursor + kGatherChunk);
+      const unsigned int cnt = (counts.x & 0xFFFFu) + (counts.x >> 16) + (counts.y & 0xFFFFu) + (counts.y >> 16) +
+                               (counts.z & 0xFFFFu) + (counts.z >> 16) + (counts.w & 0xFFFFu) + (counts.w >> 16);
+      unsigned int chunk_total;
+      const unsigned int off = block_excl_scan(cnt, chunk_total, sh);
+      __syncthreads();  // sh.off / sh.cnt8 of the previous chunk have been read
+      sh.off[threadIdx.x] = off;
+      sh.cnt8[threadIdx.x] = counts;
+      __syncthreads();
+      // entries of this chunk that fall in the block's share
+      const unsigned long long from_pos = max(pos_cursor, share_lo), to_pos = min(pos_cursor + chunk_total, share_hi);
+      for (unsigned long long g = from_pos + threadIdx.x; g < to_pos; g += kFinThreads) {
+        const unsigned int j = (unsigned int)(g - pos_cursor);
+        int lo = 0, hi = kFinThreads - 1;  // last thread slot of the chunk whose offset is <= j
+        while (lo < hi) {
+          const int mid = (lo + hi + 1) >> 1;
+          if (sh.off[mid] <= j) lo = mid; else hi = mid - 1;
+        }
+        unsigned int within = j - sh.off[lo];
+        const uint4 c8 = sh.cnt8[lo];
+        const uint32_t words[4] = {c8.x, c8.y, c8.z, c8.w};
+        int e = 0;
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+          const unsigned int c = (words[q >> 1] >> ((q & 1) * 16)) & 0xFFFFu;
+          if (q == e && within >= c) { within -= c; ++e; }
+        }
+        const unsigned long long from = (seg_cursor + lo * 8ull + e) * kSegElems + within;
+        const uint32_t val = p.seg_val[from];
+        const uint32_t key = val & 0x7FFFFFFFu;
+        put_entry((unsigned int)(g - share_lo), p.seg_idx[from], val);
         nonfinite |= key >= kInfKey;
         atomicAdd(&sh.hist[key >> digit_shift(0)], 1u);
       }
-      if (lane == 0) mine += cnt;
+      pos_cursor += chunk_total;
+      seg_cursor += kGatherChunk;
+      counts = next_counts;
     }
     if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
-    const unsigned long long block_total = block_sum(mine, sh);
-    if (threadIdx.x == 0) totals[blk] = block_total;
-    flush_hist<kMaxBins>(sh, ghist0);
+    flush_hist<kMaxBins>(sh, p.hist);
     if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
+  }
+  const unsigned int* ghist0 = p.hist;
 
-    unsigned long long part = 0;
-    for (unsigned int b = threadIdx.x; b < G; b += kCta) part += ld_cg_u64(totals + b);
-    list_total = block_sum(part, sh);
-    used_attempt = attempt;
-    if (list_total >= p.k) break;
-    if (attempt == 1) {  // cannot happen: the rebuilt list holds at least k entries
-      if (threadIdx.x == 0) set_status(&p.ctl->status, NSML_ERR_INTERNAL);
-      return;
-    }
-
-    // ---- slow path: rebuild own segments as (all non-zero keys) + (zeros within budget) ----
+  if (list_total < p.k) {
+    // ---- slow path: this block's array becomes (all non-zero keys) + (zeros within budget) ----
+    const unsigned long long r_lo = seg_first * (unsigned long long)kSegElems;
+    const unsigned long long r_hi = min(seg_last * (unsigned long long)kSegElems, p.n);
+    my_idx = p.list_idx + r_lo;  // a block's range has room for all of its elements
+    my_val = p.list_val + r_lo;
     unsigned long long nnz = 0, zeros = 0;
-    for (unsigned int seg = s0 + warp; seg < s1; seg += kCta / 32) {
-      const unsigned long long first = warp_first_round(seg, p.segments, rounds);
-      const unsigned long long last = warp_first_round(seg + 1ull, p.segments, rounds);
-      unsigned int seg_nnz = 0, seg_zero = 0;
-      for (unsigned long long rd = first; rd < last; ++rd) {
-        uint32_t bits[4];
-        const int cnt = src.load_vals4(rd * kRound + lane * 4, p.n, bits);
+    for (unsigned long long i0 = r_lo + threadIdx.x * 4ull; i0 < r_hi; i0 += kFinThreads * 4ull) {
+      uint32_t bits[4];
+      const int cnt = src.load_vals4(i0, p.n, bits);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (e < cnt) {
-            if ((bits[e] & 0x7FFFFFFFu) != 0) ++seg_nnz; else ++seg_zero;
-          }
+      for (int e = 0; e < 4; ++e) {
+        if (e < cnt) {
+          if ((bits[e] & 0x7FFFFFFFu) != 0) ++nnz; else ++zeros;
         }
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        seg_nnz += __shfl_xor_sync(0xFFFFFFFFu, seg_nnz, o);
-        seg_zero += __shfl_xor_sync(0xFFFFFFFFu, seg_zero, o);
-      }
-      if (lane == 0) {
-        p.seg_zeros[seg] = seg_zero;
-        nnz += seg_nnz;
-        zeros += seg_zero;
       }
     }
     const unsigned long long block_nnz = block_sum(nnz, sh);
@@ -202,123 +317,108 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
 
     unsigned long long all_nnz = 0, zeros_before = 0;
-    for (unsigned int b = threadIdx.x; b < G; b += kCta) {
-      const unsigned long long w = ld_cg_u64(nz_counts + b);
+    for (unsigned int b = threadIdx.x; b < G; b += kFinThreads) {
+      const unsigned long long w = __ldcg(nz_counts + b);
       all_nnz += w >> 32;
       if (b < blk) zeros_before += w & 0xFFFFFFFFull;
     }
     all_nnz = block_sum(all_nnz, sh);
     zeros_before = block_sum(zeros_before, sh);
     const unsigned long long zero_budget = (p.k > all_nnz) ? p.k - all_nnz : 0;
+    // zeros of this block to keep, lowest index first
+    const unsigned long long allowed = (zero_budget > zeros_before) ? min(block_zeros, zero_budget - zeros_before) : 0ull;
 
-    for (unsigned int seg = s0 + warp; seg < s1; seg += kCta / 32) {
-      unsigned long long before = zeros_before;
-      for (unsigned int s = s0; s < seg; ++s) before += __ldcg(p.seg_zeros + s);
-      const unsigned long long seg_zero = __ldcg(p.seg_zeros + seg);
-      const unsigned long long allowed =
-          (zero_budget > before) ? min(seg_zero, zero_budget - before) : 0ull;  // zeros of this segment to keep
-      const unsigned long long first = warp_first_round(seg, p.segments, rounds);
-      const unsigned long long last = warp_first_round(seg + 1ull, p.segments, rounds);
-      const unsigned long long seg_base = first * kRound;
-      unsigned int kept = 0, zeros_seen = 0;
-      for (unsigned long long rd = first; rd < last; ++rd) {
-        uint32_t bits[4];
-        const int cnt = src.load_vals4(rd * kRound + lane * 4, p.n, bits);
-        unsigned int fz = 0, fn = 0;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (e < cnt) {
-            if ((bits[e] & 0x7FFFFFFFu) != 0) fn |= 1u << e; else fz |= 1u << e;
-          }
-        }
-        // zeros before this lane's quad in the round, then which of its zeros are within budget
-        const unsigned int zmine = __popc(fz);
-        unsigned int zincl = zmine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-          const unsigned int up = __shfl_up_sync(0xFFFFFFFFu, zincl, o);
-          if (lane >= o) zincl += up;
-        }
-        unsigned long long zrank = zeros_seen + zincl - zmine;
-        unsigned int f = fn;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (fz & (1u << e)) {
-            if (zrank < allowed) f |= 1u << e;
-            ++zrank;
-          }
-        }
-        zeros_seen += __shfl_sync(0xFFFFFFFFu, zincl, 31);
-        if (__any_sync(0xFFFFFFFFu, f != 0))
-          kept += append_round(f, bits, (uint32_t)(rd * kRound), seg_base + kept, p.seg_idx, p.seg_val);
-      }
-      if (lane == 0) p.seg_count[seg] = kept;
-    }
-    __threadfence();
     __syncthreads();
+    for (int b = threadIdx.x; b < kMaxBins; b += kFinThreads) sh.hist[b] = 0;
+    E = 0;
+    unsigned long long zeros_seen = 0;
+    nonfinite = false;
+    for (unsigned long long base = r_lo; base < r_hi; base += kFinThreads * 4ull) {
+      const unsigned long long i0 = base + threadIdx.x * 4ull;
+      uint32_t bits[4] = {0, 0, 0, 0};
+      const int cnt = (i0 < r_hi) ? src.load_vals4(i0, p.n, bits) : 0;
+      unsigned int fz = 0, fn = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (e < cnt) {
+          if ((bits[e] & 0x7FFFFFFFu) != 0) fn |= 1u << e; else fz |= 1u << e;
+        }
+      }
+      unsigned int z_total, keep_total;
+      unsigned long long zrank = zeros_seen + block_excl_scan(__popc(fz), z_total, sh);
+      unsigned int f = fn;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (fz & (1u << e)) {
+          if (zrank < allowed) f |= 1u << e;
+          ++zrank;
+        }
+      }
+      unsigned int pos = E + block_excl_scan(__popc(f), keep_total, sh);
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (f & (1u << e)) {
+          const uint32_t key = bits[e] & 0x7FFFFFFFu;
+          put_entry(pos, (uint32_t)(i0 + e), bits[e]);
+          nonfinite |= key >= kInfKey;
+          atomicAdd(&sh.hist[key >> digit_shift(0)], 1u);
+          ++pos;
+        }
+      }
+      zeros_seen += z_total;
+      E += keep_total;
+    }
+    if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
+    unsigned long long* totals2 = p.block_counts + 3 * kMaxFinalizeBlocks;
+    if (threadIdx.x == 0) totals2[blk] = E;
+    flush_hist<kMaxBins>(sh, p.hist + 3 * kMaxBins);
+    if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
+    unsigned long long part = 0;
+    for (unsigned int b = threadIdx.x; b < G; b += kFinThreads) part += __ldcg(totals2 + b);
+    if (block_sum(part, sh) < p.k) {  // cannot happen: the rebuilt list holds at least k entries
+      if (threadIdx.x == 0) set_status(&p.ctl->status, NSML_ERR_INTERNAL);
+      return;
+    }
+    ghist0 = p.hist + 3 * kMaxBins;
   }
+  __syncthreads();  // the block's array (shared copy and global) is complete
 
-  const unsigned int* ghist0_final = p.hist + (used_attempt == 0 ? 0 : 3) * kMaxBins;
-
-  // ---------------- phase 2: resolve digit 0, histogram of digit 1 ----------------
-  resolve_digit<kMaxBins>(ghist0_final, (unsigned int)p.k, sh);
+  // ---------------- phase 1: resolve digit 0, histogram of digit 1 ----------------
+  resolve_digit<kMaxBins>(ghist0, (unsigned int)p.k, sh);
   const unsigned int d0 = sh.out[0];
   unsigned int rem = sh.out[1];
-  for (int b = threadIdx.x; b < kMaxBins; b += kCta) sh.hist[b] = 0;
+  for (int b = threadIdx.x; b < kMaxBins; b += kFinThreads) sh.hist[b] = 0;
   __syncthreads();
-  for (unsigned int seg = s0 + warp; seg < s1; seg += kCta / 32) {
-    const unsigned int cnt = __ldcg(p.seg_count + seg);
-    const unsigned long long base = warp_first_round(seg, p.segments, rounds) * kRound;
-    for (unsigned int i = lane; i < cnt; i += 32) {
-      const uint32_t key = __ldcg(p.seg_val + base + i) & 0x7FFFFFFFu;
-      if ((key >> 19) == d0) atomicAdd(&sh.hist[(key >> 7) & 0xFFFu], 1u);
-    }
+  for (unsigned int j = threadIdx.x; j < E; j += kFinThreads) {
+    const uint32_t key = entry_val(j) & 0x7FFFFFFFu;
+    if ((key >> 19) == d0) atomicAdd(&sh.hist[(key >> 7) & 0xFFFu], 1u);
   }
   flush_hist<kMaxBins>(sh, p.hist + 1 * kMaxBins);
   if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
 
-  // ---------------- phase 3: resolve digit 1, histogram of digit 2 ----------------
+  // ---------------- phase 2: resolve digit 1, histogram of digit 2 ----------------
   resolve_digit<kMaxBins>(p.hist + 1 * kMaxBins, rem, sh);
   const unsigned int prefix24 = (d0 << 12) | sh.out[0];
   rem = sh.out[1];
-  for (int b = threadIdx.x; b < 128; b += kCta) sh.hist[b] = 0;
   __syncthreads();
-  for (unsigned int seg = s0 + warp; seg < s1; seg += kCta / 32) {
-    const unsigned int cnt = __ldcg(p.seg_count + seg);
-    const unsigned long long base = warp_first_round(seg, p.segments, rounds) * kRound;
-    for (unsigned int i = lane; i < cnt; i += 32) {
-      const uint32_t key = __ldcg(p.seg_val + base + i) & 0x7FFFFFFFu;
-      if ((key >> 7) == prefix24) atomicAdd(&sh.hist[key & 0x7Fu], 1u);
-    }
+  for (int b = threadIdx.x; b < 128; b += kFinThreads) sh.hist[b] = 0;
+  __syncthreads();
+  for (unsigned int j = threadIdx.x; j < E; j += kFinThreads) {
+    const uint32_t key = entry_val(j) & 0x7FFFFFFFu;
+    if ((key >> 7) == prefix24) atomicAdd(&sh.hist[key & 0x7Fu], 1u);
   }
   flush_hist<128>(sh, p.hist + 2 * kMaxBins);
   if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
 
-  // ---------------- phase 4: T and r; count own keys > T and == T ----------------
+  // ---------------- phase 3: T and r; count own keys > T and == T ----------------
   resolve_digit<128>(p.hist + 2 * kMaxBins, rem, sh);
   const uint32_t T = (prefix24 << 7) | sh.out[0];
   const unsigned long long r = sh.out[1];  // ties (key == T) to keep, lowest index first
   unsigned long long mine_a = 0, mine_c = 0;
-  for (unsigned int seg = s0 + warp; seg < s1; seg += kCta / 32) {
-    const unsigned int cnt = __ldcg(p.seg_count + seg);
-    const unsigned long long base = warp_first_round(seg, p.segments, rounds) * kRound;
-    unsigned int a = 0, c = 0;
-    for (unsigned int i = lane; i < cnt; i += 32) {
-      const uint32_t key = __ldcg(p.seg_val + base + i) & 0x7FFFFFFFu;
-      a += key > T;
-      c += key == T;
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      a += __shfl_xor_sync(0xFFFFFFFFu, a, o);
-      c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
-    }
-    if (lane == 0) {
-      sh.seg_a[seg - s0] = a;
-      sh.seg_c[seg - s0] = c;
-      mine_a += a;
-      mine_c += c;
-    }
+  for (unsigned int j = threadIdx.x; j < E; j += kFinThreads) {
+    const uint32_t key = entry_val(j) & 0x7FFFFFFFu;
+    mine_a += key > T;
+    mine_c += key == T;
   }
   const unsigned long long block_a = block_sum(mine_a, sh);
   const unsigned long long block_c = block_sum(mine_c, sh);
@@ -326,10 +426,10 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   if (threadIdx.x == 0) ac_counts[blk] = (block_a << 32) | block_c;
   if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
 
-  // ---------------- phase 5: write the survivors in index order ----------------
+  // ---------------- phase 4: write the survivors in index order ----------------
   unsigned long long a_before = 0, c_before = 0, a_all = 0, c_all = 0;
-  for (unsigned int b = threadIdx.x; b < G; b += kCta) {
-    const unsigned long long w = ld_cg_u64(ac_counts + b);
+  for (unsigned int b = threadIdx.x; b < G; b += kFinThreads) {
+    const unsigned long long w = __ldcg(ac_counts + b);
     a_all += w >> 32;
     c_all += w & 0xFFFFFFFFull;
     if (b < blk) {
@@ -346,40 +446,30 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     return;
   }
   uint32_t* out_idx = reinterpret_cast<uint32_t*>(p.payload + p.P.idx_off);
-  const unsigned int lt = (1u << lane) - 1u;
-  for (unsigned int seg = s0 + warp; seg < s1; seg += kCta / 32) {
-    unsigned long long a_done = a_before, c_done = c_before;
-    for (unsigned int s = 0; s < seg - s0; ++s) {
-      a_done += sh.seg_a[s];
-      c_done += sh.seg_c[s];
+  for (unsigned int base = 0; base < E; base += kFinThreads) {
+    const unsigned int j = base + threadIdx.x;
+    uint32_t bits = 0, key = 0;
+    if (j < E) {
+      bits = entry_val(j);
+      key = bits & 0x7FFFFFFFu;
     }
-    const unsigned int cnt = __ldcg(p.seg_count + seg);
-    const unsigned long long base = warp_first_round(seg, p.segments, rounds) * kRound;
-    for (unsigned int i0 = 0; i0 < cnt; i0 += 32) {
-      const unsigned int i = i0 + lane;
-      uint32_t bits = 0, key = 0;
-      if (i < cnt) {
-        bits = __ldcg(p.seg_val + base + i);
-        key = bits & 0x7FFFFFFFu;
-      }
-      const bool a = i < cnt && key > T;
-      const bool c = i < cnt && key == T;
-      const unsigned int ba = __ballot_sync(0xFFFFFFFFu, a);
-      const unsigned int bc = __ballot_sync(0xFFFFFFFFu, c);
-      const unsigned long long a_here = a_done + __popc(ba & lt);
-      const unsigned long long c_here = c_done + __popc(bc & lt);
-      if (a || (c && c_here < r)) {
-        const unsigned long long pos = a_here + min(c_here, r);
-        out_idx[pos] = __ldcg(p.seg_idx + base + i);
-        p.raw_val[pos] = __uint_as_float(bits);
-      }
-      a_done += __popc(ba);
-      c_done += __popc(bc);
+    const bool a = j < E && key > T;
+    const bool c = j < E && key == T;
+    unsigned int chunk_ac;
+    const unsigned int before = block_excl_scan((unsigned)a | ((unsigned)c << 16), chunk_ac, sh);  // counts <= 1024 each
+    const unsigned long long a_here = a_before + (before & 0xFFFFu);
+    const unsigned long long c_here = c_before + (before >> 16);
+    if (a || (c && c_here < r)) {
+      const unsigned long long pos = a_here + min(c_here, r);
+      out_idx[pos] = entry_idx(j);
+      p.raw_val[pos] = __uint_as_float(bits);
     }
+    a_before += chunk_ac & 0xFFFFu;
+    c_before += chunk_ac >> 16;
   }
   if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
 
-  // ---------------- phase 6: quantise, write the header ----------------
+  // ---------------- phase 5: quantise, write the header ----------------
   if (blk == 0 && threadIdx.x == 0) {
     nsml_payload_header h;
     h.magic = NSML_PAYLOAD_MAGIC;
@@ -394,18 +484,23 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     h.scale_off = p.P.scale_off;
     *reinterpret_cast<nsml_payload_header*>(p.payload) = h;
   }
+  // a group of 256 threads (8 warps) quantises one block of 1024 survivors at a time
   const unsigned long long qblocks = (p.k + NSML_QBLOCK - 1) / NSML_QBLOCK;
-  for (unsigned long long qb = blk; qb < qblocks; qb += G) {
-    const unsigned long long j0 = qb * NSML_QBLOCK + threadIdx.x * 4;
+  const int group = threadIdx.x >> 8, gtid = threadIdx.x & 255;
+  for (unsigned long long q0 = (unsigned long long)blk * 4; q0 < qblocks; q0 += (unsigned long long)G * 4) {
+    const unsigned long long qb = q0 + group;
+    const unsigned long long j0 = qb * NSML_QBLOCK + gtid * 4;
     float v[4] = {0.f, 0.f, 0.f, 0.f};
     int cnt = 0;
-    if (j0 + 4 <= p.k) {
-      const float4 f = __ldcg(reinterpret_cast<const float4*>(p.raw_val + j0));
-      v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
-      cnt = 4;
-    } else if (j0 < p.k) {
-      cnt = (int)(p.k - j0);
-      for (int e = 0; e < cnt; ++e) v[e] = __ldcg(p.raw_val + j0 + e);
+    if (qb < qblocks) {
+      if (j0 + 4 <= p.k) {
+        const float4 f = __ldcg(reinterpret_cast<const float4*>(p.raw_val + j0));
+        v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
+        cnt = 4;
+      } else if (j0 < p.k) {
+        cnt = (int)(p.k - j0);
+        for (int e = 0; e < cnt; ++e) v[e] = __ldcg(p.raw_val + j0 + e);
+      }
     }
     if (p.bits == NSML_BITS_FP16) {
       uint16_t* out = reinterpret_cast<uint16_t*>(p.payload + p.P.val_off);
@@ -419,26 +514,28 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
       }
       continue;
     }
-    // block max-abs: warp shuffles, then one value per warp through shared memory
+    // max-abs of the 1024 survivors: warp shuffles, then one value per warp through shared memory
     float m = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-    __syncthreads();  // qmax of the previous block of survivors has been read
-    if (lane == 0) sh.qmax[warp] = m;
+    __syncthreads();  // qmax of the previous round has been read
+    if (lane == 0) sh.qmax[threadIdx.x >> 5] = m;
     __syncthreads();
-    m = sh.qmax[0];
+    m = sh.qmax[group * 8];
 #pragma unroll
-    for (int w = 1; w < kCta / 32; ++w) m = fmaxf(m, sh.qmax[w]);
+    for (int w = 1; w < 8; ++w) m = fmaxf(m, sh.qmax[group * 8 + w]);
     const float scale = __fdiv_rn(m, 127.0f);
-    if (threadIdx.x == 0) reinterpret_cast<float*>(p.payload + p.P.scale_off)[qb] = scale;
-    signed char* out = reinterpret_cast<signed char*>(p.payload + p.P.val_off);
-    if (cnt == 4) {
-      uint32_t w = 0;
+    if (qb < qblocks) {
+      if (gtid == 0) reinterpret_cast<float*>(p.payload + p.P.scale_off)[qb] = scale;
+      signed char* out = reinterpret_cast<signed char*>(p.payload + p.P.val_off);
+      if (cnt == 4) {
+        uint32_t w = 0;
 #pragma unroll
-      for (int e = 0; e < 4; ++e) w |= ((uint32_t)encode_i8(v[e], scale) & 0xFFu) << (8 * e);
-      *reinterpret_cast<uint32_t*>(out + j0) = w;
-    } else {
-      for (int e = 0; e < cnt; ++e) out[j0 + e] = (signed char)encode_i8(v[e], scale);
+        for (int e = 0; e < 4; ++e) w |= ((uint32_t)encode_i8(v[e], scale) & 0xFFu) << (8 * e);
+        *reinterpret_cast<uint32_t*>(out + j0) = w;
+      } else {
+        for (int e = 0; e < cnt; ++e) out[j0 + e] = (signed char)encode_i8(v[e], scale);
+      }
     }
   }
 }

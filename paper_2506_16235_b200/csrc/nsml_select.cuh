@@ -3,22 +3,28 @@
 //
 // The bucket is streamed exactly once, by the compaction pass, which needs a
 // key `lo` such that a little more than k keys are >= lo.  k_sample draws one
-// element from each of 8192 equal strata of the bucket and radix-selects,
-// inside one thread block, the sample key whose rank leaves a six-sigma margin
-// above the expected rank of the k-th largest; lo is that key rounded down to
-// its top 24 bits.  The exact threshold is found afterwards on the short
-// candidate list (nsml_finalize.cuh), which also repairs the rare case of a
-// misleading sample, so the sample only decides how much work is done, never
-// the result.
+// element from each of 8192 equal strata of the bucket and radix-selects the
+// sample key whose rank leaves a six-sigma margin above the expected rank of
+// the k-th largest; lo is that key rounded down to its top 24 bits.  The exact
+// threshold is found afterwards on the short candidate list
+// (nsml_finalize.cuh), which also repairs the rare case of a misleading
+// sample, so the sample only decides how much work is done, never the result.
+//
+// The kernel is one cluster of eight blocks: 8192 threads fetch one scattered
+// element each (one round of memory latency, spread over eight SMs), write the
+// keys into block 0's shared memory through the cluster's distributed shared
+// memory, meet at the cluster barrier, and block 0 selects.
 #pragma once
+
+#include <cooperative_groups.h>
 
 #include "nsml_common.cuh"
 
 namespace nsml {
 
 constexpr int kSampleThreads = 1024;
-constexpr int kSamplesPerThread = 8;
-constexpr int kSamples = kSampleThreads * kSamplesPerThread;  // 8192 strata
+constexpr int kSampleBlocks = 8;
+constexpr int kSamples = kSampleThreads * kSampleBlocks;  // 8192 strata
 
 __device__ __forceinline__ uint32_t mix32(uint32_t x) {
   x ^= x >> 16; x *= 0x7FEB352Du;
@@ -27,8 +33,8 @@ __device__ __forceinline__ uint32_t mix32(uint32_t x) {
   return x;
 }
 
-// Block-wide search from the top over NB bins, PER consecutive bins per thread
-// (own[] holds this thread's bins, lowest first): leaves in s_out the digit d
+// Block-wide search from the top over bins held PER per thread (own[] holds
+// this thread's consecutive bins, lowest first): leaves in s_out the digit d
 // with #{digit > d} < rem <= #{digit >= d} and the rank left inside bin d.
 // Called by every thread of the block; s_tot needs one word per warp.
 template <int PER, int THREADS>
@@ -63,40 +69,51 @@ __device__ __forceinline__ void find_digit_from_top(const unsigned int (&own)[PE
   __syncthreads();
 }
 
-// One block.  Clears the per-call control region, then sets ctl->lo from a
-// stratified sample.  rank_from_top == 0 means "no sampling" (small bucket, or
-// nearly everything is kept): lo = 0.
+// Clears the per-call control region and sets ctl->lo from a stratified
+// sample.  rank_from_top == 0 means "no sampling" (small bucket, or nearly
+// everything is kept): lo = 0.
 template <int DTYPE>
-__global__ void __launch_bounds__(kSampleThreads)
+__global__ void __cluster_dims__(kSampleBlocks, 1, 1) __launch_bounds__(kSampleThreads)
 k_sample(BucketSrc<DTYPE> src, unsigned long long n, unsigned int rank_from_top, Ctl* ctl, uint4* zero_base,
          unsigned int zero_vec16) {
-  __shared__ unsigned int s_hist[kMaxBins];
+  namespace cg = cooperative_groups;
+  __shared__ unsigned int s_keys[kSamples];  // block 0: the sample keys, then (first 4096 words) the histogram
+  unsigned int* s_hist = s_keys;
   __shared__ unsigned int s_tot[kSampleThreads / 32];
   __shared__ unsigned int s_out[2];
+  cg::cluster_group cluster = cg::this_cluster();
+  const unsigned int rank = cluster.block_rank();
 
-  uint32_t keys[kSamplesPerThread];
   if (rank_from_top != 0) {
-#pragma unroll
-    for (int s = 0; s < kSamplesPerThread; ++s) {
-      const unsigned long long stratum = (unsigned long long)s * kSampleThreads + threadIdx.x;
-      const unsigned long long begin = stratum * n / kSamples;
-      const unsigned long long end = (stratum + 1) * n / kSamples;  // > begin because n >= 2 * kSamples
-      const unsigned long long pos = begin + mix32((uint32_t)stratum * 0x9E3779B1u + 0x85EBCA6Bu) % (uint32_t)(end - begin);
-      keys[s] = src.load1(pos) & 0x7FFFFFFFu;
-    }
+    const unsigned long long stratum = (unsigned long long)rank * kSampleThreads + threadIdx.x;
+    const unsigned long long begin = stratum * n / kSamples;
+    const unsigned long long end = (stratum + 1) * n / kSamples;  // > begin because n >= 2 * kSamples
+    const unsigned long long pos = begin + mix32((uint32_t)stratum * 0x9E3779B1u + 0x85EBCA6Bu) % (uint32_t)(end - begin);
+    const uint32_t key = src.load1(pos) & 0x7FFFFFFFu;
+    unsigned int* remote = cluster.map_shared_rank(s_keys, 0);
+    remote[stratum] = key;
   }
-  for (unsigned int i = threadIdx.x; i < zero_vec16; i += kSampleThreads) zero_base[i] = make_uint4(0, 0, 0, 0);
+  for (unsigned int i = rank * kSampleThreads + threadIdx.x; i < zero_vec16; i += kSamples)
+    zero_base[i] = make_uint4(0, 0, 0, 0);
+  __threadfence();
+  cluster.sync();  // keys have landed in block 0; the control region is cleared
+  if (rank != 0) return;
 
   unsigned int lo = 0;
   if (rank_from_top != 0) {
+    uint32_t keys[kSampleBlocks];
+#pragma unroll
+    for (int s = 0; s < kSampleBlocks; ++s) keys[s] = s_keys[s * kSampleThreads + threadIdx.x];
+    __syncthreads();  // every key is in registers: the buffer becomes the histogram
     unsigned int prefix = 0, rem = rank_from_top;
 #pragma unroll
     for (int level = 0; level < 2; ++level) {  // 12 + 12 bits
       const int shift = digit_shift(level);
+      __syncthreads();  // the previous level's bins have been read
       for (int b = threadIdx.x; b < kMaxBins; b += kSampleThreads) s_hist[b] = 0;
       __syncthreads();
 #pragma unroll
-      for (int s = 0; s < kSamplesPerThread; ++s)
+      for (int s = 0; s < kSampleBlocks; ++s)
         if (level == 0 || (keys[s] >> 19) == prefix) atomicAdd(&s_hist[(keys[s] >> shift) & (kMaxBins - 1)], 1u);
       __syncthreads();
       unsigned int own[4];
@@ -108,7 +125,6 @@ k_sample(BucketSrc<DTYPE> src, unsigned long long n, unsigned int rank_from_top,
     }
     lo = prefix << 7;
   }
-  __syncthreads();  // the control block was cleared above by other threads
   if (threadIdx.x == 0) ctl->lo = lo;
 }
 
