@@ -446,23 +446,34 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     return;
   }
   uint32_t* out_idx = reinterpret_cast<uint32_t*>(p.payload + p.P.idx_off);
-  for (unsigned int base = 0; base < E; base += kFinThreads) {
-    const unsigned int j = base + threadIdx.x;
-    uint32_t bits = 0, key = 0;
-    if (j < E) {
-      bits = entry_val(j);
-      key = bits & 0x7FFFFFFFu;
+  for (unsigned int base = 0; base < E; base += kFinThreads * 4) {  // four consecutive candidates per thread
+    const unsigned int j0 = base + threadIdx.x * 4;
+    uint32_t bits[4];
+    unsigned int fa = 0, fc = 0;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      bits[e] = 0;
+      if (j0 + e < E) {
+        bits[e] = entry_val(j0 + e);
+        const uint32_t key = bits[e] & 0x7FFFFFFFu;
+        fa |= (unsigned)(key > T) << e;
+        fc |= (unsigned)(key == T) << e;
+      }
     }
-    const bool a = j < E && key > T;
-    const bool c = j < E && key == T;
-    unsigned int chunk_ac;
-    const unsigned int before = block_excl_scan((unsigned)a | ((unsigned)c << 16), chunk_ac, sh);  // counts <= 1024 each
-    const unsigned long long a_here = a_before + (before & 0xFFFFu);
-    const unsigned long long c_here = c_before + (before >> 16);
-    if (a || (c && c_here < r)) {
-      const unsigned long long pos = a_here + min(c_here, r);
-      out_idx[pos] = entry_idx(j);
-      p.raw_val[pos] = __uint_as_float(bits);
+    unsigned int chunk_ac;  // counts per chunk are at most 4096 each: 16 bits are enough
+    const unsigned int before = block_excl_scan((unsigned)__popc(fa) | ((unsigned)__popc(fc) << 16), chunk_ac, sh);
+    unsigned long long a_here = a_before + (before & 0xFFFFu);
+    unsigned long long c_here = c_before + (before >> 16);
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      const bool a = (fa >> e) & 1u, c = (fc >> e) & 1u;
+      if (a || (c && c_here < r)) {
+        const unsigned long long pos = a_here + min(c_here, r);
+        out_idx[pos] = entry_idx(j0 + e);
+        p.raw_val[pos] = __uint_as_float(bits[e]);
+      }
+      a_here += a;
+      c_here += c;
     }
     a_before += chunk_ac & 0xFFFFu;
     c_before += chunk_ac >> 16;
@@ -486,8 +497,9 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   }
   // a group of 256 threads (8 warps) quantises one block of 1024 survivors at a time
   const unsigned long long qblocks = (p.k + NSML_QBLOCK - 1) / NSML_QBLOCK;
+  constexpr int kQGroups = kFinThreads / 256;
   const int group = threadIdx.x >> 8, gtid = threadIdx.x & 255;
-  for (unsigned long long q0 = (unsigned long long)blk * 4; q0 < qblocks; q0 += (unsigned long long)G * 4) {
+  for (unsigned long long q0 = (unsigned long long)blk * kQGroups; q0 < qblocks; q0 += (unsigned long long)G * kQGroups) {
     const unsigned long long qb = q0 + group;
     const unsigned long long j0 = qb * NSML_QBLOCK + gtid * 4;
     float v[4] = {0.f, 0.f, 0.f, 0.f};
