@@ -36,9 +36,9 @@
 
 namespace nsml {
 
-constexpr int kFinThreads = 1024;
+constexpr int kFinThreads = 512;
 constexpr int kFinWarps = kFinThreads / 32;
-constexpr int kCacheEntries = 20480;  // candidates a block keeps in shared memory (index + value: 160 KB)
+constexpr int kCacheEntries = 12288;  // candidates a block keeps in shared memory (index + value: 96 KB)
 constexpr size_t kFinalizeDynSmem = (size_t)kCacheEntries * 8;
 constexpr int kGatherChunk = kFinThreads * 8;  // segments per gather step
 
@@ -171,12 +171,13 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
 
   auto entry_val = [&](unsigned int j) -> uint32_t { return j < (unsigned)kCacheEntries ? cache_val[j] : __ldcg(my_val + j); };
   auto entry_idx = [&](unsigned int j) -> uint32_t { return j < (unsigned)kCacheEntries ? cache_idx[j] : __ldcg(my_idx + j); };
-  auto put_entry = [&](unsigned int j, uint32_t idx, uint32_t val) {
-    my_idx[j] = idx;
-    my_val[j] = val;
+  auto put_entry = [&](unsigned int j, uint32_t idx, uint32_t val) {  // shared memory first, global memory for the overflow
     if (j < (unsigned)kCacheEntries) {
       cache_idx[j] = idx;
       cache_val[j] = val;
+    } else {
+      my_idx[j] = idx;
+      my_val[j] = val;
     }
   };
 
@@ -260,28 +261,43 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
       __syncthreads();
       // entries of this chunk that fall in the block's share
       const unsigned long long from_pos = max(pos_cursor, share_lo), to_pos = min(pos_cursor + chunk_total, share_hi);
-      for (unsigned long long g = from_pos + threadIdx.x; g < to_pos; g += kFinThreads) {
-        const unsigned int j = (unsigned int)(g - pos_cursor);
-        int lo = 0, hi = kFinThreads - 1;  // last thread slot of the chunk whose offset is <= j
-        while (lo < hi) {
-          const int mid = (lo + hi + 1) >> 1;
-          if (sh.off[mid] <= j) lo = mid; else hi = mid - 1;
-        }
-        unsigned int within = j - sh.off[lo];
-        const uint4 c8 = sh.cnt8[lo];
-        const uint32_t words[4] = {c8.x, c8.y, c8.z, c8.w};
-        int e = 0;
+      const unsigned short* cnt16 = reinterpret_cast<const unsigned short*>(sh.cnt8);  // count of segment q of the chunk
+      for (unsigned long long g0 = from_pos + threadIdx.x * 4ull; g0 < to_pos; g0 += kFinThreads * 4ull) {
+        // four consecutive entries per thread, each located by a search over the thread slots
+        unsigned long long from[4];
+        const int cnt = (int)min(4ull, to_pos - g0);
 #pragma unroll
-        for (int q = 0; q < 8; ++q) {
-          const unsigned int c = (words[q >> 1] >> ((q & 1) * 16)) & 0xFFFFu;
-          if (q == e && within >= c) { within -= c; ++e; }
+        for (int e = 0; e < 4; ++e) {
+          if (e < cnt) {
+            const unsigned int j = (unsigned int)(g0 + e - pos_cursor);
+            int lo = 0, hi = kFinThreads - 1;  // last thread slot of the chunk whose offset is <= j
+            while (lo < hi) {
+              const int mid = (lo + hi + 1) >> 1;
+              if (sh.off[mid] <= j) lo = mid; else hi = mid - 1;
+            }
+            unsigned int within = j - sh.off[lo];
+            unsigned int q = lo * 8;  // at most 8 steps: the entry lies in this slot's segments
+            while (within >= cnt16[q]) { within -= cnt16[q]; ++q; }
+            from[e] = (seg_cursor + q) * kSegElems + within;
+          }
         }
-        const unsigned long long from = (seg_cursor + lo * 8ull + e) * kSegElems + within;
-        const uint32_t val = p.seg_val[from];
-        const uint32_t key = val & 0x7FFFFFFFu;
-        put_entry((unsigned int)(g - share_lo), p.seg_idx[from], val);
-        nonfinite |= key >= kInfKey;
-        atomicAdd(&sh.hist[key >> digit_shift(0)], 1u);
+        uint32_t vals[4], idxs[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (e < cnt) {
+            vals[e] = p.seg_val[from[e]];
+            idxs[e] = p.seg_idx[from[e]];
+          }
+        }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (e < cnt) {
+            const uint32_t key = vals[e] & 0x7FFFFFFFu;
+            put_entry((unsigned int)(g0 + e - share_lo), idxs[e], vals[e]);
+            nonfinite |= key >= kInfKey;
+            atomicAdd(&sh.hist[key >> digit_shift(0)], 1u);
+          }
+        }
       }
       pos_cursor += chunk_total;
       seg_cursor += kGatherChunk;
