@@ -16,6 +16,7 @@
 namespace nsml {
 
 constexpr int kDenseTile = 8192;  // dense elements per block iteration (32 KB of shared memory)
+constexpr int kMergeRound = 4 * kCta;  // payload entries a block loads before applying them
 
 struct PayloadTable {
   const unsigned char* p[NSML_MAX_WORKERS];
@@ -49,27 +50,39 @@ __device__ inline bool header_ok(const nsml_payload_header* h, unsigned long lon
 }
 
 // offsets[w][b] = first payload entry of worker w whose index is >= b*kDenseTile.
+// One warp per (worker, boundary): a 33-way search, every lane probing one
+// position per step, so a boundary costs about log33(k) memory round trips
+// instead of log2(k).
 __global__ void __launch_bounds__(kCta)
 k_partition(PayloadTable table, int W, unsigned long long n, unsigned int tiles, unsigned int* offsets, int* status) {
-  const unsigned long long g = (unsigned long long)blockIdx.x * kCta + threadIdx.x;
+  const int lane = threadIdx.x & 31;
+  const unsigned long long g = ((unsigned long long)blockIdx.x * kCta + threadIdx.x) >> 5;  // one warp per offset
   const unsigned long long per = (unsigned long long)tiles + 1;
-  if (g >= per * W) return;
+  if (g >= per * W) return;  // whole warps leave together
   const int w = (int)(g / per);
   const unsigned long long b = g % per;
   const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(table.p[w]);
   if (!header_ok(h, n)) {
-    if (b == 0) set_status(status, NSML_ERR_PAYLOAD);
-    offsets[g] = 0;
+    if (b == 0 && lane == 0) set_status(status, NSML_ERR_PAYLOAD);
+    if (lane == 0) offsets[g] = 0;
     return;
   }
   const uint32_t* idx = reinterpret_cast<const uint32_t*>(table.p[w] + h->idx_off);
   const unsigned long long target = b * kDenseTile;
-  unsigned long long lo = 0, hi = h->k;  // lower bound
-  while (lo < hi) {
-    const unsigned long long mid = (lo + hi) >> 1;
-    if (idx[mid] < target) lo = mid + 1; else hi = mid;
+  unsigned long long lo = 0, hi = h->k;  // the answer lies in [lo, hi]
+  while (hi - lo > 32) {
+    const unsigned long long width = hi - lo;
+    const unsigned long long probe = lo + (lane + 1) * width / 33;  // lo < probe < hi, ascending with the lane
+    const unsigned int below = __ballot_sync(0xFFFFFFFFu, idx[probe] < target);
+    const int c = __popc(below);  // ascending indices: the lanes below the target form a prefix
+    const unsigned long long new_lo = (c == 0) ? lo : lo + (unsigned long long)c * width / 33 + 1;
+    const unsigned long long new_hi = (c == 32) ? hi : lo + (unsigned long long)(c + 1) * width / 33;
+    lo = new_lo;
+    hi = new_hi;
   }
-  offsets[g] = (unsigned int)lo;
+  const bool below = (lo + lane < hi) && idx[lo + lane] < target;
+  const unsigned int rest = __ballot_sync(0xFFFFFFFFu, below);
+  if (lane == 0) offsets[g] = (unsigned int)(lo + __popc(rest));
 }
 
 __global__ void __launch_bounds__(kCta)
@@ -115,27 +128,62 @@ k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long
       __syncthreads();
     }
 
-    for (int w = 0; w < W; ++w) {
-      const unsigned int from = s_from[w], to = s_to[w];
-      if (to > from) {
-        const unsigned char* base = table.p[w];
-        const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(base);
-        const uint32_t* idx = reinterpret_cast<const uint32_t*>(base + h->idx_off);
-        const bool int8 = (h->bits == NSML_BITS_INT8);
-        const signed char* codes = reinterpret_cast<const signed char*>(base + h->val_off);
-        const uint16_t* halves = reinterpret_cast<const uint16_t*>(base + h->val_off);
-        const float* scales = reinterpret_cast<const float*>(base + h->scale_off);
-        for (unsigned int j = from + threadIdx.x; j < to; j += kCta) {
-          const unsigned long long off = (unsigned long long)idx[j] - lo;  // wraps if idx < lo
-          const float v = int8 ? decode_i8(codes[j], scales[j >> 10]) : decode_f16(halves[j]);
-          if (off < len) {
-            if (staged) s_acc[off] += v; else dense[lo + off] += v;
+    // The tile's entries of all workers, taken as one worker-major sequence of
+    // `total` entries, are processed kMergeRound at a time: every thread first
+    // loads its (up to 4) entries, so that one round costs one memory latency,
+    // then the adds are applied worker by worker (an element may receive one
+    // add per worker; within a worker indices are distinct).
+    for (unsigned int base = 0; base < total; base += kMergeRound) {
+      unsigned int off[4];
+      float val[4];
+      int wk[4];
+      int w_min = W, w_max = -1;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const unsigned int f = base + e * kCta + threadIdx.x;  // position in the flattened sequence
+        wk[e] = -1;
+        if (f < total) {
+          int w = 0;
+          unsigned int before = 0;
+          while (before + (s_to[w] - s_from[w]) <= f) { before += s_to[w] - s_from[w]; ++w; }  // w < W because f < total
+          const unsigned int j = s_from[w] + (f - before);
+          const unsigned char* pbase = table.p[w];
+          const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(pbase);
+          const unsigned long long o = (unsigned long long)reinterpret_cast<const uint32_t*>(pbase + h->idx_off)[j] - lo;  // wraps if idx < lo
+          float v;
+          if (h->bits == NSML_BITS_INT8)
+            v = decode_i8(reinterpret_cast<const signed char*>(pbase + h->val_off)[j],
+                          reinterpret_cast<const float*>(pbase + h->scale_off)[j >> 10]);
+          else
+            v = decode_f16(reinterpret_cast<const uint16_t*>(pbase + h->val_off)[j]);
+          if (o < len) {
+            wk[e] = w;
+            off[e] = (unsigned int)o;
+            val[e] = v;
           } else {
             bad = true;
           }
         }
       }
-      __syncthreads();  // worker w is done before worker w+1 adds to the same elements
+      // workers present in this round (the sequence is worker-major, so they form a range)
+      {
+        const unsigned int f_lo = base, f_hi = min(total, base + kMergeRound) - 1;
+        unsigned int before = 0;
+        for (int w = 0; w < W; ++w) {
+          const unsigned int c = s_to[w] - s_from[w];
+          if (c && before <= f_hi && before + c > f_lo) { w_min = min(w_min, w); w_max = max(w_max, w); }
+          before += c;
+        }
+      }
+      for (int w = w_min; w <= w_max; ++w) {
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (wk[e] == w) {
+            if (staged) s_acc[off[e]] += val[e]; else dense[lo + off[e]] += val[e];
+          }
+        }
+        __syncthreads();  // worker w is done before worker w+1 adds to the same elements
+      }
     }
 
     if (staged) {

@@ -235,7 +235,7 @@ static int accumulate_impl(const void* const* payloads, int W, float* dense, int
   if (cudaMemsetAsync(ws, 0, 256, st) != cudaSuccess) return NSML_ERR_CUDA;
   {
     LaunchScope scope(K_PARTITION, st);
-    unsigned long long threads = (unsigned long long)W * (tiles + 1ull);
+    unsigned long long threads = (unsigned long long)W * (tiles + 1ull) * 32;  // a warp per offset
     unsigned int grid = (unsigned int)((threads + kCta - 1) / kCta);
     k_partition<<<grid, kCta, 0, st>>>(table, W, (unsigned long long)n, tiles, offsets, status);
   }
