@@ -85,6 +85,32 @@ k_partition(PayloadTable table, int W, unsigned long long n, unsigned int tiles,
   if (lane == 0) offsets[g] = (unsigned int)(lo + __popc(rest));
 }
 
+// The same table with one thread per offset and a plain binary search: less
+// latency-efficient per offset, but with hundreds of thousands of offsets the
+// searches hide each other's latency and 32 times fewer threads are needed.
+__global__ void __launch_bounds__(kCta)
+k_partition_wide(PayloadTable table, int W, unsigned long long n, unsigned int tiles, unsigned int* offsets, int* status) {
+  const unsigned long long g = (unsigned long long)blockIdx.x * kCta + threadIdx.x;
+  const unsigned long long per = (unsigned long long)tiles + 1;
+  if (g >= per * W) return;
+  const int w = (int)(g / per);
+  const unsigned long long b = g % per;
+  const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(table.p[w]);
+  if (!header_ok(h, n)) {
+    if (b == 0) set_status(status, NSML_ERR_PAYLOAD);
+    offsets[g] = 0;
+    return;
+  }
+  const uint32_t* idx = reinterpret_cast<const uint32_t*>(table.p[w] + h->idx_off);
+  const unsigned long long target = b * kDenseTile;
+  unsigned long long lo = 0, hi = h->k;
+  while (lo < hi) {
+    const unsigned long long mid = (lo + hi) >> 1;
+    if (idx[mid] < target) lo = mid + 1; else hi = mid;
+  }
+  offsets[g] = (unsigned int)lo;
+}
+
 __global__ void __launch_bounds__(kCta)
 k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long n, int zero_first,
         unsigned int tiles, const unsigned int* __restrict__ offsets, int* status) {
@@ -111,9 +137,18 @@ k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long
     __syncthreads();
     const unsigned int total = s_total;
     if (total == 0 && !zero_first) continue;
-    // Accumulate mode with few entries: touch only their elements.  Otherwise
-    // stage the whole tile in shared memory and write it back in one sweep.
-    const bool staged = zero_first || (unsigned long long)total * 16 > len;
+    // Few entries: touch only their elements in global memory (after zero-filling
+    // the tile there in overwrite mode).  Many entries: stage the whole tile in
+    // shared memory and write it back in one sweep.
+    const bool staged = (unsigned long long)total * 16 > len;
+    if (!staged && zero_first) {
+      float* dtile = dense + lo;
+      for (unsigned int i = threadIdx.x * 4; i < len; i += kCta * 4) {
+        if (i + 4 <= len) *reinterpret_cast<float4*>(dtile + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+        else for (unsigned int e = i; e < len; ++e) dtile[e] = 0.f;
+      }
+      __syncthreads();  // the zeros are in place before any add reads them
+    }
 
     if (staged) {
       float* dtile = dense + lo;

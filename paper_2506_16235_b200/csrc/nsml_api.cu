@@ -235,9 +235,14 @@ static int accumulate_impl(const void* const* payloads, int W, float* dense, int
   if (cudaMemsetAsync(ws, 0, 256, st) != cudaSuccess) return NSML_ERR_CUDA;
   {
     LaunchScope scope(K_PARTITION, st);
-    unsigned long long threads = (unsigned long long)W * (tiles + 1ull) * 32;  // a warp per offset
-    unsigned int grid = (unsigned int)((threads + kCta - 1) / kCta);
-    k_partition<<<grid, kCta, 0, st>>>(table, W, (unsigned long long)n, tiles, offsets, status);
+    const unsigned long long offsets_needed = (unsigned long long)W * (tiles + 1ull);
+    if (offsets_needed <= 32768) {  // few offsets: a warp each, few round trips
+      unsigned int grid = (unsigned int)((offsets_needed * 32 + kCta - 1) / kCta);
+      k_partition<<<grid, kCta, 0, st>>>(table, W, (unsigned long long)n, tiles, offsets, status);
+    } else {  // many offsets: a thread each
+      unsigned int grid = (unsigned int)((offsets_needed + kCta - 1) / kCta);
+      k_partition_wide<<<grid, kCta, 0, st>>>(table, W, (unsigned long long)n, tiles, offsets, status);
+    }
   }
   {
     LaunchScope scope(K_MERGE, st);

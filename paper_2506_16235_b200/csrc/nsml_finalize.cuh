@@ -153,7 +153,7 @@ __device__ __forceinline__ void resolve_digit(const unsigned int* ghist, unsigne
 }
 
 template <int DTYPE>
-__global__ void __launch_bounds__(kFinThreads, 1)
+__global__ void __launch_bounds__(kFinThreads, 2)  // at most 64 registers: leaves room for the next bucket's pass
 k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   __shared__ FinalizeShared sh;
   extern __shared__ __align__(16) uint32_t s_cache[];  // values [kCacheEntries], then indices [kCacheEntries]

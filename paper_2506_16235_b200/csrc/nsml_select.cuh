@@ -95,8 +95,7 @@ k_sample(BucketSrc<DTYPE> src, unsigned long long n, unsigned int rank_from_top,
   }
   for (unsigned int i = rank * kSampleThreads + threadIdx.x; i < zero_vec16; i += kSamples)
     zero_base[i] = make_uint4(0, 0, 0, 0);
-  __threadfence();
-  cluster.sync();  // keys have landed in block 0; the control region is cleared
+  cluster.sync();  // release/acquire at cluster scope: keys have landed in block 0, the control region is cleared
   if (rank != 0) return;
 
   unsigned int lo = 0;
