@@ -70,7 +70,7 @@ struct LaunchScope {  // brackets one kernel launch
 struct DeviceInfo {
   bool ready = false;
   int sms = 0;
-  int compact_bucket = 0, finalize = 0, merge = 0;  // resident blocks per SM
+  int compact_bucket = 0, finalize_small = 0, finalize_large = 0, merge = 0;  // resident blocks per SM
 };
 static DeviceInfo g_dev[64];
 static std::mutex g_dev_mutex;
@@ -84,13 +84,20 @@ static int device_info(const DeviceInfo** out) {
     if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return NSML_ERR_CUDA;
     cudaError_t e = cudaSuccess;
     e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_bucket, k_compact_bucket<NSML_F32>, kCta, 0);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finalize<NSML_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFinalizeDynSmem);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_finalize<NSML_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kFinalizeDynSmem);
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.finalize, k_finalize<NSML_F32>, kFinThreads, kFinalizeDynSmem);
+    auto prepare = [&](auto kernel, int threads, int cache, int* resident) {
+      if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)finalize_dyn_smem(cache));
+      int r = 0;
+      if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, kernel, threads, finalize_dyn_smem(cache));
+      if (*resident == 0 || r < *resident) *resident = r;
+    };
+    prepare(k_finalize<NSML_F32, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
+    prepare(k_finalize<NSML_BF16, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
+    prepare(k_finalize<NSML_F32, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache, &d.finalize_large);
+    prepare(k_finalize<NSML_BF16, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache, &d.finalize_large);
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.merge, k_merge, kCta, 0);
     int coop = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    if (e != cudaSuccess || d.compact_bucket < 1 || d.finalize < 1 || d.merge < 1 || !coop) {
+    if (e != cudaSuccess || d.compact_bucket < 1 || d.finalize_small < 1 || d.finalize_large < 1 || d.merge < 1 || !coop) {
       cudaGetLastError();
       return NSML_ERR_CUDA;
     }
@@ -154,11 +161,14 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
     k_compact_bucket<DTYPE><<<grid, kCta, 0, st>>>(src, (unsigned long long)n, ctl, seg_idx, seg_val, seg_count,
                                                    reinterpret_cast<unsigned int*>(ws + L.group_count));
   }
-  // list stage: cooperative, one block per SM, every block co-resident
-  unsigned int fgrid = (unsigned int)(dev.sms * dev.finalize);
-  if (fgrid > (unsigned int)dev.sms) fgrid = dev.sms;
+  // list stage: cooperative, one block per SM, every block co-resident.  The small shape when a block's
+  // share of the expected candidates (k plus the sampling margin) fits its shared-memory cache.
+  unsigned int fgrid = (unsigned int)dev.sms;
   if ((unsigned long long)fgrid > nseg) fgrid = (unsigned int)nseg;
   if (fgrid > (unsigned int)kMaxFinalizeBlocks) fgrid = kMaxFinalizeBlocks;
+  const double p_keep = (double)k / (double)n;
+  const double expected = (double)n * (p_keep + 6.0 * std::sqrt(p_keep * (1.0 - p_keep) / kSamples)) + 64.0;
+  const bool small_shape = expected / fgrid <= (double)kFinSmallCache;
   FinalizeParams fp;
   fp.n = (unsigned long long)n;
   fp.k = (unsigned long long)k;
@@ -179,9 +189,14 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
   {
     LaunchScope scope(K_FINALIZE, st);
     void* args[] = {&src, &fp};
-    if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_finalize<DTYPE>), dim3(fgrid), dim3(kFinThreads), args,
-                                    kFinalizeDynSmem, st) != cudaSuccess)
-      return NSML_ERR_CUDA;
+    cudaError_t le;
+    if (small_shape)
+      le = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_finalize<DTYPE, kFinSmallThreads, kFinSmallCache>), dim3(fgrid),
+                                       dim3(kFinSmallThreads), args, finalize_dyn_smem(kFinSmallCache), st);
+    else
+      le = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_finalize<DTYPE, kFinLargeThreads, kFinLargeCache>), dim3(fgrid),
+                                       dim3(kFinLargeThreads), args, finalize_dyn_smem(kFinLargeCache), st);
+    if (le != cudaSuccess) return NSML_ERR_CUDA;
   }
   return NSML_OK;
 }

@@ -36,11 +36,13 @@
 
 namespace nsml {
 
-constexpr int kFinThreads = 512;
-constexpr int kFinWarps = kFinThreads / 32;
-constexpr int kCacheEntries = 12288;  // candidates a block keeps in shared memory (index + value: 96 KB)
-constexpr size_t kFinalizeDynSmem = (size_t)kCacheEntries * 8;
-constexpr int kGatherChunk = kFinThreads * 8;  // segments per gather step
+// Two shapes of the kernel.  The small one (256 threads, 4096 cached candidates,
+// ~53 KB of shared memory, 16K registers) lets several list stages, and the
+// next bucket's streaming pass, share an SM when buckets are compressed on
+// several streams; the large one is for long candidate lists.
+constexpr int kFinSmallThreads = 256, kFinSmallCache = 4096;
+constexpr int kFinLargeThreads = 1024, kFinLargeCache = 20480;
+constexpr size_t finalize_dyn_smem(int cache_entries) { return (size_t)cache_entries * 8; }
 
 struct FinalizeParams {
   unsigned long long n, k;
@@ -60,21 +62,23 @@ struct FinalizeParams {
   PayloadLayout P;
 };
 
+template <int THREADS>
 struct FinalizeShared {
   unsigned int hist[kMaxBins];
-  unsigned int off[kFinThreads];  // gather: exclusive offset of each thread's 8 segments within the chunk
-  uint4 cnt8[kFinThreads];        // gather: the 8 segment counts of each thread (16 bits each)
-  unsigned long long red[kFinWarps];
-  unsigned int scan[kFinWarps];
-  unsigned int tot[kFinWarps];
+  unsigned int off[THREADS];  // gather: exclusive offset of each thread's 8 segments within the chunk
+  uint4 cnt8[THREADS];        // gather: the 8 segment counts of each thread (16 bits each)
+  unsigned long long red[(THREADS / 32)];
+  unsigned int scan[(THREADS / 32)];
+  unsigned int tot[(THREADS / 32)];
   unsigned int out[2];
   unsigned long long start[2];  // gather: first group of this block's share, list position where that group starts
-  float qmax[kFinWarps];
+  float qmax[(THREADS / 32)];
   int ok;
 };
 
 // Sum over the block; every thread gets the result.
-__device__ __forceinline__ unsigned long long block_sum(unsigned long long v, FinalizeShared& sh) {
+template <int THREADS>
+__device__ __forceinline__ unsigned long long block_sum(unsigned long long v, FinalizeShared<THREADS>& sh) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
   __syncthreads();  // sh.red may still be read from an earlier call
@@ -82,12 +86,13 @@ __device__ __forceinline__ unsigned long long block_sum(unsigned long long v, Fi
   __syncthreads();
   unsigned long long s = 0;
 #pragma unroll
-  for (int w = 0; w < kFinWarps; ++w) s += sh.red[w];
+  for (int w = 0; w < (THREADS / 32); ++w) s += sh.red[w];
   return s;
 }
 
 // Exclusive prefix over the block in thread order; `total` = sum over the block.
-__device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned int& total, FinalizeShared& sh) {
+template <int THREADS>
+__device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned int& total, FinalizeShared<THREADS>& sh) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   unsigned int incl = v;
 #pragma unroll
@@ -100,7 +105,7 @@ __device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned
   __syncthreads();
   unsigned int before = 0, all = 0;
 #pragma unroll
-  for (int w = 0; w < kFinWarps; ++w) {
+  for (int w = 0; w < (THREADS / 32); ++w) {
     const unsigned int c = sh.scan[w];
     if (w < warp) before += c;
     all += c;
@@ -110,7 +115,8 @@ __device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned
 }
 
 // All blocks arrive, then all leave.  `target` = barrier ordinal * gridDim.x.
-__device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, FinalizeShared& sh) {
+template <int THREADS>
+__device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, FinalizeShared<THREADS>& sh) {
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
@@ -129,10 +135,10 @@ __device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, Fina
 }
 
 // Adds the block's shared histogram into the global one (non-empty bins only).
-template <int NB>
-__device__ __forceinline__ void flush_hist(FinalizeShared& sh, unsigned int* ghist) {
+template <int NB, int THREADS>
+__device__ __forceinline__ void flush_hist(FinalizeShared<THREADS>& sh, unsigned int* ghist) {
   __syncthreads();
-  for (int b = threadIdx.x; b < NB; b += kFinThreads) {
+  for (int b = threadIdx.x; b < NB; b += THREADS) {
     const unsigned int c = sh.hist[b];
     if (c) atomicAdd(&ghist[b], c);
   }
@@ -140,25 +146,25 @@ __device__ __forceinline__ void flush_hist(FinalizeShared& sh, unsigned int* ghi
 
 // Every block reads the global histogram of a level and finds the digit that
 // holds the rem-th largest key; digit and the rank left inside land in sh.out.
-template <int NB>
-__device__ __forceinline__ void resolve_digit(const unsigned int* ghist, unsigned int rem, FinalizeShared& sh) {
-  constexpr int PER = (NB + kFinThreads - 1) / kFinThreads;
+template <int NB, int THREADS>
+__device__ __forceinline__ void resolve_digit(const unsigned int* ghist, unsigned int rem, FinalizeShared<THREADS>& sh) {
+  constexpr int PER = (NB + THREADS - 1) / THREADS;
   unsigned int own[PER];
 #pragma unroll
   for (int b = 0; b < PER; ++b) {
     const int bin = threadIdx.x * PER + b;
     own[b] = (bin < NB) ? __ldcg(ghist + bin) : 0u;
   }
-  find_digit_from_top<PER, kFinThreads>(own, rem, sh.tot, sh.out);
+  find_digit_from_top<PER, THREADS>(own, rem, sh.tot, sh.out);
 }
 
-template <int DTYPE>
-__global__ void __launch_bounds__(kFinThreads, 2)  // at most 64 registers: leaves room for the next bucket's pass
+template <int DTYPE, int THREADS, int CACHE>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS)  // at most 64 registers per thread
 k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
-  __shared__ FinalizeShared sh;
-  extern __shared__ __align__(16) uint32_t s_cache[];  // values [kCacheEntries], then indices [kCacheEntries]
+  __shared__ FinalizeShared<THREADS> sh;
+  extern __shared__ __align__(16) uint32_t s_cache[];  // values [CACHE], then indices [CACHE]
   uint32_t* cache_val = s_cache;
-  uint32_t* cache_idx = s_cache + kCacheEntries;
+  uint32_t* cache_idx = s_cache + CACHE;
   const int lane = threadIdx.x & 31;
   const unsigned int G = gridDim.x, blk = blockIdx.x;
   // Index-range ownership (used by the slow path only) and the block's array.
@@ -169,10 +175,10 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   unsigned int barriers = 0;
   unsigned int E = 0;  // candidates this block owns
 
-  auto entry_val = [&](unsigned int j) -> uint32_t { return j < (unsigned)kCacheEntries ? cache_val[j] : __ldcg(my_val + j); };
-  auto entry_idx = [&](unsigned int j) -> uint32_t { return j < (unsigned)kCacheEntries ? cache_idx[j] : __ldcg(my_idx + j); };
+  auto entry_val = [&](unsigned int j) -> uint32_t { return j < (unsigned)CACHE ? cache_val[j] : __ldcg(my_val + j); };
+  auto entry_idx = [&](unsigned int j) -> uint32_t { return j < (unsigned)CACHE ? cache_idx[j] : __ldcg(my_idx + j); };
   auto put_entry = [&](unsigned int j, uint32_t idx, uint32_t val) {  // shared memory first, global memory for the overflow
-    if (j < (unsigned)kCacheEntries) {
+    if (j < (unsigned)CACHE) {
       cache_idx[j] = idx;
       cache_val[j] = val;
     } else {
@@ -185,7 +191,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   // Every block reads the per-group candidate counts the bucket pass left and
   // scans them, which gives the list position of every group and the total.
   const unsigned long long ngroups = (p.nseg + kGroupSegs - 1) / kGroupSegs;
-  const unsigned long long per_thread = (ngroups + kFinThreads - 1) / kFinThreads;
+  const unsigned long long per_thread = (ngroups + THREADS - 1) / THREADS;
   const unsigned long long g_begin = min(ngroups, threadIdx.x * per_thread);
   const unsigned long long g_end = min(ngroups, g_begin + per_thread);
   unsigned long long thread_sum = 0;
@@ -205,7 +211,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     __syncthreads();
     unsigned long long before = 0, all = 0;
 #pragma unroll
-    for (int w = 0; w < kFinWarps; ++w) {
+    for (int w = 0; w < (THREADS / 32); ++w) {
       const unsigned long long c = sh.red[w];
       if (w < warp) before += c;
       all += c;
@@ -215,7 +221,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   }
   const unsigned long long share_lo = (unsigned long long)blk * list_total / G;
   const unsigned long long share_hi = (unsigned long long)(blk + 1) * list_total / G;
-  for (int b = threadIdx.x; b < kMaxBins; b += kFinThreads) sh.hist[b] = 0;
+  for (int b = threadIdx.x; b < kMaxBins; b += THREADS) sh.hist[b] = 0;
   bool nonfinite = false;
   if (list_total >= p.k) {
     my_idx = p.list_idx + share_lo;
@@ -250,7 +256,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     };
     uint4 counts = load_counts(seg_cursor);
     while (pos_cursor < share_hi && seg_cursor < p.nseg) {
-      const uint4 next_counts = load_counts(seg_cursor + kGatherChunk);
+      const uint4 next_counts = load_counts(seg_cursor + (THREADS * 8));
       const unsigned int cnt = (counts.x & 0xFFFFu) + (counts.x >> 16) + (counts.y & 0xFFFFu) + (counts.y >> 16) +
                                (counts.z & 0xFFFFu) + (counts.z >> 16) + (counts.w & 0xFFFFu) + (counts.w >> 16);
       unsigned int chunk_total;
@@ -262,7 +268,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
       // entries of this chunk that fall in the block's share
       const unsigned long long from_pos = max(pos_cursor, share_lo), to_pos = min(pos_cursor + chunk_total, share_hi);
       const unsigned short* cnt16 = reinterpret_cast<const unsigned short*>(sh.cnt8);  // count of segment q of the chunk
-      for (unsigned long long g0 = from_pos + threadIdx.x * 4ull; g0 < to_pos; g0 += kFinThreads * 4ull) {
+      for (unsigned long long g0 = from_pos + threadIdx.x * 4ull; g0 < to_pos; g0 += THREADS * 4ull) {
         // four consecutive entries per thread, each located by a search over the thread slots
         unsigned long long from[4];
         const int cnt = (int)min(4ull, to_pos - g0);
@@ -270,7 +276,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
         for (int e = 0; e < 4; ++e) {
           if (e < cnt) {
             const unsigned int j = (unsigned int)(g0 + e - pos_cursor);
-            int lo = 0, hi = kFinThreads - 1;  // last thread slot of the chunk whose offset is <= j
+            int lo = 0, hi = THREADS - 1;  // last thread slot of the chunk whose offset is <= j
             while (lo < hi) {
               const int mid = (lo + hi + 1) >> 1;
               if (sh.off[mid] <= j) lo = mid; else hi = mid - 1;
@@ -300,11 +306,11 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
         }
       }
       pos_cursor += chunk_total;
-      seg_cursor += kGatherChunk;
+      seg_cursor += (THREADS * 8);
       counts = next_counts;
     }
     if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
-    flush_hist<kMaxBins>(sh, p.hist);
+    flush_hist<kMaxBins, THREADS>(sh, p.hist);
     if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
   }
   const unsigned int* ghist0 = p.hist;
@@ -316,7 +322,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     my_idx = p.list_idx + r_lo;  // a block's range has room for all of its elements
     my_val = p.list_val + r_lo;
     unsigned long long nnz = 0, zeros = 0;
-    for (unsigned long long i0 = r_lo + threadIdx.x * 4ull; i0 < r_hi; i0 += kFinThreads * 4ull) {
+    for (unsigned long long i0 = r_lo + threadIdx.x * 4ull; i0 < r_hi; i0 += THREADS * 4ull) {
       uint32_t bits[4];
       const int cnt = src.load_vals4(i0, p.n, bits);
 #pragma unroll
@@ -333,7 +339,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
 
     unsigned long long all_nnz = 0, zeros_before = 0;
-    for (unsigned int b = threadIdx.x; b < G; b += kFinThreads) {
+    for (unsigned int b = threadIdx.x; b < G; b += THREADS) {
       const unsigned long long w = __ldcg(nz_counts + b);
       all_nnz += w >> 32;
       if (b < blk) zeros_before += w & 0xFFFFFFFFull;
@@ -345,11 +351,11 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     const unsigned long long allowed = (zero_budget > zeros_before) ? min(block_zeros, zero_budget - zeros_before) : 0ull;
 
     __syncthreads();
-    for (int b = threadIdx.x; b < kMaxBins; b += kFinThreads) sh.hist[b] = 0;
+    for (int b = threadIdx.x; b < kMaxBins; b += THREADS) sh.hist[b] = 0;
     E = 0;
     unsigned long long zeros_seen = 0;
     nonfinite = false;
-    for (unsigned long long base = r_lo; base < r_hi; base += kFinThreads * 4ull) {
+    for (unsigned long long base = r_lo; base < r_hi; base += THREADS * 4ull) {
       const unsigned long long i0 = base + threadIdx.x * 4ull;
       uint32_t bits[4] = {0, 0, 0, 0};
       const int cnt = (i0 < r_hi) ? src.load_vals4(i0, p.n, bits) : 0;
@@ -387,10 +393,10 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
     unsigned long long* totals2 = p.block_counts + 3 * kMaxFinalizeBlocks;
     if (threadIdx.x == 0) totals2[blk] = E;
-    flush_hist<kMaxBins>(sh, p.hist + 3 * kMaxBins);
+    flush_hist<kMaxBins, THREADS>(sh, p.hist + 3 * kMaxBins);
     if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
     unsigned long long part = 0;
-    for (unsigned int b = threadIdx.x; b < G; b += kFinThreads) part += __ldcg(totals2 + b);
+    for (unsigned int b = threadIdx.x; b < G; b += THREADS) part += __ldcg(totals2 + b);
     if (block_sum(part, sh) < p.k) {  // cannot happen: the rebuilt list holds at least k entries
       if (threadIdx.x == 0) set_status(&p.ctl->status, NSML_ERR_INTERNAL);
       return;
@@ -400,38 +406,38 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   __syncthreads();  // the block's array (shared copy and global) is complete
 
   // ---------------- phase 1: resolve digit 0, histogram of digit 1 ----------------
-  resolve_digit<kMaxBins>(ghist0, (unsigned int)p.k, sh);
+  resolve_digit<kMaxBins, THREADS>(ghist0, (unsigned int)p.k, sh);
   const unsigned int d0 = sh.out[0];
   unsigned int rem = sh.out[1];
-  for (int b = threadIdx.x; b < kMaxBins; b += kFinThreads) sh.hist[b] = 0;
+  for (int b = threadIdx.x; b < kMaxBins; b += THREADS) sh.hist[b] = 0;
   __syncthreads();
-  for (unsigned int j = threadIdx.x; j < E; j += kFinThreads) {
+  for (unsigned int j = threadIdx.x; j < E; j += THREADS) {
     const uint32_t key = entry_val(j) & 0x7FFFFFFFu;
     if ((key >> 19) == d0) atomicAdd(&sh.hist[(key >> 7) & 0xFFFu], 1u);
   }
-  flush_hist<kMaxBins>(sh, p.hist + 1 * kMaxBins);
+  flush_hist<kMaxBins, THREADS>(sh, p.hist + 1 * kMaxBins);
   if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
 
   // ---------------- phase 2: resolve digit 1, histogram of digit 2 ----------------
-  resolve_digit<kMaxBins>(p.hist + 1 * kMaxBins, rem, sh);
+  resolve_digit<kMaxBins, THREADS>(p.hist + 1 * kMaxBins, rem, sh);
   const unsigned int prefix24 = (d0 << 12) | sh.out[0];
   rem = sh.out[1];
   __syncthreads();
-  for (int b = threadIdx.x; b < 128; b += kFinThreads) sh.hist[b] = 0;
+  for (int b = threadIdx.x; b < 128; b += THREADS) sh.hist[b] = 0;
   __syncthreads();
-  for (unsigned int j = threadIdx.x; j < E; j += kFinThreads) {
+  for (unsigned int j = threadIdx.x; j < E; j += THREADS) {
     const uint32_t key = entry_val(j) & 0x7FFFFFFFu;
     if ((key >> 7) == prefix24) atomicAdd(&sh.hist[key & 0x7Fu], 1u);
   }
-  flush_hist<128>(sh, p.hist + 2 * kMaxBins);
+  flush_hist<128, THREADS>(sh, p.hist + 2 * kMaxBins);
   if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
 
   // ---------------- phase 3: T and r; count own keys > T and == T ----------------
-  resolve_digit<128>(p.hist + 2 * kMaxBins, rem, sh);
+  resolve_digit<128, THREADS>(p.hist + 2 * kMaxBins, rem, sh);
   const uint32_t T = (prefix24 << 7) | sh.out[0];
   const unsigned long long r = sh.out[1];  // ties (key == T) to keep, lowest index first
   unsigned long long mine_a = 0, mine_c = 0;
-  for (unsigned int j = threadIdx.x; j < E; j += kFinThreads) {
+  for (unsigned int j = threadIdx.x; j < E; j += THREADS) {
     const uint32_t key = entry_val(j) & 0x7FFFFFFFu;
     mine_a += key > T;
     mine_c += key == T;
@@ -444,7 +450,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
 
   // ---------------- phase 4: write the survivors in index order ----------------
   unsigned long long a_before = 0, c_before = 0, a_all = 0, c_all = 0;
-  for (unsigned int b = threadIdx.x; b < G; b += kFinThreads) {
+  for (unsigned int b = threadIdx.x; b < G; b += THREADS) {
     const unsigned long long w = __ldcg(ac_counts + b);
     a_all += w >> 32;
     c_all += w & 0xFFFFFFFFull;
@@ -462,7 +468,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     return;
   }
   uint32_t* out_idx = reinterpret_cast<uint32_t*>(p.payload + p.P.idx_off);
-  for (unsigned int base = 0; base < E; base += kFinThreads * 4) {  // four consecutive candidates per thread
+  for (unsigned int base = 0; base < E; base += THREADS * 4) {  // four consecutive candidates per thread
     const unsigned int j0 = base + threadIdx.x * 4;
     uint32_t bits[4];
     unsigned int fa = 0, fc = 0;
@@ -513,7 +519,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   }
   // a group of 256 threads (8 warps) quantises one block of 1024 survivors at a time
   const unsigned long long qblocks = (p.k + NSML_QBLOCK - 1) / NSML_QBLOCK;
-  constexpr int kQGroups = kFinThreads / 256;
+  constexpr int kQGroups = THREADS / 256;
   const int group = threadIdx.x >> 8, gtid = threadIdx.x & 255;
   for (unsigned long long q0 = (unsigned long long)blk * kQGroups; q0 < qblocks; q0 += (unsigned long long)G * kQGroups) {
     const unsigned long long qb = q0 + group;
