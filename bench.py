@@ -114,8 +114,54 @@ class Workload:
     name = ""
     dtype = "f32"
 
+    use_graphs = False  # replay each job from a CUDA graph captured on its stream
+    graph_period = 1    # steps after which the set of distinct jobs repeats (all graphs exist after that many)
+    graphs_ok = True    # False where every step brings new jobs (nothing to replay)
+
     def account(self, acc, kernel, nbytes):
         acc[kernel] = acc.get(kernel, 0) + nbytes
+
+    def before_step(self, i):
+        """Host side of a step (the controller); returns nothing."""
+
+    def after_step(self, i, sent):
+        """Feeds the bytes this step would send back to the controller."""
+
+    def step(self, i, acc=None):
+        """One pass of the whole path.  Jobs (one bucket: its compress calls and the sum) are independent and
+        go to the streams round-robin; with use_graphs a job is captured once per (inputs, ratio, codec, stream)
+        and replayed, which takes the per-call launch cost off the host."""
+        torch, nsml = self.torch, self.nsml
+        self.before_step(i)
+        sent = 0
+        graphs = self.use_graphs and acc is None and self.lanes.active == len(self.lanes.all)
+        for ordinal, (key, nbytes, enqueue) in enumerate(self.jobs(i)):
+            lane = self.lanes.all[ordinal % self.lanes.active]
+            sent += nbytes
+            if not graphs:
+                enqueue(lane, acc)
+                continue
+            gkey = (key, ordinal % self.lanes.active)
+            entry = self.graph_cache.get(gkey)
+            if entry is None:
+                before = nsml.nsml_launch_count()
+                g = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(g, stream=lane.stream):
+                    enqueue(lane, None)
+                entry = (g, nsml.nsml_launch_count() - before)
+                self.graph_cache[gkey] = entry
+            torch.cuda.set_stream(lane.stream)
+            entry[0].replay()
+            self.replayed_launches += entry[1]
+        if graphs:
+            torch.cuda.set_stream(self.home_stream)
+        self.after_step(i, sent)
+
+    def init_graphs(self, use_graphs):
+        self.use_graphs = use_graphs and self.graphs_ok
+        self.graph_cache = {}
+        self.replayed_launches = 0
+        self.home_stream = self.torch.cuda.current_stream()
 
     def compress_bytes(self, acc, n, esize, k, bits):
         vb = 1 if bits == 8 else 2
@@ -177,6 +223,7 @@ class Lanes:
 class ResnetWorkload(Workload):
     name = "resnet50: 25.6M fp32 params, 4 buckets of 25 MB, ratio sweep {0.5,0.1,0.01,0.001} x {int8,fp16}, W=1"
     REPLICAS = 9  # 9 x 102 MB of inputs: a replica is reused only after > 400 MB of other inputs
+    graph_period = 9
 
     def __init__(self, nsml, torch, device, rank, nlanes=2):
         from paper_2506_16235_b200 import synth
@@ -198,24 +245,29 @@ class ResnetWorkload(Workload):
                        "sweep": [[r, b] for r, b in SWEEP], "W": 1, "streams": nlanes,
                        "l2": "inputs rotate over 9 replicas (920 MB > 126 MB L2)"}
 
-    def step(self, i, acc=None):
-        nsml = self.nsml
+    def before_step(self, i):
         # the controller runs every step (its ratio is reported, the sweep's ratios are the ones compressed with)
         self.ctrl.select_ratio(self.last[0], self.last[1], self.dense_bytes)
-        sent = 0
-        for c, (ratio, bits) in enumerate(SWEEP):
-            rep = self.replicas[(i * len(SWEEP) + c) % self.REPLICAS]
-            for g in rep:
-                n = g.numel()
-                lane = self.lanes.next()
-                p = nsml.nsml_compress(g, ratio, bits, payload=lane.payloads[0], workspace=lane.ws, stream=lane.stream)
-                nsml.nsml_decompress_accumulate([p], lane.dense[:n], zero_first=True, workspace=lane.aws, stream=lane.stream)
-                sent += p.numel()
-                if acc is not None:
-                    k = nsml.nsml_k_of(n, ratio)
-                    self.compress_bytes(acc, n, 4, k, bits)
-                    self.merge_bytes(acc, n, [(k, bits)])
+
+    def after_step(self, i, sent):
         self.last = (float(sent), 1e-3 + sent / 1.25e9)  # as if sent over a 10 Gbps link
+
+    def jobs(self, i):
+        nsml = self.nsml
+        for c, (ratio, bits) in enumerate(SWEEP):
+            r = (i * len(SWEEP) + c) % self.REPLICAS
+            for b, g in enumerate(self.replicas[r]):
+                n = g.numel()
+
+                def enqueue(lane, acc, g=g, n=n, ratio=ratio, bits=bits):
+                    p = nsml.nsml_compress(g, ratio, bits, payload=lane.payloads[0], workspace=lane.ws, stream=lane.stream)
+                    nsml.nsml_decompress_accumulate([p], lane.dense[:n], zero_first=True, workspace=lane.aws, stream=lane.stream)
+                    if acc is not None:
+                        k = nsml.nsml_k_of(n, ratio)
+                        self.compress_bytes(acc, n, 4, k, bits)
+                        self.merge_bytes(acc, n, [(k, bits)])
+
+                yield (r, b, ratio, bits), nsml.nsml_payload_bytes(n, ratio, bits), enqueue
 
     # ---- host-buffer variant for the end-to-end number ----
     def setup_host(self):
@@ -300,33 +352,28 @@ class Gpt2Workload(Workload):
                        "ratio": self.RATIO, "bits": self.BITS, "W": self.W, "streams": nlanes,
                        "l2": "inputs are 2 GB per step, far larger than the 126 MB L2"}
 
-    def step(self, i, acc=None):
-        nsml = self.nsml
+    def before_step(self, i):
         self.ctrl.select_ratio(self.last[0], self.last[1], self.dense_bytes)
-        sent = 0
-        for b, n in enumerate(self.sizes):
-            # the W workers of a bucket are independent until they are summed: they alternate between the
-            # streams, each with a workspace of its own, and the sum waits for both
-            home = self.lanes.next()
-            ps = []
-            for w in range(self.W):
-                lane = self.lanes.all[(self.lanes.turn + w) % self.lanes.active]
-                p = nsml.nsml_compress(self.workers[w][b], self.RATIO, self.BITS, payload=home.payloads[w],
-                                       workspace=lane.ws, stream=lane.stream)
-                ps.append(p)
-                sent += p.numel()
-            for lane in self.lanes.all[:self.lanes.active]:
-                if lane is not home:
-                    ev = self.torch.cuda.Event()
-                    ev.record(lane.stream)
-                    home.stream.wait_event(ev)
-            nsml.nsml_decompress_accumulate(ps, home.dense[:n], zero_first=True, workspace=home.aws, stream=home.stream)
-            if acc is not None:
-                k = nsml.nsml_k_of(n, self.RATIO)
-                for w in range(self.W):
-                    self.compress_bytes(acc, n, 4, k, self.BITS)
-                self.merge_bytes(acc, n, [(k, self.BITS)] * self.W)
+
+    def after_step(self, i, sent):
         self.last = (float(sent), 1e-3 + sent / 1.25e9)
+
+    def jobs(self, i):
+        nsml = self.nsml
+        for b, n in enumerate(self.sizes):
+            def enqueue(lane, acc, b=b, n=n):
+                # the W workers' buckets are compressed one after the other on this job's stream, then summed;
+                # other buckets run on the other streams meanwhile
+                ps = [nsml.nsml_compress(self.workers[w][b], self.RATIO, self.BITS, payload=lane.payloads[w],
+                                         workspace=lane.ws, stream=lane.stream) for w in range(self.W)]
+                nsml.nsml_decompress_accumulate(ps, lane.dense[:n], zero_first=True, workspace=lane.aws, stream=lane.stream)
+                if acc is not None:
+                    k = nsml.nsml_k_of(n, self.RATIO)
+                    for w in range(self.W):
+                        self.compress_bytes(acc, n, 4, k, self.BITS)
+                    self.merge_bytes(acc, n, [(k, self.BITS)] * self.W)
+
+            yield (b,), self.W * nsml.nsml_payload_bytes(n, self.RATIO, self.BITS), enqueue
 
     def setup_host(self):
         torch, nsml = self.torch, self.nsml
@@ -364,6 +411,7 @@ class Gpt2Workload(Workload):
 class DecoderWorkload(Workload):
     name = "decoder-1.3B: bf16 grads, 64M-element buckets, fp16 values, ratio from the controller on a 100/10/1 Gbps trace"
     dtype = "bf16"
+    graphs_ok = False  # the controller emits a new ratio every step
 
     def __init__(self, nsml, torch, device, rank, nlanes=2):
         from paper_2506_16235_b200 import synth
@@ -397,23 +445,29 @@ class DecoderWorkload(Workload):
                        "controller": {"ratio_init": 0.1, "ratio_min": 0.001, "ratio_max": 0.1}, "streams": nlanes,
                        "l2": "inputs are 2.6 GB per step"}
 
-    def step(self, i, acc=None):
-        nsml = self.nsml
-        ratio = self.ctrl.select_ratio(self.last[0], self.last[1], self.dense_bytes)
-        self.ratios.append(ratio)
-        sent = 0
-        for g in self.buckets:
-            n = g.numel()
-            lane = self.lanes.next()
-            p = nsml.nsml_compress(g, ratio, 16, payload=lane.payloads[0], workspace=lane.ws, stream=lane.stream)
-            nsml.nsml_decompress_accumulate([p], lane.dense[:n], zero_first=True, workspace=lane.aws, stream=lane.stream)
-            sent += p.numel()
-            if acc is not None:
-                k = nsml.nsml_k_of(n, ratio)
-                self.compress_bytes(acc, n, 2, k, 16)
-                self.merge_bytes(acc, n, [(k, 16)])
+    def before_step(self, i):
+        self.ratio = self.ctrl.select_ratio(self.last[0], self.last[1], self.dense_bytes)
+        self.ratios.append(self.ratio)
+
+    def after_step(self, i, sent):
         bw = (100e9, 10e9, 1e9)[min(2, i // 30)] / 8.0  # bytes/s of the synthetic link
         self.last = (float(sent), 1e-3 + sent / bw)
+
+    def jobs(self, i):
+        nsml = self.nsml
+        ratio = self.ratio
+        for b, g in enumerate(self.buckets):
+            n = g.numel()
+
+            def enqueue(lane, acc, g=g, n=n, ratio=ratio):
+                p = nsml.nsml_compress(g, ratio, 16, payload=lane.payloads[0], workspace=lane.ws, stream=lane.stream)
+                nsml.nsml_decompress_accumulate([p], lane.dense[:n], zero_first=True, workspace=lane.aws, stream=lane.stream)
+                if acc is not None:
+                    k = nsml.nsml_k_of(n, ratio)
+                    self.compress_bytes(acc, n, 2, k, 16)
+                    self.merge_bytes(acc, n, [(k, 16)])
+
+            yield (b, ratio), nsml.nsml_payload_bytes(n, ratio, 16), enqueue
 
     def setup_host(self):
         torch, nsml = self.torch, self.nsml
@@ -464,11 +518,13 @@ class AggWorkload(Workload):
         self.config = {"workload": self.name, "n": self.N, "k": self.k, "W": self.W,
                        "l2": "payloads 700 MB + dense 1.4 GB per step"}
 
-    def step(self, i, acc=None):
-        lane = self.lanes.all[0]
-        self.nsml.nsml_decompress_accumulate(self.payloads, self.dense, zero_first=True, workspace=self.aws, stream=lane.stream)
-        if acc is not None:
-            self.merge_bytes(acc, self.N, [(self.k, 8)] * self.W)
+    def jobs(self, i):
+        def enqueue(lane, acc):
+            self.nsml.nsml_decompress_accumulate(self.payloads, lane.dense, zero_first=True, workspace=lane.aws, stream=lane.stream)
+            if acc is not None:
+                self.merge_bytes(acc, self.N, [(self.k, 8)] * self.W)
+
+        yield (0,), sum(p.numel() for p in self.payloads), enqueue
 
     def setup_host(self):
         torch, nsml = self.torch, self.nsml
@@ -548,7 +604,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="nsml", choices=["nsml", "reference"])
-    ap.add_argument("--streams", type=int, default=2, help="CUDA streams that independent buckets alternate between")
+    ap.add_argument("--streams", type=int, default=4, help="CUDA streams that independent buckets alternate between")
+    ap.add_argument("--no-graphs", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-large-bucket-leg", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (e2e is then null)")
@@ -585,6 +642,10 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     wl = WORKLOADS[args.workload](nsml, torch, device, rank, nlanes=max(1, args.streams))
+    wl.init_graphs(not args.no_graphs)
+    if wl.use_graphs:
+        warmup = max(warmup, wl.graph_period)  # every job has been captured before the timed region starts
+    wl.config["cuda_graphs"] = bool(wl.use_graphs)
 
     def barrier():
         if dist is not None:
@@ -597,7 +658,7 @@ def main():
         wl.step(i)
     wl.lanes.join()
     barrier()
-    launches0 = nsml.nsml_launch_count()
+    launches0, replayed0 = nsml.nsml_launch_count(), wl.replayed_launches
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local_rank) as clocks:
         ev0.record()
@@ -608,7 +669,7 @@ def main():
         ev1.record()
         torch.cuda.synchronize()
     elapsed_ms = ev0.elapsed_time(ev1)
-    launches = nsml.nsml_launch_count() - launches0
+    launches = nsml.nsml_launch_count() - launches0 + wl.replayed_launches - replayed0
     barrier()
     if dist is not None:
         t = torch.tensor([elapsed_ms], device=device, dtype=torch.float64)
@@ -678,7 +739,8 @@ def main():
 
     # ---- a 25M-element bucket, where the 60 %-of-HBM target applies ----
     if rank == 0 and args.workload == "resnet50" and not args.no_large_bucket_leg:
-        big = Gpt2Workload(nsml, torch, device, rank, buckets=[2], nlanes=max(1, args.streams))
+        big = Gpt2Workload(nsml, torch, device, rank, buckets=[2, 3, 2, 3], nlanes=max(1, args.streams))
+        big.init_graphs(not args.no_graphs)
         big.lanes.fork()
         for i in range(3):
             big.step(i)
@@ -708,7 +770,7 @@ def main():
                 gbs = acc2.get(name, 0) / (ms * 1e-3) / 1e9
                 per[name] = {"us_per_launch": 1e3 * ms / cnt, "algorithmic_GBps": gbs, "frac_of_peak": gbs / peak,
                              "frac_of_nominal_8TBps": gbs / 8000.0}
-        out["bucket_25M"] = {"workload": "one 25M-element fp32 bucket, ratio 0.01, int8, W=4",
+        out["bucket_25M"] = {"workload": "four 25M-element fp32 buckets, ratio 0.01, int8, W=4 workers each",
                              "value": big.input_bytes_per_step / (big_ms * 1e-3) / 1e9, "unit": UNIT,
                              "ms_per_step": big_ms, "kernels": per}
         del big

@@ -468,37 +468,48 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     return;
   }
   uint32_t* out_idx = reinterpret_cast<uint32_t*>(p.payload + p.P.idx_off);
-  for (unsigned int base = 0; base < E; base += THREADS * 4) {  // four consecutive candidates per thread
-    const unsigned int j0 = base + threadIdx.x * 4;
-    uint32_t bits[4];
-    unsigned int fa = 0, fc = 0;
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      bits[e] = 0;
-      if (j0 + e < E) {
-        bits[e] = entry_val(j0 + e);
-        const uint32_t key = bits[e] & 0x7FFFFFFFu;
-        fa |= (unsigned)(key > T) << e;
-        fc |= (unsigned)(key == T) << e;
-      }
+  {
+    // Each warp owns a contiguous run of the block's candidates.  First pass: count its keys > T and == T;
+    // one exchange of the warp totals through shared memory; second pass: ranks by ballot, coalesced writes.
+    constexpr int NW = THREADS / 32;
+    const int warp = threadIdx.x >> 5;
+    const unsigned int lt = (1u << lane) - 1u;
+    const unsigned int per_warp = ((E + NW - 1) / NW + 31) / 32 * 32;
+    const unsigned int w_lo = min(E, warp * per_warp), w_hi = min(E, w_lo + per_warp);
+    unsigned int wa = 0, wc = 0;
+    for (unsigned int j0 = w_lo; j0 < w_hi; j0 += 32) {
+      const unsigned int j = j0 + lane;
+      const uint32_t key = (j < w_hi) ? (entry_val(j) & 0x7FFFFFFFu) : 0u;
+      wa += __popc(__ballot_sync(0xFFFFFFFFu, j < w_hi && key > T));
+      wc += __popc(__ballot_sync(0xFFFFFFFFu, j < w_hi && key == T));
     }
-    unsigned int chunk_ac;  // counts per chunk are at most 4096 each: 16 bits are enough
-    const unsigned int before = block_excl_scan((unsigned)__popc(fa) | ((unsigned)__popc(fc) << 16), chunk_ac, sh);
-    unsigned long long a_here = a_before + (before & 0xFFFFu);
-    unsigned long long c_here = c_before + (before >> 16);
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-      const bool a = (fa >> e) & 1u, c = (fc >> e) & 1u;
-      if (a || (c && c_here < r)) {
-        const unsigned long long pos = a_here + min(c_here, r);
-        out_idx[pos] = entry_idx(j0 + e);
-        p.raw_val[pos] = __uint_as_float(bits[e]);
-      }
-      a_here += a;
-      c_here += c;
+    __syncthreads();  // sh.red may still be read by the block sums above
+    if (lane == 0) sh.red[warp] = ((unsigned long long)wa << 32) | wc;
+    __syncthreads();
+    unsigned long long a_here = a_before, c_here = c_before;
+    for (int w = 0; w < warp; ++w) {
+      a_here += sh.red[w] >> 32;
+      c_here += sh.red[w] & 0xFFFFFFFFull;
     }
-    a_before += chunk_ac & 0xFFFFu;
-    c_before += chunk_ac >> 16;
+    for (unsigned int j0 = w_lo; j0 < w_hi; j0 += 32) {
+      const unsigned int j = j0 + lane;
+      uint32_t bits = 0, key = 0;
+      if (j < w_hi) {
+        bits = entry_val(j);
+        key = bits & 0x7FFFFFFFu;
+      }
+      const bool a = j < w_hi && key > T;
+      const bool c = j < w_hi && key == T;
+      const unsigned int ba = __ballot_sync(0xFFFFFFFFu, a), bc = __ballot_sync(0xFFFFFFFFu, c);
+      const unsigned long long a_mine = a_here + __popc(ba & lt), c_mine = c_here + __popc(bc & lt);
+      if (a || (c && c_mine < r)) {
+        const unsigned long long pos = a_mine + min(c_mine, r);
+        out_idx[pos] = entry_idx(j);
+        p.raw_val[pos] = __uint_as_float(bits);
+      }
+      a_here += __popc(ba);
+      c_here += __popc(bc);
+    }
   }
   if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
 
