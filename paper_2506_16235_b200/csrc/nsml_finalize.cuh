@@ -36,13 +36,13 @@
 
 namespace nsml {
 
-// Two shapes of the kernel.  The small one (256 threads, 4096 cached candidates,
-// ~53 KB of shared memory, 16K registers) lets several list stages, and the
+// Two shapes of the kernel.  The small one (256 threads, 8192 cached candidate
+// values, ~53 KB of shared memory, 16K registers) lets several list stages, and the
 // next bucket's streaming pass, share an SM when buckets are compressed on
 // several streams; the large one is for long candidate lists.
-constexpr int kFinSmallThreads = 256, kFinSmallCache = 4096;
-constexpr int kFinLargeThreads = 1024, kFinLargeCache = 20480;
-constexpr size_t finalize_dyn_smem(int cache_entries) { return (size_t)cache_entries * 8; }
+constexpr int kFinSmallThreads = 256, kFinSmallCache = 8192;
+constexpr int kFinLargeThreads = 1024, kFinLargeCache = 40960;
+constexpr size_t finalize_dyn_smem(int cache_entries) { return (size_t)cache_entries * 4; }  // values only
 
 struct FinalizeParams {
   unsigned long long n, k;
@@ -162,9 +162,8 @@ template <int DTYPE, int THREADS, int CACHE>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS)  // at most 64 registers per thread
 k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   __shared__ FinalizeShared<THREADS> sh;
-  extern __shared__ __align__(16) uint32_t s_cache[];  // values [CACHE], then indices [CACHE]
+  extern __shared__ __align__(16) uint32_t s_cache[];  // the first CACHE candidate values of this block
   uint32_t* cache_val = s_cache;
-  uint32_t* cache_idx = s_cache + CACHE;
   const int lane = threadIdx.x & 31;
   const unsigned int G = gridDim.x, blk = blockIdx.x;
   // Index-range ownership (used by the slow path only) and the block's array.
@@ -176,14 +175,24 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   unsigned int E = 0;  // candidates this block owns
 
   auto entry_val = [&](unsigned int j) -> uint32_t { return j < (unsigned)CACHE ? cache_val[j] : __ldcg(my_val + j); };
-  auto entry_idx = [&](unsigned int j) -> uint32_t { return j < (unsigned)CACHE ? cache_idx[j] : __ldcg(my_idx + j); };
-  auto put_entry = [&](unsigned int j, uint32_t idx, uint32_t val) {  // shared memory first, global memory for the overflow
-    if (j < (unsigned)CACHE) {
-      cache_idx[j] = idx;
-      cache_val[j] = val;
-    } else {
-      my_idx[j] = idx;
-      my_val[j] = val;
+  auto put_entry = [&](unsigned int j, uint32_t idx, uint32_t val) {
+    my_idx[j] = idx;  // indices are needed once, at the end: they stay in global memory
+    if (j < (unsigned)CACHE) cache_val[j] = val; else my_val[j] = val;
+  };
+
+  // Calls f(key) for each of the block's candidates, four loads in flight per thread (the values beyond the
+  // shared-memory cache come from global memory, where one load at a time would cost a round trip each).
+  auto for_each_key = [&](auto f) {
+    for (unsigned int j0 = threadIdx.x; j0 < E; j0 += THREADS * 4) {
+      uint32_t v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const unsigned int j = j0 + u * THREADS;
+        v[u] = (j < E) ? entry_val(j) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (j0 + u * THREADS < E) f(v[u] & 0x7FFFFFFFu);
     }
   };
 
@@ -411,10 +420,9 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   unsigned int rem = sh.out[1];
   for (int b = threadIdx.x; b < kMaxBins; b += THREADS) sh.hist[b] = 0;
   __syncthreads();
-  for (unsigned int j = threadIdx.x; j < E; j += THREADS) {
-    const uint32_t key = entry_val(j) & 0x7FFFFFFFu;
+  for_each_key([&](uint32_t key) {
     if ((key >> 19) == d0) atomicAdd(&sh.hist[(key >> 7) & 0xFFFu], 1u);
-  }
+  });
   flush_hist<kMaxBins, THREADS>(sh, p.hist + 1 * kMaxBins);
   if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
 
@@ -425,10 +433,9 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   __syncthreads();
   for (int b = threadIdx.x; b < 128; b += THREADS) sh.hist[b] = 0;
   __syncthreads();
-  for (unsigned int j = threadIdx.x; j < E; j += THREADS) {
-    const uint32_t key = entry_val(j) & 0x7FFFFFFFu;
+  for_each_key([&](uint32_t key) {
     if ((key >> 7) == prefix24) atomicAdd(&sh.hist[key & 0x7Fu], 1u);
-  }
+  });
   flush_hist<128, THREADS>(sh, p.hist + 2 * kMaxBins);
   if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
 
@@ -437,11 +444,10 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   const uint32_t T = (prefix24 << 7) | sh.out[0];
   const unsigned long long r = sh.out[1];  // ties (key == T) to keep, lowest index first
   unsigned long long mine_a = 0, mine_c = 0;
-  for (unsigned int j = threadIdx.x; j < E; j += THREADS) {
-    const uint32_t key = entry_val(j) & 0x7FFFFFFFu;
+  for_each_key([&](uint32_t key) {
     mine_a += key > T;
     mine_c += key == T;
-  }
+  });
   const unsigned long long block_a = block_sum(mine_a, sh);
   const unsigned long long block_c = block_sum(mine_c, sh);
   unsigned long long* ac_counts = p.block_counts + 1 * kMaxFinalizeBlocks;
@@ -477,11 +483,19 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
     const unsigned int per_warp = ((E + NW - 1) / NW + 31) / 32 * 32;
     const unsigned int w_lo = min(E, warp * per_warp), w_hi = min(E, w_lo + per_warp);
     unsigned int wa = 0, wc = 0;
-    for (unsigned int j0 = w_lo; j0 < w_hi; j0 += 32) {
-      const unsigned int j = j0 + lane;
-      const uint32_t key = (j < w_hi) ? (entry_val(j) & 0x7FFFFFFFu) : 0u;
-      wa += __popc(__ballot_sync(0xFFFFFFFFu, j < w_hi && key > T));
-      wc += __popc(__ballot_sync(0xFFFFFFFFu, j < w_hi && key == T));
+    for (unsigned int j0 = w_lo; j0 < w_hi; j0 += 128) {  // four rounds of 32, their loads issued together
+      uint32_t key[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const unsigned int j = j0 + u * 32 + lane;
+        key[u] = (j < w_hi) ? (entry_val(j) & 0x7FFFFFFFu) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const bool live = j0 + u * 32 + lane < w_hi;
+        wa += __popc(__ballot_sync(0xFFFFFFFFu, live && key[u] > T));
+        wc += __popc(__ballot_sync(0xFFFFFFFFu, live && key[u] == T));
+      }
     }
     __syncthreads();  // sh.red may still be read by the block sums above
     if (lane == 0) sh.red[warp] = ((unsigned long long)wa << 32) | wc;
@@ -491,24 +505,30 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
       a_here += sh.red[w] >> 32;
       c_here += sh.red[w] & 0xFFFFFFFFull;
     }
-    for (unsigned int j0 = w_lo; j0 < w_hi; j0 += 32) {
-      const unsigned int j = j0 + lane;
-      uint32_t bits = 0, key = 0;
-      if (j < w_hi) {
-        bits = entry_val(j);
-        key = bits & 0x7FFFFFFFu;
+    for (unsigned int j0 = w_lo; j0 < w_hi; j0 += 128) {
+      uint32_t bits[4], idx[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const unsigned int j = j0 + u * 32 + lane;
+        bits[u] = (j < w_hi) ? entry_val(j) : 0u;
+        idx[u] = (j < w_hi) ? my_idx[j] : 0u;  // coalesced; read whether or not the entry survives
       }
-      const bool a = j < w_hi && key > T;
-      const bool c = j < w_hi && key == T;
-      const unsigned int ba = __ballot_sync(0xFFFFFFFFu, a), bc = __ballot_sync(0xFFFFFFFFu, c);
-      const unsigned long long a_mine = a_here + __popc(ba & lt), c_mine = c_here + __popc(bc & lt);
-      if (a || (c && c_mine < r)) {
-        const unsigned long long pos = a_mine + min(c_mine, r);
-        out_idx[pos] = entry_idx(j);
-        p.raw_val[pos] = __uint_as_float(bits);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const bool live = j0 + u * 32 + lane < w_hi;
+        const uint32_t key = bits[u] & 0x7FFFFFFFu;
+        const bool a = live && key > T;
+        const bool c = live && key == T;
+        const unsigned int ba = __ballot_sync(0xFFFFFFFFu, a), bc = __ballot_sync(0xFFFFFFFFu, c);
+        const unsigned long long a_mine = a_here + __popc(ba & lt), c_mine = c_here + __popc(bc & lt);
+        if (a || (c && c_mine < r)) {
+          const unsigned long long pos = a_mine + min(c_mine, r);
+          out_idx[pos] = idx[u];
+          p.raw_val[pos] = __uint_as_float(bits[u]);
+        }
+        a_here += __popc(ba);
+        c_here += __popc(bc);
       }
-      a_here += __popc(ba);
-      c_here += __popc(bc);
     }
   }
   if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
