@@ -38,6 +38,12 @@ METRIC = "compress+decompress input-gradient GB/s per bucket; % of B200 HBM roof
 UNIT = "GB/s"
 SWEEP = [(r, b) for r in (0.5, 0.1, 0.01, 0.001) for b in (8, 16)]
 
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
+# profiles/compress_kernels_gpt2_25M_ncu_full.md: 25M-element fp32 buckets, ratio 0.01, int8, W = 4.  Only valid
+# for that workload and for the kernels as they were when the capture was taken.
+NCU_TRAFFIC_25M = {"k_sample": 1.06e6, "k_compact_bucket": 103.9e6, "k_finalize": 4.6e6, "k_partition": 3.9e6,
+                   "k_merge": 46.9e6}
+
 
 def measured_peak_gbs():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -604,7 +610,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="nsml", choices=["nsml", "reference"])
-    ap.add_argument("--streams", type=int, default=4, help="CUDA streams that independent buckets alternate between")
+    ap.add_argument("--streams", type=int, default=8, help="CUDA streams that independent buckets alternate between")
     ap.add_argument("--no-graphs", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-large-bucket-leg", action="store_true")
@@ -701,7 +707,8 @@ def main():
         d = kernels[dominant]
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": d["algorithmic_GBps"], "peak": peak,
                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": d["algorithmic_GBps"] / peak,
-                    "frac_of_nominal_8TBps": d["algorithmic_GBps"] / 8000.0, "traffic": None,
+                    "frac_of_nominal_8TBps": d["algorithmic_GBps"] / 8000.0,
+                    "traffic": NCU_TRAFFIC_25M.get(dominant) if args.workload == "gpt2" else None,
                     "us_per_launch": d["us_per_launch"]}
 
     # ---- end to end through the host-buffer entry points ----
@@ -769,7 +776,7 @@ def main():
             if cnt:
                 gbs = acc2.get(name, 0) / (ms * 1e-3) / 1e9
                 per[name] = {"us_per_launch": 1e3 * ms / cnt, "algorithmic_GBps": gbs, "frac_of_peak": gbs / peak,
-                             "frac_of_nominal_8TBps": gbs / 8000.0}
+                             "frac_of_nominal_8TBps": gbs / 8000.0, "traffic": NCU_TRAFFIC_25M.get(name)}
         out["bucket_25M"] = {"workload": "four 25M-element fp32 buckets, ratio 0.01, int8, W=4 workers each",
                              "value": big.input_bytes_per_step / (big_ms * 1e-3) / 1e9, "unit": UNIT,
                              "ms_per_step": big_ms, "kernels": per}
