@@ -169,6 +169,16 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
   const double p_keep = (double)k / (double)n;
   const double expected = (double)n * (p_keep + 6.0 * std::sqrt(p_keep * (1.0 - p_keep) / kSamples)) + 64.0;
   const bool small_shape = expected / fgrid <= (double)kFinSmallCache;
+  if (small_shape) {  // short lists: no more blocks than about 4096 candidates each (cheaper barriers, one block = none)
+    unsigned int want = (unsigned int)(expected / 4096.0) + 1;
+    if (want < fgrid) fgrid = want;
+  }
+  if (!small_shape) {  // long lists: as many blocks as stay co-resident (two per SM)
+    unsigned int cap = (unsigned int)(dev.sms * (dev.finalize_large < 2 ? dev.finalize_large : 2));
+    if ((unsigned long long)cap > nseg) cap = (unsigned int)nseg;
+    if (cap > (unsigned int)kMaxFinalizeBlocks) cap = kMaxFinalizeBlocks;
+    if (cap > fgrid) fgrid = cap;
+  }
   FinalizeParams fp;
   fp.n = (unsigned long long)n;
   fp.k = (unsigned long long)k;

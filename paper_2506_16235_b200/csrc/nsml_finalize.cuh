@@ -41,7 +41,7 @@ namespace nsml {
 // next bucket's streaming pass, share an SM when buckets are compressed on
 // several streams; the large one is for long candidate lists.
 constexpr int kFinSmallThreads = 256, kFinSmallCache = 8192;
-constexpr int kFinLargeThreads = 1024, kFinLargeCache = 40960;
+constexpr int kFinLargeThreads = 512, kFinLargeCache = 20480;
 constexpr size_t finalize_dyn_smem(int cache_entries) { return (size_t)cache_entries * 4; }  // values only
 
 struct FinalizeParams {
