@@ -169,9 +169,15 @@ class Workload:
         self.replayed_launches = 0
         self.home_stream = self.torch.cuda.current_stream()
 
-    def compress_bytes(self, acc, n, esize, k, bits):
+    def compress_bytes(self, acc, n, esize, ratio, bits):
+        k = self.nsml.nsml_k_of(n, ratio)
         vb = 1 if bits == 8 else 2
         s = 4 * ((k + 1023) // 1024) if bits == 8 else 0
+        if self.nsml.nsml_compress_strategy(n, ratio) == 1:
+            # dense strategy: the select reads the bucket itself once, survivors written and re-read
+            self.account(acc, "k_clear", 256 + 4 * 4 * 4096)
+            self.account(acc, "k_finalize_dense", esize * n + 8 * k + 4 * k + vb * k + s)
+            return
         self.account(acc, "k_sample", 4 * 8192)
         self.account(acc, "k_compact_bucket", esize * n + 8 * k)
         # list stage: candidates read once per phase (5 x 4k keys + 4k indices), survivors written and re-read
@@ -270,7 +276,7 @@ class ResnetWorkload(Workload):
                     nsml.nsml_decompress_accumulate([p], lane.dense[:n], zero_first=True, workspace=lane.aws, stream=lane.stream)
                     if acc is not None:
                         k = nsml.nsml_k_of(n, ratio)
-                        self.compress_bytes(acc, n, 4, k, bits)
+                        self.compress_bytes(acc, n, 4, ratio, bits)
                         self.merge_bytes(acc, n, [(k, bits)])
 
                 yield (r, b, ratio, bits), nsml.nsml_payload_bytes(n, ratio, bits), enqueue
@@ -301,17 +307,19 @@ class ResnetWorkload(Workload):
         return h2d, d2h
 
     def oracle_sample(self):
-        """One bucket through the whole sweep on the CPU oracle."""
+        """One gradient set (its four buckets) through the whole sweep on the CPU oracle."""
         import oracle
 
-        g = self.replicas[0][0].cpu().numpy()
-        n = g.size
+        grads = [g.cpu().numpy() for g in self.replicas[0]]
         t0 = time.perf_counter()
+        nbytes = 0.0
         for ratio, bits in SWEEP:
-            p = oracle.compress(g, ratio, bits)
-            oracle.decompress_sum([p], n)
+            for g in grads:
+                p = oracle.compress(g, ratio, bits)
+                oracle.decompress_sum([p], g.size)
+                nbytes += 4.0 * g.size
         dt = time.perf_counter() - t0
-        return len(SWEEP) * 4.0 * n, dt, f"bucket 0 ({n} elements) through the 8-point ratio x codec sweep"
+        return nbytes, dt, f"one gradient set ({len(grads)} buckets, {sum(g.size for g in grads)} elements) through the 8-point ratio x codec sweep"
 
 
 class Gpt2Workload(Workload):
@@ -376,7 +384,7 @@ class Gpt2Workload(Workload):
                 if acc is not None:
                     k = nsml.nsml_k_of(n, self.RATIO)
                     for w in range(self.W):
-                        self.compress_bytes(acc, n, 4, k, self.BITS)
+                        self.compress_bytes(acc, n, 4, self.RATIO, self.BITS)
                     self.merge_bytes(acc, n, [(k, self.BITS)] * self.W)
 
             yield (b,), self.W * nsml.nsml_payload_bytes(n, self.RATIO, self.BITS), enqueue
@@ -470,7 +478,7 @@ class DecoderWorkload(Workload):
                 nsml.nsml_decompress_accumulate([p], lane.dense[:n], zero_first=True, workspace=lane.aws, stream=lane.stream)
                 if acc is not None:
                     k = nsml.nsml_k_of(n, ratio)
-                    self.compress_bytes(acc, n, 2, k, 16)
+                    self.compress_bytes(acc, n, 2, ratio, 16)
                     self.merge_bytes(acc, n, [(k, 16)])
 
             yield (b, ratio), nsml.nsml_payload_bytes(n, ratio, 16), enqueue

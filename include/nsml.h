@@ -202,6 +202,19 @@ int nsml_compress(const void* grad, int64_t n, int grad_dtype, double ratio, int
                   const uint32_t* prune_mask, void* payload, size_t payload_capacity,
                   void* workspace, size_t workspace_bytes, void* stream);
 
+/* Which of its two internal strategies nsml_compress takes for (n, ratio) on
+ * the current device.  Both give the same payload; this is information for
+ * byte accounting (the paper prescribes no strategy).
+ *   NSML_STRATEGY_LIST   a stratified sample bounds the threshold from below,
+ *                        one streaming pass keeps the candidates above the
+ *                        bound, an exact radix select runs on that list
+ *   NSML_STRATEGY_DENSE  the radix select runs over the bucket itself (high
+ *                        kept fractions, and buckets too small to sample)
+ * Returns the strategy, or NSML_ERR_ARG / NSML_ERR_CUDA. */
+#define NSML_STRATEGY_LIST 0
+#define NSML_STRATEGY_DENSE 1
+int nsml_compress_strategy(int64_t n, double ratio);
+
 /* ------------------------------------------------------------------------
  * nsml_decompress_accumulate -- dense += sum over W payloads (plain sum, no
  * averaging), after optionally zeroing dense.

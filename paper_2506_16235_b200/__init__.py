@@ -90,6 +90,7 @@ def _load() -> ctypes.CDLL:
         "nsml_ctrl_save": (ci, [vp, vp, sz]),
         "nsml_ctrl_load": (ci, [vp, vp, sz]),
         "nsml_k_of": (i64, [i64, dbl]),
+        "nsml_compress_strategy": (ci, [i64, dbl]),
         "nsml_payload_bytes": (sz, [i64, dbl, ci]),
         "nsml_workspace_bytes": (sz, [i64, ci]),
         "nsml_accumulate_workspace_bytes": (sz, [i64, ci]),
@@ -185,6 +186,14 @@ def nsml_select_ratio(ctrl: Controller, last_bytes: float, last_seconds: float, 
 # --------------------------------------------------------------------------
 def nsml_k_of(n: int, ratio: float) -> int:
     return int(lib.nsml_k_of(int(n), float(ratio)))
+
+
+def nsml_compress_strategy(n: int, ratio: float) -> int:
+    """0 = sampled candidate list, 1 = dense select over the bucket (current device)."""
+    rc = int(lib.nsml_compress_strategy(int(n), float(ratio)))
+    if rc < 0:
+        raise NsmlError(rc, "nsml_compress_strategy")
+    return rc
 
 
 def nsml_payload_bytes(n: int, ratio: float, bits: int) -> int:

@@ -11,13 +11,15 @@
 #include "nsml_common.cuh"
 #include "nsml_compact.cuh"
 #include "nsml_finalize.cuh"
+#include "nsml_dense.cuh"
 #include "nsml_select.cuh"
 
 namespace nsml {
 
-enum KernelId { K_SAMPLE = 0, K_COMPACT_BUCKET, K_FINALIZE, K_PARTITION, K_MERGE, K_COUNT };
+enum KernelId { K_SAMPLE = 0, K_COMPACT_BUCKET, K_FINALIZE, K_PARTITION, K_MERGE, K_CLEAR, K_FINALIZE_DENSE, K_COUNT };
 
-static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_compact_bucket", "k_finalize", "k_partition", "k_merge"};
+static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_compact_bucket", "k_finalize", "k_partition", "k_merge",
+                                                  "k_clear", "k_finalize_dense"};
 
 static std::atomic<int64_t> g_launches{0};
 
@@ -92,8 +94,12 @@ static int device_info(const DeviceInfo** out) {
     };
     prepare(k_finalize<NSML_F32, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
     prepare(k_finalize<NSML_BF16, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
+    prepare(k_finalize_dense<NSML_F32, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
+    prepare(k_finalize_dense<NSML_BF16, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
     prepare(k_finalize<NSML_F32, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache, &d.finalize_large);
     prepare(k_finalize<NSML_BF16, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache, &d.finalize_large);
+    prepare(k_finalize_dense<NSML_F32, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache, &d.finalize_large);
+    prepare(k_finalize_dense<NSML_BF16, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache, &d.finalize_large);
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.merge, k_merge, kCta, 0);
     int coop = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
@@ -137,6 +143,25 @@ static unsigned int sample_rank(int64_t n, int64_t k) {
   return (unsigned int)j;
 }
 
+// Kept fractions from which the dense mode of the finalize kernel is used: for any bucket, and for a bucket
+// that fits the shared-memory caches of one co-resident grid.
+constexpr double kDenseRatioAny = 0.25;
+constexpr double kDenseRatioOnChip = 0.25;
+
+static unsigned long long finalize_large_blocks(const DeviceInfo& dev) {
+  return (unsigned long long)dev.sms * (dev.finalize_large < 2 ? dev.finalize_large : 2);
+}
+
+// Dense mode: the finalize kernel selects over the bucket itself, with no sample and no bucket pass.
+// Taken when the bucket cannot be sampled, when the candidate list (8 bytes per entry) would be about
+// as large as the bucket, and for moderate kept fractions when the whole bucket fits the shared-memory
+// caches of one co-resident grid (it is then read from memory once).
+static bool use_dense(int64_t n, int64_t k, const DeviceInfo& dev) {
+  const double p_keep = (double)k / (double)n;
+  const bool fits_on_chip = (unsigned long long)n <= finalize_large_blocks(dev) * (unsigned long long)kFinDenseLargeCache;
+  return sample_rank(n, k) == 0 || p_keep >= kDenseRatioAny || (fits_on_chip && p_keep >= kDenseRatioOnChip);
+}
+
 template <int DTYPE>
 static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, int64_t k, int bits, unsigned char* ws,
                            unsigned char* payload, const CompressLayout& L, const PayloadLayout& P,
@@ -147,37 +172,51 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
   unsigned short* seg_count = reinterpret_cast<unsigned short*>(ws + L.seg_count);
   const unsigned long long nseg = ((unsigned long long)n + kSegElems - 1) / kSegElems;
   BucketSrc<DTYPE> src{grad, mask};
-  {
-    LaunchScope scope(K_SAMPLE, st);  // one cluster of kSampleBlocks blocks
-    k_sample<DTYPE><<<kSampleBlocks, kSampleThreads, 0, st>>>(src, (unsigned long long)n, sample_rank(n, k), ctl,
-                                                              reinterpret_cast<uint4*>(ws),
-                                                              (unsigned int)(L.zero_bytes / 16));
-  }
-  {
-    // bucket pass: a block takes 8 segments per step; at most 4 resident blocks per SM
-    LaunchScope scope(K_COMPACT_BUCKET, st);
-    const int per_sm = dev.compact_bucket < 4 ? dev.compact_bucket : 4;
-    const unsigned int grid = grid_for(nseg, kCta / 32, dev.sms * per_sm);
-    k_compact_bucket<DTYPE><<<grid, kCta, 0, st>>>(src, (unsigned long long)n, ctl, seg_idx, seg_val, seg_count,
-                                                   reinterpret_cast<unsigned int*>(ws + L.group_count));
-  }
-  // list stage: cooperative, one block per SM, every block co-resident.  The small shape when a block's
-  // share of the expected candidates (k plus the sampling margin) fits its shared-memory cache.
-  unsigned int fgrid = (unsigned int)dev.sms;
-  if ((unsigned long long)fgrid > nseg) fgrid = (unsigned int)nseg;
-  if (fgrid > (unsigned int)kMaxFinalizeBlocks) fgrid = kMaxFinalizeBlocks;
   const double p_keep = (double)k / (double)n;
-  const double expected = (double)n * (p_keep + 6.0 * std::sqrt(p_keep * (1.0 - p_keep) / kSamples)) + 64.0;
-  const bool small_shape = expected / fgrid <= (double)kFinSmallCache;
-  if (small_shape) {  // short lists: no more blocks than about 4096 candidates each (cheaper barriers, one block = none)
-    unsigned int want = (unsigned int)(expected / 4096.0) + 1;
-    if (want < fgrid) fgrid = want;
-  }
-  if (!small_shape) {  // long lists: as many blocks as stay co-resident (two per SM)
-    unsigned int cap = (unsigned int)(dev.sms * (dev.finalize_large < 2 ? dev.finalize_large : 2));
-    if ((unsigned long long)cap > nseg) cap = (unsigned int)nseg;
-    if (cap > (unsigned int)kMaxFinalizeBlocks) cap = kMaxFinalizeBlocks;
-    if (cap > fgrid) fgrid = cap;
+  const unsigned long long large_cap_blocks = finalize_large_blocks(dev);
+  const bool dense = use_dense(n, k, dev);
+  unsigned int fgrid;
+  bool small_shape;
+  if (dense) {
+    small_shape = (unsigned long long)n <= (unsigned long long)dev.sms * kFinSmallCache;
+    unsigned long long cap = small_shape ? (unsigned long long)dev.sms : large_cap_blocks;
+    if (cap > (unsigned long long)kMaxFinalizeBlocks) cap = kMaxFinalizeBlocks;
+    unsigned long long want = (unsigned long long)n / 4096 + 1;  // at least about 4096 elements per block
+    if (want > nseg) want = nseg;
+    fgrid = (unsigned int)(want < cap ? want : cap);
+    LaunchScope scope(K_CLEAR, st);
+    k_clear<<<4, kCta, 0, st>>>(reinterpret_cast<uint4*>(ws), (unsigned int)(L.group_count / 16));
+  } else {
+    {
+      LaunchScope scope(K_SAMPLE, st);  // one cluster of kSampleBlocks blocks
+      k_sample<DTYPE><<<kSampleBlocks, kSampleThreads, 0, st>>>(src, (unsigned long long)n, sample_rank(n, k), ctl,
+                                                                reinterpret_cast<uint4*>(ws),
+                                                                (unsigned int)(L.zero_bytes / 16));
+    }
+    {
+      // bucket pass: a block takes 8 segments per step; at most 4 resident blocks per SM
+      LaunchScope scope(K_COMPACT_BUCKET, st);
+      const int per_sm = dev.compact_bucket < 4 ? dev.compact_bucket : 4;
+      const unsigned int grid = grid_for(nseg, kCta / 32, dev.sms * per_sm);
+      k_compact_bucket<DTYPE><<<grid, kCta, 0, st>>>(src, (unsigned long long)n, ctl, seg_idx, seg_val, seg_count,
+                                                     reinterpret_cast<unsigned int*>(ws + L.group_count));
+    }
+    // list stage: cooperative, every block co-resident.  The small shape when a block's share of the
+    // expected candidates (k plus the sampling margin) fits its shared-memory cache.
+    fgrid = (unsigned int)dev.sms;
+    if ((unsigned long long)fgrid > nseg) fgrid = (unsigned int)nseg;
+    if (fgrid > (unsigned int)kMaxFinalizeBlocks) fgrid = kMaxFinalizeBlocks;
+    const double expected = (double)n * (p_keep + 6.0 * std::sqrt(p_keep * (1.0 - p_keep) / kSamples)) + 64.0;
+    small_shape = expected / fgrid <= (double)kFinSmallCache;
+    if (small_shape) {  // short lists: no more blocks than about 4096 candidates each (cheaper barriers, one block = none)
+      unsigned int want = (unsigned int)(expected / 4096.0) + 1;
+      if (want < fgrid) fgrid = want;
+    } else {  // long lists: as many blocks as stay co-resident (two per SM)
+      unsigned long long cap = large_cap_blocks;
+      if (cap > nseg) cap = nseg;
+      if (cap > (unsigned long long)kMaxFinalizeBlocks) cap = kMaxFinalizeBlocks;
+      if (cap > fgrid) fgrid = (unsigned int)cap;
+    }
   }
   FinalizeParams fp;
   fp.n = (unsigned long long)n;
@@ -197,15 +236,17 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
   fp.payload = payload;
   fp.P = P;
   {
-    LaunchScope scope(K_FINALIZE, st);
+    LaunchScope scope(dense ? K_FINALIZE_DENSE : K_FINALIZE, st);
     void* args[] = {&src, &fp};
     cudaError_t le;
-    if (small_shape)
-      le = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_finalize<DTYPE, kFinSmallThreads, kFinSmallCache>), dim3(fgrid),
-                                       dim3(kFinSmallThreads), args, finalize_dyn_smem(kFinSmallCache), st);
-    else
-      le = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_finalize<DTYPE, kFinLargeThreads, kFinLargeCache>), dim3(fgrid),
-                                       dim3(kFinLargeThreads), args, finalize_dyn_smem(kFinLargeCache), st);
+    auto launch = [&](auto kernel, int threads, int cache) {
+      return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(fgrid), dim3(threads), args,
+                                         finalize_dyn_smem(cache), st);
+    };
+    if (small_shape && dense) le = launch(k_finalize_dense<DTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
+    else if (small_shape) le = launch(k_finalize<DTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
+    else if (dense) le = launch(k_finalize_dense<DTYPE, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache);
+    else le = launch(k_finalize<DTYPE, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache);
     if (le != cudaSuccess) return NSML_ERR_CUDA;
   }
   return NSML_OK;
@@ -310,6 +351,15 @@ using namespace nsml;
 extern "C" {
 
 int64_t nsml_k_of(int64_t n, double ratio) { return k_of(n, ratio); }
+
+int nsml_compress_strategy(int64_t n, double ratio) {
+  const int64_t k = k_of(n, ratio);
+  if (k == 0) return NSML_ERR_ARG;
+  const DeviceInfo* dev = nullptr;
+  const int rc = device_info(&dev);
+  if (rc != NSML_OK) return rc;
+  return use_dense(n, k, *dev) ? NSML_STRATEGY_DENSE : NSML_STRATEGY_LIST;
+}
 
 size_t nsml_payload_bytes(int64_t n, double ratio, int bits) {
   if (bits != NSML_BITS_INT8 && bits != NSML_BITS_FP16) return 0;

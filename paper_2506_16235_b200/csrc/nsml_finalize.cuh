@@ -25,6 +25,9 @@
 // an index range and rebuilds its array from the bucket: every non-zero key
 // plus the first k - nnz zeros in index order (one more barrier).
 //
+// Calls in which the list would be about as large as the bucket take k_finalize_dense
+// (nsml_dense.cuh) instead, which shares this file's helpers and the quantise phase.
+//
 // Every barrier wait is bounded: when it runs out the block records
 // NSML_ERR_TIMEOUT and leaves; the others then time out as well.
 #pragma once
@@ -42,6 +45,9 @@ namespace nsml {
 // several streams; the large one is for long candidate lists.
 constexpr int kFinSmallThreads = 256, kFinSmallCache = 8192;
 constexpr int kFinLargeThreads = 512, kFinLargeCache = 20480;
+// The dense kernel needs no gather scratch, which leaves room for a larger cache in the large shape: two
+// blocks per SM then hold 2 x 23040 values, 6.8M elements over 148 SMs (a 25 MB float32 bucket stays on chip).
+constexpr int kFinDenseLargeCache = 23040;
 constexpr size_t finalize_dyn_smem(int cache_entries) { return (size_t)cache_entries * 4; }  // values only
 
 struct FinalizeParams {
@@ -62,12 +68,23 @@ struct FinalizeParams {
   PayloadLayout P;
 };
 
+template <int THREADS, bool DENSE>
+struct GatherScratch {
+  unsigned int off[THREADS];  // exclusive offset of each thread's 8 segments within the chunk
+  uint4 cnt8[THREADS];        // the 8 segment counts of each thread (16 bits each)
+};
+constexpr int kUndCap = 192;  // undecided entries a warp of the dense kernel can list
 template <int THREADS>
+struct GatherScratch<THREADS, true> {  // the dense kernel gathers nothing; it lists undecided entries per warp
+  unsigned short und[THREADS / 32][kUndCap];
+};
+
+template <int THREADS, bool DENSE>
 struct FinalizeShared {
   unsigned int hist[kMaxBins];
-  unsigned int off[THREADS];  // gather: exclusive offset of each thread's 8 segments within the chunk
-  uint4 cnt8[THREADS];        // gather: the 8 segment counts of each thread (16 bits each)
+  GatherScratch<THREADS, DENSE> g;
   unsigned long long red[(THREADS / 32)];
+  unsigned long long run[2 * (THREADS / 32)];  // write phase: survivors per (warp, run)
   unsigned int scan[(THREADS / 32)];
   unsigned int tot[(THREADS / 32)];
   unsigned int out[2];
@@ -77,8 +94,8 @@ struct FinalizeShared {
 };
 
 // Sum over the block; every thread gets the result.
-template <int THREADS>
-__device__ __forceinline__ unsigned long long block_sum(unsigned long long v, FinalizeShared<THREADS>& sh) {
+template <int THREADS, bool D>
+__device__ __forceinline__ unsigned long long block_sum(unsigned long long v, FinalizeShared<THREADS, D>& sh) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
   __syncthreads();  // sh.red may still be read from an earlier call
@@ -91,8 +108,8 @@ __device__ __forceinline__ unsigned long long block_sum(unsigned long long v, Fi
 }
 
 // Exclusive prefix over the block in thread order; `total` = sum over the block.
-template <int THREADS>
-__device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned int& total, FinalizeShared<THREADS>& sh) {
+template <int THREADS, bool D>
+__device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned int& total, FinalizeShared<THREADS, D>& sh) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   unsigned int incl = v;
 #pragma unroll
@@ -115,8 +132,8 @@ __device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned
 }
 
 // All blocks arrive, then all leave.  `target` = barrier ordinal * gridDim.x.
-template <int THREADS>
-__device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, FinalizeShared<THREADS>& sh) {
+template <int THREADS, bool D>
+__device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, FinalizeShared<THREADS, D>& sh) {
   __syncthreads();
   if (threadIdx.x == 0) {
     __threadfence();
@@ -135,8 +152,8 @@ __device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, Fina
 }
 
 // Adds the block's shared histogram into the global one (non-empty bins only).
-template <int NB, int THREADS>
-__device__ __forceinline__ void flush_hist(FinalizeShared<THREADS>& sh, unsigned int* ghist) {
+template <int NB, int THREADS, bool D>
+__device__ __forceinline__ void flush_hist(FinalizeShared<THREADS, D>& sh, unsigned int* ghist) {
   __syncthreads();
   for (int b = threadIdx.x; b < NB; b += THREADS) {
     const unsigned int c = sh.hist[b];
@@ -146,8 +163,8 @@ __device__ __forceinline__ void flush_hist(FinalizeShared<THREADS>& sh, unsigned
 
 // Every block reads the global histogram of a level and finds the digit that
 // holds the rem-th largest key; digit and the rank left inside land in sh.out.
-template <int NB, int THREADS>
-__device__ __forceinline__ void resolve_digit(const unsigned int* ghist, unsigned int rem, FinalizeShared<THREADS>& sh) {
+template <int NB, int THREADS, bool D>
+__device__ __forceinline__ void resolve_digit(const unsigned int* ghist, unsigned int rem, FinalizeShared<THREADS, D>& sh) {
   constexpr int PER = (NB + THREADS - 1) / THREADS;
   unsigned int own[PER];
 #pragma unroll
@@ -158,382 +175,19 @@ __device__ __forceinline__ void resolve_digit(const unsigned int* ghist, unsigne
   find_digit_from_top<PER, THREADS>(own, rem, sh.tot, sh.out);
 }
 
-template <int DTYPE, int THREADS, int CACHE>
-__global__ void __launch_bounds__(THREADS, 1024 / THREADS)  // at most 64 registers per thread
-k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
-  __shared__ FinalizeShared<THREADS> sh;
-  extern __shared__ __align__(16) uint32_t s_cache[];  // the first CACHE candidate values of this block
-  uint32_t* cache_val = s_cache;
-  const int lane = threadIdx.x & 31;
+// Clears the control block and the histograms of a workspace (what the sample
+// kernel does on the list path) ahead of a dense-mode finalize.
+__global__ void __launch_bounds__(kCta) k_clear(uint4* __restrict__ region, unsigned int count16) {
+  for (unsigned int i = blockIdx.x * kCta + threadIdx.x; i < count16; i += gridDim.x * kCta)
+    region[i] = make_uint4(0u, 0u, 0u, 0u);
+}
+
+// Phase 5 of both finalize kernels: quantises the k survivors left in raw_val (int8 per block of 1024
+// with a max-abs scale, or fp16) into the payload and writes the payload header.
+template <int THREADS, bool D>
+__device__ __forceinline__ void quantize_phase(const FinalizeParams& p, FinalizeShared<THREADS, D>& sh) {
   const unsigned int G = gridDim.x, blk = blockIdx.x;
-  // Index-range ownership (used by the slow path only) and the block's array.
-  const unsigned long long seg_first = (unsigned long long)blk * p.nseg / G;
-  const unsigned long long seg_last = (unsigned long long)(blk + 1) * p.nseg / G;
-  uint32_t* my_idx = p.list_idx;  // set below
-  uint32_t* my_val = p.list_val;
-  unsigned int barriers = 0;
-  unsigned int E = 0;  // candidates this block owns
-
-  auto entry_val = [&](unsigned int j) -> uint32_t { return j < (unsigned)CACHE ? cache_val[j] : __ldcg(my_val + j); };
-  auto put_entry = [&](unsigned int j, uint32_t idx, uint32_t val) {
-    my_idx[j] = idx;  // indices are needed once, at the end: they stay in global memory
-    if (j < (unsigned)CACHE) cache_val[j] = val; else my_val[j] = val;
-  };
-
-  // Calls f(key) for each of the block's candidates, four loads in flight per thread (the values beyond the
-  // shared-memory cache come from global memory, where one load at a time would cost a round trip each).
-  auto for_each_key = [&](auto f) {
-    for (unsigned int j0 = threadIdx.x; j0 < E; j0 += THREADS * 4) {
-      uint32_t v[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const unsigned int j = j0 + u * THREADS;
-        v[u] = (j < E) ? entry_val(j) : 0u;
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u)
-        if (j0 + u * THREADS < E) f(v[u] & 0x7FFFFFFFu);
-    }
-  };
-
-  // ---------------- phase 0: take an equal share of the candidates, histogram of digit 0 ----------------
-  // Every block reads the per-group candidate counts the bucket pass left and
-  // scans them, which gives the list position of every group and the total.
-  const unsigned long long ngroups = (p.nseg + kGroupSegs - 1) / kGroupSegs;
-  const unsigned long long per_thread = (ngroups + THREADS - 1) / THREADS;
-  const unsigned long long g_begin = min(ngroups, threadIdx.x * per_thread);
-  const unsigned long long g_end = min(ngroups, g_begin + per_thread);
-  unsigned long long thread_sum = 0;
-  for (unsigned long long gi = g_begin; gi < g_end; ++gi) thread_sum += p.group_count[gi];
-  unsigned long long list_total;
-  unsigned long long thread_pos;  // list position where this thread's first group starts
-  {
-    // 64-bit exclusive scan over the block
-    const int warp = threadIdx.x >> 5;
-    unsigned long long incl = thread_sum;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-      if (lane >= o) incl += up;
-    }
-    if (lane == 31) sh.red[warp] = incl;
-    __syncthreads();
-    unsigned long long before = 0, all = 0;
-#pragma unroll
-    for (int w = 0; w < (THREADS / 32); ++w) {
-      const unsigned long long c = sh.red[w];
-      if (w < warp) before += c;
-      all += c;
-    }
-    list_total = all;
-    thread_pos = before + incl - thread_sum;
-  }
-  const unsigned long long share_lo = (unsigned long long)blk * list_total / G;
-  const unsigned long long share_hi = (unsigned long long)(blk + 1) * list_total / G;
-  for (int b = threadIdx.x; b < kMaxBins; b += THREADS) sh.hist[b] = 0;
-  bool nonfinite = false;
-  if (list_total >= p.k) {
-    my_idx = p.list_idx + share_lo;
-    my_val = p.list_val + share_lo;
-    E = (unsigned int)(share_hi - share_lo);
-    if (E > 0 && thread_pos <= share_lo && share_lo < thread_pos + thread_sum) {  // exactly one thread
-      unsigned long long pos = thread_pos, gi = g_begin;
-      for (; gi < g_end; ++gi) {
-        const unsigned long long c = p.group_count[gi];
-        if (share_lo < pos + c) break;
-        pos += c;
-      }
-      sh.start[0] = gi;
-      sh.start[1] = pos;
-    }
-    __syncthreads();
-    unsigned long long seg_cursor = (E > 0) ? sh.start[0] * kGroupSegs : p.nseg;
-    unsigned long long pos_cursor = (E > 0) ? sh.start[1] : 0;
-    // A chunk is 8 segments per thread.  Thin stretches of the bucket make a
-    // share span many chunks, so the next chunk's counts are fetched before
-    // the current chunk's entries are copied.
-    auto load_counts = [&](unsigned long long first_seg) -> uint4 {
-      const unsigned long long s = first_seg + threadIdx.x * 8ull;  // a multiple of 8: the 16-byte load is aligned
-      if (s + 8 <= p.nseg) return *reinterpret_cast<const uint4*>(p.seg_count + s);
-      unsigned short c[8];
-#pragma unroll
-      for (int e = 0; e < 8; ++e) c[e] = (s + e < p.nseg) ? p.seg_count[s + e] : (unsigned short)0;
-      uint4 v;
-      v.x = c[0] | ((uint32_t)c[1] << 16); v.y = c[2] | ((uint32_t)c[3] << 16);
-      v.z = c[4] | ((uint32_t)c[5] << 16); v.w = c[6] | ((uint32_t)c[7] << 16);
-      return v;
-    };
-    uint4 counts = load_counts(seg_cursor);
-    while (pos_cursor < share_hi && seg_cursor < p.nseg) {
-      const uint4 next_counts = load_counts(seg_cursor + (THREADS * 8));
-      const unsigned int cnt = (counts.x & 0xFFFFu) + (counts.x >> 16) + (counts.y & 0xFFFFu) + (counts.y >> 16) +
-                               (counts.z & 0xFFFFu) + (counts.z >> 16) + (counts.w & 0xFFFFu) + (counts.w >> 16);
-      unsigned int chunk_total;
-      const unsigned int off = block_excl_scan(cnt, chunk_total, sh);
-      __syncthreads();  // sh.off / sh.cnt8 of the previous chunk have been read
-      sh.off[threadIdx.x] = off;
-      sh.cnt8[threadIdx.x] = counts;
-      __syncthreads();
-      // entries of this chunk that fall in the block's share
-      const unsigned long long from_pos = max(pos_cursor, share_lo), to_pos = min(pos_cursor + chunk_total, share_hi);
-      const unsigned short* cnt16 = reinterpret_cast<const unsigned short*>(sh.cnt8);  // count of segment q of the chunk
-      for (unsigned long long g0 = from_pos + threadIdx.x * 4ull; g0 < to_pos; g0 += THREADS * 4ull) {
-        // four consecutive entries per thread, each located by a search over the thread slots
-        unsigned long long from[4];
-        const int cnt = (int)min(4ull, to_pos - g0);
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (e < cnt) {
-            const unsigned int j = (unsigned int)(g0 + e - pos_cursor);
-            int lo = 0, hi = THREADS - 1;  // last thread slot of the chunk whose offset is <= j
-            while (lo < hi) {
-              const int mid = (lo + hi + 1) >> 1;
-              if (sh.off[mid] <= j) lo = mid; else hi = mid - 1;
-            }
-            unsigned int within = j - sh.off[lo];
-            unsigned int q = lo * 8;  // at most 8 steps: the entry lies in this slot's segments
-            while (within >= cnt16[q]) { within -= cnt16[q]; ++q; }
-            from[e] = (seg_cursor + q) * kSegElems + within;
-          }
-        }
-        uint32_t vals[4], idxs[4];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (e < cnt) {
-            vals[e] = p.seg_val[from[e]];
-            idxs[e] = p.seg_idx[from[e]];
-          }
-        }
-#pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (e < cnt) {
-            const uint32_t key = vals[e] & 0x7FFFFFFFu;
-            put_entry((unsigned int)(g0 + e - share_lo), idxs[e], vals[e]);
-            nonfinite |= key >= kInfKey;
-            atomicAdd(&sh.hist[key >> digit_shift(0)], 1u);
-          }
-        }
-      }
-      pos_cursor += chunk_total;
-      seg_cursor += (THREADS * 8);
-      counts = next_counts;
-    }
-    if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
-    flush_hist<kMaxBins, THREADS>(sh, p.hist);
-    if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
-  }
-  const unsigned int* ghist0 = p.hist;
-
-  if (list_total < p.k) {
-    // ---- slow path: this block's array becomes (all non-zero keys) + (zeros within budget) ----
-    const unsigned long long r_lo = seg_first * (unsigned long long)kSegElems;
-    const unsigned long long r_hi = min(seg_last * (unsigned long long)kSegElems, p.n);
-    my_idx = p.list_idx + r_lo;  // a block's range has room for all of its elements
-    my_val = p.list_val + r_lo;
-    unsigned long long nnz = 0, zeros = 0;
-    for (unsigned long long i0 = r_lo + threadIdx.x * 4ull; i0 < r_hi; i0 += THREADS * 4ull) {
-      uint32_t bits[4];
-      const int cnt = src.load_vals4(i0, p.n, bits);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (e < cnt) {
-          if ((bits[e] & 0x7FFFFFFFu) != 0) ++nnz; else ++zeros;
-        }
-      }
-    }
-    const unsigned long long block_nnz = block_sum(nnz, sh);
-    const unsigned long long block_zeros = block_sum(zeros, sh);
-    unsigned long long* nz_counts = p.block_counts + 2 * kMaxFinalizeBlocks;
-    if (threadIdx.x == 0) nz_counts[blk] = (block_nnz << 32) | block_zeros;
-    if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
-
-    unsigned long long all_nnz = 0, zeros_before = 0;
-    for (unsigned int b = threadIdx.x; b < G; b += THREADS) {
-      const unsigned long long w = __ldcg(nz_counts + b);
-      all_nnz += w >> 32;
-      if (b < blk) zeros_before += w & 0xFFFFFFFFull;
-    }
-    all_nnz = block_sum(all_nnz, sh);
-    zeros_before = block_sum(zeros_before, sh);
-    const unsigned long long zero_budget = (p.k > all_nnz) ? p.k - all_nnz : 0;
-    // zeros of this block to keep, lowest index first
-    const unsigned long long allowed = (zero_budget > zeros_before) ? min(block_zeros, zero_budget - zeros_before) : 0ull;
-
-    __syncthreads();
-    for (int b = threadIdx.x; b < kMaxBins; b += THREADS) sh.hist[b] = 0;
-    E = 0;
-    unsigned long long zeros_seen = 0;
-    nonfinite = false;
-    for (unsigned long long base = r_lo; base < r_hi; base += THREADS * 4ull) {
-      const unsigned long long i0 = base + threadIdx.x * 4ull;
-      uint32_t bits[4] = {0, 0, 0, 0};
-      const int cnt = (i0 < r_hi) ? src.load_vals4(i0, p.n, bits) : 0;
-      unsigned int fz = 0, fn = 0;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (e < cnt) {
-          if ((bits[e] & 0x7FFFFFFFu) != 0) fn |= 1u << e; else fz |= 1u << e;
-        }
-      }
-      unsigned int z_total, keep_total;
-      unsigned long long zrank = zeros_seen + block_excl_scan(__popc(fz), z_total, sh);
-      unsigned int f = fn;
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (fz & (1u << e)) {
-          if (zrank < allowed) f |= 1u << e;
-          ++zrank;
-        }
-      }
-      unsigned int pos = E + block_excl_scan(__popc(f), keep_total, sh);
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (f & (1u << e)) {
-          const uint32_t key = bits[e] & 0x7FFFFFFFu;
-          put_entry(pos, (uint32_t)(i0 + e), bits[e]);
-          nonfinite |= key >= kInfKey;
-          atomicAdd(&sh.hist[key >> digit_shift(0)], 1u);
-          ++pos;
-        }
-      }
-      zeros_seen += z_total;
-      E += keep_total;
-    }
-    if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
-    unsigned long long* totals2 = p.block_counts + 3 * kMaxFinalizeBlocks;
-    if (threadIdx.x == 0) totals2[blk] = E;
-    flush_hist<kMaxBins, THREADS>(sh, p.hist + 3 * kMaxBins);
-    if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
-    unsigned long long part = 0;
-    for (unsigned int b = threadIdx.x; b < G; b += THREADS) part += __ldcg(totals2 + b);
-    if (block_sum(part, sh) < p.k) {  // cannot happen: the rebuilt list holds at least k entries
-      if (threadIdx.x == 0) set_status(&p.ctl->status, NSML_ERR_INTERNAL);
-      return;
-    }
-    ghist0 = p.hist + 3 * kMaxBins;
-  }
-  __syncthreads();  // the block's array (shared copy and global) is complete
-
-  // ---------------- phase 1: resolve digit 0, histogram of digit 1 ----------------
-  resolve_digit<kMaxBins, THREADS>(ghist0, (unsigned int)p.k, sh);
-  const unsigned int d0 = sh.out[0];
-  unsigned int rem = sh.out[1];
-  for (int b = threadIdx.x; b < kMaxBins; b += THREADS) sh.hist[b] = 0;
-  __syncthreads();
-  for_each_key([&](uint32_t key) {
-    if ((key >> 19) == d0) atomicAdd(&sh.hist[(key >> 7) & 0xFFFu], 1u);
-  });
-  flush_hist<kMaxBins, THREADS>(sh, p.hist + 1 * kMaxBins);
-  if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
-
-  // ---------------- phase 2: resolve digit 1, histogram of digit 2 ----------------
-  resolve_digit<kMaxBins, THREADS>(p.hist + 1 * kMaxBins, rem, sh);
-  const unsigned int prefix24 = (d0 << 12) | sh.out[0];
-  rem = sh.out[1];
-  __syncthreads();
-  for (int b = threadIdx.x; b < 128; b += THREADS) sh.hist[b] = 0;
-  __syncthreads();
-  for_each_key([&](uint32_t key) {
-    if ((key >> 7) == prefix24) atomicAdd(&sh.hist[key & 0x7Fu], 1u);
-  });
-  flush_hist<128, THREADS>(sh, p.hist + 2 * kMaxBins);
-  if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
-
-  // ---------------- phase 3: T and r; count own keys > T and == T ----------------
-  resolve_digit<128, THREADS>(p.hist + 2 * kMaxBins, rem, sh);
-  const uint32_t T = (prefix24 << 7) | sh.out[0];
-  const unsigned long long r = sh.out[1];  // ties (key == T) to keep, lowest index first
-  unsigned long long mine_a = 0, mine_c = 0;
-  for_each_key([&](uint32_t key) {
-    mine_a += key > T;
-    mine_c += key == T;
-  });
-  const unsigned long long block_a = block_sum(mine_a, sh);
-  const unsigned long long block_c = block_sum(mine_c, sh);
-  unsigned long long* ac_counts = p.block_counts + 1 * kMaxFinalizeBlocks;
-  if (threadIdx.x == 0) ac_counts[blk] = (block_a << 32) | block_c;
-  if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
-
-  // ---------------- phase 4: write the survivors in index order ----------------
-  unsigned long long a_before = 0, c_before = 0, a_all = 0, c_all = 0;
-  for (unsigned int b = threadIdx.x; b < G; b += THREADS) {
-    const unsigned long long w = __ldcg(ac_counts + b);
-    a_all += w >> 32;
-    c_all += w & 0xFFFFFFFFull;
-    if (b < blk) {
-      a_before += w >> 32;
-      c_before += w & 0xFFFFFFFFull;
-    }
-  }
-  a_before = block_sum(a_before, sh);
-  c_before = block_sum(c_before, sh);
-  a_all = block_sum(a_all, sh);
-  c_all = block_sum(c_all, sh);
-  if (a_all + min(c_all, r) != p.k) {
-    if (threadIdx.x == 0) set_status(&p.ctl->status, NSML_ERR_INTERNAL);
-    return;
-  }
-  uint32_t* out_idx = reinterpret_cast<uint32_t*>(p.payload + p.P.idx_off);
-  {
-    // Each warp owns a contiguous run of the block's candidates.  First pass: count its keys > T and == T;
-    // one exchange of the warp totals through shared memory; second pass: ranks by ballot, coalesced writes.
-    constexpr int NW = THREADS / 32;
-    const int warp = threadIdx.x >> 5;
-    const unsigned int lt = (1u << lane) - 1u;
-    const unsigned int per_warp = ((E + NW - 1) / NW + 31) / 32 * 32;
-    const unsigned int w_lo = min(E, warp * per_warp), w_hi = min(E, w_lo + per_warp);
-    unsigned int wa = 0, wc = 0;
-    for (unsigned int j0 = w_lo; j0 < w_hi; j0 += 128) {  // four rounds of 32, their loads issued together
-      uint32_t key[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const unsigned int j = j0 + u * 32 + lane;
-        key[u] = (j < w_hi) ? (entry_val(j) & 0x7FFFFFFFu) : 0u;
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const bool live = j0 + u * 32 + lane < w_hi;
-        wa += __popc(__ballot_sync(0xFFFFFFFFu, live && key[u] > T));
-        wc += __popc(__ballot_sync(0xFFFFFFFFu, live && key[u] == T));
-      }
-    }
-    __syncthreads();  // sh.red may still be read by the block sums above
-    if (lane == 0) sh.red[warp] = ((unsigned long long)wa << 32) | wc;
-    __syncthreads();
-    unsigned long long a_here = a_before, c_here = c_before;
-    for (int w = 0; w < warp; ++w) {
-      a_here += sh.red[w] >> 32;
-      c_here += sh.red[w] & 0xFFFFFFFFull;
-    }
-    for (unsigned int j0 = w_lo; j0 < w_hi; j0 += 128) {
-      uint32_t bits[4], idx[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const unsigned int j = j0 + u * 32 + lane;
-        bits[u] = (j < w_hi) ? entry_val(j) : 0u;
-        idx[u] = (j < w_hi) ? my_idx[j] : 0u;  // coalesced; read whether or not the entry survives
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const bool live = j0 + u * 32 + lane < w_hi;
-        const uint32_t key = bits[u] & 0x7FFFFFFFu;
-        const bool a = live && key > T;
-        const bool c = live && key == T;
-        const unsigned int ba = __ballot_sync(0xFFFFFFFFu, a), bc = __ballot_sync(0xFFFFFFFFu, c);
-        const unsigned long long a_mine = a_here + __popc(ba & lt), c_mine = c_here + __popc(bc & lt);
-        if (a || (c && c_mine < r)) {
-          const unsigned long long pos = a_mine + min(c_mine, r);
-          out_idx[pos] = idx[u];
-          p.raw_val[pos] = __uint_as_float(bits[u]);
-        }
-        a_here += __popc(ba);
-        c_here += __popc(bc);
-      }
-    }
-  }
-  if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
-
-  // ---------------- phase 5: quantise, write the header ----------------
+  const int lane = threadIdx.x & 31;
   if (blk == 0 && threadIdx.x == 0) {
     nsml_payload_header h;
     h.magic = NSML_PAYLOAD_MAGIC;
@@ -603,6 +257,402 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
       }
     }
   }
+}
+
+template <int DTYPE, int THREADS, int CACHE>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS)  // at most 64 registers per thread
+k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
+  __shared__ FinalizeShared<THREADS, false> sh;
+  extern __shared__ __align__(16) uint32_t s_cache[];  // the first CACHE candidate values of this block
+  uint32_t* cache_val = s_cache;
+  const int lane = threadIdx.x & 31;
+  const unsigned int G = gridDim.x, blk = blockIdx.x;
+  // Index-range ownership (used by the slow path only) and the block's array.
+  const unsigned long long seg_first = (unsigned long long)blk * p.nseg / G;
+  const unsigned long long seg_last = (unsigned long long)(blk + 1) * p.nseg / G;
+  uint32_t* my_idx = p.list_idx;  // set below
+  uint32_t* my_val = p.list_val;
+  unsigned int barriers = 0;
+  unsigned int E = 0;  // candidates this block owns
+
+  auto entry_val = [&](unsigned int j) -> uint32_t { return j < (unsigned)CACHE ? cache_val[j] : __ldcg(my_val + j); };
+  auto put_entry = [&](unsigned int j, uint32_t idx, uint32_t val) {
+    my_idx[j] = idx;  // indices are needed once, at the end: they stay in global memory
+    if (j < (unsigned)CACHE) cache_val[j] = val; else my_val[j] = val;
+  };
+
+  // Calls f(key) for each of the block's candidates, four loads in flight per thread (the values beyond the
+  // shared-memory cache come from global memory, where one load at a time would cost a round trip each).
+  auto for_each_key = [&](auto f) {
+    for (unsigned int j0 = threadIdx.x; j0 < E; j0 += THREADS * 4) {
+      uint32_t v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const unsigned int j = j0 + u * THREADS;
+        v[u] = (j < E) ? entry_val(j) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u)
+        if (j0 + u * THREADS < E) f(v[u] & 0x7FFFFFFFu);
+    }
+  };
+
+  // ---------------- phase 0: take an equal share of the candidates, histogram of digit 0 ----------------
+  const unsigned int* ghist0 = p.hist;
+  for (int b = threadIdx.x; b < kMaxBins; b += THREADS) sh.hist[b] = 0;
+  bool nonfinite = false;
+  {
+    // Every block reads the per-group candidate counts the bucket pass left and
+    // scans them, which gives the list position of every group and the total.
+    const unsigned long long ngroups = (p.nseg + kGroupSegs - 1) / kGroupSegs;
+    const unsigned long long per_thread = (ngroups + THREADS - 1) / THREADS;
+    const unsigned long long g_begin = min(ngroups, threadIdx.x * per_thread);
+    const unsigned long long g_end = min(ngroups, g_begin + per_thread);
+    unsigned long long thread_sum = 0;
+    for (unsigned long long gi = g_begin; gi < g_end; ++gi) thread_sum += p.group_count[gi];
+    unsigned long long list_total;
+    unsigned long long thread_pos;  // list position where this thread's first group starts
+    {
+      // 64-bit exclusive scan over the block
+      const int warp = threadIdx.x >> 5;
+      unsigned long long incl = thread_sum;
+  #pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned long long up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= o) incl += up;
+      }
+      if (lane == 31) sh.red[warp] = incl;
+      __syncthreads();
+      unsigned long long before = 0, all = 0;
+  #pragma unroll
+      for (int w = 0; w < (THREADS / 32); ++w) {
+        const unsigned long long c = sh.red[w];
+        if (w < warp) before += c;
+        all += c;
+      }
+      list_total = all;
+      thread_pos = before + incl - thread_sum;
+    }
+    const unsigned long long share_lo = (unsigned long long)blk * list_total / G;
+    const unsigned long long share_hi = (unsigned long long)(blk + 1) * list_total / G;
+    if (list_total >= p.k) {
+      my_idx = p.list_idx + share_lo;
+      my_val = p.list_val + share_lo;
+      E = (unsigned int)(share_hi - share_lo);
+      if (E > 0 && thread_pos <= share_lo && share_lo < thread_pos + thread_sum) {  // exactly one thread
+        unsigned long long pos = thread_pos, gi = g_begin;
+        for (; gi < g_end; ++gi) {
+          const unsigned long long c = p.group_count[gi];
+          if (share_lo < pos + c) break;
+          pos += c;
+        }
+        sh.start[0] = gi;
+        sh.start[1] = pos;
+      }
+      __syncthreads();
+      unsigned long long seg_cursor = (E > 0) ? sh.start[0] * kGroupSegs : p.nseg;
+      unsigned long long pos_cursor = (E > 0) ? sh.start[1] : 0;
+      // A chunk is 8 segments per thread.  Thin stretches of the bucket make a
+      // share span many chunks, so the next chunk's counts are fetched before
+      // the current chunk's entries are copied.
+      auto load_counts = [&](unsigned long long first_seg) -> uint4 {
+        const unsigned long long s = first_seg + threadIdx.x * 8ull;  // a multiple of 8: the 16-byte load is aligned
+        if (s + 8 <= p.nseg) return *reinterpret_cast<const uint4*>(p.seg_count + s);
+        unsigned short c[8];
+  #pragma unroll
+        for (int e = 0; e < 8; ++e) c[e] = (s + e < p.nseg) ? p.seg_count[s + e] : (unsigned short)0;
+        uint4 v;
+        v.x = c[0] | ((uint32_t)c[1] << 16); v.y = c[2] | ((uint32_t)c[3] << 16);
+        v.z = c[4] | ((uint32_t)c[5] << 16); v.w = c[6] | ((uint32_t)c[7] << 16);
+        return v;
+      };
+      uint4 counts = load_counts(seg_cursor);
+      while (pos_cursor < share_hi && seg_cursor < p.nseg) {
+        const uint4 next_counts = load_counts(seg_cursor + (THREADS * 8));
+        const unsigned int cnt = (counts.x & 0xFFFFu) + (counts.x >> 16) + (counts.y & 0xFFFFu) + (counts.y >> 16) +
+                                 (counts.z & 0xFFFFu) + (counts.z >> 16) + (counts.w & 0xFFFFu) + (counts.w >> 16);
+        unsigned int chunk_total;
+        const unsigned int off = block_excl_scan(cnt, chunk_total, sh);
+        __syncthreads();  // sh.off / sh.cnt8 of the previous chunk have been read
+        sh.g.off[threadIdx.x] = off;
+        sh.g.cnt8[threadIdx.x] = counts;
+        __syncthreads();
+        // entries of this chunk that fall in the block's share
+        const unsigned long long from_pos = max(pos_cursor, share_lo), to_pos = min(pos_cursor + chunk_total, share_hi);
+        const unsigned short* cnt16 = reinterpret_cast<const unsigned short*>(sh.g.cnt8);  // count of segment q of the chunk
+        for (unsigned long long g0 = from_pos + threadIdx.x * 4ull; g0 < to_pos; g0 += THREADS * 4ull) {
+          // four consecutive entries per thread, each located by a search over the thread slots
+          unsigned long long from[4];
+          const int cnt = (int)min(4ull, to_pos - g0);
+  #pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            if (e < cnt) {
+              const unsigned int j = (unsigned int)(g0 + e - pos_cursor);
+              int lo = 0, hi = THREADS - 1;  // last thread slot of the chunk whose offset is <= j
+              while (lo < hi) {
+                const int mid = (lo + hi + 1) >> 1;
+                if (sh.g.off[mid] <= j) lo = mid; else hi = mid - 1;
+              }
+              unsigned int within = j - sh.g.off[lo];
+              unsigned int q = lo * 8;  // at most 8 steps: the entry lies in this slot's segments
+              while (within >= cnt16[q]) { within -= cnt16[q]; ++q; }
+              from[e] = (seg_cursor + q) * kSegElems + within;
+            }
+          }
+          uint32_t vals[4], idxs[4];
+  #pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            if (e < cnt) {
+              vals[e] = p.seg_val[from[e]];
+              idxs[e] = p.seg_idx[from[e]];
+            }
+          }
+  #pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            if (e < cnt) {
+              const uint32_t key = vals[e] & 0x7FFFFFFFu;
+              put_entry((unsigned int)(g0 + e - share_lo), idxs[e], vals[e]);
+              nonfinite |= key >= kInfKey;
+              atomicAdd(&sh.hist[key >> digit_shift(0)], 1u);
+            }
+          }
+        }
+        pos_cursor += chunk_total;
+        seg_cursor += (THREADS * 8);
+        counts = next_counts;
+      }
+      if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
+      flush_hist<kMaxBins>(sh, p.hist);
+      if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
+    }
+
+    if (list_total < p.k) {
+      // ---- slow path: this block's array becomes (all non-zero keys) + (zeros within budget) ----
+      const unsigned long long r_lo = seg_first * (unsigned long long)kSegElems;
+      const unsigned long long r_hi = min(seg_last * (unsigned long long)kSegElems, p.n);
+      my_idx = p.list_idx + r_lo;  // a block's range has room for all of its elements
+      my_val = p.list_val + r_lo;
+      unsigned long long nnz = 0, zeros = 0;
+      for (unsigned long long i0 = r_lo + threadIdx.x * 4ull; i0 < r_hi; i0 += THREADS * 4ull) {
+        uint32_t bits[4];
+        const int cnt = src.load_vals4(i0, p.n, bits);
+  #pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (e < cnt) {
+            if ((bits[e] & 0x7FFFFFFFu) != 0) ++nnz; else ++zeros;
+          }
+        }
+      }
+      const unsigned long long block_nnz = block_sum(nnz, sh);
+      const unsigned long long block_zeros = block_sum(zeros, sh);
+      unsigned long long* nz_counts = p.block_counts + 2 * kMaxFinalizeBlocks;
+      if (threadIdx.x == 0) nz_counts[blk] = (block_nnz << 32) | block_zeros;
+      if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
+
+      unsigned long long all_nnz = 0, zeros_before = 0;
+      for (unsigned int b = threadIdx.x; b < G; b += THREADS) {
+        const unsigned long long w = __ldcg(nz_counts + b);
+        all_nnz += w >> 32;
+        if (b < blk) zeros_before += w & 0xFFFFFFFFull;
+      }
+      all_nnz = block_sum(all_nnz, sh);
+      zeros_before = block_sum(zeros_before, sh);
+      const unsigned long long zero_budget = (p.k > all_nnz) ? p.k - all_nnz : 0;
+      // zeros of this block to keep, lowest index first
+      const unsigned long long allowed = (zero_budget > zeros_before) ? min(block_zeros, zero_budget - zeros_before) : 0ull;
+
+      __syncthreads();
+      for (int b = threadIdx.x; b < kMaxBins; b += THREADS) sh.hist[b] = 0;
+      E = 0;
+      unsigned long long zeros_seen = 0;
+      nonfinite = false;
+      for (unsigned long long base = r_lo; base < r_hi; base += THREADS * 4ull) {
+        const unsigned long long i0 = base + threadIdx.x * 4ull;
+        uint32_t bits[4] = {0, 0, 0, 0};
+        const int cnt = (i0 < r_hi) ? src.load_vals4(i0, p.n, bits) : 0;
+        unsigned int fz = 0, fn = 0;
+  #pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (e < cnt) {
+            if ((bits[e] & 0x7FFFFFFFu) != 0) fn |= 1u << e; else fz |= 1u << e;
+          }
+        }
+        unsigned int z_total, keep_total;
+        unsigned long long zrank = zeros_seen + block_excl_scan(__popc(fz), z_total, sh);
+        unsigned int f = fn;
+  #pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (fz & (1u << e)) {
+            if (zrank < allowed) f |= 1u << e;
+            ++zrank;
+          }
+        }
+        unsigned int pos = E + block_excl_scan(__popc(f), keep_total, sh);
+  #pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (f & (1u << e)) {
+            const uint32_t key = bits[e] & 0x7FFFFFFFu;
+            put_entry(pos, (uint32_t)(i0 + e), bits[e]);
+            nonfinite |= key >= kInfKey;
+            atomicAdd(&sh.hist[key >> digit_shift(0)], 1u);
+            ++pos;
+          }
+        }
+        zeros_seen += z_total;
+        E += keep_total;
+      }
+      if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
+      unsigned long long* totals2 = p.block_counts + 3 * kMaxFinalizeBlocks;
+      if (threadIdx.x == 0) totals2[blk] = E;
+      flush_hist<kMaxBins>(sh, p.hist + 3 * kMaxBins);
+      if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
+      unsigned long long part = 0;
+      for (unsigned int b = threadIdx.x; b < G; b += THREADS) part += __ldcg(totals2 + b);
+      if (block_sum(part, sh) < p.k) {  // cannot happen: the rebuilt list holds at least k entries
+        if (threadIdx.x == 0) set_status(&p.ctl->status, NSML_ERR_INTERNAL);
+        return;
+      }
+      ghist0 = p.hist + 3 * kMaxBins;
+    }
+  }
+  __syncthreads();  // the block's array (shared copy and global) is complete
+
+  // ---------------- phase 1: resolve digit 0, histogram of digit 1 ----------------
+  resolve_digit<kMaxBins>(ghist0, (unsigned int)p.k, sh);
+  const unsigned int d0 = sh.out[0];
+  unsigned int rem = sh.out[1];
+  for (int b = threadIdx.x; b < kMaxBins; b += THREADS) sh.hist[b] = 0;
+  __syncthreads();
+  for_each_key([&](uint32_t key) {
+    if ((key >> 19) == d0) atomicAdd(&sh.hist[(key >> 7) & 0xFFFu], 1u);
+  });
+  flush_hist<kMaxBins>(sh, p.hist + 1 * kMaxBins);
+  if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
+
+  // ---------------- phase 2: resolve digit 1, histogram of digit 2 ----------------
+  resolve_digit<kMaxBins>(p.hist + 1 * kMaxBins, rem, sh);
+  const unsigned int prefix24 = (d0 << 12) | sh.out[0];
+  rem = sh.out[1];
+  __syncthreads();
+  for (int b = threadIdx.x; b < 128; b += THREADS) sh.hist[b] = 0;
+  __syncthreads();
+  for_each_key([&](uint32_t key) {
+    if ((key >> 7) == prefix24) atomicAdd(&sh.hist[key & 0x7Fu], 1u);
+  });
+  flush_hist<128>(sh, p.hist + 2 * kMaxBins);
+  if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
+
+  // ---------------- phase 3: T and r; count own keys > T and == T ----------------
+  resolve_digit<128>(p.hist + 2 * kMaxBins, rem, sh);
+  const uint32_t T = (prefix24 << 7) | sh.out[0];
+  const unsigned long long r = sh.out[1];  // ties (key == T) to keep, lowest index first
+  unsigned long long mine_a = 0, mine_c = 0;
+  for_each_key([&](uint32_t key) {
+    mine_a += key > T;
+    mine_c += key == T;
+  });
+  const unsigned long long block_a = block_sum(mine_a, sh);
+  const unsigned long long block_c = block_sum(mine_c, sh);
+  unsigned long long* ac_counts = p.block_counts + 1 * kMaxFinalizeBlocks;
+  if (threadIdx.x == 0) ac_counts[blk] = (block_a << 32) | block_c;
+  if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
+
+  // ---------------- phase 4: write the survivors in index order ----------------
+  unsigned long long a_before = 0, c_before = 0, a_all = 0, c_all = 0;
+  for (unsigned int b = threadIdx.x; b < G; b += THREADS) {
+    const unsigned long long w = __ldcg(ac_counts + b);
+    a_all += w >> 32;
+    c_all += w & 0xFFFFFFFFull;
+    if (b < blk) {
+      a_before += w >> 32;
+      c_before += w & 0xFFFFFFFFull;
+    }
+  }
+  a_before = block_sum(a_before, sh);
+  c_before = block_sum(c_before, sh);
+  a_all = block_sum(a_all, sh);
+  c_all = block_sum(c_all, sh);
+  if (a_all + min(c_all, r) != p.k) {
+    if (threadIdx.x == 0) set_status(&p.ctl->status, NSML_ERR_INTERNAL);
+    return;
+  }
+  uint32_t* out_idx = reinterpret_cast<uint32_t*>(p.payload + p.P.idx_off);
+  {
+    // Each warp owns two contiguous runs of the block's candidates: its slice of those cached in shared
+    // memory and its slice of the rest (so that the slow loads of uncached values are spread over all
+    // warps).  First pass: count the keys > T and == T of each run; one exchange of the run totals through
+    // shared memory; second pass: ranks by ballot, coalesced writes.
+    constexpr int NW = THREADS / 32;
+    const int warp = threadIdx.x >> 5;
+    const unsigned int lt = (1u << lane) - 1u;
+    const unsigned int cached = min(E, (unsigned int)CACHE);
+    unsigned int run_lo[2], run_hi[2];
+    {
+      const unsigned int per_a = ((cached + NW - 1) / NW + 31) / 32 * 32;
+      const unsigned int per_b = ((E - cached + NW - 1) / NW + 31) / 32 * 32;
+      run_lo[0] = min(cached, warp * per_a);
+      run_hi[0] = min(cached, run_lo[0] + per_a);
+      run_lo[1] = min(E, cached + warp * per_b);
+      run_hi[1] = min(E, run_lo[1] + per_b);
+    }
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      unsigned int wa = 0, wc = 0;
+      for (unsigned int j0 = run_lo[q]; j0 < run_hi[q]; j0 += 128) {  // four rounds of 32, their loads issued together
+        uint32_t key[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const unsigned int j = j0 + u * 32 + lane;
+          key[u] = (j < run_hi[q]) ? (entry_val(j) & 0x7FFFFFFFu) : 0u;
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const bool live = j0 + u * 32 + lane < run_hi[q];
+          wa += __popc(__ballot_sync(0xFFFFFFFFu, live && key[u] > T));
+          wc += __popc(__ballot_sync(0xFFFFFFFFu, live && key[u] == T));
+        }
+      }
+      if (lane == 0) sh.run[q * NW + warp] = ((unsigned long long)wa << 32) | wc;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+      unsigned long long a_here = a_before, c_here = c_before;
+      for (int w = 0; w < q * NW + warp; ++w) {  // runs in index order: every warp's cached run, then the others
+        a_here += sh.run[w] >> 32;
+        c_here += sh.run[w] & 0xFFFFFFFFull;
+      }
+      for (unsigned int j0 = run_lo[q]; j0 < run_hi[q]; j0 += 128) {
+        uint32_t bits[4], idx[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const unsigned int j = j0 + u * 32 + lane;
+          bits[u] = (j < run_hi[q]) ? entry_val(j) : 0u;
+          idx[u] = (j < run_hi[q]) ? my_idx[j] : 0u;  // coalesced; read whether or not the entry survives
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const bool live = j0 + u * 32 + lane < run_hi[q];
+          const uint32_t key = bits[u] & 0x7FFFFFFFu;
+          const bool a = live && key > T;
+          const bool c = live && key == T;
+          const unsigned int ba = __ballot_sync(0xFFFFFFFFu, a), bc = __ballot_sync(0xFFFFFFFFu, c);
+          const unsigned long long a_mine = a_here + __popc(ba & lt), c_mine = c_here + __popc(bc & lt);
+          if (a || (c && c_mine < r)) {
+            const unsigned long long pos = a_mine + min(c_mine, r);
+            out_idx[pos] = idx[u];
+            p.raw_val[pos] = __uint_as_float(bits[u]);
+          }
+          a_here += __popc(ba);
+          c_here += __popc(bc);
+        }
+      }
+    }
+  }
+  if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
+
+  // ---------------- phase 5: quantise, write the header ----------------
+  quantize_phase(p, sh);
 }
 
 }  // namespace nsml

@@ -183,3 +183,38 @@ def test_runtime_argument_errors():
     with pytest.raises(nsml.NsmlError) as e:
         nsml.nsml_compress(grad[1:], 0.5, 8)  # 4-byte offset: not 16-byte aligned
     assert e.value.status == nsml.NSML_ERR_ARG
+
+
+# ---- the dense strategy (high kept fractions; no sample, no bucket pass) at sizes that use the large
+# kernel shape, with and without values beyond a block's shared-memory cache ----
+@pytest.mark.parametrize("n,ratio", [(2_000_003, 0.5), (3_100_000, 0.26), (9_000_001, 0.3)])
+def test_dense_strategy_large_buckets(n, ratio):
+    assert nsml.nsml_compress_strategy(n, ratio) == 1
+    rng = np.random.default_rng(n)
+    g = (rng.standard_normal(n) * 10.0 ** rng.uniform(-4, -1, n)).astype(np.float32)
+    g[rng.random(n) < 0.2] = 0.0
+    check_compress(g, ratio, 8)
+    mask = rng.random(n) < 0.5 * (1.0 - ratio)
+    check_compress(g, ratio, 16, mask_bool=mask)
+    check_compress(synth.f32_to_bf16_bits(g), ratio, 8, mask_bool=mask)
+
+
+@pytest.mark.parametrize("kind", ["equal", "zero", "ties", "sparse", "denormal"])
+def test_dense_strategy_degenerate_values(kind):
+    # every key equal / mostly zeros: the selection is decided by the index tie-break across blocks
+    n = 2_500_000 + 13
+    g = make(kind, n, np.random.default_rng(17))
+    for ratio in (0.25, 0.6, 1.0):
+        assert nsml.nsml_compress_strategy(n, ratio) == 1
+        check_compress(g, ratio, 8)
+
+
+def test_strategy_switch_is_invisible():
+    # the same bucket just below and just above the kept fraction at which the strategy changes
+    n = 1_500_000
+    g = synth.config1_bucket(n=n, seed=11)
+    seen = set()
+    for ratio in (0.049, 0.051, 0.249, 0.2499, 0.25, 0.251):
+        seen.add(nsml.nsml_compress_strategy(n, ratio))
+        check_compress(g, ratio, 8)
+    assert seen == {0, 1}
