@@ -323,6 +323,9 @@ k_finalize_dense(BucketSrc<DTYPE> src, FinalizeParams p) {
     return;
   }
   uint32_t* out_idx = reinterpret_cast<uint32_t*>(p.payload + p.P.idx_off);
+  static_assert(kMaxBins * 4 >= NW * 128 * 8, "the staging areas of all warps fit the histogram");
+  uint32_t* stage_idx = sh.hist + warp * 256;  // 128 indices, then 128 values, per warp
+  uint32_t* stage_val = stage_idx + 128;
 #pragma unroll
   for (int q = 0; q < 2; ++q) {
     // survivors before this slice: every warp's cached slice comes before any uncached one
@@ -361,26 +364,34 @@ k_finalize_dense(BucketSrc<DTYPE> src, FinalizeParams p) {
         if (lane >= o) incl += up;
       }
       const unsigned int total = __shfl_sync(FULL, incl, 31);
-      unsigned int a_rank = a_here + ((incl - mine) & 0xFFFFu);
-      unsigned int c_rank = c_here + ((incl - mine) >> 16);
-      if (fa | fc) {
-        const uint32_t first_index = (uint32_t)(range_lo + 4ull * w);
+      const unsigned int a_lane = (incl - mine) & 0xFFFFu, c_lane = (incl - mine) >> 16;  // of this step, in lower lanes
+      // Survivors of this step go to consecutive payload positions.  They are first put in order into the
+      // warp's staging area (the histogram's shared memory, free in this phase), then written 32 at a time.
+      const unsigned int c_room = r > c_here ? r - c_here : 0u;           // ties still to keep from here on
+      const unsigned int ta = total & 0xFFFFu, tc = min(total >> 16, c_room);
+      const unsigned int step_base = a_here + min(c_here, r);              // payload position of the step's first survivor
+      if (ta + tc != 0) {  // warp-uniform
+        if (fa | fc) {
+          unsigned int a_rank = a_lane, c_rank = c_lane;  // within the step
+          const uint32_t first_index = (uint32_t)(range_lo + 4ull * w);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (fa & (1u << e)) {
-            const unsigned int pos = a_rank + min(c_rank, r);
-            out_idx[pos] = first_index + e;
-            p.raw_val[pos] = __uint_as_float(bits[e]);
-            ++a_rank;
-          } else if (fc & (1u << e)) {
-            if (c_rank < r) {
-              const unsigned int pos = a_rank + c_rank;
-              out_idx[pos] = first_index + e;
-              p.raw_val[pos] = __uint_as_float(bits[e]);
+          for (int e = 0; e < 4; ++e) {
+            const bool is_a = fa & (1u << e), is_c = fc & (1u << e);
+            if (is_a || (is_c && c_rank < c_room)) {
+              const unsigned int slot = a_rank + min(c_rank, c_room);
+              stage_idx[slot] = first_index + e;
+              stage_val[slot] = bits[e];
             }
-            ++c_rank;
+            a_rank += is_a;
+            c_rank += is_c;
           }
         }
+        __syncwarp();
+        for (unsigned int i = lane; i < ta + tc; i += 32) {
+          out_idx[step_base + i] = stage_idx[i];
+          p.raw_val[step_base + i] = __uint_as_float(stage_val[i]);
+        }
+        __syncwarp();  // the staging area is read before the next step overwrites it
       }
       a_here += total & 0xFFFFu;
       c_here += total >> 16;
