@@ -50,12 +50,17 @@ __device__ inline bool header_ok(const nsml_payload_header* h, unsigned long lon
 }
 
 // offsets[w][b] = first payload entry of worker w whose index is >= b*kDenseTile.
+// The partition kernels also clear the call's status word (no separate clearing
+// step is needed); payload errors are therefore reported by the merge kernel,
+// which starts only after every block here has finished: a worker with a bad
+// header gets all-zero offsets, so nothing of its payload is read.
 // One warp per (worker, boundary): a 33-way search, every lane probing one
 // position per step, so a boundary costs about log33(k) memory round trips
 // instead of log2(k).
 __global__ void __launch_bounds__(kCta)
 k_partition(PayloadTable table, int W, unsigned long long n, unsigned int tiles, unsigned int* offsets, int* status) {
   const int lane = threadIdx.x & 31;
+  if (blockIdx.x == 0 && threadIdx.x == 0) *status = NSML_OK;
   const unsigned long long g = ((unsigned long long)blockIdx.x * kCta + threadIdx.x) >> 5;  // one warp per offset
   const unsigned long long per = (unsigned long long)tiles + 1;
   if (g >= per * W) return;  // whole warps leave together
@@ -63,7 +68,6 @@ k_partition(PayloadTable table, int W, unsigned long long n, unsigned int tiles,
   const unsigned long long b = g % per;
   const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(table.p[w]);
   if (!header_ok(h, n)) {
-    if (b == 0 && lane == 0) set_status(status, NSML_ERR_PAYLOAD);
     if (lane == 0) offsets[g] = 0;
     return;
   }
@@ -90,6 +94,7 @@ k_partition(PayloadTable table, int W, unsigned long long n, unsigned int tiles,
 // searches hide each other's latency and 32 times fewer threads are needed.
 __global__ void __launch_bounds__(kCta)
 k_partition_wide(PayloadTable table, int W, unsigned long long n, unsigned int tiles, unsigned int* offsets, int* status) {
+  if (blockIdx.x == 0 && threadIdx.x == 0) *status = NSML_OK;
   const unsigned long long g = (unsigned long long)blockIdx.x * kCta + threadIdx.x;
   const unsigned long long per = (unsigned long long)tiles + 1;
   if (g >= per * W) return;
@@ -97,7 +102,6 @@ k_partition_wide(PayloadTable table, int W, unsigned long long n, unsigned int t
   const unsigned long long b = g % per;
   const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(table.p[w]);
   if (!header_ok(h, n)) {
-    if (b == 0) set_status(status, NSML_ERR_PAYLOAD);
     offsets[g] = 0;
     return;
   }
@@ -119,6 +123,8 @@ k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long
   __shared__ unsigned int s_total;
   const unsigned long long per = (unsigned long long)tiles + 1;
   bool bad = false;
+  if (blockIdx.x == 0 && threadIdx.x < W)  // headers are checked here; the partition kernel cleared the status
+    bad = !header_ok(reinterpret_cast<const nsml_payload_header*>(table.p[threadIdx.x]), n);
 
   for (unsigned int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
     const unsigned long long lo = (unsigned long long)tile * kDenseTile;

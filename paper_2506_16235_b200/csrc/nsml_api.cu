@@ -298,9 +298,8 @@ static int accumulate_impl(const void* const* payloads, int W, float* dense, int
   int* status = reinterpret_cast<int*>(ws);
   unsigned int* offsets = reinterpret_cast<unsigned int*>(ws + L.offsets);
   const unsigned int tiles = (unsigned int)((n + kDenseTile - 1) / kDenseTile);
-  if (cudaMemsetAsync(ws, 0, 256, st) != cudaSuccess) return NSML_ERR_CUDA;
   {
-    LaunchScope scope(K_PARTITION, st);
+    LaunchScope scope(K_PARTITION, st);  // also clears the status word
     const unsigned long long offsets_needed = (unsigned long long)W * (tiles + 1ull);
     if (offsets_needed <= 32768) {  // few offsets: a warp each, few round trips
       unsigned int grid = (unsigned int)((offsets_needed * 32 + kCta - 1) / kCta);

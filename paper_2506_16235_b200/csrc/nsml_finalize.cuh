@@ -136,14 +136,17 @@ template <int THREADS, bool D>
 __device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, FinalizeShared<THREADS, D>& sh) {
   __syncthreads();
   if (threadIdx.x == 0) {
-    __threadfence();
-    atomicAdd(&ctl->barrier, 1u);
+    // Arrive with release, wait with acquire (both at device scope): what the block wrote before the
+    // __syncthreads above is visible to every block that leaves the wait, without full fences.
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(&ctl->barrier), "r"(1u) : "memory");
     int ok = 1, polls = 0;
-    while (*reinterpret_cast<volatile unsigned int*>(&ctl->barrier) < target) {
+    for (;;) {
+      unsigned int seen;
+      asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&ctl->barrier) : "memory");
+      if (seen >= target) break;
       if (++polls > kMaxPolls) { ok = 0; break; }
       if (polls > 256) __nanosleep(64);
     }
-    __threadfence();
     if (!ok) set_status(&ctl->status, NSML_ERR_TIMEOUT);
     sh.ok = ok;
   }
