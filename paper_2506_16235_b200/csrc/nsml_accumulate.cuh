@@ -16,7 +16,6 @@
 namespace nsml {
 
 constexpr int kDenseTile = 8192;  // dense elements per block iteration (32 KB of shared memory)
-constexpr int kMergeRound = 4 * kCta;  // payload entries a block loads before applying them
 
 struct PayloadTable {
   const unsigned char* p[NSML_MAX_WORKERS];
@@ -115,49 +114,82 @@ k_partition_wide(PayloadTable table, int W, unsigned long long n, unsigned int t
   offsets[g] = (unsigned int)lo;
 }
 
-__global__ void __launch_bounds__(kCta)
+// What a block needs to know about one worker's payload, read from its header once per block.
+struct WorkerView {
+  const uint32_t* idx;
+  const unsigned char* val;  // int8 codes or binary16 bit patterns
+  const float* scale;
+  int bits;
+};
+
+constexpr int kMergeUnits = 8;  // (worker, 256-entry chunk) units a thread loads before the adds are applied
+
+__global__ void __launch_bounds__(kCta, 6)
 k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long n, int zero_first,
         unsigned int tiles, const unsigned int* __restrict__ offsets, int* status) {
   __shared__ __align__(16) float s_acc[kDenseTile];
-  __shared__ unsigned int s_from[NSML_MAX_WORKERS], s_to[NSML_MAX_WORKERS];
-  __shared__ unsigned int s_total;
+  __shared__ WorkerView s_view[NSML_MAX_WORKERS];
+  __shared__ unsigned int s_from[NSML_MAX_WORKERS], s_to[NSML_MAX_WORKERS], s_pref[NSML_MAX_WORKERS + 1];
   const unsigned long long per = (unsigned long long)tiles + 1;
   bool bad = false;
-  if (blockIdx.x == 0 && threadIdx.x < W)  // headers are checked here; the partition kernel cleared the status
-    bad = !header_ok(reinterpret_cast<const nsml_payload_header*>(table.p[threadIdx.x]), n);
+  if (threadIdx.x < W) {
+    // Headers are checked here (the partition kernel cleared the status word).  A worker with a bad
+    // header has all-zero offsets, so its view is never used.
+    const unsigned char* pbase = table.p[threadIdx.x];
+    const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(pbase);
+    WorkerView v = {nullptr, nullptr, nullptr, 0};
+    if (header_ok(h, n)) {
+      v.idx = reinterpret_cast<const uint32_t*>(pbase + h->idx_off);
+      v.val = pbase + h->val_off;
+      v.scale = reinterpret_cast<const float*>(pbase + h->scale_off);
+      v.bits = (int)h->bits;
+    } else {
+      bad = blockIdx.x == 0;
+    }
+    s_view[threadIdx.x] = v;
+  }
 
   for (unsigned int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
     const unsigned long long lo = (unsigned long long)tile * kDenseTile;
     const unsigned int len = (unsigned int)min((unsigned long long)kDenseTile, n - lo);
-    __syncthreads();  // the previous tile is fully written out
-    if (threadIdx.x == 0) s_total = 0;
-    __syncthreads();
-    if (threadIdx.x < W) {
-      unsigned int a = offsets[threadIdx.x * per + tile];
-      unsigned int b = offsets[threadIdx.x * per + tile + 1];
-      if (b < a) b = a;  // only a corrupt (unsorted) payload gets here
-      s_from[threadIdx.x] = a;
-      s_to[threadIdx.x] = b;
-      if (b > a) atomicAdd(&s_total, b - a);
+    __syncthreads();  // the previous tile is fully written out (first tile: the views are in place)
+    if (threadIdx.x < 32) {
+      // the first warp reads the tile's offsets (two workers per lane) and scans the counts
+      unsigned int cnt[2];
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const int w = threadIdx.x * 2 + h;
+        cnt[h] = 0;
+        if (w < W) {
+          unsigned int a = offsets[w * per + tile];
+          unsigned int b = offsets[w * per + tile + 1];
+          if (b < a) b = a;  // only a corrupt (unsorted) payload gets here
+          s_from[w] = a;
+          s_to[w] = b;
+          cnt[h] = b - a;
+        }
+      }
+      unsigned int incl = cnt[0] + cnt[1];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if ((int)threadIdx.x >= o) incl += up;
+      }
+      const unsigned int before = incl - cnt[0] - cnt[1];
+      if ((int)threadIdx.x * 2 < W) s_pref[threadIdx.x * 2] = before;
+      if ((int)threadIdx.x * 2 + 1 < W) s_pref[threadIdx.x * 2 + 1] = before + cnt[0];
+      static_assert(NSML_MAX_WORKERS == 64, "two workers per lane of the first warp");
+      if (threadIdx.x == 31) s_pref[W] = incl;
     }
     __syncthreads();
-    const unsigned int total = s_total;
+    const unsigned int total = s_pref[W];
     if (total == 0 && !zero_first) continue;
     // Few entries: touch only their elements in global memory (after zero-filling
-    // the tile there in overwrite mode).  Many entries: stage the whole tile in
+    // the tile there in overwrite mode).  Many entries: stage the tile in
     // shared memory and write it back in one sweep.
     const bool staged = (unsigned long long)total * 16 > len;
-    if (!staged && zero_first) {
-      float* dtile = dense + lo;
-      for (unsigned int i = threadIdx.x * 4; i < len; i += kCta * 4) {
-        if (i + 4 <= len) *reinterpret_cast<float4*>(dtile + i) = make_float4(0.f, 0.f, 0.f, 0.f);
-        else for (unsigned int e = i; e < len; ++e) dtile[e] = 0.f;
-      }
-      __syncthreads();  // the zeros are in place before any add reads them
-    }
-
+    float* dtile = dense + lo;
     if (staged) {
-      float* dtile = dense + lo;
       for (unsigned int i = threadIdx.x * 4; i < len; i += kCta * 4) {
         if (i + 4 <= len) {
           float4 v = zero_first ? make_float4(0.f, 0.f, 0.f, 0.f) : *reinterpret_cast<const float4*>(dtile + i);
@@ -166,69 +198,70 @@ k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long
           for (unsigned int e = i; e < len; ++e) s_acc[e] = zero_first ? 0.f : dtile[e];
         }
       }
-      __syncthreads();
+    } else if (zero_first) {
+      for (unsigned int i = threadIdx.x * 4; i < len; i += kCta * 4) {
+        if (i + 4 <= len) *reinterpret_cast<float4*>(dtile + i) = make_float4(0.f, 0.f, 0.f, 0.f);
+        else for (unsigned int e = i; e < len; ++e) dtile[e] = 0.f;
+      }
     }
+    __syncthreads();  // the tile's starting values are in place before any add reads them
 
-    // The tile's entries of all workers, taken as one worker-major sequence of
-    // `total` entries, are processed kMergeRound at a time: every thread first
-    // loads its (up to 4) entries, so that one round costs one memory latency,
-    // then the adds are applied worker by worker (an element may receive one
-    // add per worker; within a worker indices are distinct).
-    for (unsigned int base = 0; base < total; base += kMergeRound) {
-      unsigned int off[4];
-      float val[4];
-      int wk[4];
-      int w_min = W, w_max = -1;
+    // The tile's entries are taken worker by worker in units of kCta consecutive entries, one per
+    // thread.  A thread first issues the loads of its entries of the next kMergeUnits units and
+    // touches none of the results, so that a group of units costs one memory latency; then the adds
+    // are applied unit by unit with a block barrier wherever the worker changes: an element gets at
+    // most one add per worker, always in worker order.
+    float* acc = staged ? s_acc : dtile;
+    int w = 0;           // current worker (uniform over the block)
+    unsigned int c = 0;  // entries of worker w already taken
+    while (w < W && s_to[w] == s_from[w]) ++w;
+    while (w < W) {
+      uint32_t raw_idx[kMergeUnits];  // 0xFFFFFFFF = no entry (indices are below 2^31)
+      int raw_val[kMergeUnits];
+      float raw_scale[kMergeUnits];
+      int unit_w[kMergeUnits], unit_bits[kMergeUnits];
 #pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        const unsigned int f = base + e * kCta + threadIdx.x;  // position in the flattened sequence
-        wk[e] = -1;
-        if (f < total) {
-          int w = 0;
-          unsigned int before = 0;
-          while (before + (s_to[w] - s_from[w]) <= f) { before += s_to[w] - s_from[w]; ++w; }  // w < W because f < total
-          const unsigned int j = s_from[w] + (f - before);
-          const unsigned char* pbase = table.p[w];
-          const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(pbase);
-          const unsigned long long o = (unsigned long long)reinterpret_cast<const uint32_t*>(pbase + h->idx_off)[j] - lo;  // wraps if idx < lo
-          float v;
-          if (h->bits == NSML_BITS_INT8)
-            v = decode_i8(reinterpret_cast<const signed char*>(pbase + h->val_off)[j],
-                          reinterpret_cast<const float*>(pbase + h->scale_off)[j >> 10]);
-          else
-            v = decode_f16(reinterpret_cast<const uint16_t*>(pbase + h->val_off)[j]);
-          if (o < len) {
-            wk[e] = w;
-            off[e] = (unsigned int)o;
-            val[e] = v;
-          } else {
-            bad = true;
+      for (int u = 0; u < kMergeUnits; ++u) {
+        unit_w[u] = w;
+        unit_bits[u] = 0;
+        raw_idx[u] = 0xFFFFFFFFu;
+        raw_val[u] = 0;
+        raw_scale[u] = 0.f;
+        if (w < W) {
+          const unsigned int to = s_to[w];
+          const unsigned int j = s_from[w] + c + threadIdx.x;
+          const WorkerView v = s_view[w];
+          unit_bits[u] = v.bits;
+          if (j < to) {
+            raw_idx[u] = v.idx[j];
+            if (v.bits == NSML_BITS_INT8) {
+              raw_val[u] = reinterpret_cast<const signed char*>(v.val)[j];
+              raw_scale[u] = v.scale[j >> 10];
+            } else {
+              raw_val[u] = reinterpret_cast<const uint16_t*>(v.val)[j];
+            }
+          }
+          c += kCta;
+          if (s_from[w] + c >= to) {  // worker w is used up: on to the next one that has entries here
+            c = 0;
+            do ++w; while (w < W && s_to[w] == s_from[w]);
           }
         }
       }
-      // workers present in this round (the sequence is worker-major, so they form a range)
-      {
-        const unsigned int f_lo = base, f_hi = min(total, base + kMergeRound) - 1;
-        unsigned int before = 0;
-        for (int w = 0; w < W; ++w) {
-          const unsigned int c = s_to[w] - s_from[w];
-          if (c && before <= f_hi && before + c > f_lo) { w_min = min(w_min, w); w_max = max(w_max, w); }
-          before += c;
-        }
-      }
-      for (int w = w_min; w <= w_max; ++w) {
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          if (wk[e] == w) {
-            if (staged) s_acc[off[e]] += val[e]; else dense[lo + off[e]] += val[e];
-          }
+      for (int u = 0; u < kMergeUnits; ++u) {
+        if (unit_w[u] >= W) break;
+        if (raw_idx[u] != 0xFFFFFFFFu) {
+          const unsigned long long o = (unsigned long long)raw_idx[u] - lo;  // wraps if idx < lo
+          const float v = unit_bits[u] == NSML_BITS_INT8 ? decode_i8(raw_val[u], raw_scale[u])
+                                                         : decode_f16((uint16_t)raw_val[u]);
+          if (o < len) acc[o] += v; else bad = true;
         }
-        __syncthreads();  // worker w is done before worker w+1 adds to the same elements
+        if (u + 1 == kMergeUnits || unit_w[u + 1] != unit_w[u]) __syncthreads();  // uniform over the block
       }
     }
 
     if (staged) {
-      float* dtile = dense + lo;
       for (unsigned int i = threadIdx.x * 4; i < len; i += kCta * 4) {
         if (i + 4 <= len) {
           *reinterpret_cast<float4*>(dtile + i) = *reinterpret_cast<const float4*>(s_acc + i);
