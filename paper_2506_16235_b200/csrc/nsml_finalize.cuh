@@ -48,6 +48,7 @@ constexpr int kFinLargeThreads = 512, kFinLargeCache = 20480;
 // The dense kernel needs no gather scratch, which leaves room for a larger cache in the large shape: two
 // blocks per SM then hold 2 x 23040 values, 6.8M elements over 148 SMs (a 25 MB float32 bucket stays on chip).
 constexpr int kFinDenseLargeCache = 23040;
+constexpr int kGatherRun = 4;  // consecutive candidates a thread of the gather copies per step
 constexpr size_t finalize_dyn_smem(int cache_entries) { return (size_t)cache_entries * 4; }  // values only
 
 struct FinalizeParams {
@@ -383,35 +384,47 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
         // entries of this chunk that fall in the block's share
         const unsigned long long from_pos = max(pos_cursor, share_lo), to_pos = min(pos_cursor + chunk_total, share_hi);
         const unsigned short* cnt16 = reinterpret_cast<const unsigned short*>(sh.g.cnt8);  // count of segment q of the chunk
-        for (unsigned long long g0 = from_pos + threadIdx.x * 4ull; g0 < to_pos; g0 += THREADS * 4ull) {
-          // four consecutive entries per thread, each located by a search over the thread slots
-          unsigned long long from[4];
-          const int cnt = (int)min(4ull, to_pos - g0);
-  #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            if (e < cnt) {
-              const unsigned int j = (unsigned int)(g0 + e - pos_cursor);
-              int lo = 0, hi = THREADS - 1;  // last thread slot of the chunk whose offset is <= j
+        for (unsigned long long g0 = from_pos + threadIdx.x * (unsigned long long)kGatherRun; g0 < to_pos;
+             g0 += THREADS * (unsigned long long)kGatherRun) {
+          // kGatherRun consecutive entries per thread: the first is located by a search over the thread
+          // slots, the others by stepping on from it; all their loads are issued together.
+          const int cnt = (int)min((unsigned long long)kGatherRun, to_pos - g0);
+          uint32_t from[kGatherRun];  // list slot of each entry (below 2^31)
+          {
+            unsigned int q = 0, within = 0;
+            auto locate = [&](unsigned int j) {  // segment q of the chunk and place in it of the chunk's entry j
+              int lo = 0, hi = THREADS - 1;      // last thread slot of the chunk whose offset is <= j
               while (lo < hi) {
                 const int mid = (lo + hi + 1) >> 1;
                 if (sh.g.off[mid] <= j) lo = mid; else hi = mid - 1;
               }
-              unsigned int within = j - sh.g.off[lo];
-              unsigned int q = lo * 8;  // at most 8 steps: the entry lies in this slot's segments
+              within = j - sh.g.off[lo];
+              q = lo * 8;  // at most 8 steps: the entry lies in this slot's segments
               while (within >= cnt16[q]) { within -= cnt16[q]; ++q; }
-              from[e] = (seg_cursor + q) * kSegElems + within;
+            };
+            const unsigned int j0 = (unsigned int)(g0 - pos_cursor);
+            locate(j0);
+#pragma unroll
+            for (int e = 0; e < kGatherRun; ++e) {
+              from[e] = 0;
+              if (e < cnt) {
+                from[e] = (uint32_t)((seg_cursor + q) * kSegElems + within);
+                // the next entry is the next one of this segment, else it is searched for (a walk could
+                // cross any number of empty segments)
+                if (e + 1 < cnt && ++within >= cnt16[q]) locate(j0 + e + 1);
+              }
             }
           }
-          uint32_t vals[4], idxs[4];
-  #pragma unroll
-          for (int e = 0; e < 4; ++e) {
+          uint32_t vals[kGatherRun], idxs[kGatherRun];
+#pragma unroll
+          for (int e = 0; e < kGatherRun; ++e) {
             if (e < cnt) {
               vals[e] = p.seg_val[from[e]];
               idxs[e] = p.seg_idx[from[e]];
             }
           }
-  #pragma unroll
-          for (int e = 0; e < 4; ++e) {
+#pragma unroll
+          for (int e = 0; e < kGatherRun; ++e) {
             if (e < cnt) {
               const uint32_t key = vals[e] & 0x7FFFFFFFu;
               put_entry((unsigned int)(g0 + e - share_lo), idxs[e], vals[e]);
