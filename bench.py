@@ -516,7 +516,7 @@ class DecoderWorkload(Workload):
 
 
 class AggWorkload(Workload):
-    name = "aggregation stress: W=8 int8 payloads (ratio 0.05) for a 350M-element bucket, decompress + sum only"
+    name = "aggregation stress: W=8 int8 payloads (ratio 0.05) for one dense bucket (350M elements unless --agg-elements), decompress + sum only"
     W, N, RATIO = 8, 350_000_000, 0.05
 
     def __init__(self, nsml, torch, device, rank, nlanes=1):
@@ -626,6 +626,8 @@ def main():
     ap.add_argument("--no-large-bucket-leg", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (e2e is then null)")
     ap.add_argument("--no-kernel-times", action="store_true", help="skip the event-bracketed per-kernel pass")
+    ap.add_argument("--agg-elements", type=int, default=None,
+                    help="agg workload only: dense elements (default 350M; smaller sizes are for profiler captures)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -657,6 +659,8 @@ def main():
         dist = dist_mod
         dist.init_process_group("nccl", device_id=device)
 
+    if args.workload == "agg" and args.agg_elements:
+        AggWorkload.N = int(args.agg_elements)
     wl = WORKLOADS[args.workload](nsml, torch, device, rank, nlanes=max(1, args.streams))
     wl.init_graphs(not args.no_graphs)
     if wl.use_graphs:
