@@ -16,6 +16,14 @@ Pins (what each function is checked against, independently of itself):
                      bit patterns
   decompress_sum     closed forms (identical payloads, disjoint payloads),
                      dense brute-force loop
+  l2_norm            closed forms (constant vectors, 3-4-5), math.fsum of exact
+                     rational squares, the library norm in float64
+  quantize_gate      the four branches of Alg. 2 Step 1 written out by hand
+  prune_mask         brute force over all m-subsets, worked example, library
+                     partial sort on distinct keys, the paper's rate formula,
+                     invariants (count, order, tie rule)
+  error_feedback_step  worked two-step example, conservation (what is sent
+                     plus what is kept equals the accumulated gradient)
   Controller (NetSense phase)  hand trace from Eq. 1-3, closed forms for the
                      multiplicative-decrease / additive-increase recurrences
   Controller (start-up phase)  parity unpinned: the paper gives neither the
@@ -37,5 +45,14 @@ from .compress import (  # noqa: F401
     compress,
     decompress_sum,
     Payload,
+)
+from .adaptive import (  # noqa: F401
+    l2_norm,
+    quantize_gate,
+    pruning_rate,
+    pruned_count,
+    prune_mask,
+    netsense_compression,
+    error_feedback_step,
 )
 from .controller import Controller, ControllerParams  # noqa: F401

@@ -16,6 +16,8 @@ What is computed, and where the paper states it:
   nearest even; magnitudes that would round to infinity saturate to the
   largest finite half (65504).  The int8 codec (symmetric, one max-abs scale
   per block of 1024 consecutive survivors) is an addition to the paper.
+  When Step 1 does not quantise, the survivors travel as the 32-bit floats
+  they are (bits = 32).
 * Section 4.2 Step 3 / Section 5.3: every worker receives all workers'
   sparse payloads (AllGather pattern) and sums them into a dense gradient.
   The sum is a plain sum (no averaging), taken in fp64 and rounded once.
@@ -201,7 +203,7 @@ class Payload:
 
     n: int
     k: int
-    bits: int  # 8 -> int8 codes + per-block scales; 16 -> fp16 bit patterns
+    bits: int  # 8 -> int8 codes + per-block scales; 16 -> fp16 bit patterns; 32 -> the raw float32 values
     idx: np.ndarray  # uint32[k], strictly ascending
     raw: np.ndarray  # float32[k], survivor values before quantisation
     codes: Optional[np.ndarray] = None  # int8[k]       (bits == 8)
@@ -212,6 +214,8 @@ class Payload:
         """Dequantised float32 values v'."""
         if self.bits == 8:
             return dequantize_int8(self.codes, self.scales)
+        if self.bits == 32:
+            return self.raw.copy()
         return f16_bits_to_f32(self.half)
 
 
@@ -226,8 +230,8 @@ def compress(
     A bf16 bucket is widened with widen_bf16 first.  `prune_mask[i]` true
     means parameter i is pruned this step.
     """
-    if bits not in (8, 16):
-        raise ValueError("bits must be 8 (int8) or 16 (fp16)")
+    if bits not in (8, 16, 32):
+        raise ValueError("bits must be 8 (int8), 16 (fp16) or 32 (float32 as is)")
     v = _apply_mask(grad, prune_mask)
     n = v.size
     k = k_of(ratio, n)
@@ -236,7 +240,7 @@ def compress(
     p = Payload(n=n, k=k, bits=bits, idx=idx, raw=raw)
     if bits == 8:
         p.codes, p.scales = quantize_int8(raw)
-    else:
+    elif bits == 16:
         p.half = f32_to_f16_bits(raw)
     return p
 
