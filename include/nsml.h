@@ -52,7 +52,7 @@ enum {
 };
 
 enum { NSML_F32 = 0, NSML_BF16 = 1 };              /* gradient element type */
-enum { NSML_BITS_INT8 = 8, NSML_BITS_FP16 = 16 };  /* value codec ("bits") */
+enum { NSML_BITS_INT8 = 8, NSML_BITS_FP16 = 16, NSML_BITS_FP32 = 32 }; /* value codec ("bits") */
 
 #define NSML_QBLOCK 1024         /* survivors per int8 scale block */
 #define NSML_MAX_WORKERS 64      /* largest W of nsml_decompress_accumulate */
@@ -63,8 +63,8 @@ enum { NSML_BITS_INT8 = 8, NSML_BITS_FP16 = 16 };  /* value codec ("bits") */
 /* ------------------------------------------------------------------------
  * Payload: one worker's compressed bucket, one contiguous buffer, every
  * section 16-byte aligned:
- *   header (64 B) | idx: u32[k] strictly ascending | val: i8[k] or f16[k]
- *   | scale: f32[nblocks] (int8 only; block b covers payload entries
+ *   header (64 B) | idx: u32[k] strictly ascending | val: i8[k], f16[k] or
+ *   f32[k] | scale: f32[nblocks] (int8 only; block b covers payload entries
  *   [b*1024, (b+1)*1024))
  * The paper leaves the layout of Com_grads open (Alg. 2 names only
  * top_k(grads, ratio)); this one is defined here.
@@ -74,12 +74,12 @@ typedef struct nsml_payload_header {
   uint32_t version;   /* NSML_PAYLOAD_VERSION */
   uint64_t n;         /* elements in the dense bucket */
   uint64_t k;         /* survivors = ceil(ratio*n) */
-  uint32_t bits;      /* NSML_BITS_INT8 or NSML_BITS_FP16 */
+  uint32_t bits;      /* NSML_BITS_INT8, NSML_BITS_FP16 or NSML_BITS_FP32 */
   uint32_t qblock;    /* NSML_QBLOCK */
-  uint64_t nblocks;   /* ceil(k/qblock) for int8, 0 for fp16 */
+  uint64_t nblocks;   /* ceil(k/qblock) for int8, else 0 */
   uint64_t idx_off;   /* byte offsets from the start of the payload */
   uint64_t val_off;
-  uint64_t scale_off; /* 0 for fp16 */
+  uint64_t scale_off; /* int8 only, else 0 */
 } nsml_payload_header;
 
 /* ------------------------------------------------------------------------
@@ -183,6 +183,8 @@ size_t nsml_accumulate_workspace_bytes(int64_t n, int W);
  *               scale 0 gives codes 0.  (Not in the paper.)
  *               NSML_BITS_FP16: float32 -> binary16, round to nearest even
  *               (Alg. 2 Step 1 "quantize"); |v| >= 65520 saturates to +-65504.
+ *               NSML_BITS_FP32: the survivors' float32 values as they are
+ *               (Alg. 2 when Step 1 does not quantise).
  *   prune_mask  device pointer (4-byte aligned) to ceil(n/32) words, bit (i&31)
  *               of word i>>5 set = parameter i is pruned: its gradient counts as
  *               +0.0 (Alg. 2 Step 2).  NULL = nothing pruned.
@@ -221,7 +223,7 @@ int nsml_compress_strategy(int64_t n, double ratio);
  *
  *   payloads    HOST array of W device pointers (16-byte aligned), each a payload
  *               written by nsml_compress (or laid out the same way) for this n;
- *               int8 and fp16 payloads may be mixed; 1 <= W <= NSML_MAX_WORKERS
+ *               payloads of different codecs may be mixed; 1 <= W <= NSML_MAX_WORKERS
  *   dense       device pointer, 16-byte aligned, n float32; read unless
  *               zero_first, always written
  *   zero_first  non-zero: dense is overwritten by the sum; zero: the sum is
@@ -229,8 +231,8 @@ int nsml_compress_strategy(int64_t n, double ratio);
  *   workspace   device pointer, 256-byte aligned, >=
  *               nsml_accumulate_workspace_bytes(n, W)
  *
- * Values are dequantised as float(code)*scale (one float32 multiply) or
- * float(half), and added in float32 in worker order w = 0..W-1, each dense
+ * Values are dequantised as float(code)*scale (one float32 multiply),
+ * float(half) or taken as they are, and added in float32 in worker order w = 0..W-1, each dense
  * element by one thread: the result is deterministic.  Device-detected:
  * NSML_ERR_PAYLOAD if a header does not match (magic, version, n, bits, k) or
  * an index is >= n; nothing is written out of range.
@@ -272,6 +274,98 @@ int nsml_decompress_accumulate(const void* const* payloads, int W, float* dense,
 #define NSML_STATIC_SCRATCH_BYTES 66048 /* 256 + 8 * (2^24 / 8192 + 1) * 4, rounded up to 256 */
 int nsml_decompress_accumulate_static(const void* const* payloads, int W, float* dense, int64_t n,
                                       int zero_first, void* stream, int* status_out);
+
+/* ------------------------------------------------------------------------
+ * The rest of Alg. 2 around the top-k step.
+ * ---------------------------------------------------------------------- */
+
+/* nsml_grad_l2 -- the L2 norm of Alg. 2 Step 1 ("calculate_L2_norm(grads)"):
+ * sqrt(sum g_i^2), every square and the sum in float64.
+ *   grad, n, grad_dtype   as for nsml_compress (no pruning mask: Step 1 comes
+ *                         before Step 2)
+ *   workspace   device pointer, 256-byte aligned, >= nsml_l2_workspace_bytes()
+ *   l2_out      host pointer or NULL.  NULL: the call returns after enqueueing
+ *               and the sum of squares (float64) is left at byte offset 8 of
+ *               `workspace`.  Non-NULL: the call synchronises `stream` and
+ *               stores the norm there.
+ * The adds follow a fixed order for a given device, so the value is
+ * reproducible run to run.  NSML_ERR_NONFINITE if the bucket holds NaN or Inf
+ * (returned when l2_out is given, else left in the status word). */
+size_t nsml_l2_workspace_bytes(void);
+int nsml_grad_l2(const void* grad, int64_t n, int grad_dtype, void* workspace, size_t workspace_bytes,
+                 void* stream, double* l2_out);
+
+/* nsml_quantize_gate -- the decision of Alg. 2 Step 1, host arithmetic only:
+ * if ratio < tr_q and l2 > tr_d the values are sent as 16-bit floats and the
+ * ratio is doubled (capped at 1; the paper states no cap), else the values are
+ * sent with `plain_bits` (NSML_BITS_FP32 is the paper's case) at the ratio
+ * given.  tr_q ("quantization check threshold") and tr_d ("gradient density
+ * threshold") are inputs of Alg. 2; the paper gives no values for them.
+ * NSML_ERR_ARG for NULL outputs, a ratio outside (0, 1], NaN thresholds or a
+ * negative norm. */
+int nsml_quantize_gate(double ratio, double l2, double tr_q, double tr_d, int plain_bits,
+                       double* ratio_out, int* bits_out);
+
+/* Alg. 2 Step 2: pruning_rate = 0.5 * (1 - ratio).  The number of parameters
+ * that rate stands for is read as m = ceil(pruning_rate * n) in IEEE double
+ * (0 for arguments out of range). */
+int64_t nsml_pruned_count(int64_t n, double ratio);
+size_t nsml_prune_workspace_bytes(int64_t n);
+
+/* nsml_prune_mask_build -- Alg. 2 Step 2 ("prune_weights(pruning_rate)"): marks
+ * the m = nsml_pruned_count(n, ratio) parameters of smallest magnitude
+ * (compared on the float32 bit pattern with the sign cleared; ties: smaller
+ * magnitude first, then lower index -- the paper states no tie rule).
+ *   weights     device pointer, 16-byte aligned, n finite float32
+ *   prune_mask  device pointer (4-byte aligned), ceil(n/32) words, written in
+ *               the layout nsml_compress reads; bits past n are 0
+ *   workspace   device pointer, 256-byte aligned, >= nsml_prune_workspace_bytes(n)
+ * Nothing is remembered between calls: the mask is rebuilt from the weights
+ * every time (pruned parameters "are not permanently removed").
+ * Device-detected: NSML_ERR_NONFINITE. */
+int nsml_prune_mask_build(const float* weights, int64_t n, double ratio, uint32_t* prune_mask,
+                          void* workspace, size_t workspace_bytes, void* stream);
+
+/* nsml_compress_feedback -- nsml_compress with the local accumulation of the
+ * gradients that sparsification filters out (Section 4.2 Step 3: "accumulate
+ * the local filtered gradients for further aggregation and transmission"),
+ * read as a residual kept by the caller between steps:
+ *   acc      = grad + residual          (one float32 add per element)
+ *   payload  = nsml_compress(acc, ratio, bits, prune_mask)
+ *   residual = acc, and at every selected index i: acc[i] - v'_i, v' being the
+ *              value nsml_decompress_accumulate reconstructs (one float32
+ *              subtraction), so that the quantisation error is carried too
+ *   residual    device pointer, 16-byte aligned, n float32, read and written;
+ *               zero it before the first step
+ *   all other arguments as for nsml_compress (workspace of
+ *   nsml_workspace_bytes(n, NSML_F32) bytes).
+ * A pruned parameter is not sent but keeps accumulating in the residual. */
+int nsml_compress_feedback(const void* grad, float* residual, int64_t n, int grad_dtype, double ratio,
+                           int bits, const uint32_t* prune_mask, void* payload, size_t payload_capacity,
+                           void* workspace, size_t workspace_bytes, void* stream);
+
+/* nsml_compress_adaptive -- Alg. 2 as a whole, in its order:
+ *   Step 1  if ratio < tr_q: L2 norm (device), gate (host; the call waits for
+ *           the norm, so it synchronises `stream` once in that case)
+ *   Step 2  if weights != NULL: prune_mask is rebuilt from them at the ratio
+ *           Step 1 left (prune_mask must then be writable, ceil(n/32) words);
+ *           if weights == NULL: prune_mask is used as given (may be NULL)
+ *   Step 3  nsml_compress at that ratio and codec
+ *   payload_capacity >= nsml_adaptive_payload_bytes(n, ratio, tr_q, plain_bits)
+ *   (the larger of the two outcomes); workspace >=
+ *   nsml_adaptive_workspace_bytes(n, grad_dtype)
+ *   ratio_used, bits_used   host pointers, receive what Steps 2-3 used
+ *   l2_out      host pointer or NULL: the norm, or -1 when it was not needed
+ * Selection is on the float32 magnitudes and only the survivors are converted
+ * to 16 bits (Alg. 2 converts before selecting; the survivors differ only
+ * where the conversion creates ties). */
+size_t nsml_adaptive_payload_bytes(int64_t n, double ratio, double tr_q, int plain_bits);
+size_t nsml_adaptive_workspace_bytes(int64_t n, int grad_dtype);
+int nsml_compress_adaptive(const void* grad, int64_t n, int grad_dtype, double ratio, double tr_q,
+                           double tr_d, int plain_bits, const float* weights, uint32_t* prune_mask,
+                           void* payload, size_t payload_capacity, void* workspace,
+                           size_t workspace_bytes, void* stream, double* ratio_used, int* bits_used,
+                           double* l2_out);
 
 /* Host-buffer variants: the same operations for callers whose gradients and
  * payloads live in host memory (pinned memory gives asynchronous copies).

@@ -34,6 +34,7 @@ NSML_F32 = 0
 NSML_BF16 = 1
 NSML_BITS_INT8 = 8
 NSML_BITS_FP16 = 16
+NSML_BITS_FP32 = 32
 NSML_QBLOCK = 1024
 NSML_MAX_WORKERS = 64
 NSML_PAYLOAD_MAGIC = 0x4C4D534E
@@ -101,6 +102,17 @@ def _load() -> ctypes.CDLL:
         "nsml_compress_host": (ci, [vp, i64, ci, dbl, ci, vp, vp, sz, vp, sz, vp]),
         "nsml_accumulate_host_scratch_bytes": (sz, [i64, ci, sz]),
         "nsml_decompress_accumulate_host": (ci, [ctypes.POINTER(vp), ctypes.POINTER(sz), ci, vp, i64, ci, vp, sz, vp]),
+        "nsml_l2_workspace_bytes": (sz, []),
+        "nsml_grad_l2": (ci, [vp, i64, ci, vp, sz, vp, ctypes.POINTER(dbl)]),
+        "nsml_quantize_gate": (ci, [dbl, dbl, dbl, dbl, ci, ctypes.POINTER(dbl), ctypes.POINTER(ci)]),
+        "nsml_pruned_count": (i64, [i64, dbl]),
+        "nsml_prune_workspace_bytes": (sz, [i64]),
+        "nsml_prune_mask_build": (ci, [vp, i64, dbl, vp, vp, sz, vp]),
+        "nsml_compress_feedback": (ci, [vp, vp, i64, ci, dbl, ci, vp, vp, sz, vp, sz, vp]),
+        "nsml_adaptive_payload_bytes": (sz, [i64, dbl, dbl, ci]),
+        "nsml_adaptive_workspace_bytes": (sz, [i64, ci]),
+        "nsml_compress_adaptive": (ci, [vp, i64, ci, dbl, dbl, dbl, ci, vp, vp, vp, sz, vp, sz, vp,
+                                        ctypes.POINTER(dbl), ctypes.POINTER(ci), ctypes.POINTER(dbl)]),
         "nsml_last_status": (ci, [vp, vp, ctypes.POINTER(ci)]),
         "nsml_strerror": (ctypes.c_char_p, [ci]),
         "nsml_kernel_count": (ci, []),
@@ -310,6 +322,106 @@ def nsml_decompress_accumulate_static(payloads: Sequence, dense, zero_first: boo
     return status.value if want_status else None
 
 
+def _check_bucket(t, what="grad"):
+    if not (t.is_cuda and t.is_contiguous() and t.dim() == 1):
+        raise ValueError(f"{what} must be a contiguous 1-D CUDA tensor")
+
+
+def nsml_grad_l2(grad, workspace=None, stream=None) -> float:
+    """L2 norm of a bucket (Alg. 2 Step 1), float64; synchronises the stream."""
+    _check_bucket(grad)
+    if workspace is None:
+        workspace = alloc_bytes(lib.nsml_l2_workspace_bytes(), grad.device)
+    out = ctypes.c_double()
+    rc = lib.nsml_grad_l2(grad.data_ptr(), grad.numel(), _grad_dtype(grad), workspace.data_ptr(), workspace.numel(),
+                          _stream_ptr(stream), ctypes.byref(out))
+    _check(rc, "nsml_grad_l2")
+    return out.value
+
+
+def nsml_quantize_gate(ratio: float, l2: float, tr_q: float, tr_d: float, plain_bits: int = NSML_BITS_FP32):
+    """Alg. 2 Step 1 decision: (ratio to use, value codec to use)."""
+    r, b = ctypes.c_double(), ctypes.c_int()
+    _check(lib.nsml_quantize_gate(float(ratio), float(l2), float(tr_q), float(tr_d), int(plain_bits),
+                                  ctypes.byref(r), ctypes.byref(b)), "nsml_quantize_gate")
+    return r.value, b.value
+
+
+def nsml_pruned_count(n: int, ratio: float) -> int:
+    return int(lib.nsml_pruned_count(int(n), float(ratio)))
+
+
+def nsml_prune_workspace_bytes(n: int) -> int:
+    return int(lib.nsml_prune_workspace_bytes(int(n)))
+
+
+def nsml_prune_mask_build(weights, ratio: float, prune_mask=None, workspace=None, stream=None):
+    """Pruning mask from the weights (Alg. 2 Step 2): int32 CUDA tensor of ceil(n/32) words."""
+    _check_bucket(weights, "weights")
+    torch = _torch()
+    if weights.dtype != torch.float32:
+        raise TypeError("weights must be float32")
+    n = weights.numel()
+    if prune_mask is None:
+        prune_mask = torch.empty((n + 31) // 32, dtype=torch.int32, device=weights.device)
+    if workspace is None:
+        workspace = alloc_bytes(nsml_prune_workspace_bytes(n), weights.device)
+    rc = lib.nsml_prune_mask_build(weights.data_ptr(), n, float(ratio), prune_mask.data_ptr(), workspace.data_ptr(),
+                                   workspace.numel(), _stream_ptr(stream))
+    _check(rc, "nsml_prune_mask_build")
+    return prune_mask
+
+
+def nsml_compress_feedback(grad, residual, ratio: float, bits: int = NSML_BITS_INT8, prune_mask=None, payload=None,
+                           workspace=None, stream=None):
+    """nsml_compress of grad + residual; residual (float32 CUDA tensor) is updated in place."""
+    _check_bucket(grad)
+    _check_bucket(residual, "residual")
+    torch = _torch()
+    n = grad.numel()
+    if residual.dtype != torch.float32 or residual.numel() != n:
+        raise ValueError("residual must be float32 with one element per gradient element")
+    need = nsml_payload_bytes(n, ratio, bits)
+    if need == 0:
+        raise NsmlError(NSML_ERR_ARG, "nsml_compress_feedback")
+    if payload is None:
+        payload = alloc_bytes(need, grad.device)
+    if workspace is None:
+        workspace = alloc_bytes(nsml_workspace_bytes(n, NSML_F32), grad.device)
+    rc = lib.nsml_compress_feedback(grad.data_ptr(), residual.data_ptr(), n, _grad_dtype(grad), float(ratio), int(bits),
+                                    None if prune_mask is None else prune_mask.data_ptr(), payload.data_ptr(),
+                                    payload.numel(), workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    _check(rc, "nsml_compress_feedback")
+    return payload[:need]
+
+
+def nsml_compress_adaptive(grad, ratio: float, tr_q: float, tr_d: float, plain_bits: int = NSML_BITS_FP32,
+                           weights=None, prune_mask=None, payload=None, workspace=None, stream=None):
+    """Alg. 2 as a whole.  Returns (payload, ratio used, bits used, L2 norm or None, prune mask or None)."""
+    _check_bucket(grad)
+    torch = _torch()
+    n = grad.numel()
+    dtype = _grad_dtype(grad)
+    cap = int(lib.nsml_adaptive_payload_bytes(n, float(ratio), float(tr_q), int(plain_bits)))
+    if cap == 0:
+        raise NsmlError(NSML_ERR_ARG, "nsml_compress_adaptive")
+    if payload is None:
+        payload = alloc_bytes(cap, grad.device)
+    if workspace is None:
+        workspace = alloc_bytes(int(lib.nsml_adaptive_workspace_bytes(n, dtype)), grad.device)
+    if weights is not None and prune_mask is None:
+        prune_mask = torch.empty((n + 31) // 32, dtype=torch.int32, device=grad.device)
+    r, b, l2 = ctypes.c_double(), ctypes.c_int(), ctypes.c_double()
+    rc = lib.nsml_compress_adaptive(grad.data_ptr(), n, dtype, float(ratio), float(tr_q), float(tr_d), int(plain_bits),
+                                    None if weights is None else weights.data_ptr(),
+                                    None if prune_mask is None else prune_mask.data_ptr(),
+                                    payload.data_ptr(), payload.numel(), workspace.data_ptr(), workspace.numel(),
+                                    _stream_ptr(stream), ctypes.byref(r), ctypes.byref(b), ctypes.byref(l2))
+    _check(rc, "nsml_compress_adaptive")
+    need = nsml_payload_bytes(n, r.value, b.value)
+    return payload[:need], r.value, b.value, (l2.value if l2.value >= 0.0 else None), prune_mask
+
+
 def nsml_last_status(workspace, stream=None) -> int:
     out = ctypes.c_int()
     _check(lib.nsml_last_status(workspace.data_ptr(), _stream_ptr(stream), ctypes.byref(out)), "nsml_last_status")
@@ -352,7 +464,7 @@ def _align16(x: int) -> int:
 
 def unpack_payload(payload) -> dict:
     """Split a payload (CUDA/CPU uint8 tensor, bytes or uint8 ndarray) into its
-    sections as numpy arrays: n, k, bits, idx, and codes+scales or half."""
+    sections as numpy arrays: n, k, bits, idx, and codes+scales, half or f32."""
     if hasattr(payload, "detach"):
         raw = payload.detach().cpu().numpy()
     else:
@@ -368,12 +480,14 @@ def unpack_payload(payload) -> dict:
     if bits == NSML_BITS_INT8:
         out["codes"] = raw[val_off:val_off + k].view(np.int8).copy()
         out["scales"] = raw[scale_off:scale_off + 4 * nblocks].view(np.float32).copy()
-    else:
+    elif bits == NSML_BITS_FP16:
         out["half"] = raw[val_off:val_off + 2 * k].view(np.uint16).copy()
+    else:
+        out["f32"] = raw[val_off:val_off + 4 * k].view(np.float32).copy()
     return out
 
 
-def pack_payload(n: int, bits: int, idx, codes=None, scales=None, half=None) -> np.ndarray:
+def pack_payload(n: int, bits: int, idx, codes=None, scales=None, half=None, f32=None) -> np.ndarray:
     """Lay out payload sections as nsml_compress would (uint8 ndarray)."""
     idx = np.ascontiguousarray(idx, dtype=np.uint32)
     k = idx.size
@@ -384,7 +498,7 @@ def pack_payload(n: int, bits: int, idx, codes=None, scales=None, half=None) -> 
         total = scale_off + _align16(4 * nblocks)
     else:
         nblocks, scale_off = 0, 0
-        total = val_off + _align16(2 * k)
+        total = val_off + _align16((4 if bits == NSML_BITS_FP32 else 2) * k)
     raw = np.zeros(total, dtype=np.uint8)
     raw[0:8].view(np.uint32)[:] = (NSML_PAYLOAD_MAGIC, 1)
     raw[8:24].view(np.uint64)[:] = (n, k)
@@ -394,8 +508,10 @@ def pack_payload(n: int, bits: int, idx, codes=None, scales=None, half=None) -> 
     if bits == NSML_BITS_INT8:
         raw[val_off:val_off + k] = np.ascontiguousarray(codes, dtype=np.int8).view(np.uint8)
         raw[scale_off:scale_off + 4 * nblocks] = np.ascontiguousarray(scales, dtype=np.float32).view(np.uint8)
-    else:
+    elif bits == NSML_BITS_FP16:
         raw[val_off:val_off + 2 * k] = np.ascontiguousarray(half, dtype=np.uint16).view(np.uint8)
+    else:
+        raw[val_off:val_off + 4 * k] = np.ascontiguousarray(f32, dtype=np.float32).view(np.uint8)
     return raw
 
 

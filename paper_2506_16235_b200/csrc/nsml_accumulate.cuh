@@ -37,7 +37,7 @@ inline AccumulateLayout accumulate_layout(int64_t n, int W) {
 __device__ inline bool header_ok(const nsml_payload_header* h, unsigned long long n) {
   if (h->magic != NSML_PAYLOAD_MAGIC || h->version != NSML_PAYLOAD_VERSION) return false;
   if (h->n != n || h->k < 1 || h->k > n || h->qblock != NSML_QBLOCK) return false;
-  if (h->bits != NSML_BITS_INT8 && h->bits != NSML_BITS_FP16) return false;
+  if (h->bits != NSML_BITS_INT8 && h->bits != NSML_BITS_FP16 && h->bits != NSML_BITS_FP32) return false;
   const unsigned long long k = h->k;
   const unsigned long long val_off = 64 + (k * 4 + 15) / 16 * 16;
   if (h->idx_off != 64 || h->val_off != val_off) return false;
@@ -117,7 +117,7 @@ k_partition_wide(PayloadTable table, int W, unsigned long long n, unsigned int t
 // What a block needs to know about one worker's payload, read from its header once per block.
 struct WorkerView {
   const uint32_t* idx;
-  const unsigned char* val;  // int8 codes or binary16 bit patterns
+  const unsigned char* val;  // int8 codes, binary16 bit patterns or float32 values
   const float* scale;
   int bits;
 };
@@ -237,8 +237,10 @@ k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long
             if (v.bits == NSML_BITS_INT8) {
               raw_val[u] = reinterpret_cast<const signed char*>(v.val)[j];
               raw_scale[u] = v.scale[j >> 10];
-            } else {
+            } else if (v.bits == NSML_BITS_FP16) {
               raw_val[u] = reinterpret_cast<const uint16_t*>(v.val)[j];
+            } else {
+              raw_val[u] = reinterpret_cast<const int*>(v.val)[j];  // float32 bit pattern
             }
           }
           c += kCta;
@@ -253,8 +255,9 @@ k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long
         if (unit_w[u] >= W) break;
         if (raw_idx[u] != 0xFFFFFFFFu) {
           const unsigned long long o = (unsigned long long)raw_idx[u] - lo;  // wraps if idx < lo
-          const float v = unit_bits[u] == NSML_BITS_INT8 ? decode_i8(raw_val[u], raw_scale[u])
-                                                         : decode_f16((uint16_t)raw_val[u]);
+          const float v = unit_bits[u] == NSML_BITS_INT8   ? decode_i8(raw_val[u], raw_scale[u])
+                          : unit_bits[u] == NSML_BITS_FP16 ? decode_f16((uint16_t)raw_val[u])
+                                                           : __int_as_float(raw_val[u]);
           if (o < len) acc[o] += v; else bad = true;
         }
         if (u + 1 == kMergeUnits || unit_w[u + 1] != unit_w[u]) __syncthreads();  // uniform over the block

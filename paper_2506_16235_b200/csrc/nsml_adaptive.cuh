@@ -1,0 +1,418 @@
+// The steps of Alg. 2 around the top-k selection:
+//   Step 1  the gradient's L2 norm for the adaptive-quantisation gate (k_sumsq)
+//   Step 2  the pruning mask built from the weights: the ceil(0.5*(1-ratio)*n)
+//           parameters of smallest magnitude, ties by lower index
+//           (k_prune_hist, k_prune_ties, k_prune_write)
+//   Step 3  "accumulate the local filtered gradients": the bucket that is
+//           compressed is gradient + residual, and the residual keeps what the
+//           payload does not carry (k_feedback_add, k_feedback_subtract)
+// All of them stream the bucket with 16-byte loads, block-cyclically, so that
+// the grid reads one moving window of memory.
+#pragma once
+
+#include "nsml_accumulate.cuh"
+#include "nsml_codec.cuh"
+#include "nsml_common.cuh"
+#include "nsml_select.cuh"
+
+namespace nsml {
+
+constexpr int kStreamTile = kCta * 16;  // elements a block takes per step: four 4-element loads per thread
+
+// ------------------------------------------------------------------------
+// Step 1: sum of squares in float64.  Every square is exact in float64 (a
+// float32 has 24 significant bits), the adds follow a fixed order for a given
+// grid (per thread, per warp, per block, then the last block to finish adds
+// the per-block sums in block order), so the result is reproducible.
+// ------------------------------------------------------------------------
+struct SumsqCtl {
+  int status;
+  unsigned int ticket;  // blocks that have delivered their partial sum
+  double sumsq;
+};
+constexpr int kSumsqMaxBlocks = 4096;
+constexpr size_t kSumsqWorkspace = 256 + (size_t)kSumsqMaxBlocks * 8;
+
+__device__ __forceinline__ double block_sum_f64(double t, double* s_red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) t += __shfl_xor_sync(0xFFFFFFFFu, t, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) s_red[threadIdx.x >> 5] = t;
+  __syncthreads();
+  double b = 0.0;
+#pragma unroll
+  for (int w = 0; w < kCta / 32; ++w) b += s_red[w];
+  return b;
+}
+
+template <int DTYPE>
+__global__ void __launch_bounds__(kCta)
+k_sumsq(BucketSrc<DTYPE> src, unsigned long long n, SumsqCtl* ctl, double* __restrict__ partials) {
+  __shared__ double s_red[kCta / 32];
+  __shared__ unsigned int s_last;
+  const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
+  double acc[4] = {0.0, 0.0, 0.0, 0.0};
+  uint32_t worst = 0;  // largest magnitude key seen
+  for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    const unsigned long long base = tile * kStreamTile;
+    uint32_t bits[4][4];
+    if (base + kStreamTile <= n) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) src.load_full4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, bits[u]);
+    } else {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) src.load_vals4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, n, bits[u]);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const double v = (double)__uint_as_float(bits[u][e]);
+        acc[u] = fma(v, v, acc[u]);  // the product is exact, so this is one rounding, of the add
+        worst = max(worst, bits[u][e] & 0x7FFFFFFFu);
+      }
+    }
+  }
+  if (worst >= kInfKey) set_status(&ctl->status, NSML_ERR_NONFINITE);
+  const double block_total = block_sum_f64((acc[0] + acc[1]) + (acc[2] + acc[3]), s_red);
+  if (threadIdx.x == 0) {
+    partials[blockIdx.x] = block_total;
+    __threadfence();
+    s_last = atomicAdd(&ctl->ticket, 1u) == gridDim.x - 1;
+  }
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();  // the other blocks' partial sums are visible
+  double p = 0.0;
+  for (unsigned int i = threadIdx.x; i < gridDim.x; i += kCta) p += __ldcg(partials + i);
+  const double total = block_sum_f64(p, s_red);
+  if (threadIdx.x == 0) {
+    ctl->sumsq = total;
+    ctl->ticket = 0;
+  }
+}
+
+// ------------------------------------------------------------------------
+// Step 3, local accumulation.  residual <- gradient + residual (one float32
+// add per element); the sum is what gets compressed.
+// ------------------------------------------------------------------------
+template <int DTYPE>
+__global__ void __launch_bounds__(kCta)
+k_feedback_add(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned long long n) {
+  const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
+  for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    const unsigned long long base = tile * kStreamTile;
+    if (base + kStreamTile <= n) {
+      uint32_t g[4][4];
+      float4 r[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const unsigned long long i0 = base + (unsigned long long)(u * kCta + threadIdx.x) * 4;
+        src.load_full4(i0, g[u]);
+        r[u] = *reinterpret_cast<const float4*>(residual + i0);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const unsigned long long i0 = base + (unsigned long long)(u * kCta + threadIdx.x) * 4;
+        float4 s;
+        s.x = __fadd_rn(__uint_as_float(g[u][0]), r[u].x);
+        s.y = __fadd_rn(__uint_as_float(g[u][1]), r[u].y);
+        s.z = __fadd_rn(__uint_as_float(g[u][2]), r[u].z);
+        s.w = __fadd_rn(__uint_as_float(g[u][3]), r[u].w);
+        *reinterpret_cast<float4*>(residual + i0) = s;
+      }
+    } else {
+      for (unsigned long long i = base + threadIdx.x; i < n; i += kCta)
+        residual[i] = __fadd_rn(__uint_as_float(src.load1(i)), residual[i]);
+    }
+  }
+}
+
+// residual[idx_j] <- residual[idx_j] - v'_j for every payload entry, v' being the
+// value a receiver reconstructs (one float32 subtraction).  Indices are unique,
+// so entries do not interfere.
+__global__ void __launch_bounds__(kCta)
+k_feedback_subtract(const unsigned char* __restrict__ payload, float* __restrict__ residual, unsigned long long n,
+                    int* status) {
+  const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(payload);
+  if (!header_ok(h, n)) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) set_status(status, NSML_ERR_PAYLOAD);
+    return;
+  }
+  const unsigned long long k = h->k;
+  const uint32_t* idx = reinterpret_cast<const uint32_t*>(payload + h->idx_off);
+  const unsigned char* val = payload + h->val_off;
+  const float* scale = reinterpret_cast<const float*>(payload + h->scale_off);
+  const int bits = (int)h->bits;
+  for (unsigned long long j = (unsigned long long)blockIdx.x * kCta + threadIdx.x; j < k;
+       j += (unsigned long long)gridDim.x * kCta) {
+    const uint32_t i = idx[j];
+    float v;
+    if (bits == NSML_BITS_INT8) v = decode_i8(reinterpret_cast<const signed char*>(val)[j], scale[j >> 10]);
+    else if (bits == NSML_BITS_FP16) v = decode_f16(reinterpret_cast<const uint16_t*>(val)[j]);
+    else v = reinterpret_cast<const float*>(val)[j];
+    if (i < n) residual[i] = __fsub_rn(residual[i], v);
+    else set_status(status, NSML_ERR_PAYLOAD);
+  }
+}
+
+// ------------------------------------------------------------------------
+// Step 2: pruning mask from the weights.  The m parameters of smallest
+// magnitude, ties by lower index, are the m LARGEST under the complemented
+// key (~bits & 0x7FFFFFFF) with the same tie rule, so this is the radix select
+// of the top-k step on complemented keys: three histogram passes (12 + 12 + 7
+// bits; each pass first resolves the previous level from the global
+// histogram, every block for itself), an optional pass that counts the keys
+// equal to the threshold per tile (needed only when not all of them are
+// pruned), and the pass that writes the mask bits.
+// ------------------------------------------------------------------------
+struct PruneCtl {
+  int status;
+  unsigned int d0, rem1;       // digit 0 of the threshold, rank left inside its bin
+  unsigned int prefix24, rem2; // digits 0-1, rank left
+  unsigned int T, r, cT;       // threshold key (complemented), ties to prune, ties in all
+};
+
+struct PruneLayout {
+  size_t hist;       // u32[3][kMaxBins]
+  size_t tile_ties;  // u32[tiles]
+  size_t total;
+};
+
+inline PruneLayout prune_layout(int64_t n) {
+  PruneLayout L;
+  const size_t tiles = ((size_t)n + kStreamTile - 1) / kStreamTile;
+  L.hist = 256;
+  L.tile_ties = L.hist + 3 * kMaxBins * sizeof(unsigned int);
+  L.total = L.tile_ties + align_up(tiles * 4, 256);
+  return L;
+}
+
+__device__ __forceinline__ uint32_t prune_key(uint32_t bits) { return ~bits & 0x7FFFFFFFu; }
+
+// Loads the block's share of one tile: bits[u][e] = element base + (u*kCta + t)*4 + e, cnt[u] of them exist.
+__device__ __forceinline__ void load_tile(const BucketSrc<NSML_F32>& src, unsigned long long base, unsigned long long n,
+                                          uint32_t (&bits)[4][4], int (&cnt)[4]) {
+  if (base + kStreamTile <= n) {
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      src.load_full4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, bits[u]);
+      cnt[u] = 4;
+    }
+  } else {
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+      cnt[u] = src.load_vals4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, n, bits[u]);
+  }
+}
+
+// Resolves one level from its global histogram; every thread returns (digit, rank left).
+template <int NB>
+__device__ __forceinline__ void prune_resolve(const unsigned int* ghist, unsigned int rem, unsigned int* s_tot,
+                                              unsigned int* s_out) {
+  constexpr int PER = (NB + kCta - 1) / kCta;
+  unsigned int own[PER];
+#pragma unroll
+  for (int b = 0; b < PER; ++b) {
+    const int bin = threadIdx.x * PER + b;
+    own[b] = (bin < NB) ? ghist[bin] : 0u;
+  }
+  find_digit_from_top<PER, kCta>(own, rem, s_tot, s_out);
+}
+
+template <int LEVEL>
+__global__ void __launch_bounds__(kCta)
+k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, PruneCtl* ctl, unsigned int* __restrict__ hist) {
+  constexpr int NB = (LEVEL == 2) ? 128 : kMaxBins;
+  __shared__ unsigned int s_hist[NB];
+  __shared__ unsigned int s_tot[kCta / 32], s_out[2];
+  unsigned int prefix = 0;
+  if (LEVEL == 1) {
+    prune_resolve<kMaxBins>(hist, m, s_tot, s_out);
+    prefix = s_out[0];
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      ctl->d0 = s_out[0];
+      ctl->rem1 = s_out[1];
+    }
+  } else if (LEVEL == 2) {
+    prune_resolve<kMaxBins>(hist + kMaxBins, ctl->rem1, s_tot, s_out);
+    prefix = (ctl->d0 << 12) | s_out[0];
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+      ctl->prefix24 = prefix;
+      ctl->rem2 = s_out[1];
+    }
+  }
+  for (int b = threadIdx.x; b < NB; b += kCta) s_hist[b] = 0;
+  __syncthreads();
+  const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
+  bool nonfinite = false;
+  for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    uint32_t bits[4][4];
+    int cnt[4];
+    load_tile(src, tile * kStreamTile, n, bits, cnt);
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (e < cnt[u]) {
+          const uint32_t key = prune_key(bits[u][e]);
+          if (LEVEL == 0) {
+            nonfinite |= key <= 0x007FFFFFu;  // magnitude bits >= 0x7F800000
+            atomicAdd(&s_hist[key >> 19], 1u);
+          } else if (LEVEL == 1) {
+            if ((key >> 19) == prefix) atomicAdd(&s_hist[(key >> 7) & 0xFFFu], 1u);
+          } else {
+            if ((key >> 7) == prefix) atomicAdd(&s_hist[key & 0x7Fu], 1u);
+          }
+        }
+      }
+    }
+  }
+  if (nonfinite) set_status(&ctl->status, NSML_ERR_NONFINITE);
+  __syncthreads();
+  unsigned int* ghist = hist + LEVEL * kMaxBins;
+  for (int b = threadIdx.x; b < NB; b += kCta) {
+    const unsigned int c = s_hist[b];
+    if (c) atomicAdd(&ghist[b], c);
+  }
+}
+
+// Resolves the last digit: threshold T, ties to prune r, ties in all cT.  When r < cT the ties are pruned
+// in index order, which needs their count per tile.
+__global__ void __launch_bounds__(kCta)
+k_prune_ties(BucketSrc<NSML_F32> src, unsigned long long n, PruneCtl* ctl, const unsigned int* __restrict__ hist,
+             unsigned int* __restrict__ tile_ties) {
+  __shared__ unsigned int s_tot[kCta / 32], s_out[2];
+  __shared__ unsigned int s_cnt[kCta / 32];
+  prune_resolve<128>(hist + 2 * kMaxBins, ctl->rem2, s_tot, s_out);
+  const uint32_t T = (ctl->prefix24 << 7) | s_out[0];
+  const unsigned int r = s_out[1], cT = hist[2 * kMaxBins + s_out[0]];
+  if (blockIdx.x == 0 && threadIdx.x == 0) {
+    ctl->T = T;
+    ctl->r = r;
+    ctl->cT = cT;
+  }
+  if (r >= cT) return;  // every key equal to T is pruned: no ranks needed
+  const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
+  for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    uint32_t bits[4][4];
+    int cnt[4];
+    load_tile(src, tile * kStreamTile, n, bits, cnt);
+    unsigned int c = 0;
+#pragma unroll
+    for (int u = 0; u < 4; ++u)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) c += (e < cnt[u]) && prune_key(bits[u][e]) == T;
+    c = __reduce_add_sync(0xFFFFFFFFu, c);
+    __syncthreads();  // s_cnt of the previous tile has been read
+    if ((threadIdx.x & 31) == 0) s_cnt[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      unsigned int t = 0;
+#pragma unroll
+      for (int w = 0; w < kCta / 32; ++w) t += s_cnt[w];
+      tile_ties[tile] = t;
+    }
+  }
+}
+
+// Writes the mask: bit (i & 31) of word i >> 5 set = parameter i pruned.  Bits past n in the last word are 0.
+__global__ void __launch_bounds__(kCta)
+k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl, const unsigned int* __restrict__ tile_ties,
+              uint32_t* __restrict__ mask) {
+  __shared__ unsigned int s_scan[kCta / 32];
+  __shared__ unsigned long long s_red[kCta / 32];
+  const uint32_t T = ctl->T;
+  const unsigned int r = ctl->r, cT = ctl->cT;
+  const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
+  const unsigned long long nwords = (n + 31) / 32;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  if (r >= cT) {
+    // every key >= T is pruned.  A warp's load covers 128 consecutive elements = 4 mask words; the 4-bit
+    // flags of 8 neighbouring lanes are combined into one word.
+    for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+      const unsigned long long base = tile * kStreamTile;
+      uint32_t bits[4][4];
+      int cnt[4];
+      load_tile(src, base, n, bits, cnt);
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        unsigned int f = 0;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) f |= (unsigned)((e < cnt[u]) && prune_key(bits[u][e]) >= T) << e;
+        unsigned int x = f << (4 * (lane & 7));
+        x |= __shfl_xor_sync(0xFFFFFFFFu, x, 1);
+        x |= __shfl_xor_sync(0xFFFFFFFFu, x, 2);
+        x |= __shfl_xor_sync(0xFFFFFFFFu, x, 4);
+        const unsigned long long word = (base + (unsigned long long)(u * kCta + warp * 32) * 4) / 32 + (lane >> 3);
+        if ((lane & 7) == 0 && word < nwords) mask[word] = x;
+      }
+    }
+    return;
+  }
+  // Some of the keys equal to T stay unpruned: the first r of them in index order are pruned.  A block
+  // takes a contiguous range of tiles and carries the number of ties seen so far; within a tile a thread
+  // owns one mask word (32 consecutive elements).
+  const unsigned long long t_first = (unsigned long long)blockIdx.x * tiles / gridDim.x;
+  const unsigned long long t_last = (unsigned long long)(blockIdx.x + 1) * tiles / gridDim.x;
+  unsigned long long before = 0;
+  for (unsigned long long t = threadIdx.x; t < t_first; t += kCta) before += tile_ties[t];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xFFFFFFFFu, before, o);
+  if (lane == 0) s_red[warp] = before;
+  __syncthreads();
+  before = 0;
+#pragma unroll
+  for (int w = 0; w < kCta / 32; ++w) before += s_red[w];
+  constexpr int kWordsPerTile = kStreamTile / 32;  // 128: the first 128 threads own a word each
+  for (unsigned long long tile = t_first; tile < t_last; ++tile) {
+    const unsigned long long i0 = tile * kStreamTile + (unsigned long long)threadIdx.x * 32;
+    uint32_t key[32];
+    unsigned int ties = 0;
+    const bool owner = threadIdx.x < kWordsPerTile && i0 < n;
+    if (owner) {
+#pragma unroll
+      for (int q = 0; q < 8; ++q) {
+        uint32_t b4[4];
+        const int c = src.load_vals4(i0 + q * 4, n, b4);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          key[q * 4 + e] = (e < c) ? prune_key(b4[e]) : 0u;  // key 0 = missing (a real key 0 would be NaN)
+          ties += (e < c) && key[q * 4 + e] == T;
+        }
+      }
+    }
+    // exclusive scan of the per-thread tie counts over the block
+    unsigned int incl = ties;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    __syncthreads();  // s_scan of the previous tile has been read
+    if (lane == 31) s_scan[warp] = incl;
+    __syncthreads();
+    unsigned int warps_before = 0, all = 0;
+#pragma unroll
+    for (int w = 0; w < kCta / 32; ++w) {
+      const unsigned int c = s_scan[w];
+      if (w < warp) warps_before += c;
+      all += c;
+    }
+    if (owner) {
+      unsigned long long rank = before + warps_before + incl - ties;
+      uint32_t word = 0;
+#pragma unroll
+      for (int e = 0; e < 32; ++e) {
+        const bool tie = key[e] == T && T != 0u;
+        const bool pruned = key[e] > T || (tie && rank < r);
+        rank += tie;
+        word |= (uint32_t)pruned << e;
+      }
+      mask[i0 / 32] = word;
+    }
+    before += all;
+  }
+}
+
+}  // namespace nsml

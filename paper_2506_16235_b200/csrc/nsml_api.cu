@@ -7,6 +7,7 @@
 #include <vector>
 
 #include "nsml_accumulate.cuh"
+#include "nsml_adaptive.cuh"
 #include "nsml_codec.cuh"
 #include "nsml_common.cuh"
 #include "nsml_compact.cuh"
@@ -16,10 +17,14 @@
 
 namespace nsml {
 
-enum KernelId { K_SAMPLE = 0, K_COMPACT_BUCKET, K_FINALIZE, K_PARTITION, K_MERGE, K_CLEAR, K_FINALIZE_DENSE, K_COUNT };
+enum KernelId {
+  K_SAMPLE = 0, K_COMPACT_BUCKET, K_FINALIZE, K_PARTITION, K_MERGE, K_CLEAR, K_FINALIZE_DENSE,
+  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_COUNT
+};
 
 static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_compact_bucket", "k_finalize", "k_partition", "k_merge",
-                                                  "k_clear", "k_finalize_dense"};
+                                                  "k_clear", "k_finalize_dense", "k_sumsq", "k_feedback_add",
+                                                  "k_feedback_subtract", "k_prune_hist", "k_prune_ties", "k_prune_write"};
 
 static std::atomic<int64_t> g_launches{0};
 
@@ -113,6 +118,7 @@ static int device_info(const DeviceInfo** out) {
   return NSML_OK;
 }
 
+static inline bool valid_bits(int bits) { return bits == NSML_BITS_INT8 || bits == NSML_BITS_FP16 || bits == NSML_BITS_FP32; }
 static inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 static inline unsigned int grid_for(unsigned long long work_items, unsigned long long per_block, int cap) {
@@ -257,7 +263,7 @@ static int compress_impl(const void* grad, int64_t n, int grad_dtype, double rat
                          size_t workspace_bytes, cudaStream_t st) {
   if (grad == nullptr || payload == nullptr || workspace == nullptr) return NSML_ERR_ARG;
   if (grad_dtype != NSML_F32 && grad_dtype != NSML_BF16) return NSML_ERR_ARG;
-  if (bits != NSML_BITS_INT8 && bits != NSML_BITS_FP16) return NSML_ERR_ARG;
+  if (!valid_bits(bits)) return NSML_ERR_ARG;
   const int64_t k = k_of(n, ratio);
   if (k == 0) return NSML_ERR_ARG;
   if (!aligned(grad, 16) || !aligned(payload, 16) || !aligned(workspace, 256)) return NSML_ERR_ARG;
@@ -318,6 +324,156 @@ static int accumulate_impl(const void* const* payloads, int W, float* dense, int
   return NSML_OK;
 }
 
+// ---- Alg. 2 Step 1: L2 norm and gate ----------------------------------------
+// Blocks of the streaming kernels of nsml_adaptive.cuh: enough to keep every SM's loads in flight.
+static unsigned int stream_grid(int64_t n, const DeviceInfo& dev, int per_sm, unsigned int cap) {
+  unsigned int g = grid_for(((unsigned long long)n + kStreamTile - 1) / kStreamTile, 1, dev.sms * per_sm);
+  return g < cap ? g : cap;
+}
+
+static int sumsq_impl(const void* grad, int64_t n, int grad_dtype, void* workspace, size_t workspace_bytes,
+                      cudaStream_t st) {
+  if (grad == nullptr || workspace == nullptr) return NSML_ERR_ARG;
+  if (grad_dtype != NSML_F32 && grad_dtype != NSML_BF16) return NSML_ERR_ARG;
+  if (n < 1 || n > NSML_MAX_N) return NSML_ERR_ARG;
+  if (!aligned(grad, 16) || !aligned(workspace, 256)) return NSML_ERR_ARG;
+  if (workspace_bytes < kSumsqWorkspace) return NSML_ERR_CAPACITY;
+  const DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != NSML_OK) return rc;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  if (cudaMemsetAsync(ws, 0, 256, st) != cudaSuccess) return NSML_ERR_CUDA;
+  SumsqCtl* ctl = reinterpret_cast<SumsqCtl*>(ws);
+  double* partials = reinterpret_cast<double*>(ws + 256);
+  const unsigned int grid = stream_grid(n, *dev, 8, kSumsqMaxBlocks);
+  {
+    LaunchScope scope(K_SUMSQ, st);
+    if (grad_dtype == NSML_F32)
+      k_sumsq<NSML_F32><<<grid, kCta, 0, st>>>(BucketSrc<NSML_F32>{grad, nullptr}, (unsigned long long)n, ctl, partials);
+    else
+      k_sumsq<NSML_BF16><<<grid, kCta, 0, st>>>(BucketSrc<NSML_BF16>{grad, nullptr}, (unsigned long long)n, ctl, partials);
+  }
+  if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
+  return NSML_OK;
+}
+
+// Synchronises the stream and reads the status word and the sum of squares left by sumsq_impl.
+static int sumsq_read(const void* workspace, cudaStream_t st, double* sumsq) {
+  SumsqCtl host;
+  if (cudaMemcpyAsync(&host, workspace, sizeof(host), cudaMemcpyDeviceToHost, st) != cudaSuccess) return NSML_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return NSML_ERR_CUDA;
+  if (host.status != NSML_OK) return host.status;
+  *sumsq = host.sumsq;
+  return NSML_OK;
+}
+
+static int gate(double ratio, double l2, double tr_q, double tr_d, int plain_bits, double* ratio_out, int* bits_out) {
+  if (!(ratio > 0.0) || !(ratio <= 1.0) || !valid_bits(plain_bits) || !(l2 >= 0.0) || tr_q != tr_q || tr_d != tr_d)
+    return NSML_ERR_ARG;
+  if (ratio < tr_q && l2 > tr_d) {
+    const double doubled = 2.0 * ratio;
+    *ratio_out = doubled < 1.0 ? doubled : 1.0;
+    *bits_out = NSML_BITS_FP16;
+  } else {
+    *ratio_out = ratio;
+    *bits_out = plain_bits;
+  }
+  return NSML_OK;
+}
+
+// ---- Alg. 2 Step 2: pruning mask from the weights ---------------------------
+static int64_t pruned_count(int64_t n, double ratio) {
+  if (n < 1 || n > NSML_MAX_N || !(ratio > 0.0) || !(ratio <= 1.0)) return -1;
+  const double rate = 0.5 * (1.0 - ratio);
+  int64_t m = (int64_t)std::ceil(rate * (double)n);
+  if (m < 0) m = 0;
+  if (m > n) m = n;
+  return m;
+}
+
+static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* mask, void* workspace,
+                      size_t workspace_bytes, cudaStream_t st) {
+  if (weights == nullptr || mask == nullptr || workspace == nullptr) return NSML_ERR_ARG;
+  const int64_t m = pruned_count(n, ratio);
+  if (m < 0) return NSML_ERR_ARG;
+  if (!aligned(weights, 16) || !aligned(mask, 4) || !aligned(workspace, 256)) return NSML_ERR_ARG;
+  const PruneLayout L = prune_layout(n);
+  if (workspace_bytes < L.total) return NSML_ERR_CAPACITY;
+  const DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != NSML_OK) return rc;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  if (cudaMemsetAsync(ws, 0, L.tile_ties, st) != cudaSuccess) return NSML_ERR_CUDA;  // status, ctl, histograms
+  if (m == 0) {  // ratio 1: nothing is pruned
+    if (cudaMemsetAsync(mask, 0, (size_t)((n + 31) / 32) * 4, st) != cudaSuccess) return NSML_ERR_CUDA;
+    return NSML_OK;
+  }
+  PruneCtl* ctl = reinterpret_cast<PruneCtl*>(ws);
+  unsigned int* hist = reinterpret_cast<unsigned int*>(ws + L.hist);
+  unsigned int* tile_ties = reinterpret_cast<unsigned int*>(ws + L.tile_ties);
+  const BucketSrc<NSML_F32> src{weights, nullptr};
+  const unsigned int grid = stream_grid(n, *dev, 6, 1u << 16);
+  const unsigned long long un = (unsigned long long)n;
+  {
+    LaunchScope scope(K_PRUNE_HIST, st);
+    k_prune_hist<0><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist);
+  }
+  {
+    LaunchScope scope(K_PRUNE_HIST, st);
+    k_prune_hist<1><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist);
+  }
+  {
+    LaunchScope scope(K_PRUNE_HIST, st);
+    k_prune_hist<2><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist);
+  }
+  {
+    LaunchScope scope(K_PRUNE_TIES, st);
+    k_prune_ties<<<grid, kCta, 0, st>>>(src, un, ctl, hist, tile_ties);
+  }
+  {
+    LaunchScope scope(K_PRUNE_WRITE, st);
+    k_prune_write<<<grid, kCta, 0, st>>>(src, un, ctl, tile_ties, mask);
+  }
+  if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
+  return NSML_OK;
+}
+
+// ---- Section 4.2 Step 3: local accumulation of the filtered gradients ---------
+static int feedback_impl(const void* grad, float* residual, int64_t n, int grad_dtype, double ratio, int bits,
+                         const uint32_t* prune_mask, void* payload, size_t payload_capacity, void* workspace,
+                         size_t workspace_bytes, cudaStream_t st) {
+  if (grad == nullptr || residual == nullptr) return NSML_ERR_ARG;
+  if (grad_dtype != NSML_F32 && grad_dtype != NSML_BF16) return NSML_ERR_ARG;
+  const int64_t k = k_of(n, ratio);
+  if (k == 0 || !valid_bits(bits)) return NSML_ERR_ARG;
+  if (!aligned(grad, 16) || !aligned(residual, 16)) return NSML_ERR_ARG;
+  if (payload == nullptr || workspace == nullptr || !aligned(payload, 16) || !aligned(workspace, 256)) return NSML_ERR_ARG;
+  if (payload_capacity < payload_layout(k, bits).total || workspace_bytes < compress_layout(n).total)
+    return NSML_ERR_CAPACITY;
+  const DeviceInfo* dev = nullptr;
+  int rc = device_info(&dev);
+  if (rc != NSML_OK) return rc;
+  const unsigned int grid = stream_grid(n, *dev, 8, 1u << 16);
+  {
+    LaunchScope scope(K_FEEDBACK_ADD, st);
+    if (grad_dtype == NSML_F32)
+      k_feedback_add<NSML_F32><<<grid, kCta, 0, st>>>(BucketSrc<NSML_F32>{grad, nullptr}, residual, (unsigned long long)n);
+    else
+      k_feedback_add<NSML_BF16><<<grid, kCta, 0, st>>>(BucketSrc<NSML_BF16>{grad, nullptr}, residual, (unsigned long long)n);
+  }
+  rc = compress_impl(residual, n, NSML_F32, ratio, bits, prune_mask, payload, payload_capacity, workspace,
+                     workspace_bytes, st);
+  if (rc != NSML_OK) return rc;
+  {
+    LaunchScope scope(K_FEEDBACK_SUBTRACT, st);
+    const unsigned int sgrid = grid_for((unsigned long long)k, kCta, dev->sms * 8);
+    k_feedback_subtract<<<sgrid, kCta, 0, st>>>(static_cast<const unsigned char*>(payload), residual,
+                                                (unsigned long long)n, static_cast<int*>(workspace));
+  }
+  if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
+  return NSML_OK;
+}
+
 // ---- scratch for nsml_decompress_accumulate_static --------------------------
 // Part of the library image: every device that loads the library holds this
 // array until exit.  In host code the name below is only a handle; the device
@@ -361,7 +517,7 @@ int nsml_compress_strategy(int64_t n, double ratio) {
 }
 
 size_t nsml_payload_bytes(int64_t n, double ratio, int bits) {
-  if (bits != NSML_BITS_INT8 && bits != NSML_BITS_FP16) return 0;
+  if (!valid_bits(bits)) return 0;
   const int64_t k = k_of(n, ratio);
   if (k == 0) return 0;
   return payload_layout(k, bits).total;
@@ -405,6 +561,105 @@ int nsml_decompress_accumulate_static(const void* const* payloads, int W, float*
   if (cudaStreamSynchronize(st) != cudaSuccess) return NSML_ERR_CUDA;
   *status_out = value;
   return NSML_OK;
+}
+
+// ---- Alg. 2 Steps 1-2 and the local accumulation of Step 3 --------------------
+size_t nsml_l2_workspace_bytes(void) { return kSumsqWorkspace; }
+
+int nsml_grad_l2(const void* grad, int64_t n, int grad_dtype, void* workspace, size_t workspace_bytes, void* stream,
+                 double* l2_out) {
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  int rc = sumsq_impl(grad, n, grad_dtype, workspace, workspace_bytes, st);
+  if (rc != NSML_OK || l2_out == nullptr) return rc;
+  double sumsq = 0.0;
+  rc = sumsq_read(workspace, st, &sumsq);
+  if (rc != NSML_OK) return rc;
+  *l2_out = std::sqrt(sumsq);
+  return NSML_OK;
+}
+
+int nsml_quantize_gate(double ratio, double l2, double tr_q, double tr_d, int plain_bits, double* ratio_out,
+                       int* bits_out) {
+  if (ratio_out == nullptr || bits_out == nullptr) return NSML_ERR_ARG;
+  return gate(ratio, l2, tr_q, tr_d, plain_bits, ratio_out, bits_out);
+}
+
+int64_t nsml_pruned_count(int64_t n, double ratio) {
+  const int64_t m = pruned_count(n, ratio);
+  return m < 0 ? 0 : m;
+}
+
+size_t nsml_prune_workspace_bytes(int64_t n) {
+  if (n < 1 || n > NSML_MAX_N) return 0;
+  return prune_layout(n).total;
+}
+
+int nsml_prune_mask_build(const float* weights, int64_t n, double ratio, uint32_t* prune_mask, void* workspace,
+                          size_t workspace_bytes, void* stream) {
+  return prune_impl(weights, n, ratio, prune_mask, workspace, workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+int nsml_compress_feedback(const void* grad, float* residual, int64_t n, int grad_dtype, double ratio, int bits,
+                           const uint32_t* prune_mask, void* payload, size_t payload_capacity, void* workspace,
+                           size_t workspace_bytes, void* stream) {
+  return feedback_impl(grad, residual, n, grad_dtype, ratio, bits, prune_mask, payload, payload_capacity, workspace,
+                       workspace_bytes, static_cast<cudaStream_t>(stream));
+}
+
+size_t nsml_adaptive_payload_bytes(int64_t n, double ratio, double tr_q, int plain_bits) {
+  size_t need = nsml_payload_bytes(n, ratio, plain_bits);
+  if (need == 0) return 0;
+  if (ratio < tr_q) {
+    const double doubled = 2.0 * ratio;
+    const size_t q = nsml_payload_bytes(n, doubled < 1.0 ? doubled : 1.0, NSML_BITS_FP16);
+    if (q > need) need = q;
+  }
+  return need;
+}
+
+size_t nsml_adaptive_workspace_bytes(int64_t n, int grad_dtype) {
+  size_t need = nsml_workspace_bytes(n, grad_dtype);
+  if (need == 0) return 0;
+  if (need < kSumsqWorkspace) need = kSumsqWorkspace;
+  const size_t p = prune_layout(n).total;
+  return need < p ? p : need;
+}
+
+int nsml_compress_adaptive(const void* grad, int64_t n, int grad_dtype, double ratio, double tr_q, double tr_d,
+                           int plain_bits, const float* weights, uint32_t* prune_mask, void* payload,
+                           size_t payload_capacity, void* workspace, size_t workspace_bytes, void* stream,
+                           double* ratio_used, int* bits_used, double* l2_out) {
+  if (ratio_used == nullptr || bits_used == nullptr) return NSML_ERR_ARG;
+  if (!(ratio > 0.0) || !(ratio <= 1.0) || !valid_bits(plain_bits) || tr_q != tr_q || tr_d != tr_d) return NSML_ERR_ARG;
+  if (weights != nullptr && prune_mask == nullptr) return NSML_ERR_ARG;
+  const size_t need_ws = nsml_adaptive_workspace_bytes(n, grad_dtype);
+  if (need_ws == 0) return NSML_ERR_ARG;
+  if (workspace_bytes < need_ws) return NSML_ERR_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  // Step 1: the norm is needed only when the ratio is below the quantisation check threshold
+  double use_ratio = ratio, l2 = -1.0;
+  int use_bits = plain_bits;
+  if (ratio < tr_q) {
+    int rc = sumsq_impl(grad, n, grad_dtype, workspace, workspace_bytes, st);
+    if (rc != NSML_OK) return rc;
+    double sumsq = 0.0;
+    rc = sumsq_read(workspace, st, &sumsq);
+    if (rc != NSML_OK) return rc;
+    l2 = std::sqrt(sumsq);
+    rc = gate(ratio, l2, tr_q, tr_d, plain_bits, &use_ratio, &use_bits);
+    if (rc != NSML_OK) return rc;
+  }
+  if (l2_out != nullptr) *l2_out = l2;
+  *ratio_used = use_ratio;
+  *bits_used = use_bits;
+  // Step 2: the mask follows the ratio Step 1 left
+  if (weights != nullptr) {
+    const int rc = prune_impl(weights, n, use_ratio, prune_mask, workspace, workspace_bytes, st);
+    if (rc != NSML_OK) return rc;
+  }
+  // Step 3
+  return compress_impl(grad, n, grad_dtype, use_ratio, use_bits, prune_mask, payload, payload_capacity, workspace,
+                       workspace_bytes, st);
 }
 
 // ---- host-buffer variants --------------------------------------------------

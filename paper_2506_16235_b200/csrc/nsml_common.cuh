@@ -84,10 +84,10 @@ inline PayloadLayout payload_layout(int64_t k, int bits) {
     P.nblocks = (size_t)((k + NSML_QBLOCK - 1) / NSML_QBLOCK);
     P.scale_off = P.val_off + align_up((size_t)k, 16);
     P.total = P.scale_off + align_up(P.nblocks * 4, 16);
-  } else {
+  } else {  // fp16: 2 bytes per value; float32 as is: 4
     P.nblocks = 0;
     P.scale_off = 0;
-    P.total = P.val_off + align_up((size_t)k * 2, 16);
+    P.total = P.val_off + align_up((size_t)k * (bits == NSML_BITS_FP32 ? 4 : 2), 16);
   }
   return P;
 }

@@ -225,6 +225,15 @@ __device__ __forceinline__ void quantize_phase(const FinalizeParams& p, Finalize
         for (int e = 0; e < cnt; ++e) v[e] = __ldcg(p.raw_val + j0 + e);
       }
     }
+    if (p.bits == NSML_BITS_FP32) {  // values travel as they are (Alg. 2 when Step 1 does not quantise)
+      float* out = reinterpret_cast<float*>(p.payload + p.P.val_off);
+      if (cnt == 4) {
+        *reinterpret_cast<float4*>(out + j0) = make_float4(v[0], v[1], v[2], v[3]);
+      } else {
+        for (int e = 0; e < cnt; ++e) out[j0 + e] = v[e];
+      }
+      continue;
+    }
     if (p.bits == NSML_BITS_FP16) {
       uint16_t* out = reinterpret_cast<uint16_t*>(p.payload + p.P.val_off);
       if (cnt == 4) {

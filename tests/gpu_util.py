@@ -52,8 +52,10 @@ def assert_payload_equal(payload, want: oracle.Payload):
     if want.bits == 8:
         assert np.array_equal(got["scales"].view(np.uint32), want.scales.view(np.uint32)), "scales differ"
         assert np.array_equal(got["codes"], want.codes), "int8 codes differ"
-    else:
+    elif want.bits == 16:
         assert np.array_equal(got["half"], want.half), "fp16 bit patterns differ"
+    else:
+        assert np.array_equal(got["f32"].view(np.uint32), want.raw.view(np.uint32)), "float32 values differ"
     return got
 
 
@@ -66,7 +68,8 @@ def check_compress(g, ratio, bits, mask_bool=None):
 
 
 def payload_to_device(want: oracle.Payload) -> torch.Tensor:
-    raw = nsml.pack_payload(want.n, want.bits, want.idx, codes=want.codes, scales=want.scales, half=want.half)
+    raw = nsml.pack_payload(want.n, want.bits, want.idx, codes=want.codes, scales=want.scales, half=want.half,
+                            f32=want.raw if want.bits == 32 else None)
     return torch.from_numpy(raw).cuda()
 
 
