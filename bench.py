@@ -575,6 +575,70 @@ WORKLOADS = {"resnet50": ResnetWorkload, "gpt2": Gpt2Workload, "decoder": Decode
 # --------------------------------------------------------------------------
 # reference arm: the CPU oracle, timed as it stands
 # --------------------------------------------------------------------------
+def alg2_leg(nsml, torch, device, big, peak):
+    """The other steps of Alg. 2 on 25M-element buckets: L2 norm (Step 1), pruning mask from synthetic
+    Gaussian weights (Step 2), compress with local accumulation (Step 3), ratio 0.01, int8.  Inputs rotate
+    over sixteen gradient buckets and four weight / residual buffers (each 100 MB)."""
+    ratio, bits = 0.01, 8
+    n = big.sizes[0]
+    k = nsml.nsml_k_of(n, ratio)
+    grads = [big.workers[w][b] for b in range(len(big.sizes)) for w in range(big.W) if big.sizes[b] == n]
+    gen = torch.Generator(device=device)
+    gen.manual_seed(77)
+    weights = [torch.empty(n, device=device).normal_(0.0, 0.02, generator=gen) for _ in range(4)]
+    residual = [torch.zeros(n, device=device) for _ in range(4)]
+    lane = big.lanes.all[0]
+    l2ws = nsml.alloc_bytes(nsml.lib.nsml_l2_workspace_bytes(), device)
+    pws = nsml.alloc_bytes(nsml.nsml_prune_workspace_bytes(n), device)
+    mask = torch.empty((n + 31) // 32, dtype=torch.int32, device=device)
+
+    def one(i):
+        g = grads[i % len(grads)]
+        nsml.nsml_grad_l2(g, workspace=l2ws, sync=False)
+        nsml.nsml_prune_mask_build(weights[i % 4], ratio, prune_mask=mask, workspace=pws)
+        nsml.nsml_compress_feedback(g, residual[i % 4], ratio, bits, prune_mask=mask, payload=lane.payloads[0],
+                                    workspace=lane.ws)
+
+    for i in range(3):
+        one(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = 12
+    e0.record()
+    for i in range(reps):
+        one(3 + i)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / reps
+    nsml.nsml_prof_reset()
+    nsml.nsml_prof_enable(True)
+    for i in range(8):
+        one(i)
+    torch.cuda.synchronize()
+    prof = nsml.nsml_prof_read()
+    nsml.nsml_prof_enable(False)
+    per_launch = {  # algorithmic bytes per launch
+        "k_sumsq": 4 * n,
+        "k_prune_hist": 4 * n,
+        "k_prune_ties": 3 * 4096 * 4,
+        "k_prune_write": 4 * n + n // 8,
+        "k_feedback_add": 12 * n,
+        "k_feedback_subtract": 13 * k,
+        "k_sample": 4 * 8192,
+        "k_compact_bucket": 4 * n + n // 8 + 8 * k,
+        "k_finalize": 24 * k + 8 * k + 4 * k + k + 4 * ((k + 1023) // 1024),
+    }
+    per = {}
+    for name, (t, cnt) in prof.items():
+        if cnt and name in per_launch:
+            gbs = per_launch[name] * cnt / (t * 1e-3) / 1e9
+            per[name] = {"launches_per_step": cnt / 8, "us_per_launch": 1e3 * t / cnt, "algorithmic_GBps": gbs,
+                         "frac_of_peak": gbs / peak, "frac_of_nominal_8TBps": gbs / 8000.0}
+    return {"workload": "one 25M-element fp32 bucket per step: L2 norm, pruning mask from weights, compress with "
+                        "local accumulation (ratio 0.01, int8, mask applied), one stream, eager",
+            "value": 4.0 * n / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms, "kernels": per}
+
+
 def run_reference(args, rank):
     if rank != 0:
         return
@@ -794,6 +858,7 @@ def main():
         out["bucket_25M"] = {"workload": "four 25M-element fp32 buckets, ratio 0.01, int8, W=4 workers each",
                              "value": big.input_bytes_per_step / (big_ms * 1e-3) / 1e9, "unit": UNIT,
                              "ms_per_step": big_ms, "kernels": per}
+        out["alg2_25M"] = alg2_leg(nsml, torch, device, big, peak)
         del big
 
     if rank == 0 and not args.no_cpu_baseline:

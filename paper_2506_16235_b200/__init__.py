@@ -327,16 +327,18 @@ def _check_bucket(t, what="grad"):
         raise ValueError(f"{what} must be a contiguous 1-D CUDA tensor")
 
 
-def nsml_grad_l2(grad, workspace=None, stream=None) -> float:
-    """L2 norm of a bucket (Alg. 2 Step 1), float64; synchronises the stream."""
+def nsml_grad_l2(grad, workspace=None, stream=None, sync: bool = True):
+    """L2 norm of a bucket (Alg. 2 Step 1), float64.  sync=True synchronises the
+    stream and returns the norm; sync=False only enqueues (the float64 sum of
+    squares is then left at byte offset 8 of `workspace`) and returns None."""
     _check_bucket(grad)
     if workspace is None:
         workspace = alloc_bytes(lib.nsml_l2_workspace_bytes(), grad.device)
     out = ctypes.c_double()
     rc = lib.nsml_grad_l2(grad.data_ptr(), grad.numel(), _grad_dtype(grad), workspace.data_ptr(), workspace.numel(),
-                          _stream_ptr(stream), ctypes.byref(out))
+                          _stream_ptr(stream), ctypes.byref(out) if sync else None)
     _check(rc, "nsml_grad_l2")
-    return out.value
+    return out.value if sync else None
 
 
 def nsml_quantize_gate(ratio: float, l2: float, tr_q: float, tr_d: float, plain_bits: int = NSML_BITS_FP32):

@@ -17,7 +17,8 @@
 
 namespace nsml {
 
-constexpr int kStreamTile = kCta * 16;  // elements a block takes per step: four 4-element loads per thread
+constexpr int kStreamLoads = 4;  // 16-byte loads a thread keeps in flight
+constexpr int kStreamTile = kCta * 4 * kStreamLoads;  // elements a block takes per step
 
 // ------------------------------------------------------------------------
 // Step 1: sum of squares in float64.  Every square is exact in float64 (a
@@ -55,20 +56,20 @@ k_sumsq(BucketSrc<DTYPE> src, unsigned long long n, SumsqCtl* ctl, double* __res
   uint32_t worst = 0;  // largest magnitude key seen
   for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
     const unsigned long long base = tile * kStreamTile;
-    uint32_t bits[4][4];
+    uint32_t bits[kStreamLoads][4];
     if (base + kStreamTile <= n) {
 #pragma unroll
-      for (int u = 0; u < 4; ++u) src.load_full4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, bits[u]);
+      for (int u = 0; u < kStreamLoads; ++u) src.load_full4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, bits[u]);
     } else {
 #pragma unroll
-      for (int u = 0; u < 4; ++u) src.load_vals4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, n, bits[u]);
+      for (int u = 0; u < kStreamLoads; ++u) src.load_vals4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, n, bits[u]);
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kStreamLoads; ++u) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const double v = (double)__uint_as_float(bits[u][e]);
-        acc[u] = fma(v, v, acc[u]);  // the product is exact, so this is one rounding, of the add
+        acc[u & 3] = fma(v, v, acc[u & 3]);  // the product is exact, so this is one rounding, of the add
         worst = max(worst, bits[u][e] & 0x7FFFFFFFu);
       }
     }
@@ -103,16 +104,16 @@ k_feedback_add(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned long
   for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
     const unsigned long long base = tile * kStreamTile;
     if (base + kStreamTile <= n) {
-      uint32_t g[4][4];
-      float4 r[4];
+      uint32_t g[kStreamLoads][4];
+      float4 r[kStreamLoads];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < kStreamLoads; ++u) {
         const unsigned long long i0 = base + (unsigned long long)(u * kCta + threadIdx.x) * 4;
         src.load_full4(i0, g[u]);
         r[u] = *reinterpret_cast<const float4*>(residual + i0);
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < kStreamLoads; ++u) {
         const unsigned long long i0 = base + (unsigned long long)(u * kCta + threadIdx.x) * 4;
         float4 s;
         s.x = __fadd_rn(__uint_as_float(g[u][0]), r[u].x);
@@ -192,16 +193,16 @@ __device__ __forceinline__ uint32_t prune_key(uint32_t bits) { return ~bits & 0x
 
 // Loads the block's share of one tile: bits[u][e] = element base + (u*kCta + t)*4 + e, cnt[u] of them exist.
 __device__ __forceinline__ void load_tile(const BucketSrc<NSML_F32>& src, unsigned long long base, unsigned long long n,
-                                          uint32_t (&bits)[4][4], int (&cnt)[4]) {
+                                          uint32_t (&bits)[kStreamLoads][4], int (&cnt)[kStreamLoads]) {
   if (base + kStreamTile <= n) {
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kStreamLoads; ++u) {
       src.load_full4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, bits[u]);
       cnt[u] = 4;
     }
   } else {
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < kStreamLoads; ++u)
       cnt[u] = src.load_vals4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, n, bits[u]);
   }
 }
@@ -247,11 +248,11 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
   const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
   bool nonfinite = false;
   for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-    uint32_t bits[4][4];
-    int cnt[4];
+    uint32_t bits[kStreamLoads][4];
+    int cnt[kStreamLoads];
     load_tile(src, tile * kStreamTile, n, bits, cnt);
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
+    for (int u = 0; u < kStreamLoads; ++u) {
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         if (e < cnt[u]) {
@@ -295,12 +296,12 @@ k_prune_ties(BucketSrc<NSML_F32> src, unsigned long long n, PruneCtl* ctl, const
   if (r >= cT) return;  // every key equal to T is pruned: no ranks needed
   const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
   for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-    uint32_t bits[4][4];
-    int cnt[4];
+    uint32_t bits[kStreamLoads][4];
+    int cnt[kStreamLoads];
     load_tile(src, tile * kStreamTile, n, bits, cnt);
     unsigned int c = 0;
 #pragma unroll
-    for (int u = 0; u < 4; ++u)
+    for (int u = 0; u < kStreamLoads; ++u)
 #pragma unroll
       for (int e = 0; e < 4; ++e) c += (e < cnt[u]) && prune_key(bits[u][e]) == T;
     c = __reduce_add_sync(0xFFFFFFFFu, c);
@@ -332,11 +333,11 @@ k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl
     // flags of 8 neighbouring lanes are combined into one word.
     for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
       const unsigned long long base = tile * kStreamTile;
-      uint32_t bits[4][4];
-      int cnt[4];
+      uint32_t bits[kStreamLoads][4];
+      int cnt[kStreamLoads];
       load_tile(src, base, n, bits, cnt);
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < kStreamLoads; ++u) {
         unsigned int f = 0;
 #pragma unroll
         for (int e = 0; e < 4; ++e) f |= (unsigned)((e < cnt[u]) && prune_key(bits[u][e]) >= T) << e;
@@ -364,7 +365,8 @@ k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl
   before = 0;
 #pragma unroll
   for (int w = 0; w < kCta / 32; ++w) before += s_red[w];
-  constexpr int kWordsPerTile = kStreamTile / 32;  // 128: the first 128 threads own a word each
+  constexpr int kWordsPerTile = kStreamTile / 32;  // a thread owns one word of the tile
+  static_assert(kWordsPerTile <= kCta, "one mask word per thread");
   for (unsigned long long tile = t_first; tile < t_last; ++tile) {
     const unsigned long long i0 = tile * kStreamTile + (unsigned long long)threadIdx.x * 32;
     uint32_t key[32];
