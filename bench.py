@@ -18,6 +18,9 @@ Workloads (value distributions are described in paper_2506_16235_b200/synth.py):
             every step by the controller from a synthetic 100/10/1 Gbps link trace
   agg       8 workers x int8 payloads for a 350M-element bucket (ratio 0.05),
             decompress + sum only
+  alg2      the whole of Alg. 2 on 25M-element fp32 buckets: L2 norm, pruning mask
+            built from synthetic weights, compress of gradient + residual (ratio
+            0.01, int8), sum, W = 1
 """
 from __future__ import annotations
 
@@ -569,74 +572,129 @@ class AggWorkload(Workload):
         return 4.0 * n, dt, f"the same payload recipe at one tenth of the size (n={n}, k={k}, W=8)"
 
 
-WORKLOADS = {"resnet50": ResnetWorkload, "gpt2": Gpt2Workload, "decoder": DecoderWorkload, "agg": AggWorkload}
+class Alg2Workload(Workload):
+    """The whole of Alg. 2 per bucket, with the local accumulation of Section 4.2 Step 3: L2 norm of the gradient
+    (Step 1; enqueued, not waited for), pruning mask from the weights at the step's ratio (Step 2), compress of
+    gradient + residual under that mask (Step 3), and the receiver's decompress + sum (W = 1)."""
+
+    name = "alg2: 25M-element fp32 buckets, L2 norm + pruning mask from weights + compress with local accumulation (ratio 0.01, int8) + sum, W=1"
+    RATIO, BITS, N = 0.01, 8, 25_000_000
+    GRADS, STATE = 8, 4  # gradient buckets and weight / residual buffers the steps rotate over (100 MB each)
+    has_host = False     # no host-buffer entry points for these steps
+    graph_period = 8
+
+    def __init__(self, nsml, torch, device, rank, nlanes=2):
+        self.nsml, self.torch = nsml, torch
+        n = self.N
+        gen = torch.Generator(device=device)
+        gen.manual_seed(500 + rank)
+        rs = np.random.default_rng([500, rank])
+        self.grads = []
+        for _ in range(self.GRADS):  # a bucket = 50 equal "tensors", per-tensor sigma log-uniform [1e-4, 1e-2]
+            g = torch.empty(n, dtype=torch.float32, device=device)
+            for t in range(50):
+                g[t * (n // 50):(t + 1) * (n // 50)].normal_(0.0, 10.0 ** rs.uniform(-4.0, -2.0), generator=gen)
+            self.grads.append(g)
+        self.weights = [torch.empty(n, dtype=torch.float32, device=device).normal_(0.0, 0.02, generator=gen)
+                        for _ in range(self.STATE)]
+        self.residual = [torch.zeros(n, dtype=torch.float32, device=device) for _ in range(self.STATE)]
+        self.lanes = Lanes(torch, nsml, device, nlanes, nsml.nsml_workspace_bytes(n), nsml.nsml_accumulate_workspace_bytes(n, 1),
+                           nsml.nsml_payload_bytes(n, self.RATIO, self.BITS), 1, n)
+        for lane in self.lanes.all:
+            lane.l2ws = nsml.alloc_bytes(nsml.lib.nsml_l2_workspace_bytes(), device)
+            lane.pws = nsml.alloc_bytes(nsml.nsml_prune_workspace_bytes(n), device)
+            lane.mask = torch.empty((n + 31) // 32, dtype=torch.int32, device=device)
+        self.dense = self.lanes.all[0].dense
+        self.sizes = [n] * self.STATE
+        self.input_bytes_per_step = 4.0 * n * self.STATE
+        self.config = {"workload": self.name, "buckets": self.STATE, "bucket_elems": self.sizes, "ratio": self.RATIO,
+                       "bits": self.BITS, "W": 1, "streams": nlanes,
+                       "l2": "gradients rotate over 8 buckets (800 MB), weights and residuals over 4 each"}
+
+    def jobs(self, i):
+        nsml, n = self.nsml, self.N
+        k = nsml.nsml_k_of(n, self.RATIO)
+        for b in range(self.STATE):
+            def enqueue(lane, acc, b=b, g=self.grads[(i * self.STATE + b) % self.GRADS]):
+                nsml.nsml_grad_l2(g, workspace=lane.l2ws, stream=lane.stream, sync=False)
+                nsml.nsml_prune_mask_build(self.weights[b], self.RATIO, prune_mask=lane.mask, workspace=lane.pws,
+                                           stream=lane.stream)
+                p = nsml.nsml_compress_feedback(g, self.residual[b], self.RATIO, self.BITS, prune_mask=lane.mask,
+                                                payload=lane.payloads[0], workspace=lane.ws, stream=lane.stream)
+                nsml.nsml_decompress_accumulate([p], lane.dense, zero_first=True, workspace=lane.aws, stream=lane.stream)
+                if acc is not None:
+                    self.account(acc, "k_sumsq", 4 * n)
+                    self.account(acc, "k_prune_hist", 3 * 4 * n)
+                    self.account(acc, "k_prune_ties", 3 * 4096 * 4)
+                    self.account(acc, "k_prune_write", 4 * n + n // 8)
+                    self.account(acc, "k_feedback_add", 12 * n)
+                    self.account(acc, "k_feedback_subtract", 13 * k)
+                    self.compress_bytes(acc, n, 4, self.RATIO, self.BITS)
+                    self.account(acc, "k_compact_bucket", n // 8)  # the mask
+                    self.merge_bytes(acc, n, [(k, self.BITS)])
+
+            yield ((i * self.STATE + b) % self.GRADS, b), nsml.nsml_payload_bytes(n, self.RATIO, self.BITS), enqueue
+
+    def oracle_sample(self):
+        import oracle
+
+        n = 4_000_000
+        g = self.grads[0][:n].cpu().numpy()
+        w = self.weights[0][:n].cpu().numpy()
+        r = np.zeros(n, dtype=np.float32)
+        t0 = time.perf_counter()
+        oracle.l2_norm(g)
+        mask = oracle.prune_mask(w, self.RATIO)
+        p, r = oracle.error_feedback_step(g, r, self.RATIO, self.BITS, mask)
+        oracle.decompress_sum([p], n)
+        dt = time.perf_counter() - t0
+        return 4.0 * n, dt, f"first {n} elements of one bucket: L2 norm, mask, compress with residual, sum"
+
+
+WORKLOADS = {"resnet50": ResnetWorkload, "gpt2": Gpt2Workload, "decoder": DecoderWorkload, "agg": AggWorkload,
+             "alg2": Alg2Workload}
 
 
 # --------------------------------------------------------------------------
 # reference arm: the CPU oracle, timed as it stands
 # --------------------------------------------------------------------------
-def alg2_leg(nsml, torch, device, big, peak):
-    """The other steps of Alg. 2 on 25M-element buckets: L2 norm (Step 1), pruning mask from synthetic
-    Gaussian weights (Step 2), compress with local accumulation (Step 3), ratio 0.01, int8.  Inputs rotate
-    over sixteen gradient buckets and four weight / residual buffers (each 100 MB)."""
-    ratio, bits = 0.01, 8
-    n = big.sizes[0]
-    k = nsml.nsml_k_of(n, ratio)
-    grads = [big.workers[w][b] for b in range(len(big.sizes)) for w in range(big.W) if big.sizes[b] == n]
-    gen = torch.Generator(device=device)
-    gen.manual_seed(77)
-    weights = [torch.empty(n, device=device).normal_(0.0, 0.02, generator=gen) for _ in range(4)]
-    residual = [torch.zeros(n, device=device) for _ in range(4)]
-    lane = big.lanes.all[0]
-    l2ws = nsml.alloc_bytes(nsml.lib.nsml_l2_workspace_bytes(), device)
-    pws = nsml.alloc_bytes(nsml.nsml_prune_workspace_bytes(n), device)
-    mask = torch.empty((n + 31) // 32, dtype=torch.int32, device=device)
-
-    def one(i):
-        g = grads[i % len(grads)]
-        nsml.nsml_grad_l2(g, workspace=l2ws, sync=False)
-        nsml.nsml_prune_mask_build(weights[i % 4], ratio, prune_mask=mask, workspace=pws)
-        nsml.nsml_compress_feedback(g, residual[i % 4], ratio, bits, prune_mask=mask, payload=lane.payloads[0],
-                                    workspace=lane.ws)
-
-    for i in range(3):
-        one(i)
+def run_leg(nsml, torch, wl, peak, use_graphs, traffic=None, steps=10):
+    """A second workload measured inside the default run: device time of `steps` steps, then per-kernel
+    device time with every launch bracketed by CUDA events (one stream, eager)."""
+    wl.init_graphs(use_graphs)
+    warm = max(3, wl.graph_period if wl.use_graphs else 3)
+    wl.lanes.fork()
+    for i in range(warm):
+        wl.step(i)
+    wl.lanes.join()
     torch.cuda.synchronize()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    reps = 12
-    e0.record()
-    for i in range(reps):
-        one(3 + i)
-    e1.record()
+    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    b0.record()
+    wl.lanes.fork()
+    for i in range(steps):
+        wl.step(warm + i)
+    wl.lanes.join()
+    b1.record()
     torch.cuda.synchronize()
-    ms = e0.elapsed_time(e1) / reps
+    ms = b0.elapsed_time(b1) / steps
+    acc = {}
     nsml.nsml_prof_reset()
     nsml.nsml_prof_enable(True)
-    for i in range(8):
-        one(i)
+    wl.lanes.active = 1
+    for i in range(5):
+        wl.step(i, acc)
     torch.cuda.synchronize()
     prof = nsml.nsml_prof_read()
     nsml.nsml_prof_enable(False)
-    per_launch = {  # algorithmic bytes per launch
-        "k_sumsq": 4 * n,
-        "k_prune_hist": 4 * n,
-        "k_prune_ties": 3 * 4096 * 4,
-        "k_prune_write": 4 * n + n // 8,
-        "k_feedback_add": 12 * n,
-        "k_feedback_subtract": 13 * k,
-        "k_sample": 4 * 8192,
-        "k_compact_bucket": 4 * n + n // 8 + 8 * k,
-        "k_finalize": 24 * k + 8 * k + 4 * k + k + 4 * ((k + 1023) // 1024),
-    }
     per = {}
     for name, (t, cnt) in prof.items():
-        if cnt and name in per_launch:
-            gbs = per_launch[name] * cnt / (t * 1e-3) / 1e9
-            per[name] = {"launches_per_step": cnt / 8, "us_per_launch": 1e3 * t / cnt, "algorithmic_GBps": gbs,
-                         "frac_of_peak": gbs / peak, "frac_of_nominal_8TBps": gbs / 8000.0}
-    return {"workload": "one 25M-element fp32 bucket per step: L2 norm, pruning mask from weights, compress with "
-                        "local accumulation (ratio 0.01, int8, mask applied), one stream, eager",
-            "value": 4.0 * n / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms, "kernels": per}
+        if cnt:
+            gbs = acc.get(name, 0) / (t * 1e-3) / 1e9
+            per[name] = {"launches_per_step": cnt / 5, "us_per_launch": 1e3 * t / cnt, "algorithmic_GBps": gbs,
+                         "frac_of_peak": gbs / peak, "frac_of_nominal_8TBps": gbs / 8000.0,
+                         "traffic": (traffic or {}).get(name)}
+    return {"workload": wl.name, "value": wl.input_bytes_per_step / (ms * 1e-3) / 1e9, "unit": UNIT,
+            "ms_per_step": ms, "kernels": per}
 
 
 def run_reference(args, rank):
@@ -710,7 +768,7 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    defaults = {"resnet50": (100, 5), "gpt2": (20, 3), "decoder": (90, 3), "agg": (50, 3)}[args.workload]
+    defaults = {"resnet50": (100, 5), "gpt2": (20, 3), "decoder": (90, 3), "agg": (50, 3), "alg2": (20, 8)}[args.workload]
     steps = args.steps or defaults[0]
     warmup = max(3, defaults[1] if args.warmup is None else args.warmup)
 
@@ -791,7 +849,7 @@ def main():
 
     # ---- end to end through the host-buffer entry points ----
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and getattr(wl, "has_host", True):
         wl.setup_host()
         host_steps = max(1, min(steps, 5))
         for i in range(2):
@@ -825,41 +883,14 @@ def main():
     # ---- a 25M-element bucket, where the 60 %-of-HBM target applies ----
     if rank == 0 and args.workload == "resnet50" and not args.no_large_bucket_leg:
         big = Gpt2Workload(nsml, torch, device, rank, buckets=[2, 3, 2, 3], nlanes=max(1, args.streams))
-        big.init_graphs(not args.no_graphs)
-        big.lanes.fork()
-        for i in range(3):
-            big.step(i)
-        big.lanes.join()
-        torch.cuda.synchronize()
-        b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        b0.record()
-        big.lanes.fork()
-        for i in range(10):
-            big.step(i)
-        big.lanes.join()
-        b1.record()
-        torch.cuda.synchronize()
-        big_ms = b0.elapsed_time(b1) / 10
-        acc2 = {}
-        nsml.nsml_prof_reset()
-        nsml.nsml_prof_enable(True)
-        big.lanes.active = 1
-        for i in range(5):
-            big.step(i, acc2)
-        torch.cuda.synchronize()
-        prof2 = nsml.nsml_prof_read()
-        nsml.nsml_prof_enable(False)
-        per = {}
-        for name, (ms, cnt) in prof2.items():
-            if cnt:
-                gbs = acc2.get(name, 0) / (ms * 1e-3) / 1e9
-                per[name] = {"us_per_launch": 1e3 * ms / cnt, "algorithmic_GBps": gbs, "frac_of_peak": gbs / peak,
-                             "frac_of_nominal_8TBps": gbs / 8000.0, "traffic": NCU_TRAFFIC_25M.get(name)}
-        out["bucket_25M"] = {"workload": "four 25M-element fp32 buckets, ratio 0.01, int8, W=4 workers each",
-                             "value": big.input_bytes_per_step / (big_ms * 1e-3) / 1e9, "unit": UNIT,
-                             "ms_per_step": big_ms, "kernels": per}
-        out["alg2_25M"] = alg2_leg(nsml, torch, device, big, peak)
+        big.name = "four 25M-element fp32 buckets, ratio 0.01, int8, W=4 workers each"
+        out["bucket_25M"] = run_leg(nsml, torch, big, peak, not args.no_graphs, NCU_TRAFFIC_25M)
         del big
+        torch.cuda.empty_cache()
+        # the other steps of Alg. 2 (L2 norm, mask from weights, local accumulation) on buckets of that size
+        alg2 = Alg2Workload(nsml, torch, device, rank, nlanes=max(1, args.streams))
+        out["alg2_25M"] = run_leg(nsml, torch, alg2, peak, not args.no_graphs)
+        del alg2
 
     if rank == 0 and not args.no_cpu_baseline:
         nbytes, dt, sample = wl.oracle_sample()

@@ -172,10 +172,16 @@ struct PruneCtl {
   unsigned int d0, rem1;       // digit 0 of the threshold, rank left inside its bin
   unsigned int prefix24, rem2; // digits 0-1, rank left
   unsigned int T, r, cT;       // threshold key (complemented), ties to prune, ties in all
+  unsigned int list_count;     // entries appended to the tie list by the last histogram pass
+  unsigned int list_ok;        // the tie list holds every key that shares the threshold's 24-bit prefix
+  unsigned int use_limit;      // ties are decided by index: pruned iff index <= idx_limit
+  unsigned int idx_limit;
 };
+constexpr unsigned int kTieCap = 1024;  // keys sharing the threshold's 24-bit prefix that the tie list can hold
 
 struct PruneLayout {
   size_t hist;       // u32[3][kMaxBins]
+  size_t tie_list;   // uint2[kTieCap]: (index, last key digit) of the keys that share the threshold's 24-bit prefix
   size_t tile_ties;  // u32[tiles]
   size_t total;
 };
@@ -184,7 +190,8 @@ inline PruneLayout prune_layout(int64_t n) {
   PruneLayout L;
   const size_t tiles = ((size_t)n + kStreamTile - 1) / kStreamTile;
   L.hist = 256;
-  L.tile_ties = L.hist + 3 * kMaxBins * sizeof(unsigned int);
+  L.tie_list = L.hist + 3 * kMaxBins * sizeof(unsigned int);
+  L.tile_ties = L.tie_list + kTieCap * sizeof(uint2);
   L.total = L.tile_ties + align_up(tiles * 4, 256);
   return L;
 }
@@ -223,11 +230,13 @@ __device__ __forceinline__ void prune_resolve(const unsigned int* ghist, unsigne
 
 template <int LEVEL>
 __global__ void __launch_bounds__(kCta)
-k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, PruneCtl* ctl, unsigned int* __restrict__ hist) {
+k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, PruneCtl* ctl, unsigned int* __restrict__ hist,
+             uint2* __restrict__ tie_list) {
   constexpr int NB = (LEVEL == 2) ? 128 : kMaxBins;
   __shared__ unsigned int s_hist[NB];
   __shared__ unsigned int s_tot[kCta / 32], s_out[2];
   unsigned int prefix = 0;
+  bool collect = false;
   if (LEVEL == 1) {
     prune_resolve<kMaxBins>(hist, m, s_tot, s_out);
     prefix = s_out[0];
@@ -238,9 +247,13 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
   } else if (LEVEL == 2) {
     prune_resolve<kMaxBins>(hist + kMaxBins, ctl->rem1, s_tot, s_out);
     prefix = (ctl->d0 << 12) | s_out[0];
+    // Few keys share the threshold's first 24 bits (their number is the bin's count): this pass lists
+    // them, so that ties at the threshold can be ranked by index without another pass over the weights.
+    collect = hist[kMaxBins + s_out[0]] <= kTieCap;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       ctl->prefix24 = prefix;
       ctl->rem2 = s_out[1];
+      ctl->list_ok = collect;
     }
   }
   for (int b = threadIdx.x; b < NB; b += kCta) s_hist[b] = 0;
@@ -263,7 +276,13 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
           } else if (LEVEL == 1) {
             if ((key >> 19) == prefix) atomicAdd(&s_hist[(key >> 7) & 0xFFFu], 1u);
           } else {
-            if ((key >> 7) == prefix) atomicAdd(&s_hist[key & 0x7Fu], 1u);
+            if ((key >> 7) == prefix) {
+              atomicAdd(&s_hist[key & 0x7Fu], 1u);
+              if (collect) {
+                const unsigned long long i = tile * kStreamTile + (unsigned long long)(u * kCta + threadIdx.x) * 4 + e;
+                tie_list[atomicAdd(&ctl->list_count, 1u)] = make_uint2((uint32_t)i, key & 0x7Fu);
+              }
+            }
           }
         }
       }
@@ -278,13 +297,17 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
   }
 }
 
-// Resolves the last digit: threshold T, ties to prune r, ties in all cT.  When r < cT the ties are pruned
-// in index order, which needs their count per tile.
+// Resolves the last digit: threshold T, ties to prune r, ties in all cT.  When r < cT only the r ties of
+// lowest index are pruned.  Usually the last histogram pass has listed them: block 0 then finds the
+// r-th smallest index among them and the mask pass compares indices with it.  Otherwise (more keys share
+// the threshold's prefix than the list holds) the ties are counted per tile for a ranked mask pass.
 __global__ void __launch_bounds__(kCta)
 k_prune_ties(BucketSrc<NSML_F32> src, unsigned long long n, PruneCtl* ctl, const unsigned int* __restrict__ hist,
-             unsigned int* __restrict__ tile_ties) {
+             const uint2* __restrict__ tie_list, unsigned int* __restrict__ tile_ties) {
   __shared__ unsigned int s_tot[kCta / 32], s_out[2];
   __shared__ unsigned int s_cnt[kCta / 32];
+  __shared__ uint32_t s_tied[kTieCap];
+  __shared__ unsigned int s_ntied;
   prune_resolve<128>(hist + 2 * kMaxBins, ctl->rem2, s_tot, s_out);
   const uint32_t T = (ctl->prefix24 << 7) | s_out[0];
   const unsigned int r = s_out[1], cT = hist[2 * kMaxBins + s_out[0]];
@@ -294,6 +317,28 @@ k_prune_ties(BucketSrc<NSML_F32> src, unsigned long long n, PruneCtl* ctl, const
     ctl->cT = cT;
   }
   if (r >= cT) return;  // every key equal to T is pruned: no ranks needed
+  if (ctl->list_ok) {
+    if (blockIdx.x != 0) return;
+    if (threadIdx.x == 0) s_ntied = 0;
+    __syncthreads();
+    const unsigned int listed = min(ctl->list_count, kTieCap);
+    for (unsigned int j = threadIdx.x; j < listed; j += kCta) {
+      const uint2 e = tie_list[j];
+      if (e.y == s_out[0]) s_tied[atomicAdd(&s_ntied, 1u)] = e.x;
+    }
+    __syncthreads();
+    const unsigned int ntied = s_ntied;  // == cT
+    for (unsigned int j = threadIdx.x; j < ntied; j += kCta) {
+      const uint32_t mine = s_tied[j];
+      unsigned int below = 0;
+      for (unsigned int q = 0; q < ntied; ++q) below += s_tied[q] < mine;
+      if (below == r - 1) {  // indices are distinct: exactly one entry has r - 1 below it
+        ctl->idx_limit = mine;
+        ctl->use_limit = 1;
+      }
+    }
+    return;
+  }
   const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
   for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
     uint32_t bits[kStreamLoads][4];
@@ -325,11 +370,13 @@ k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl
   __shared__ unsigned long long s_red[kCta / 32];
   const uint32_t T = ctl->T;
   const unsigned int r = ctl->r, cT = ctl->cT;
+  const bool by_index = ctl->use_limit != 0;  // ties pruned iff their index is <= idx_limit
+  const uint32_t idx_limit = ctl->idx_limit;
   const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
   const unsigned long long nwords = (n + 31) / 32;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (r >= cT) {
-    // every key >= T is pruned.  A warp's load covers 128 consecutive elements = 4 mask words; the 4-bit
+  if (r >= cT || by_index) {
+    // every key > T is pruned, and every key == T (or those up to idx_limit).  A warp's load covers 128 consecutive elements = 4 mask words; the 4-bit
     // flags of 8 neighbouring lanes are combined into one word.
     for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
       const unsigned long long base = tile * kStreamTile;
@@ -340,7 +387,13 @@ k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl
       for (int u = 0; u < kStreamLoads; ++u) {
         unsigned int f = 0;
 #pragma unroll
-        for (int e = 0; e < 4; ++e) f |= (unsigned)((e < cnt[u]) && prune_key(bits[u][e]) >= T) << e;
+        for (int e = 0; e < 4; ++e) {
+          const uint32_t key = prune_key(bits[u][e]);
+          bool pruned = key > T;
+          if (key == T)  // rare: the index is worked out only here (indices are below 2^31)
+            pruned = !by_index || (uint32_t)base + (uint32_t)((u * kCta + threadIdx.x) * 4 + e) <= idx_limit;
+          f |= (unsigned)((e < cnt[u]) && pruned) << e;
+        }
         unsigned int x = f << (4 * (lane & 7));
         x |= __shfl_xor_sync(0xFFFFFFFFu, x, 1);
         x |= __shfl_xor_sync(0xFFFFFFFFu, x, 2);

@@ -403,7 +403,7 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
   int rc = device_info(&dev);
   if (rc != NSML_OK) return rc;
   unsigned char* ws = static_cast<unsigned char*>(workspace);
-  if (cudaMemsetAsync(ws, 0, L.tile_ties, st) != cudaSuccess) return NSML_ERR_CUDA;  // status, ctl, histograms
+  if (cudaMemsetAsync(ws, 0, L.tie_list, st) != cudaSuccess) return NSML_ERR_CUDA;  // status, ctl, histograms
   if (m == 0) {  // ratio 1: nothing is pruned
     if (cudaMemsetAsync(mask, 0, (size_t)((n + 31) / 32) * 4, st) != cudaSuccess) return NSML_ERR_CUDA;
     return NSML_OK;
@@ -411,24 +411,25 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
   PruneCtl* ctl = reinterpret_cast<PruneCtl*>(ws);
   unsigned int* hist = reinterpret_cast<unsigned int*>(ws + L.hist);
   unsigned int* tile_ties = reinterpret_cast<unsigned int*>(ws + L.tile_ties);
+  uint2* tie_list = reinterpret_cast<uint2*>(ws + L.tie_list);
   const BucketSrc<NSML_F32> src{weights, nullptr};
   const unsigned int grid = stream_grid(n, *dev, 6, 1u << 16);
   const unsigned long long un = (unsigned long long)n;
   {
     LaunchScope scope(K_PRUNE_HIST, st);
-    k_prune_hist<0><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist);
+    k_prune_hist<0><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
     LaunchScope scope(K_PRUNE_HIST, st);
-    k_prune_hist<1><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist);
+    k_prune_hist<1><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
     LaunchScope scope(K_PRUNE_HIST, st);
-    k_prune_hist<2><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist);
+    k_prune_hist<2><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
     LaunchScope scope(K_PRUNE_TIES, st);
-    k_prune_ties<<<grid, kCta, 0, st>>>(src, un, ctl, hist, tile_ties);
+    k_prune_ties<<<grid, kCta, 0, st>>>(src, un, ctl, hist, tie_list, tile_ties);
   }
   {
     LaunchScope scope(K_PRUNE_WRITE, st);

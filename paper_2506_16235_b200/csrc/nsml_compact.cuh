@@ -106,6 +106,11 @@ k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, uint32_t*
       cp_async_lane<LANE_BYTES>(fifo + r * 32 * LANE_BYTES, g + (seg * kSegElems + r * kRound) * ESIZE);
   }
   cp_async_commit();
+  // The segment's 16 words of the pruning mask (64 bytes) are fetched by lanes 0-15 one segment ahead, like
+  // the data, and handed to the lanes by shuffle.
+  constexpr int kSegMaskWords = kSegElems / 32;
+  uint32_t mask_words = 0, mask_words_next = 0;
+  if (src.mask != nullptr && seg < nseg_full && lane < kSegMaskWords) mask_words = __ldg(src.mask + seg * kSegMaskWords + lane);
   // Zeros are never candidates here; if they are needed (fewer than k non-zero
   // keys) the list comes out short and the finalize kernel's slow path adds them.
   const float t = __uint_as_float(max(ctl->lo, 1u));
@@ -119,6 +124,8 @@ k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, uint32_t*
         cp_async_lane<LANE_BYTES>(fifo + ((buf ^ 1) * kSegRounds + r) * 32 * LANE_BYTES,
                                   g + (next * kSegElems + r * kRound) * ESIZE);
     }
+    if (src.mask != nullptr && next < nseg_full && lane < kSegMaskWords)
+      mask_words_next = __ldg(src.mask + next * kSegMaskWords + lane);
     cp_async_commit();
     cp_async_wait<1>();  // this segment's copies have landed; the next segment's stay in flight
 
@@ -138,8 +145,8 @@ k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, uint32_t*
           bits[2] = v.y << 16; bits[3] = v.y & 0xFFFF0000u;
         }
         if (src.mask != nullptr) {
-          const unsigned long long i0 = seg_base + r * kRound + lane * 4;
-          const uint32_t m = (src.mask[i0 >> 5] >> (unsigned)(i0 & 31)) & 0xFu;
+          const uint32_t word = __shfl_sync(0xFFFFFFFFu, mask_words, r * (kRound / 32) + (lane >> 3));
+          const uint32_t m = (word >> (unsigned)((lane & 7) * 4)) & 0xFu;
 #pragma unroll
           for (int e = 0; e < 4; ++e)
             if (m & (1u << e)) bits[e] = 0;
@@ -158,6 +165,7 @@ k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, uint32_t*
     }
     seg = next;
     buf ^= 1;
+    mask_words = mask_words_next;
   }
   cp_async_wait<0>();
 }

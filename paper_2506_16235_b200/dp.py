@@ -42,3 +42,63 @@ def payload_slots(world: int, payload_bytes: int):
     """Byte ranges of the W equal-size payloads inside an all-gather buffer (16-byte aligned slots)."""
     slot = (payload_bytes + 15) // 16 * 16
     return [(r * slot, r * slot + payload_bytes) for r in range(world)], slot * world
+
+
+def exchange_payloads(payload: torch.Tensor, group=None):
+    """The exchange step of the sparse path (Section 5.3: top-k payloads travel by AllGather):
+    every rank contributes its payload (uint8 tensor; all ranks' payloads have the same size because
+    they compressed equally long buckets at the agreed ratio) and receives all of them.
+    Returns (buffer, [one view per rank]); view r is rank r's payload, 16-byte aligned, ready for
+    nsml_decompress_accumulate.  One fixed-size all-gather, NCCL on CUDA tensors, gloo on CPU ones."""
+    world = dist.get_world_size(group) if dist.is_initialized() else 1
+    nbytes = payload.numel()
+    slots, total = payload_slots(world, nbytes)
+    slot = total // world
+    buf = torch.empty(total, dtype=torch.uint8, device=payload.device)
+    if world == 1:
+        buf[:nbytes].copy_(payload)
+    else:
+        rank = dist.get_rank(group)
+        mine = buf[rank * slot:(rank + 1) * slot]
+        mine[:nbytes].copy_(payload)
+        if slot > nbytes:
+            mine[nbytes:].zero_()
+        dist.all_gather_into_tensor(buf, mine.clone(), group=group)
+    return buf, [buf[a:b] for a, b in slots]
+
+
+class GradientExchange:
+    """One bucket's data-parallel gradient exchange, every step (Fig. 1 and Alg. 1-2 of the paper put
+    together): rank 0's controller picks the ratio from the last measured transfer, every rank compresses
+    its bucket at that ratio, the payloads are all-gathered, every rank sums them into its dense
+    gradient, and the measured transfer (bytes of all payloads, slowest rank's device time of the
+    all-gather) is what the controller sees next step.  CUDA only: the compression and the sum run in
+    libnsml."""
+
+    def __init__(self, n: int, bits: int = 8, group=None, device=None, **ctrl_overrides):
+        import paper_2506_16235_b200 as nsml
+
+        self.nsml, self.n, self.bits, self.group = nsml, int(n), int(bits), group
+        self.device = device if device is not None else torch.device("cuda", torch.cuda.current_device())
+        self.world = dist.get_world_size(group) if dist.is_initialized() else 1
+        self.ctrl = nsml.Controller(**ctrl_overrides)
+        self.ws = nsml.alloc_bytes(nsml.nsml_workspace_bytes(self.n), self.device)
+        self.aws = nsml.alloc_bytes(nsml.nsml_accumulate_workspace_bytes(self.n, self.world), self.device)
+        self.last = (0.0, 0.0)
+        self.ratio = None
+
+    def step(self, grad: torch.Tensor, dense: torch.Tensor) -> float:
+        """dense <- sum over ranks of their compressed `grad`; returns the ratio used."""
+        nsml = self.nsml
+        mine = self.ctrl.select_ratio(self.last[0], self.last[1], 4.0 * self.n * self.world)
+        self.ratio = agree_ratio(mine, self.group)
+        payload = nsml.nsml_compress(grad, self.ratio, self.bits, workspace=self.ws)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ev0.record()
+        _, views = exchange_payloads(payload, self.group)
+        ev1.record()
+        nsml.nsml_decompress_accumulate(views, dense, zero_first=True, workspace=self.aws)
+        ev1.synchronize()
+        seconds = max_over_ranks(ev0.elapsed_time(ev1) * 1e-3, self.group)
+        self.last = (float(self.world * payload.numel()), max(seconds, 1e-9))
+        return self.ratio

@@ -242,3 +242,26 @@ def test_adaptive_matches_oracle(case):
     assert np.array_equal(mask.cpu().numpy().view(np.uint32), mask_words(want_mask))
     assert_payload_equal(payload, want)
     assert {"quantise": (0.04, 16), "small_norm": (0.02, 32), "gate_closed": (0.2, 32)}[case] == (got_ratio, got_bits)
+
+
+# ------------------------------------------------------------------ the exchange step around the path
+def test_gradient_exchange_single_rank_follows_the_controller():
+    # one rank (no process group): the all-gather is a copy, everything else is the real path
+    from paper_2506_16235_b200 import dp
+
+    n = 300_001
+    rng = np.random.default_rng(21)
+    ex = dp.GradientExchange(n, bits=16, startup_max_steps=0, ratio_init=0.05)
+    ora = oracle.Controller(oracle.ControllerParams(startup_max_steps=0, ratio_init=0.05))
+    dense = torch.empty(n, device="cuda")
+    last = (0.0, 0.0)
+    for step in range(4):
+        g = rng.standard_normal(n).astype(np.float32)
+        ratio = ex.step(to_device_grad(g), dense)
+        assert ratio == ora.select_ratio(last[0], last[1], 4.0 * n)
+        last = ex.last
+        assert last[0] == nsml.nsml_payload_bytes(n, ratio, 16) and last[1] > 0
+        want = oracle.compress(g, ratio, 16)
+        got = dense.cpu().numpy()
+        ref = oracle.decompress_sum([want], n)
+        assert np.max(np.abs(got.astype(np.float64) - ref.astype(np.float64))) <= 1e-6 * float(np.abs(g).max())

@@ -41,8 +41,9 @@ def _worker(rank, world, port, out):
     raw = torch.from_numpy(nsml.pack_payload(n, bits, p.idx, half=p.half))
     assert raw.numel() == nsml.nsml_payload_bytes(n, ratio, bits)
     slots, total = dp.payload_slots(world, raw.numel())
-    gathered = [torch.empty_like(raw) for _ in range(world)]
-    dist.all_gather(gathered, raw)
+    buf, gathered = dp.exchange_payloads(raw)  # the one fixed-size all-gather of the sparse path
+    assert buf.numel() == total and torch.equal(gathered[rank], raw)
+    assert all(v.data_ptr() % 16 == 0 for v in gathered)
     parts = [nsml.unpack_payload(t) for t in gathered]
     payloads = [oracle.Payload(n=n, k=q["k"], bits=bits, idx=q["idx"], raw=oracle.f16_bits_to_f32(q["half"]), half=q["half"])
                 for q in parts]
