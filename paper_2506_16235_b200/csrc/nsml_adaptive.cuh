@@ -363,11 +363,10 @@ k_prune_ties(BucketSrc<NSML_F32> src, unsigned long long n, PruneCtl* ctl, const
 }
 
 // Writes the mask: bit (i & 31) of word i >> 5 set = parameter i pruned.  Bits past n in the last word are 0.
+// Covers the two usual cases: every key equal to the threshold is pruned, or the ties are decided by index.
 __global__ void __launch_bounds__(kCta)
 k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl, const unsigned int* __restrict__ tile_ties,
               uint32_t* __restrict__ mask) {
-  __shared__ unsigned int s_scan[kCta / 32];
-  __shared__ unsigned long long s_red[kCta / 32];
   const uint32_t T = ctl->T;
   const unsigned int r = ctl->r, cT = ctl->cT;
   const bool by_index = ctl->use_limit != 0;  // ties pruned iff their index is <= idx_limit
@@ -375,8 +374,10 @@ k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl
   const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
   const unsigned long long nwords = (n + 31) / 32;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  if (r >= cT || by_index) {
-    // every key > T is pruned, and every key == T (or those up to idx_limit).  A warp's load covers 128 consecutive elements = 4 mask words; the 4-bit
+  (void)tile_ties;
+  if (r >= cT || by_index) {  // else: k_prune_write_ranked writes the mask
+    // Every key > T is pruned, and every key == T (or, by_index, those up to idx_limit).  A warp's load
+    // covers 128 consecutive elements = 4 mask words; the 4-bit
     // flags of 8 neighbouring lanes are combined into one word.
     for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
       const unsigned long long base = tile * kStreamTile;
@@ -402,10 +403,22 @@ k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl
         if ((lane & 7) == 0 && word < nwords) mask[word] = x;
       }
     }
-    return;
   }
-  // Some of the keys equal to T stay unpruned: the first r of them in index order are pruned.  A block
-  // takes a contiguous range of tiles and carries the number of ties seen so far; within a tile a thread
+}
+
+// The mask pass for the remaining case: some of the keys equal to T stay unpruned and there are too many
+// of them to list, so the first r of them in index order are found by rank.  Returns at once otherwise.
+__global__ void __launch_bounds__(kCta)
+k_prune_write_ranked(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl,
+                     const unsigned int* __restrict__ tile_ties, uint32_t* __restrict__ mask) {
+  __shared__ unsigned int s_scan[kCta / 32];
+  __shared__ unsigned long long s_red[kCta / 32];
+  const uint32_t T = ctl->T;
+  const unsigned int r = ctl->r, cT = ctl->cT;
+  if (r >= cT || ctl->use_limit != 0) return;
+  const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // A block takes a contiguous range of tiles and carries the number of ties seen so far; within a tile a thread
   // owns one mask word (32 consecutive elements).
   const unsigned long long t_first = (unsigned long long)blockIdx.x * tiles / gridDim.x;
   const unsigned long long t_last = (unsigned long long)(blockIdx.x + 1) * tiles / gridDim.x;

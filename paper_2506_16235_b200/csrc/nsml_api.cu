@@ -19,12 +19,13 @@ namespace nsml {
 
 enum KernelId {
   K_SAMPLE = 0, K_COMPACT_BUCKET, K_FINALIZE, K_PARTITION, K_MERGE, K_CLEAR, K_FINALIZE_DENSE,
-  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_COUNT
+  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_PRUNE_WRITE_RANKED, K_COUNT
 };
 
 static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_compact_bucket", "k_finalize", "k_partition", "k_merge",
                                                   "k_clear", "k_finalize_dense", "k_sumsq", "k_feedback_add",
-                                                  "k_feedback_subtract", "k_prune_hist", "k_prune_ties", "k_prune_write"};
+                                                  "k_feedback_subtract", "k_prune_hist", "k_prune_ties", "k_prune_write",
+                                                  "k_prune_write_ranked"};
 
 static std::atomic<int64_t> g_launches{0};
 
@@ -78,6 +79,7 @@ struct DeviceInfo {
   bool ready = false;
   int sms = 0;
   int compact_bucket = 0, finalize_small = 0, finalize_large = 0, merge = 0;  // resident blocks per SM
+  int sumsq = 0, feedback_add = 0, prune_hist = 0, prune_write = 0;            // the same, streaming kernels
 };
 static DeviceInfo g_dev[64];
 static std::mutex g_dev_mutex;
@@ -106,6 +108,24 @@ static int device_info(const DeviceInfo** out) {
     prepare(k_finalize_dense<NSML_F32, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache, &d.finalize_large);
     prepare(k_finalize_dense<NSML_BF16, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache, &d.finalize_large);
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.merge, k_merge, kCta, 0);
+    // The streaming kernels run as one wave of resident blocks (a second, partial wave would read
+    // with a fraction of the SMs' loads in flight).
+    auto resident = [&](auto kernel, int* out) {
+      int r = 0;
+      if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, kernel, kCta, 0);
+      if (*out == 0 || r < *out) *out = r;
+    };
+    resident(k_sumsq<NSML_F32>, &d.sumsq);
+    resident(k_sumsq<NSML_BF16>, &d.sumsq);
+    resident(k_feedback_add<NSML_F32>, &d.feedback_add);
+    resident(k_feedback_add<NSML_BF16>, &d.feedback_add);
+    resident(k_prune_hist<0>, &d.prune_hist);
+    resident(k_prune_hist<1>, &d.prune_hist);
+    resident(k_prune_hist<2>, &d.prune_hist);
+    resident(k_prune_ties, &d.prune_hist);
+    resident(k_prune_write, &d.prune_write);
+    resident(k_prune_write_ranked, &d.prune_write);
+    if (e == cudaSuccess && (d.sumsq < 1 || d.feedback_add < 1 || d.prune_hist < 1 || d.prune_write < 1)) e = cudaErrorUnknown;
     int coop = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
     if (e != cudaSuccess || d.compact_bucket < 1 || d.finalize_small < 1 || d.finalize_large < 1 || d.merge < 1 || !coop) {
@@ -345,7 +365,7 @@ static int sumsq_impl(const void* grad, int64_t n, int grad_dtype, void* workspa
   if (cudaMemsetAsync(ws, 0, 256, st) != cudaSuccess) return NSML_ERR_CUDA;
   SumsqCtl* ctl = reinterpret_cast<SumsqCtl*>(ws);
   double* partials = reinterpret_cast<double*>(ws + 256);
-  const unsigned int grid = stream_grid(n, *dev, 8, kSumsqMaxBlocks);
+  const unsigned int grid = stream_grid(n, *dev, dev->sumsq < 8 ? dev->sumsq : 8, kSumsqMaxBlocks);
   {
     LaunchScope scope(K_SUMSQ, st);
     if (grad_dtype == NSML_F32)
@@ -413,7 +433,8 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
   unsigned int* tile_ties = reinterpret_cast<unsigned int*>(ws + L.tile_ties);
   uint2* tie_list = reinterpret_cast<uint2*>(ws + L.tie_list);
   const BucketSrc<NSML_F32> src{weights, nullptr};
-  const unsigned int grid = stream_grid(n, *dev, 6, 1u << 16);
+  const unsigned int grid = stream_grid(n, *dev, dev->prune_hist < 8 ? dev->prune_hist : 8, 1u << 16);
+  const unsigned int wgrid = stream_grid(n, *dev, dev->prune_write < 8 ? dev->prune_write : 8, 1u << 16);
   const unsigned long long un = (unsigned long long)n;
   {
     LaunchScope scope(K_PRUNE_HIST, st);
@@ -433,7 +454,11 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
   }
   {
     LaunchScope scope(K_PRUNE_WRITE, st);
-    k_prune_write<<<grid, kCta, 0, st>>>(src, un, ctl, tile_ties, mask);
+    k_prune_write<<<wgrid, kCta, 0, st>>>(src, un, ctl, tile_ties, mask);
+  }
+  {
+    LaunchScope scope(K_PRUNE_WRITE_RANKED, st);  // returns at once unless ties have to be ranked
+    k_prune_write_ranked<<<wgrid, kCta, 0, st>>>(src, un, ctl, tile_ties, mask);
   }
   if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
   return NSML_OK;
@@ -454,7 +479,7 @@ static int feedback_impl(const void* grad, float* residual, int64_t n, int grad_
   const DeviceInfo* dev = nullptr;
   int rc = device_info(&dev);
   if (rc != NSML_OK) return rc;
-  const unsigned int grid = stream_grid(n, *dev, 8, 1u << 16);
+  const unsigned int grid = stream_grid(n, *dev, dev->feedback_add < 8 ? dev->feedback_add : 8, 1u << 16);
   {
     LaunchScope scope(K_FEEDBACK_ADD, st);
     if (grad_dtype == NSML_F32)
