@@ -80,6 +80,7 @@ struct DeviceInfo {
   int sms = 0;
   int compact_bucket = 0, finalize_small = 0, finalize_large = 0, merge = 0;  // resident blocks per SM
   int sumsq = 0, feedback_add = 0, prune_hist = 0, prune_write = 0;            // the same, streaming kernels
+  bool finalize_cluster = false;  // the one-cluster shape of the list stage fits an SM
 };
 static DeviceInfo g_dev[64];
 static std::mutex g_dev_mutex;
@@ -103,6 +104,10 @@ static int device_info(const DeviceInfo** out) {
     prepare(k_finalize<NSML_BF16, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
     prepare(k_finalize_dense<NSML_F32, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
     prepare(k_finalize_dense<NSML_BF16, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
+    int cluster_shape = 0;
+    prepare(k_finalize<NSML_F32, kFinClusterThreads, kFinClusterCache, true>, kFinClusterThreads, kFinClusterCache, &cluster_shape);
+    prepare(k_finalize<NSML_BF16, kFinClusterThreads, kFinClusterCache, true>, kFinClusterThreads, kFinClusterCache, &cluster_shape);
+    d.finalize_cluster = cluster_shape >= 1;
     prepare(k_finalize<NSML_F32, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache, &d.finalize_large);
     prepare(k_finalize<NSML_BF16, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache, &d.finalize_large);
     prepare(k_finalize_dense<NSML_F32, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache, &d.finalize_large);
@@ -203,6 +208,7 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
   const bool dense = use_dense(n, k, dev);
   unsigned int fgrid;
   bool small_shape;
+  bool cluster_shape = false;
   if (dense) {
     small_shape = (unsigned long long)n <= (unsigned long long)dev.sms * kFinSmallCache;
     unsigned long long cap = small_shape ? (unsigned long long)dev.sms : large_cap_blocks;
@@ -234,7 +240,10 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
     if (fgrid > (unsigned int)kMaxFinalizeBlocks) fgrid = kMaxFinalizeBlocks;
     const double expected = (double)n * (p_keep + 6.0 * std::sqrt(p_keep * (1.0 - p_keep) / kSamples)) + 64.0;
     small_shape = expected / fgrid <= (double)kFinSmallCache;
-    if (small_shape) {  // short lists: no more blocks than about 4096 candidates each (cheaper barriers, one block = none)
+    cluster_shape = dev.finalize_cluster && expected <= kFinClusterMaxCandidates && nseg >= (unsigned long long)kFinClusterBlocks;
+    if (cluster_shape) {
+      fgrid = kFinClusterBlocks;
+    } else if (small_shape) {  // short lists: no more blocks than about 4096 candidates each (cheaper barriers, one block = none)
       unsigned int want = (unsigned int)(expected / 4096.0) + 1;
       if (want < fgrid) fgrid = want;
     } else {  // long lists: as many blocks as stay co-resident (two per SM)
@@ -269,7 +278,22 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
       return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(fgrid), dim3(threads), args,
                                          finalize_dyn_smem(cache), st);
     };
-    if (small_shape && dense) le = launch(k_finalize_dense<DTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
+    if (cluster_shape) {
+      // one cluster; the blocks of a cluster are co-scheduled by the hardware, so no cooperative launch is needed
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(kFinClusterBlocks);
+      cfg.blockDim = dim3(kFinClusterThreads);
+      cfg.dynamicSmemBytes = finalize_dyn_smem(kFinClusterCache);
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = kFinClusterBlocks;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      le = cudaLaunchKernelEx(&cfg, k_finalize<DTYPE, kFinClusterThreads, kFinClusterCache, true>, src, fp);
+    } else if (small_shape && dense) le = launch(k_finalize_dense<DTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
     else if (small_shape) le = launch(k_finalize<DTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
     else if (dense) le = launch(k_finalize_dense<DTYPE, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache);
     else le = launch(k_finalize<DTYPE, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache);
