@@ -79,7 +79,7 @@ struct DeviceInfo {
   bool ready = false;
   int sms = 0;
   int compact_bucket = 0, finalize_small = 0, finalize_large = 0, merge = 0;  // resident blocks per SM
-  int sumsq = 0, feedback_add = 0, prune_hist = 0, prune_write = 0;            // the same, streaming kernels
+  int sumsq = 0, feedback_add = 0, prune_hist = 0, prune_write = 0, prune_write_ranked = 0;  // the same, streaming kernels
   bool finalize_cluster = false;  // the one-cluster shape of the list stage fits an SM
 };
 static DeviceInfo g_dev[64];
@@ -129,8 +129,8 @@ static int device_info(const DeviceInfo** out) {
     resident(k_prune_hist<2>, &d.prune_hist);
     resident(k_prune_ties, &d.prune_hist);
     resident(k_prune_write, &d.prune_write);
-    resident(k_prune_write_ranked, &d.prune_write);
-    if (e == cudaSuccess && (d.sumsq < 1 || d.feedback_add < 1 || d.prune_hist < 1 || d.prune_write < 1)) e = cudaErrorUnknown;
+    resident(k_prune_write_ranked, &d.prune_write_ranked);
+    if (e == cudaSuccess && (d.sumsq < 1 || d.feedback_add < 1 || d.prune_hist < 1 || d.prune_write < 1 || d.prune_write_ranked < 1)) e = cudaErrorUnknown;
     int coop = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
     if (e != cudaSuccess || d.compact_bucket < 1 || d.finalize_small < 1 || d.finalize_large < 1 || d.merge < 1 || !coop) {
@@ -482,7 +482,8 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
   }
   {
     LaunchScope scope(K_PRUNE_WRITE_RANKED, st);  // returns at once unless ties have to be ranked
-    k_prune_write_ranked<<<wgrid, kCta, 0, st>>>(src, un, ctl, tile_ties, mask);
+    const unsigned int rgrid = stream_grid(n, *dev, dev->prune_write_ranked < 8 ? dev->prune_write_ranked : 8, 1u << 16);
+    k_prune_write_ranked<<<rgrid, kCta, 0, st>>>(src, un, ctl, tile_ties, mask);
   }
   if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
   return NSML_OK;
