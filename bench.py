@@ -183,8 +183,10 @@ class Workload:
             return
         self.account(acc, "k_sample", 4 * 8192)
         self.account(acc, "k_compact_bucket", esize * n + 8 * k)
-        # list stage: candidates read once per phase (5 x 4k keys + 4k indices), survivors written and re-read
-        self.account(acc, "k_finalize", 24 * k + 8 * k + 4 * k + vb * k + s)
+        # gather: candidates (index + value) read from the segmented list and written contiguously
+        self.account(acc, "k_gather", 16 * k)
+        # list stage: candidate values read once per phase (4 x 4k keys), indices once, survivors written and re-read
+        self.account(acc, "k_finalize", 16 * k + 4 * k + 8 * k + 4 * k + vb * k + s)
 
     def merge_bytes(self, acc, n, ks_bits, zero_first=True):
         total = 4 * n if zero_first else 0

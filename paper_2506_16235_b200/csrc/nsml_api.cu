@@ -19,13 +19,13 @@ namespace nsml {
 
 enum KernelId {
   K_SAMPLE = 0, K_COMPACT_BUCKET, K_FINALIZE, K_PARTITION, K_MERGE, K_CLEAR, K_FINALIZE_DENSE,
-  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_PRUNE_WRITE_RANKED, K_COUNT
+  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_PRUNE_WRITE_RANKED, K_GATHER, K_COUNT
 };
 
 static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_compact_bucket", "k_finalize", "k_partition", "k_merge",
                                                   "k_clear", "k_finalize_dense", "k_sumsq", "k_feedback_add",
                                                   "k_feedback_subtract", "k_prune_hist", "k_prune_ties", "k_prune_write",
-                                                  "k_prune_write_ranked"};
+                                                  "k_prune_write_ranked", "k_gather"};
 
 static std::atomic<int64_t> g_launches{0};
 
@@ -270,6 +270,11 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
   fp.raw_val = reinterpret_cast<float*>(ws + L.raw_val);
   fp.payload = payload;
   fp.P = P;
+  if (!dense) {
+    LaunchScope scope(K_GATHER, st);  // segmented list -> contiguous list and the histogram of the first digit
+    const unsigned int ggrid = (unsigned int)((nseg + kGatherSegs - 1) / kGatherSegs);
+    k_gather<<<ggrid, kCta, 0, st>>>(fp);
+  }
   {
     LaunchScope scope(dense ? K_FINALIZE_DENSE : K_FINALIZE, st);
     void* args[] = {&src, &fp};

@@ -56,7 +56,6 @@ constexpr double kFinClusterMaxCandidates = 32768.0;  // expected candidates up 
 // The dense kernel needs no gather scratch, which leaves room for a larger cache in the large shape: two
 // blocks per SM then hold 2 x 23040 values, 6.8M elements over 148 SMs (a 25 MB float32 bucket stays on chip).
 constexpr int kFinDenseLargeCache = 23040;
-constexpr int kGatherRun = 4;  // consecutive candidates a thread of the gather copies per step
 constexpr size_t finalize_dyn_smem(int cache_entries) { return (size_t)cache_entries * 4; }  // values only
 
 struct FinalizeParams {
@@ -286,6 +285,104 @@ __device__ __forceinline__ void quantize_phase(const FinalizeParams& p, Finalize
   }
 }
 
+// Segmented candidate list -> contiguous list (list_idx / list_val, in index order) plus the global
+// histogram of the candidates' first key digit.  A plain (non-cooperative) kernel that spreads the copy
+// over all SMs: every candidate sits in another memory sector, and what bounds the copy is the rate of
+// scattered loads per SM.  A block takes kGatherSegs consecutive segments (one group); the list
+// position of its first candidate is the sum of the group counts before it; inside the block the
+// candidates are taken entry-parallel (thread t copies entries t*4..t*4+3, t*4 + 4*256.., located by a
+// search over the segments' offsets), so crowded segments are shared by all threads.
+constexpr int kGatherSegs = kGroupSegs;  // one group per block: its list position is a plain sum of group counts
+constexpr int kGatherRun = 4;      // consecutive candidates a thread copies per step
+
+__global__ void __launch_bounds__(kCta)
+k_gather(FinalizeParams p) {
+  __shared__ unsigned int s_hist[kMaxBins];
+  __shared__ unsigned int s_off[kGatherSegs + 1];  // exclusive offsets of the block's segments, total at the end
+  __shared__ unsigned long long s_red[kCta / 32];
+  __shared__ unsigned int s_scan[kCta / 32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (int b = threadIdx.x; b < kMaxBins; b += kCta) s_hist[b] = 0;
+  // list position of the block's first candidate
+  const unsigned long long first_group = (unsigned long long)blockIdx.x * (kGatherSegs / kGroupSegs);
+  unsigned long long before = 0;
+  for (unsigned long long g = threadIdx.x; g < first_group; g += kCta) before += p.group_count[g];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xFFFFFFFFu, before, o);
+  if (lane == 0) s_red[warp] = before;
+  // offsets of the block's segments
+  const unsigned long long seg0 = (unsigned long long)blockIdx.x * kGatherSegs;
+  const unsigned long long seg = seg0 + threadIdx.x;
+  const unsigned int c = (threadIdx.x < kGatherSegs && seg < p.nseg) ? p.seg_count[seg] : 0u;
+  unsigned int incl = c;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += up;
+  }
+  if (lane == 31) s_scan[warp] = incl;
+  __syncthreads();
+  unsigned long long base = 0;
+  unsigned int warps_before = 0, total = 0;
+#pragma unroll
+  for (int w = 0; w < kCta / 32; ++w) {
+    base += s_red[w];
+    if (w < warp) warps_before += s_scan[w];
+    total += s_scan[w];
+  }
+  if (threadIdx.x < kGatherSegs) s_off[threadIdx.x] = warps_before + incl - c;
+  if (threadIdx.x == 0) s_off[kGatherSegs] = total;
+  __syncthreads();
+  bool nonfinite = false;
+  for (unsigned int j0 = threadIdx.x * kGatherRun; j0 < total; j0 += kCta * kGatherRun) {
+    const int cnt = (int)min((unsigned int)kGatherRun, total - j0);
+    uint32_t from[kGatherRun];
+    {
+      // segment of entry j0: the last one whose offset is <= j0 (empty segments share an offset with their
+      // successor, so the search lands on the segment that holds the entry)
+      int lo = 0, hi = kGatherSegs - 1;
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (s_off[mid] <= j0) lo = mid; else hi = mid - 1;
+      }
+      unsigned int q = lo, within = j0 - s_off[lo];
+#pragma unroll
+      for (int e = 0; e < kGatherRun; ++e) {
+        from[e] = 0;
+        if (e < cnt) {
+          while (within >= s_off[q + 1] - s_off[q]) { within = 0; ++q; }  // entry e exists, so this ends inside the block
+          from[e] = (uint32_t)((seg0 + q) * kSegElems + within);
+          ++within;
+        }
+      }
+    }
+    uint32_t vals[kGatherRun], idxs[kGatherRun];
+#pragma unroll
+    for (int e = 0; e < kGatherRun; ++e) {
+      if (e < cnt) {
+        vals[e] = __ldg(p.seg_val + from[e]);
+        idxs[e] = __ldg(p.seg_idx + from[e]);
+      }
+    }
+#pragma unroll
+    for (int e = 0; e < kGatherRun; ++e) {
+      if (e < cnt) {
+        const uint32_t key = vals[e] & 0x7FFFFFFFu;
+        p.list_idx[base + j0 + e] = idxs[e];
+        p.list_val[base + j0 + e] = vals[e];
+        nonfinite |= key >= kInfKey;
+        atomicAdd(&s_hist[key >> digit_shift(0)], 1u);
+      }
+    }
+  }
+  if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
+  __syncthreads();
+  for (int b = threadIdx.x; b < kMaxBins; b += kCta) {
+    const unsigned int n_b = s_hist[b];
+    if (n_b) atomicAdd(&p.hist[b], n_b);
+  }
+}
+
 template <int DTYPE, int THREADS, int CACHE, bool CLUSTER = false>
 __global__ void __launch_bounds__(THREADS, 1024 / THREADS)  // at most 64 registers per thread
 k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
@@ -366,103 +463,9 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
       my_idx = p.list_idx + share_lo;
       my_val = p.list_val + share_lo;
       E = (unsigned int)(share_hi - share_lo);
-      if (E > 0 && thread_pos <= share_lo && share_lo < thread_pos + thread_sum) {  // exactly one thread
-        unsigned long long pos = thread_pos, gi = g_begin;
-        for (; gi < g_end; ++gi) {
-          const unsigned long long c = p.group_count[gi];
-          if (share_lo < pos + c) break;
-          pos += c;
-        }
-        sh.start[0] = gi;
-        sh.start[1] = pos;
-      }
-      __syncthreads();
-      unsigned long long seg_cursor = (E > 0) ? sh.start[0] * kGroupSegs : p.nseg;
-      unsigned long long pos_cursor = (E > 0) ? sh.start[1] : 0;
-      // A chunk is 8 segments per thread.  Thin stretches of the bucket make a
-      // share span many chunks, so the next chunk's counts are fetched before
-      // the current chunk's entries are copied.
-      auto load_counts = [&](unsigned long long first_seg) -> uint4 {
-        const unsigned long long s = first_seg + threadIdx.x * 8ull;  // a multiple of 8: the 16-byte load is aligned
-        if (s + 8 <= p.nseg) return *reinterpret_cast<const uint4*>(p.seg_count + s);
-        unsigned short c[8];
-  #pragma unroll
-        for (int e = 0; e < 8; ++e) c[e] = (s + e < p.nseg) ? p.seg_count[s + e] : (unsigned short)0;
-        uint4 v;
-        v.x = c[0] | ((uint32_t)c[1] << 16); v.y = c[2] | ((uint32_t)c[3] << 16);
-        v.z = c[4] | ((uint32_t)c[5] << 16); v.w = c[6] | ((uint32_t)c[7] << 16);
-        return v;
-      };
-      uint4 counts = load_counts(seg_cursor);
-      while (pos_cursor < share_hi && seg_cursor < p.nseg) {
-        const uint4 next_counts = load_counts(seg_cursor + (THREADS * 8));
-        const unsigned int cnt = (counts.x & 0xFFFFu) + (counts.x >> 16) + (counts.y & 0xFFFFu) + (counts.y >> 16) +
-                                 (counts.z & 0xFFFFu) + (counts.z >> 16) + (counts.w & 0xFFFFu) + (counts.w >> 16);
-        unsigned int chunk_total;
-        const unsigned int off = block_excl_scan(cnt, chunk_total, sh);
-        __syncthreads();  // sh.off / sh.cnt8 of the previous chunk have been read
-        sh.g.off[threadIdx.x] = off;
-        sh.g.cnt8[threadIdx.x] = counts;
-        __syncthreads();
-        // entries of this chunk that fall in the block's share
-        const unsigned long long from_pos = max(pos_cursor, share_lo), to_pos = min(pos_cursor + chunk_total, share_hi);
-        const unsigned short* cnt16 = reinterpret_cast<const unsigned short*>(sh.g.cnt8);  // count of segment q of the chunk
-        for (unsigned long long g0 = from_pos + threadIdx.x * (unsigned long long)kGatherRun; g0 < to_pos;
-             g0 += THREADS * (unsigned long long)kGatherRun) {
-          // kGatherRun consecutive entries per thread: the first is located by a search over the thread
-          // slots, the others by stepping on from it; all their loads are issued together.
-          const int cnt = (int)min((unsigned long long)kGatherRun, to_pos - g0);
-          uint32_t from[kGatherRun];  // list slot of each entry (below 2^31)
-          {
-            unsigned int q = 0, within = 0;
-            auto locate = [&](unsigned int j) {  // segment q of the chunk and place in it of the chunk's entry j
-              int lo = 0, hi = THREADS - 1;      // last thread slot of the chunk whose offset is <= j
-              while (lo < hi) {
-                const int mid = (lo + hi + 1) >> 1;
-                if (sh.g.off[mid] <= j) lo = mid; else hi = mid - 1;
-              }
-              within = j - sh.g.off[lo];
-              q = lo * 8;  // at most 8 steps: the entry lies in this slot's segments
-              while (within >= cnt16[q]) { within -= cnt16[q]; ++q; }
-            };
-            const unsigned int j0 = (unsigned int)(g0 - pos_cursor);
-            locate(j0);
-#pragma unroll
-            for (int e = 0; e < kGatherRun; ++e) {
-              from[e] = 0;
-              if (e < cnt) {
-                from[e] = (uint32_t)((seg_cursor + q) * kSegElems + within);
-                // the next entry is the next one of this segment, else it is searched for (a walk could
-                // cross any number of empty segments)
-                if (e + 1 < cnt && ++within >= cnt16[q]) locate(j0 + e + 1);
-              }
-            }
-          }
-          uint32_t vals[kGatherRun], idxs[kGatherRun];
-#pragma unroll
-          for (int e = 0; e < kGatherRun; ++e) {
-            if (e < cnt) {
-              vals[e] = p.seg_val[from[e]];
-              idxs[e] = p.seg_idx[from[e]];
-            }
-          }
-#pragma unroll
-          for (int e = 0; e < kGatherRun; ++e) {
-            if (e < cnt) {
-              const uint32_t key = vals[e] & 0x7FFFFFFFu;
-              put_entry((unsigned int)(g0 + e - share_lo), idxs[e], vals[e]);
-              nonfinite |= key >= kInfKey;
-              atomicAdd(&sh.hist[key >> digit_shift(0)], 1u);
-            }
-          }
-        }
-        pos_cursor += chunk_total;
-        seg_cursor += (THREADS * 8);
-        counts = next_counts;
-      }
-      if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
-      flush_hist<kMaxBins>(sh, p.hist);
-      if (!grid_barrier<CLUSTER>(p.ctl, ++barriers * G, sh)) return;
+      // k_gather has made the list contiguous and built the histogram of digit 0: the block's share is a
+      // plain range of it; its first CACHE values are copied into shared memory for the phases below.
+      for (unsigned int j = threadIdx.x; j < min(E, (unsigned int)CACHE); j += THREADS) cache_val[j] = __ldcg(my_val + j);
     }
 
     if (list_total < p.k) {
