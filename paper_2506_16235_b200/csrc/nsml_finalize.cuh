@@ -294,15 +294,20 @@ __device__ __forceinline__ void quantize_phase(const FinalizeParams& p, Finalize
 // search over the segments' offsets), so crowded segments are shared by all threads.
 constexpr int kGatherSegs = kGroupSegs;  // one group per block: its list position is a plain sum of group counts
 constexpr int kGatherRun = 4;      // consecutive candidates a thread copies per step
+constexpr int kGatherBins = 256;   // first-digit bins a block of the gather counts in shared memory
 
 __global__ void __launch_bounds__(kCta)
 k_gather(FinalizeParams p) {
-  __shared__ unsigned int s_hist[kMaxBins];
+  // Every candidate's key is >= the sampled bound lo, and almost all lie within a few octaves above it:
+  // the block counts first digits in a window of kGatherBins bins that starts at lo's bin (16 bins per
+  // octave); the rare key beyond the window goes to the global histogram directly.
+  __shared__ unsigned int s_hist[kGatherBins];
   __shared__ unsigned int s_off[kGatherSegs + 1];  // exclusive offsets of the block's segments, total at the end
   __shared__ unsigned long long s_red[kCta / 32];
   __shared__ unsigned int s_scan[kCta / 32];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int b = threadIdx.x; b < kMaxBins; b += kCta) s_hist[b] = 0;
+  for (int b = threadIdx.x; b < kGatherBins; b += kCta) s_hist[b] = 0;
+  const unsigned int first_bin = p.ctl->lo >> digit_shift(0);
   // list position of the block's first candidate
   const unsigned long long first_group = (unsigned long long)blockIdx.x * (kGatherSegs / kGroupSegs);
   unsigned long long before = 0;
@@ -371,15 +376,17 @@ k_gather(FinalizeParams p) {
         p.list_idx[base + j0 + e] = idxs[e];
         p.list_val[base + j0 + e] = vals[e];
         nonfinite |= key >= kInfKey;
-        atomicAdd(&s_hist[key >> digit_shift(0)], 1u);
+        const unsigned int bin = key >> digit_shift(0), rel = bin - first_bin;  // wraps only for a key below lo
+        if (rel < (unsigned int)kGatherBins) atomicAdd(&s_hist[rel], 1u);
+        else atomicAdd(&p.hist[bin], 1u);
       }
     }
   }
   if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
   __syncthreads();
-  for (int b = threadIdx.x; b < kMaxBins; b += kCta) {
+  for (int b = threadIdx.x; b < kGatherBins; b += kCta) {
     const unsigned int n_b = s_hist[b];
-    if (n_b) atomicAdd(&p.hist[b], n_b);
+    if (n_b) atomicAdd(&p.hist[first_bin + b], n_b);  // first_bin + b <= 4095: a count here came from a real key
   }
 }
 
