@@ -44,8 +44,8 @@ SWEEP = [(r, b) for r in (0.5, 0.1, 0.01, 0.001) for b in (8, 16)]
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
 # profiles/compress_kernels_gpt2_25M_ncu_full.md: 25M-element fp32 buckets, ratio 0.01, int8, W = 4.  Only valid
 # for that workload and for the kernels as they were when the capture was taken.
-NCU_TRAFFIC_25M = {"k_sample": 1.06e6, "k_compact_bucket": 104.1e6, "k_finalize": 4.5e6, "k_partition": 3.9e6,
-                   "k_merge": 49.1e6}
+NCU_TRAFFIC_25M = {"k_sample": 1.06e6, "k_compact_bucket": 103.6e6, "k_gather": 4.5e6, "k_finalize": 3.7e6,
+                   "k_partition": 3.9e6, "k_merge": 53.0e6}
 
 
 def measured_peak_gbs():
