@@ -629,10 +629,10 @@ class Alg2Workload(Workload):
                     self.account(acc, "k_prune_hist", 3 * 4 * n)
                     self.account(acc, "k_prune_ties", 3 * 4096 * 4)
                     self.account(acc, "k_prune_write", 4 * n + n // 8)
-                    self.account(acc, "k_feedback_add", 12 * n)
                     self.account(acc, "k_feedback_subtract", 13 * k)
                     self.compress_bytes(acc, n, 4, self.RATIO, self.BITS)
-                    self.account(acc, "k_compact_bucket", n // 8)  # the mask
+                    # the bucket pass also reads the mask and the residual and writes gradient + residual back
+                    self.account(acc, "k_compact_bucket", n // 8 + 8 * n)
                     self.merge_bytes(acc, n, [(k, self.BITS)])
 
             yield ((i * self.STATE + b) % self.GRADS, b), nsml.nsml_payload_bytes(n, self.RATIO, self.BITS), enqueue

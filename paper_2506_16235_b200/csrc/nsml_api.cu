@@ -78,7 +78,7 @@ struct LaunchScope {  // brackets one kernel launch
 struct DeviceInfo {
   bool ready = false;
   int sms = 0;
-  int compact_bucket = 0, finalize_small = 0, finalize_large = 0, merge = 0;  // resident blocks per SM
+  int compact_bucket = 0, compact_feedback = 0, finalize_small = 0, finalize_large = 0, merge = 0;  // resident blocks per SM
   int sumsq = 0, feedback_add = 0, prune_hist = 0, prune_write = 0, prune_write_ranked = 0;  // the same, streaming kernels
   bool finalize_cluster = false;  // the one-cluster shape of the list stage fits an SM
 };
@@ -93,7 +93,10 @@ static int device_info(const DeviceInfo** out) {
   if (!d.ready) {
     if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return NSML_ERR_CUDA;
     cudaError_t e = cudaSuccess;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_bucket, k_compact_bucket<NSML_F32>, kCta, 0);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_bucket, k_compact_bucket<NSML_F32, false>, kCta, 0);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_compact_bucket<NSML_F32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCompactFeedbackSmem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_compact_bucket<NSML_BF16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCompactFeedbackSmem);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_feedback, k_compact_bucket<NSML_F32, true>, kCta, kCompactFeedbackSmem);
     auto prepare = [&](auto kernel, int threads, int cache, int* resident) {
       if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)finalize_dyn_smem(cache));
       int r = 0;
@@ -133,7 +136,7 @@ static int device_info(const DeviceInfo** out) {
     if (e == cudaSuccess && (d.sumsq < 1 || d.feedback_add < 1 || d.prune_hist < 1 || d.prune_write < 1 || d.prune_write_ranked < 1)) e = cudaErrorUnknown;
     int coop = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    if (e != cudaSuccess || d.compact_bucket < 1 || d.finalize_small < 1 || d.finalize_large < 1 || d.merge < 1 || !coop) {
+    if (e != cudaSuccess || d.compact_bucket < 1 || d.compact_feedback < 1 || d.finalize_small < 1 || d.finalize_large < 1 || d.merge < 1 || !coop) {
       cudaGetLastError();
       return NSML_ERR_CUDA;
     }
@@ -193,9 +196,12 @@ static bool use_dense(int64_t n, int64_t k, const DeviceInfo& dev) {
   return sample_rank(n, k) == 0 || p_keep >= kDenseRatioAny || (fits_on_chip && p_keep >= kDenseRatioOnChip);
 }
 
-template <int DTYPE>
-static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, int64_t k, int bits, unsigned char* ws,
-                           unsigned char* payload, const CompressLayout& L, const PayloadLayout& P,
+// DTYPE: element type of `grad` (what the sample and the bucket pass read).  FDTYPE: element type of the
+// bucket the later stages re-read; with a residual (local accumulation fused into the bucket pass, list
+// strategy only) that bucket is the residual buffer, float32, which then holds gradient + residual.
+template <int DTYPE, int FDTYPE>
+static int launch_compress(const void* grad, float* residual, const uint32_t* mask, int64_t n, int64_t k, int bits,
+                           unsigned char* ws, unsigned char* payload, const CompressLayout& L, const PayloadLayout& P,
                            const DeviceInfo& dev, cudaStream_t st) {
   Ctl* ctl = reinterpret_cast<Ctl*>(ws);
   uint32_t* seg_idx = reinterpret_cast<uint32_t*>(ws + L.seg_idx);
@@ -203,6 +209,7 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
   unsigned short* seg_count = reinterpret_cast<unsigned short*>(ws + L.seg_count);
   const unsigned long long nseg = ((unsigned long long)n + kSegElems - 1) / kSegElems;
   BucketSrc<DTYPE> src{grad, mask};
+  BucketSrc<FDTYPE> fsrc{residual != nullptr ? static_cast<const void*>(residual) : grad, mask};
   const double p_keep = (double)k / (double)n;
   const unsigned long long large_cap_blocks = finalize_large_blocks(dev);
   const bool dense = use_dense(n, k, dev);
@@ -221,17 +228,23 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
   } else {
     {
       LaunchScope scope(K_SAMPLE, st);  // one cluster of kSampleBlocks blocks
-      k_sample<DTYPE><<<kSampleBlocks, kSampleThreads, 0, st>>>(src, (unsigned long long)n, sample_rank(n, k), ctl,
+      k_sample<DTYPE><<<kSampleBlocks, kSampleThreads, 0, st>>>(src, residual, (unsigned long long)n, sample_rank(n, k), ctl,
                                                                 reinterpret_cast<uint4*>(ws),
                                                                 (unsigned int)(L.zero_bytes / 16));
     }
     {
       // bucket pass: a block takes 8 segments per step; at most 4 resident blocks per SM
       LaunchScope scope(K_COMPACT_BUCKET, st);
-      const int per_sm = dev.compact_bucket < 4 ? dev.compact_bucket : 4;
+      const int resident = residual != nullptr ? dev.compact_feedback : dev.compact_bucket;
+      const int per_sm = resident < 4 ? resident : 4;
       const unsigned int grid = grid_for(nseg, kCta / 32, dev.sms * per_sm);
-      k_compact_bucket<DTYPE><<<grid, kCta, 0, st>>>(src, (unsigned long long)n, ctl, seg_idx, seg_val, seg_count,
-                                                     reinterpret_cast<unsigned int*>(ws + L.group_count));
+      unsigned int* group_count = reinterpret_cast<unsigned int*>(ws + L.group_count);
+      if (residual != nullptr)
+        k_compact_bucket<DTYPE, true><<<grid, kCta, kCompactFeedbackSmem, st>>>(src, residual, (unsigned long long)n, ctl, seg_idx,
+                                                                                seg_val, seg_count, group_count);
+      else
+        k_compact_bucket<DTYPE, false><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, ctl, seg_idx, seg_val,
+                                                              seg_count, group_count);
     }
     // list stage: cooperative, every block co-resident.  The small shape when a block's share of the
     // expected candidates (k plus the sampling margin) fits its shared-memory cache.
@@ -277,7 +290,7 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
   }
   {
     LaunchScope scope(dense ? K_FINALIZE_DENSE : K_FINALIZE, st);
-    void* args[] = {&src, &fp};
+    void* args[] = {&fsrc, &fp};
     cudaError_t le;
     auto launch = [&](auto kernel, int threads, int cache) {
       return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(fgrid), dim3(threads), args,
@@ -297,11 +310,11 @@ static int launch_compress(const void* grad, const uint32_t* mask, int64_t n, in
       attr[0].val.clusterDim.z = 1;
       cfg.attrs = attr;
       cfg.numAttrs = 1;
-      le = cudaLaunchKernelEx(&cfg, k_finalize<DTYPE, kFinClusterThreads, kFinClusterCache, true>, src, fp);
-    } else if (small_shape && dense) le = launch(k_finalize_dense<DTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
-    else if (small_shape) le = launch(k_finalize<DTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
-    else if (dense) le = launch(k_finalize_dense<DTYPE, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache);
-    else le = launch(k_finalize<DTYPE, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache);
+      le = cudaLaunchKernelEx(&cfg, k_finalize<FDTYPE, kFinClusterThreads, kFinClusterCache, true>, fsrc, fp);
+    } else if (small_shape && dense) le = launch(k_finalize_dense<FDTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
+    else if (small_shape) le = launch(k_finalize<FDTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
+    else if (dense) le = launch(k_finalize_dense<FDTYPE, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache);
+    else le = launch(k_finalize<FDTYPE, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache);
     if (le != cudaSuccess) return NSML_ERR_CUDA;
   }
   return NSML_OK;
@@ -325,8 +338,8 @@ static int compress_impl(const void* grad, int64_t n, int grad_dtype, double rat
   if (rc != NSML_OK) return rc;
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   unsigned char* pl = static_cast<unsigned char*>(payload);
-  if (grad_dtype == NSML_F32) rc = launch_compress<NSML_F32>(grad, prune_mask, n, k, bits, ws, pl, L, P, *dev, st);
-  else rc = launch_compress<NSML_BF16>(grad, prune_mask, n, k, bits, ws, pl, L, P, *dev, st);
+  if (grad_dtype == NSML_F32) rc = launch_compress<NSML_F32, NSML_F32>(grad, nullptr, prune_mask, n, k, bits, ws, pl, L, P, *dev, st);
+  else rc = launch_compress<NSML_BF16, NSML_BF16>(grad, nullptr, prune_mask, n, k, bits, ws, pl, L, P, *dev, st);
   if (rc != NSML_OK) return rc;
   if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
   return NSML_OK;
@@ -509,16 +522,31 @@ static int feedback_impl(const void* grad, float* residual, int64_t n, int grad_
   const DeviceInfo* dev = nullptr;
   int rc = device_info(&dev);
   if (rc != NSML_OK) return rc;
-  const unsigned int grid = stream_grid(n, *dev, dev->feedback_add < 8 ? dev->feedback_add : 8, 1u << 16);
-  {
-    LaunchScope scope(K_FEEDBACK_ADD, st);
+  if (use_dense(n, k, *dev)) {
+    // dense strategy (no bucket pass to fuse the add into): residual <- grad + residual first, then the select
+    // over the residual buffer
+    const unsigned int grid = stream_grid(n, *dev, dev->feedback_add < 8 ? dev->feedback_add : 8, 1u << 16);
+    {
+      LaunchScope scope(K_FEEDBACK_ADD, st);
+      if (grad_dtype == NSML_F32)
+        k_feedback_add<NSML_F32><<<grid, kCta, 0, st>>>(BucketSrc<NSML_F32>{grad, nullptr}, residual, (unsigned long long)n);
+      else
+        k_feedback_add<NSML_BF16><<<grid, kCta, 0, st>>>(BucketSrc<NSML_BF16>{grad, nullptr}, residual, (unsigned long long)n);
+    }
+    rc = compress_impl(residual, n, NSML_F32, ratio, bits, prune_mask, payload, payload_capacity, workspace,
+                       workspace_bytes, st);
+  } else {
+    // list strategy: the bucket pass adds the residual as it streams the gradient and leaves the sum in it
+    if (prune_mask != nullptr && !aligned(prune_mask, 4)) return NSML_ERR_ARG;
+    unsigned char* ws = static_cast<unsigned char*>(workspace);
+    unsigned char* pl = static_cast<unsigned char*>(payload);
+    const PayloadLayout P = payload_layout(k, bits);
+    const CompressLayout L = compress_layout(n);
     if (grad_dtype == NSML_F32)
-      k_feedback_add<NSML_F32><<<grid, kCta, 0, st>>>(BucketSrc<NSML_F32>{grad, nullptr}, residual, (unsigned long long)n);
+      rc = launch_compress<NSML_F32, NSML_F32>(grad, residual, prune_mask, n, k, bits, ws, pl, L, P, *dev, st);
     else
-      k_feedback_add<NSML_BF16><<<grid, kCta, 0, st>>>(BucketSrc<NSML_BF16>{grad, nullptr}, residual, (unsigned long long)n);
+      rc = launch_compress<NSML_BF16, NSML_F32>(grad, residual, prune_mask, n, k, bits, ws, pl, L, P, *dev, st);
   }
-  rc = compress_impl(residual, n, NSML_F32, ratio, bits, prune_mask, payload, payload_capacity, workspace,
-                     workspace_bytes, st);
   if (rc != NSML_OK) return rc;
   {
     LaunchScope scope(K_FEEDBACK_SUBTRACT, st);

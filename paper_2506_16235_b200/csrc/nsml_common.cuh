@@ -154,6 +154,15 @@ struct BucketSrc {
     }
   }
 
+  // element i as stored (no pruning mask applied), and whether the mask prunes it
+  __device__ __forceinline__ uint32_t raw1(unsigned long long i) const {
+    if (DTYPE == NSML_F32) return static_cast<const uint32_t*>(grad)[i];
+    return (uint32_t)static_cast<const uint16_t*>(grad)[i] << 16;
+  }
+  __device__ __forceinline__ bool pruned(unsigned long long i) const {
+    return mask != nullptr && ((mask[i >> 5] >> (unsigned)(i & 31)) & 1u);
+  }
+
   __device__ __forceinline__ uint32_t load1(unsigned long long i) const {
     if (mask != nullptr && ((mask[i >> 5] >> (unsigned)(i & 31)) & 1u)) return 0;
     if (DTYPE == NSML_F32) return static_cast<const uint32_t*>(grad)[i];

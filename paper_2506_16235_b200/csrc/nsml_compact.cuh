@@ -23,6 +23,8 @@ namespace nsml {
 
 constexpr int kRound = 128;                       // elements a warp handles per step (32 lanes x 4)
 constexpr int kSegRounds = kSegElems / kRound;    // 4
+// dynamic shared memory of the bucket pass with local accumulation: the residual's double buffers
+constexpr size_t kCompactFeedbackSmem = (size_t)(kCta / 32) * 2 * kSegRounds * 32 * 16;
 
 // Appends the kept elements of one round.  `f` holds this lane's four keep
 // flags (bit e = element lane*4+e of the round).  Returns the round's total.
@@ -82,17 +84,24 @@ __device__ __forceinline__ unsigned int keep_flags(const uint32_t (&bits)[4], fl
   return f;
 }
 
-template <int DTYPE>
+// FEEDBACK: the bucket that is compressed is gradient + residual (Section 4.2 Step 3, local accumulation of
+// the filtered gradients).  The residual is streamed beside the gradient, the sum (one float32 add per
+// element) is written back over the residual and is what the candidates are taken from; the pruning mask
+// zeroes a key, not the stored sum.
+template <int DTYPE, bool FEEDBACK = false>
 __global__ void __launch_bounds__(kCta)
-k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, uint32_t* __restrict__ seg_idx,
-                 uint32_t* __restrict__ seg_val, unsigned short* __restrict__ seg_count,
+k_compact_bucket(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned long long n, Ctl* ctl,
+                 uint32_t* __restrict__ seg_idx, uint32_t* __restrict__ seg_val, unsigned short* __restrict__ seg_count,
                  unsigned int* __restrict__ group_count) {
   constexpr int ESIZE = (DTYPE == NSML_F32) ? 4 : 2;
   constexpr int LANE_BYTES = 4 * ESIZE;
   constexpr int BUF_BYTES = kSegRounds * 32 * LANE_BYTES;  // one segment of one warp
+  constexpr int RBUF_BYTES = FEEDBACK ? kSegRounds * 32 * 16 : 0;  // the same segment of the residual
   __shared__ __align__(16) unsigned char s_fifo[(kCta / 32) * 2 * BUF_BYTES];
+  extern __shared__ __align__(16) unsigned char s_rfifo[];  // FEEDBACK only: (kCta / 32) * 2 * RBUF_BYTES bytes
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   unsigned char* fifo = s_fifo + (size_t)w * 2 * BUF_BYTES + lane * LANE_BYTES;  // round r of buffer b at + (b*kSegRounds + r)*32*LANE_BYTES
+  unsigned char* rfifo = s_rfifo + (size_t)w * 2 * RBUF_BYTES + lane * 16;       // the same for the residual: + (b*kSegRounds + r)*32*16
 
   const unsigned long long nseg = (n + kSegElems - 1) / kSegElems;
   const unsigned long long nseg_full = n / kSegElems;  // segments that need no bounds checks
@@ -102,8 +111,10 @@ k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, uint32_t*
   unsigned long long seg = (unsigned long long)blockIdx.x * (kCta / 32) + w;
   if (seg < nseg_full) {
 #pragma unroll
-    for (int r = 0; r < kSegRounds; ++r)
+    for (int r = 0; r < kSegRounds; ++r) {
       cp_async_lane<LANE_BYTES>(fifo + r * 32 * LANE_BYTES, g + (seg * kSegElems + r * kRound) * ESIZE);
+      if (FEEDBACK) cp_async_lane<16>(rfifo + r * 32 * 16, residual + seg * kSegElems + r * kRound + lane * 4);
+    }
   }
   cp_async_commit();
   // The segment's 16 words of the pruning mask (64 bytes) are fetched by lanes 0-15 one segment ahead, like
@@ -120,9 +131,12 @@ k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, uint32_t*
     const unsigned long long next = seg + step;
     if (next < nseg_full) {
 #pragma unroll
-      for (int r = 0; r < kSegRounds; ++r)
+      for (int r = 0; r < kSegRounds; ++r) {
         cp_async_lane<LANE_BYTES>(fifo + ((buf ^ 1) * kSegRounds + r) * 32 * LANE_BYTES,
                                   g + (next * kSegElems + r * kRound) * ESIZE);
+        if (FEEDBACK)
+          cp_async_lane<16>(rfifo + ((buf ^ 1) * kSegRounds + r) * 32 * 16, residual + next * kSegElems + r * kRound + lane * 4);
+      }
     }
     if (src.mask != nullptr && next < nseg_full && lane < kSegMaskWords)
       mask_words_next = __ldg(src.mask + next * kSegMaskWords + lane);
@@ -144,6 +158,17 @@ k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, uint32_t*
           bits[0] = v.x << 16; bits[1] = v.x & 0xFFFF0000u;
           bits[2] = v.y << 16; bits[3] = v.y & 0xFFFF0000u;
         }
+        if (FEEDBACK) {
+          const float4 rv = *reinterpret_cast<const float4*>(rfifo + (buf * kSegRounds + r) * 32 * 16);
+          float4 acc;
+          acc.x = __fadd_rn(__uint_as_float(bits[0]), rv.x);
+          acc.y = __fadd_rn(__uint_as_float(bits[1]), rv.y);
+          acc.z = __fadd_rn(__uint_as_float(bits[2]), rv.z);
+          acc.w = __fadd_rn(__uint_as_float(bits[3]), rv.w);
+          *reinterpret_cast<float4*>(residual + seg_base + r * kRound + lane * 4) = acc;
+          bits[0] = __float_as_uint(acc.x); bits[1] = __float_as_uint(acc.y);
+          bits[2] = __float_as_uint(acc.z); bits[3] = __float_as_uint(acc.w);
+        }
         if (src.mask != nullptr) {
           const uint32_t word = __shfl_sync(0xFFFFFFFFu, mask_words, r * (kRound / 32) + (lane >> 3));
           const uint32_t m = (word >> (unsigned)((lane & 7) * 4)) & 0xFu;
@@ -153,7 +178,20 @@ k_compact_bucket(BucketSrc<DTYPE> src, unsigned long long n, Ctl* ctl, uint32_t*
         }
       } else {
         // the bucket's ragged last segment: plain loads, missing elements read as 0 and are never kept
-        src.load_vals4(seg_base + r * kRound + lane * 4, n, bits);
+        if (FEEDBACK) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const unsigned long long i = seg_base + r * kRound + lane * 4 + e;
+            bits[e] = 0;
+            if (i < n) {
+              const float acc = __fadd_rn(__uint_as_float(src.raw1(i)), residual[i]);
+              residual[i] = acc;
+              bits[e] = src.pruned(i) ? 0u : __float_as_uint(acc);
+            }
+          }
+        } else {
+          src.load_vals4(seg_base + r * kRound + lane * 4, n, bits);
+        }
       }
       const unsigned int f = keep_flags(bits, t);
       if (!__any_sync(0xFFFFFFFFu, f != 0)) continue;

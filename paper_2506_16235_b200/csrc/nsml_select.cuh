@@ -70,12 +70,12 @@ __device__ __forceinline__ void find_digit_from_top(const unsigned int (&own)[PE
 }
 
 // Clears the per-call control region and sets ctl->lo from a stratified
-// sample.  rank_from_top == 0 means "no sampling" (small bucket, or nearly
+// sample of the bucket (of bucket + addend when an addend is given).  rank_from_top == 0 means "no sampling" (small bucket, or nearly
 // everything is kept): lo = 0.
 template <int DTYPE>
 __global__ void __cluster_dims__(kSampleBlocks, 1, 1) __launch_bounds__(kSampleThreads)
-k_sample(BucketSrc<DTYPE> src, unsigned long long n, unsigned int rank_from_top, Ctl* ctl, uint4* zero_base,
-         unsigned int zero_vec16) {
+k_sample(BucketSrc<DTYPE> src, const float* __restrict__ addend, unsigned long long n, unsigned int rank_from_top,
+         Ctl* ctl, uint4* zero_base, unsigned int zero_vec16) {
   namespace cg = cooperative_groups;
   __shared__ unsigned int s_keys[kSamples];  // block 0: the sample keys, then (first 4096 words) the histogram
   unsigned int* s_hist = s_keys;
@@ -89,7 +89,10 @@ k_sample(BucketSrc<DTYPE> src, unsigned long long n, unsigned int rank_from_top,
     const unsigned long long begin = stratum * n / kSamples;
     const unsigned long long end = (stratum + 1) * n / kSamples;  // > begin because n >= 2 * kSamples
     const unsigned long long pos = begin + mix32((uint32_t)stratum * 0x9E3779B1u + 0x85EBCA6Bu) % (uint32_t)(end - begin);
-    const uint32_t key = src.load1(pos) & 0x7FFFFFFFu;
+    // with an addend (the residual of the local accumulation) the bucket that is selected from is the sum
+    uint32_t bits = src.load1(pos);
+    if (addend != nullptr && !src.pruned(pos)) bits = __float_as_uint(__fadd_rn(__uint_as_float(src.raw1(pos)), addend[pos]));
+    const uint32_t key = bits & 0x7FFFFFFFu;
     unsigned int* remote = cluster.map_shared_rank(s_keys, 0);
     remote[stratum] = key;
   }
