@@ -259,35 +259,47 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
   for (int b = threadIdx.x; b < NB; b += kCta) s_hist[b] = 0;
   __syncthreads();
   const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
-  bool nonfinite = false;
-  for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-    uint32_t bits[kStreamLoads][4];
-    int cnt[kStreamLoads];
-    load_tile(src, tile * kStreamTile, n, bits, cnt);
-#pragma unroll
-    for (int u = 0; u < kStreamLoads; ++u) {
-#pragma unroll
-      for (int e = 0; e < 4; ++e) {
-        if (e < cnt[u]) {
-          const uint32_t key = prune_key(bits[u][e]);
-          if (LEVEL == 0) {
-            nonfinite |= key <= 0x007FFFFFu;  // magnitude bits >= 0x7F800000
-            atomicAdd(&s_hist[key >> 19], 1u);
-          } else if (LEVEL == 1) {
-            if ((key >> 19) == prefix) atomicAdd(&s_hist[(key >> 7) & 0xFFFu], 1u);
-          } else {
-            if ((key >> 7) == prefix) {
-              atomicAdd(&s_hist[key & 0x7Fu], 1u);
-              if (collect) {
-                const unsigned long long i = tile * kStreamTile + (unsigned long long)(u * kCta + threadIdx.x) * 4 + e;
-                tie_list[atomicAdd(&ctl->list_count, 1u)] = make_uint2((uint32_t)i, key & 0x7Fu);
-              }
-            }
-          }
+  uint32_t lowest = 0x7FFFFFFFu;  // smallest complemented key seen: at most 0x007FFFFF for a NaN or an infinity
+  // one key; (tile, u, e) locate it and are turned into an index only where one is needed
+  auto visit = [&](uint32_t key, unsigned long long tile, int u, int e) {
+    if (LEVEL == 0) {
+      lowest = min(lowest, key);
+      atomicAdd(&s_hist[key >> 19], 1u);
+    } else if (LEVEL == 1) {
+      if ((key >> 19) == prefix) atomicAdd(&s_hist[(key >> 7) & 0xFFFu], 1u);
+    } else {
+      if ((key >> 7) == prefix) {
+        atomicAdd(&s_hist[key & 0x7Fu], 1u);
+        if (collect) {
+          const unsigned long long i = tile * kStreamTile + (unsigned long long)(u * kCta + threadIdx.x) * 4 + e;
+          tie_list[atomicAdd(&ctl->list_count, 1u)] = make_uint2((uint32_t)i, key & 0x7Fu);
         }
       }
     }
+  };
+  for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    const unsigned long long base = tile * kStreamTile;
+    uint32_t bits[kStreamLoads][4];
+    if (base + kStreamTile <= n) {  // a whole tile: no bounds checks
+#pragma unroll
+      for (int u = 0; u < kStreamLoads; ++u) src.load_full4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, bits[u]);
+#pragma unroll
+      for (int u = 0; u < kStreamLoads; ++u)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) visit(prune_key(bits[u][e]), tile, u, e);
+    } else {
+      int cnt[kStreamLoads];
+#pragma unroll
+      for (int u = 0; u < kStreamLoads; ++u)
+        cnt[u] = src.load_vals4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, n, bits[u]);
+#pragma unroll
+      for (int u = 0; u < kStreamLoads; ++u)
+#pragma unroll
+        for (int e = 0; e < 4; ++e)
+          if (e < cnt[u]) visit(prune_key(bits[u][e]), tile, u, e);
+    }
   }
+  const bool nonfinite = LEVEL == 0 && lowest <= 0x007FFFFFu;  // magnitude bits >= 0x7F800000
   if (nonfinite) set_status(&ctl->status, NSML_ERR_NONFINITE);
   __syncthreads();
   unsigned int* ghist = hist + LEVEL * kMaxBins;
@@ -379,28 +391,48 @@ k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl
     // Every key > T is pruned, and every key == T (or, by_index, those up to idx_limit).  A warp's load
     // covers 128 consecutive elements = 4 mask words; the 4-bit
     // flags of 8 neighbouring lanes are combined into one word.
+    // flags of this thread's four elements of load u -> the word shared by eight lanes
+    auto word_of = [&](unsigned int f) {
+      unsigned int x = f << (4 * (lane & 7));
+      x |= __shfl_xor_sync(0xFFFFFFFFu, x, 1);
+      x |= __shfl_xor_sync(0xFFFFFFFFu, x, 2);
+      x |= __shfl_xor_sync(0xFFFFFFFFu, x, 4);
+      return x;
+    };
+    auto is_pruned = [&](uint32_t key, unsigned long long base, int u, int e) {
+      if (key == T)  // rare: the index is worked out only here (indices are below 2^31)
+        return !by_index || (uint32_t)base + (uint32_t)((u * kCta + threadIdx.x) * 4 + e) <= idx_limit;
+      return key > T;
+    };
     for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
       const unsigned long long base = tile * kStreamTile;
       uint32_t bits[kStreamLoads][4];
-      int cnt[kStreamLoads];
-      load_tile(src, base, n, bits, cnt);
+      uint32_t* out = mask + base / 32 + warp * 4 + (lane >> 3);  // word of load 0; load u is 32 words further
+      if (base + kStreamTile <= n) {  // a whole tile: no bounds checks
 #pragma unroll
-      for (int u = 0; u < kStreamLoads; ++u) {
-        unsigned int f = 0;
+        for (int u = 0; u < kStreamLoads; ++u) src.load_full4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, bits[u]);
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
-          const uint32_t key = prune_key(bits[u][e]);
-          bool pruned = key > T;
-          if (key == T)  // rare: the index is worked out only here (indices are below 2^31)
-            pruned = !by_index || (uint32_t)base + (uint32_t)((u * kCta + threadIdx.x) * 4 + e) <= idx_limit;
-          f |= (unsigned)((e < cnt[u]) && pruned) << e;
+        for (int u = 0; u < kStreamLoads; ++u) {
+          unsigned int f = 0;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) f |= (unsigned)is_pruned(prune_key(bits[u][e]), base, u, e) << e;
+          const unsigned int x = word_of(f);
+          if ((lane & 7) == 0) out[u * (kCta / 8)] = x;
         }
-        unsigned int x = f << (4 * (lane & 7));
-        x |= __shfl_xor_sync(0xFFFFFFFFu, x, 1);
-        x |= __shfl_xor_sync(0xFFFFFFFFu, x, 2);
-        x |= __shfl_xor_sync(0xFFFFFFFFu, x, 4);
-        const unsigned long long word = (base + (unsigned long long)(u * kCta + warp * 32) * 4) / 32 + (lane >> 3);
-        if ((lane & 7) == 0 && word < nwords) mask[word] = x;
+      } else {
+        int cnt[kStreamLoads];
+#pragma unroll
+        for (int u = 0; u < kStreamLoads; ++u)
+          cnt[u] = src.load_vals4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, n, bits[u]);
+#pragma unroll
+        for (int u = 0; u < kStreamLoads; ++u) {
+          unsigned int f = 0;
+#pragma unroll
+          for (int e = 0; e < 4; ++e) f |= (unsigned)((e < cnt[u]) && is_pruned(prune_key(bits[u][e]), base, u, e)) << e;
+          const unsigned int x = word_of(f);
+          const unsigned long long word = base / 32 + warp * 4 + (lane >> 3) + (unsigned long long)u * (kCta / 8);
+          if ((lane & 7) == 0 && word < nwords) mask[word] = x;
+        }
       }
     }
   }
