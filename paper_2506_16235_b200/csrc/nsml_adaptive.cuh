@@ -404,6 +404,9 @@ k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl
         return !by_index || (uint32_t)base + (uint32_t)((u * kCta + threadIdx.x) * 4 + e) <= idx_limit;
       return key > T;
     };
+    // The same test on the weight itself: complemented key > T  <=>  |w| < tmag, key == T  <=>  |w| == tmag
+    // (finite weights; denormals are not flushed), one compare with a free |.| instead of mask and compare.
+    const float tmag = __uint_as_float(~T & 0x7FFFFFFFu);
     for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
       const unsigned long long base = tile * kStreamTile;
       uint32_t bits[kStreamLoads][4];
@@ -414,8 +417,18 @@ k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl
 #pragma unroll
         for (int u = 0; u < kStreamLoads; ++u) {
           unsigned int f = 0;
+          bool tie = false;
 #pragma unroll
-          for (int e = 0; e < 4; ++e) f |= (unsigned)is_pruned(prune_key(bits[u][e]), base, u, e) << e;
+          for (int e = 0; e < 4; ++e) {
+            const float a = fabsf(__uint_as_float(bits[u][e]));
+            f |= (unsigned)(a < tmag) << e;
+            tie |= a == tmag;
+          }
+          if (tie) {  // rare
+            f = 0;
+#pragma unroll
+            for (int e = 0; e < 4; ++e) f |= (unsigned)is_pruned(prune_key(bits[u][e]), base, u, e) << e;
+          }
           const unsigned int x = word_of(f);
           if ((lane & 7) == 0) out[u * (kCta / 8)] = x;
         }
