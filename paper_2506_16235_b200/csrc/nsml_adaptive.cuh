@@ -237,6 +237,17 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
   __shared__ unsigned int s_tot[kCta / 32], s_out[2];
   unsigned int prefix = 0;
   bool collect = false;
+  // The block's first tile is requested before the previous level is resolved, so that the resolve (a read
+  // of the 4096 global bins and a block-wide search) runs while those loads are in flight.
+  const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
+  uint32_t bits[kStreamLoads][4];
+  bool preloaded = false;
+  if (LEVEL != 0 && ((unsigned long long)blockIdx.x + 1) * kStreamTile <= n) {
+#pragma unroll
+    for (int u = 0; u < kStreamLoads; ++u)
+      src.load_full4((unsigned long long)blockIdx.x * kStreamTile + (unsigned long long)(u * kCta + threadIdx.x) * 4, bits[u]);
+    preloaded = true;
+  }
   if (LEVEL == 1) {
     prune_resolve<kMaxBins>(hist, m, s_tot, s_out);
     prefix = s_out[0];
@@ -258,7 +269,6 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
   }
   for (int b = threadIdx.x; b < NB; b += kCta) s_hist[b] = 0;
   __syncthreads();
-  const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
   uint32_t lowest = 0x7FFFFFFFu;  // smallest complemented key seen: at most 0x007FFFFF for a NaN or an infinity
   // one key; (tile, u, e) locate it and are turned into an index only where one is needed
   auto visit = [&](uint32_t key, unsigned long long tile, int u, int e) {
@@ -279,10 +289,12 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
   };
   for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
     const unsigned long long base = tile * kStreamTile;
-    uint32_t bits[kStreamLoads][4];
     if (base + kStreamTile <= n) {  // a whole tile: no bounds checks
+      if (!preloaded) {
 #pragma unroll
-      for (int u = 0; u < kStreamLoads; ++u) src.load_full4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, bits[u]);
+        for (int u = 0; u < kStreamLoads; ++u) src.load_full4(base + (unsigned long long)(u * kCta + threadIdx.x) * 4, bits[u]);
+      }
+      preloaded = false;
 #pragma unroll
       for (int u = 0; u < kStreamLoads; ++u)
 #pragma unroll
