@@ -218,3 +218,41 @@ def test_strategy_switch_is_invisible():
         seen.add(nsml.nsml_compress_strategy(n, ratio))
         check_compress(g, ratio, 8)
     assert seen == {0, 1}
+
+
+def test_buckets_on_concurrent_streams_and_replayed_from_a_graph():
+    # independent buckets on eight streams with their own workspaces (as the benchmark runs them), nothing
+    # synchronised in between; then one of the calls captured into a CUDA graph and replayed on new data
+    rng = np.random.default_rng(77)
+    cases = []
+    for s in range(8):
+        n = int(rng.integers(200_000, 900_000))
+        g = (rng.standard_normal(n) * 10.0 ** rng.uniform(-4, -1, n)).astype(np.float32)
+        ratio, bits = [(0.01, 8), (0.001, 16), (0.1, 8), (0.5, 16), (0.03, 32), (0.01, 16), (0.3, 8), (0.002, 8)][s]
+        cases.append((g, ratio, bits))
+    streams = [torch.cuda.Stream() for _ in cases]
+    grads = [to_device_grad(g) for g, _, _ in cases]
+    wss = [nsml.alloc_bytes(nsml.nsml_workspace_bytes(g.size), "cuda") for g, _, _ in cases]
+    torch.cuda.synchronize()
+    payloads = []
+    for rep in range(3):  # the same calls again and again, still without waiting
+        payloads = [nsml.nsml_compress(grads[i], r, b, workspace=wss[i], stream=streams[i])
+                    for i, (_, r, b) in enumerate(cases)]
+    torch.cuda.synchronize()
+    for i, (g, r, b) in enumerate(cases):
+        assert nsml.nsml_last_status(wss[i]) == 0
+        assert_payload_equal(payloads[i], oracle_compress(g, r, b))
+
+    g, ratio, bits = cases[0]
+    buf, ws = grads[0], wss[0]
+    payload = nsml.alloc_bytes(nsml.nsml_payload_bytes(g.size, ratio, bits), "cuda")
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        nsml.nsml_compress(buf, ratio, bits, payload=payload, workspace=ws, stream=side)
+    for rep in range(2):
+        fresh = np.roll(g, 1234 * (rep + 1))
+        buf.copy_(torch.from_numpy(fresh))
+        graph.replay()
+        torch.cuda.synchronize()
+        assert_payload_equal(payload[:nsml.nsml_payload_bytes(g.size, ratio, bits)], oracle_compress(fresh, ratio, bits))
