@@ -595,15 +595,53 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   resolve_digit<128>(p.hist + 2 * kMaxBins, rem, sh);
   const uint32_t T = (prefix24 << 7) | sh.out[0];
   const unsigned long long r = sh.out[1];  // ties (key == T) to keep, lowest index first
-  unsigned long long mine_a = 0, mine_c = 0;
-  for_each_key([&](uint32_t key) {
-    mine_a += key > T;
-    mine_c += key == T;
-  });
-  const unsigned long long block_a = block_sum(mine_a, sh);
-  const unsigned long long block_c = block_sum(mine_c, sh);
+  // Each warp owns two contiguous runs of the block's candidates: its slice of those cached in shared
+  // memory and its slice of the rest (so that the slow loads of uncached values are spread over all
+  // warps).  Here the keys > T and == T of each run are counted; the run totals stay in shared memory for
+  // the write phase and their sum is the block's count.
+  constexpr int NW = THREADS / 32;
+  const int warp = threadIdx.x >> 5;
+  const unsigned int lt = (1u << lane) - 1u;
+  const unsigned int cached = min(E, (unsigned int)CACHE);
+  unsigned int run_lo[2], run_hi[2];
+  {
+    const unsigned int per_a = ((cached + NW - 1) / NW + 31) / 32 * 32;
+    const unsigned int per_b = ((E - cached + NW - 1) / NW + 31) / 32 * 32;
+    run_lo[0] = min(cached, warp * per_a);
+    run_hi[0] = min(cached, run_lo[0] + per_a);
+    run_lo[1] = min(E, cached + warp * per_b);
+    run_hi[1] = min(E, run_lo[1] + per_b);
+  }
+  __syncthreads();  // sh.run may still be read from an earlier call
+#pragma unroll
+  for (int q = 0; q < 2; ++q) {
+    unsigned int wa = 0, wc = 0;
+    for (unsigned int j0 = run_lo[q]; j0 < run_hi[q]; j0 += 128) {  // four rounds of 32, their loads issued together
+      uint32_t key[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const unsigned int j = j0 + u * 32 + lane;
+        key[u] = (j < run_hi[q]) ? (entry_val(j) & 0x7FFFFFFFu) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const bool live = j0 + u * 32 + lane < run_hi[q];
+        wa += __popc(__ballot_sync(0xFFFFFFFFu, live && key[u] > T));
+        wc += __popc(__ballot_sync(0xFFFFFFFFu, live && key[u] == T));
+      }
+    }
+    if (lane == 0) sh.run[q * NW + warp] = ((unsigned long long)wa << 32) | wc;
+  }
+  __syncthreads();
   unsigned long long* ac_counts = p.block_counts + 1 * kMaxFinalizeBlocks;
-  if (threadIdx.x == 0) ac_counts[blk] = (block_a << 32) | block_c;
+  if (threadIdx.x == 0) {
+    unsigned long long block_a = 0, block_c = 0;
+    for (int w = 0; w < 2 * NW; ++w) {
+      block_a += sh.run[w] >> 32;
+      block_c += sh.run[w] & 0xFFFFFFFFull;
+    }
+    ac_counts[blk] = (block_a << 32) | block_c;
+  }
   if (!grid_barrier<CLUSTER>(p.ctl, ++barriers * G, sh)) return;
 
   // ---------------- phase 4: write the survivors in index order ----------------
@@ -627,43 +665,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   }
   uint32_t* out_idx = reinterpret_cast<uint32_t*>(p.payload + p.P.idx_off);
   {
-    // Each warp owns two contiguous runs of the block's candidates: its slice of those cached in shared
-    // memory and its slice of the rest (so that the slow loads of uncached values are spread over all
-    // warps).  First pass: count the keys > T and == T of each run; one exchange of the run totals through
-    // shared memory; second pass: ranks by ballot, coalesced writes.
-    constexpr int NW = THREADS / 32;
-    const int warp = threadIdx.x >> 5;
-    const unsigned int lt = (1u << lane) - 1u;
-    const unsigned int cached = min(E, (unsigned int)CACHE);
-    unsigned int run_lo[2], run_hi[2];
-    {
-      const unsigned int per_a = ((cached + NW - 1) / NW + 31) / 32 * 32;
-      const unsigned int per_b = ((E - cached + NW - 1) / NW + 31) / 32 * 32;
-      run_lo[0] = min(cached, warp * per_a);
-      run_hi[0] = min(cached, run_lo[0] + per_a);
-      run_lo[1] = min(E, cached + warp * per_b);
-      run_hi[1] = min(E, run_lo[1] + per_b);
-    }
-#pragma unroll
-    for (int q = 0; q < 2; ++q) {
-      unsigned int wa = 0, wc = 0;
-      for (unsigned int j0 = run_lo[q]; j0 < run_hi[q]; j0 += 128) {  // four rounds of 32, their loads issued together
-        uint32_t key[4];
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const unsigned int j = j0 + u * 32 + lane;
-          key[u] = (j < run_hi[q]) ? (entry_val(j) & 0x7FFFFFFFu) : 0u;
-        }
-#pragma unroll
-        for (int u = 0; u < 4; ++u) {
-          const bool live = j0 + u * 32 + lane < run_hi[q];
-          wa += __popc(__ballot_sync(0xFFFFFFFFu, live && key[u] > T));
-          wc += __popc(__ballot_sync(0xFFFFFFFFu, live && key[u] == T));
-        }
-      }
-      if (lane == 0) sh.run[q * NW + warp] = ((unsigned long long)wa << 32) | wc;
-    }
-    __syncthreads();
+    // ranks by ballot on top of the run totals counted in phase 3, coalesced writes
 #pragma unroll
     for (int q = 0; q < 2; ++q) {
       unsigned long long a_here = a_before, c_here = c_before;
