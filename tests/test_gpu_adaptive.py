@@ -265,3 +265,47 @@ def test_gradient_exchange_single_rank_follows_the_controller():
         got = dense.cpu().numpy()
         ref = oracle.decompress_sum([want], n)
         assert np.max(np.abs(got.astype(np.float64) - ref.astype(np.float64))) <= 1e-6 * float(np.abs(g).max())
+
+
+# ------------------------------------------------------------------ corner paths of the new steps
+def test_prune_mask_small_tie_group_at_the_threshold():
+    # exactly three weights share the threshold magnitude and only some of them are pruned: decided by index
+    n = 100_001
+    rng = np.random.default_rng(31)
+    w = ((rng.permutation(n).astype(np.float32) + 1.0) * np.float32(1e-4)) * rng.choice(np.array([-1.0, 1.0], np.float32), n)
+    order = np.argsort(np.abs(w), kind="stable")
+    for ratio, extra in ((0.5, 0), (0.5, 1), (0.5, 2), (0.2, 1)):
+        m = oracle.pruned_count(ratio, n)
+        v = w.copy()
+        tied = order[m - 1 - extra:m + 2 - extra]  # three ranks around the m-th smallest
+        v[tied] = np.abs(w[order[m - 1 - extra]]) * np.array([1.0, -1.0, 1.0], np.float32)
+        check_mask(v, ratio)
+
+
+def test_feedback_when_fewer_than_k_sums_are_nonzero():
+    # list strategy whose candidate list comes out short: the list stage rebuilds it from the bucket, which
+    # here is the residual buffer holding gradient + residual
+    rng = np.random.default_rng(41)
+    n = 300_001
+    gs = []
+    for _ in range(3):
+        g = rng.standard_normal(n).astype(np.float32)
+        g[rng.random(n) < 0.93] = 0.0
+        gs.append(g)
+    run_feedback(gs[:1], 0.2, 8)   # first step: 7 % non-zero, 20 % kept
+    run_feedback(gs, 0.2, 16)      # later steps: the residual fills positions up
+
+
+def test_adaptive_bf16_gradient_with_int8_as_the_plain_codec():
+    rng = np.random.default_rng(51)
+    n = 400_003
+    bits16 = (rng.standard_normal(n).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16)
+    g = oracle.widen_bf16(bits16)
+    w = rng.standard_normal(n).astype(np.float32)
+    for ratio, tr_q in ((0.03, 0.1), (0.3, 0.1)):
+        want, want_ratio, want_bits, _, want_mask = oracle.netsense_compression(g, ratio, tr_q, 5.0, weights=w, plain_bits=8)
+        payload, got_ratio, got_bits, _, mask = nsml.nsml_compress_adaptive(
+            to_device_grad(bits16), ratio, tr_q, 5.0, plain_bits=8, weights=torch.from_numpy(w).cuda())
+        assert (got_ratio, got_bits) == (want_ratio, want_bits)
+        assert np.array_equal(mask.cpu().numpy().view(np.uint32), mask_words(want_mask))
+        assert_payload_equal(payload, want)
