@@ -187,7 +187,7 @@ k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long
     // Few entries: touch only their elements in global memory (after zero-filling
     // the tile there in overwrite mode).  Many entries: stage the tile in
     // shared memory and write it back in one sweep.
-    const bool staged = (unsigned long long)total * 16 > len;
+    const bool staged = (unsigned long long)total * 64 > len;
     float* dtile = dense + lo;
     if (staged) {
       for (unsigned int i = threadIdx.x * 4; i < len; i += kCta * 4) {
