@@ -626,7 +626,7 @@ class Alg2Workload(Workload):
                 nsml.nsml_decompress_accumulate([p], lane.dense, zero_first=True, workspace=lane.aws, stream=lane.stream)
                 if acc is not None:
                     self.account(acc, "k_sumsq", 4 * n)
-                    self.account(acc, "k_prune_hist", 2 * 4 * n)  # the third launch returns at once (k_prune_cand did its work)
+                    self.account(acc, "k_prune_hist", 3 * 4 * n)
                     self.account(acc, "k_prune_ties", 3 * 4096 * 4)
                     self.account(acc, "k_prune_write", 4 * n + n // 8)
                     self.account(acc, "k_feedback_subtract", 13 * k)

@@ -176,21 +176,15 @@ struct PruneCtl {
   unsigned int list_ok;        // the tie list holds every key that shares the threshold's 24-bit prefix
   unsigned int use_limit;      // ties are decided by index: pruned iff index <= idx_limit
   unsigned int idx_limit;
-  unsigned int cand_count;     // keys listed by the second histogram pass (those in the threshold's first-digit bin)
-  unsigned int cand_ok;        // that list is complete: the last digit is resolved from it, not from the weights
 };
 constexpr unsigned int kTieCap = 1024;  // keys sharing the threshold's 24-bit prefix that the tie list can hold
-constexpr unsigned int kCandCap = 1u << 21;  // keys of the threshold's first-digit bin that can be listed
-constexpr unsigned int kCandBuf = 1024;      // of which a block buffers this many in shared memory between flushes
 
 struct PruneLayout {
   size_t hist;       // u32[3][kMaxBins]
   size_t tie_list;   // uint2[kTieCap]: (index, last key digit) of the keys that share the threshold's 24-bit prefix
   size_t tile_ties;  // u32[tiles]
-  size_t cand;       // uint2[min(n, kCandCap)]: (index, complemented key) of the keys in the threshold's first-digit bin
   size_t total;
 };
-inline unsigned int cand_capacity(int64_t n) { return (unsigned int)((uint64_t)n < kCandCap ? (uint64_t)n : kCandCap); }
 
 inline PruneLayout prune_layout(int64_t n) {
   PruneLayout L;
@@ -198,8 +192,7 @@ inline PruneLayout prune_layout(int64_t n) {
   L.hist = 256;
   L.tie_list = L.hist + 3 * kMaxBins * sizeof(unsigned int);
   L.tile_ties = L.tie_list + kTieCap * sizeof(uint2);
-  L.cand = L.tile_ties + align_up(tiles * 4, 256);
-  L.total = L.cand + align_up((size_t)cand_capacity(n) * sizeof(uint2), 256);
+  L.total = L.tile_ties + align_up(tiles * 4, 256);
   return L;
 }
 
@@ -238,16 +231,12 @@ __device__ __forceinline__ void prune_resolve(const unsigned int* ghist, unsigne
 template <int LEVEL>
 __global__ void __launch_bounds__(kCta)
 k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, PruneCtl* ctl, unsigned int* __restrict__ hist,
-             uint2* __restrict__ tie_list, uint2* __restrict__ cand, unsigned int cand_cap) {
+             uint2* __restrict__ tie_list) {
   constexpr int NB = (LEVEL == 2) ? 128 : kMaxBins;
   __shared__ unsigned int s_hist[NB];
   __shared__ unsigned int s_tot[kCta / 32], s_out[2];
-  __shared__ uint2 s_buf[LEVEL == 1 ? kCandBuf : 1];  // level 1: keys of the threshold's bin on their way to the list
-  __shared__ unsigned int s_cnt, s_base;
-  if (LEVEL == 2 && ctl->cand_ok) return;  // the last digit comes from the list (k_prune_cand)
   unsigned int prefix = 0;
   bool collect = false;
-  bool keep = false;  // level 1: list the keys of the threshold's first-digit bin (their number is that bin's count)
   // The block's first tile is requested before the previous level is resolved, so that the resolve (a read
   // of the 4096 global bins and a block-wide search) runs while those loads are in flight.
   const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
@@ -262,12 +251,9 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
   if (LEVEL == 1) {
     prune_resolve<kMaxBins>(hist, m, s_tot, s_out);
     prefix = s_out[0];
-    keep = hist[s_out[0]] <= cand_cap;
-    if (threadIdx.x == 0) s_cnt = 0;
     if (blockIdx.x == 0 && threadIdx.x == 0) {
       ctl->d0 = s_out[0];
       ctl->rem1 = s_out[1];
-      ctl->cand_ok = keep;
     }
   } else if (LEVEL == 2) {
     prune_resolve<kMaxBins>(hist + kMaxBins, ctl->rem1, s_tot, s_out);
@@ -290,16 +276,7 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
       lowest = min(lowest, key);
       atomicAdd(&s_hist[key >> 19], 1u);
     } else if (LEVEL == 1) {
-      if ((key >> 19) == prefix) {
-        atomicAdd(&s_hist[(key >> 7) & 0xFFFu], 1u);
-        if (keep) {
-          const unsigned long long i = tile * kStreamTile + (unsigned long long)(u * kCta + threadIdx.x) * 4 + e;
-          const uint2 entry = make_uint2((uint32_t)i, key);
-          const unsigned int slot = atomicAdd(&s_cnt, 1u);
-          if (slot < kCandBuf) s_buf[slot] = entry;
-          else cand[atomicAdd(&ctl->cand_count, 1u)] = entry;  // buffer full (a tile crowded with such keys)
-        }
-      }
+      if ((key >> 19) == prefix) atomicAdd(&s_hist[(key >> 7) & 0xFFFu], 1u);
     } else {
       if ((key >> 7) == prefix) {
         atomicAdd(&s_hist[key & 0x7Fu], 1u);
@@ -310,21 +287,7 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
       }
     }
   };
-  // level 1: moves the buffered keys to the global list (one reservation per flush); block-uniform
-  auto flush_buffer = [&](unsigned int threshold) {
-    __syncthreads();
-    const unsigned int held = min(s_cnt, kCandBuf);
-    if (held > threshold) {
-      if (threadIdx.x == 0) s_base = atomicAdd(&ctl->cand_count, held);
-      __syncthreads();
-      for (unsigned int j = threadIdx.x; j < held; j += kCta) cand[s_base + j] = s_buf[j];
-      __syncthreads();
-      if (threadIdx.x == 0) s_cnt = 0;
-    }
-    __syncthreads();
-  };
   for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
-    if (LEVEL == 1 && keep) flush_buffer(kCandBuf / 2);
     const unsigned long long base = tile * kStreamTile;
     if (base + kStreamTile <= n) {  // a whole tile: no bounds checks
       if (!preloaded) {
@@ -348,7 +311,6 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
           if (e < cnt[u]) visit(prune_key(bits[u][e]), tile, u, e);
     }
   }
-  if (LEVEL == 1 && keep) flush_buffer(0);
   const bool nonfinite = LEVEL == 0 && lowest <= 0x007FFFFFu;  // magnitude bits >= 0x7F800000
   if (nonfinite) set_status(&ctl->status, NSML_ERR_NONFINITE);
   __syncthreads();
@@ -356,40 +318,6 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
   for (int b = threadIdx.x; b < NB; b += kCta) {
     const unsigned int c = s_hist[b];
     if (c) atomicAdd(&ghist[b], c);
-  }
-}
-
-// The last histogram level from the list the second pass left (the keys of the threshold's first-digit bin,
-// a few per cent of the weights) instead of from the weights: resolves digit 1, counts the last digit of
-// the keys that share the 24-bit prefix and lists those for the tie ranking.  Returns at once when the
-// list was not kept (k_prune_hist<2> then does the same from the weights).
-__global__ void __launch_bounds__(kCta)
-k_prune_cand(PruneCtl* ctl, unsigned int* __restrict__ hist, const uint2* __restrict__ cand, uint2* __restrict__ tie_list) {
-  __shared__ unsigned int s_hist[128];
-  __shared__ unsigned int s_tot[kCta / 32], s_out[2];
-  if (!ctl->cand_ok) return;
-  prune_resolve<kMaxBins>(hist + kMaxBins, ctl->rem1, s_tot, s_out);
-  const unsigned int prefix = (ctl->d0 << 12) | s_out[0];
-  const bool collect = hist[kMaxBins + s_out[0]] <= kTieCap;
-  if (blockIdx.x == 0 && threadIdx.x == 0) {
-    ctl->prefix24 = prefix;
-    ctl->rem2 = s_out[1];
-    ctl->list_ok = collect;
-  }
-  for (int b = threadIdx.x; b < 128; b += kCta) s_hist[b] = 0;
-  __syncthreads();
-  const unsigned int count = ctl->cand_count;
-  for (unsigned int j = blockIdx.x * kCta + threadIdx.x; j < count; j += gridDim.x * kCta) {
-    const uint2 e = __ldg(cand + j);
-    if ((e.y >> 7) == prefix) {
-      atomicAdd(&s_hist[e.y & 0x7Fu], 1u);
-      if (collect) tie_list[atomicAdd(&ctl->list_count, 1u)] = make_uint2(e.x, e.y & 0x7Fu);
-    }
-  }
-  __syncthreads();
-  for (int b = threadIdx.x; b < 128; b += kCta) {
-    const unsigned int c = s_hist[b];
-    if (c) atomicAdd(&hist[2 * kMaxBins + b], c);
   }
 }
 

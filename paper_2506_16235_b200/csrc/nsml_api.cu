@@ -19,13 +19,13 @@ namespace nsml {
 
 enum KernelId {
   K_SAMPLE = 0, K_COMPACT_BUCKET, K_FINALIZE, K_PARTITION, K_MERGE, K_CLEAR, K_FINALIZE_DENSE,
-  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_PRUNE_WRITE_RANKED, K_GATHER, K_PRUNE_CAND, K_COUNT
+  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_PRUNE_WRITE_RANKED, K_GATHER, K_COUNT
 };
 
 static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_compact_bucket", "k_finalize", "k_partition", "k_merge",
                                                   "k_clear", "k_finalize_dense", "k_sumsq", "k_feedback_add",
                                                   "k_feedback_subtract", "k_prune_hist", "k_prune_ties", "k_prune_write",
-                                                  "k_prune_write_ranked", "k_gather", "k_prune_cand"};
+                                                  "k_prune_write_ranked", "k_gather"};
 
 static std::atomic<int64_t> g_launches{0};
 
@@ -474,26 +474,21 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
   unsigned int* hist = reinterpret_cast<unsigned int*>(ws + L.hist);
   unsigned int* tile_ties = reinterpret_cast<unsigned int*>(ws + L.tile_ties);
   uint2* tie_list = reinterpret_cast<uint2*>(ws + L.tie_list);
-  uint2* cand = reinterpret_cast<uint2*>(ws + L.cand);
   const BucketSrc<NSML_F32> src{weights, nullptr};
   const unsigned int grid = stream_grid(n, *dev, dev->prune_hist < 8 ? dev->prune_hist : 8, 1u << 16);
   const unsigned int wgrid = stream_grid(n, *dev, dev->prune_write < 8 ? dev->prune_write : 8, 1u << 16);
   const unsigned long long un = (unsigned long long)n;
   {
     LaunchScope scope(K_PRUNE_HIST, st);
-    k_prune_hist<0><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list, cand, cand_capacity(n));
+    k_prune_hist<0><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
     LaunchScope scope(K_PRUNE_HIST, st);
-    k_prune_hist<1><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list, cand, cand_capacity(n));
+    k_prune_hist<1><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
-    LaunchScope scope(K_PRUNE_CAND, st);  // the last level from the listed keys (returns at once without a list)
-    k_prune_cand<<<dev->sms, kCta, 0, st>>>(ctl, hist, cand, tie_list);
-  }
-  {
-    LaunchScope scope(K_PRUNE_HIST, st);  // returns at once when the list was used
-    k_prune_hist<2><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list, cand, cand_capacity(n));
+    LaunchScope scope(K_PRUNE_HIST, st);
+    k_prune_hist<2><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
     LaunchScope scope(K_PRUNE_TIES, st);
