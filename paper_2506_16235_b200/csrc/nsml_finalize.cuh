@@ -339,41 +339,42 @@ k_gather(FinalizeParams p) {
   if (threadIdx.x == 0) s_off[kGatherSegs] = total;
   __syncthreads();
   bool nonfinite = false;
-  // Thread t takes entries t, t + 256, t + 512, ... of the block, kGatherRun of them per step with their loads
-  // issued together: neighbouring lanes take neighbouring entries, so where a segment holds many candidates a
-  // warp's load and its stores are contiguous.
-  for (unsigned int j0 = threadIdx.x; j0 < total; j0 += kCta * kGatherRun) {
+  for (unsigned int j0 = threadIdx.x * kGatherRun; j0 < total; j0 += kCta * kGatherRun) {
+    const int cnt = (int)min((unsigned int)kGatherRun, total - j0);
     uint32_t from[kGatherRun];
+    {
+      // segment of entry j0: the last one whose offset is <= j0 (empty segments share an offset with their
+      // successor, so the search lands on the segment that holds the entry)
+      int lo = 0, hi = kGatherSegs - 1;
+      while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (s_off[mid] <= j0) lo = mid; else hi = mid - 1;
+      }
+      unsigned int q = lo, within = j0 - s_off[lo];
 #pragma unroll
-    for (int e = 0; e < kGatherRun; ++e) {
-      const unsigned int j = j0 + e * kCta;
-      from[e] = 0xFFFFFFFFu;
-      if (j < total) {
-        // segment of entry j: the last one whose offset is <= j (empty segments share an offset with their
-        // successor, so the search lands on the segment that holds the entry)
-        int lo = 0, hi = kGatherSegs - 1;
-        while (lo < hi) {
-          const int mid = (lo + hi + 1) >> 1;
-          if (s_off[mid] <= j) lo = mid; else hi = mid - 1;
+      for (int e = 0; e < kGatherRun; ++e) {
+        from[e] = 0;
+        if (e < cnt) {
+          while (within >= s_off[q + 1] - s_off[q]) { within = 0; ++q; }  // entry e exists, so this ends inside the block
+          from[e] = (uint32_t)((seg0 + q) * kSegElems + within);
+          ++within;
         }
-        from[e] = (uint32_t)((seg0 + lo) * kSegElems + (j - s_off[lo]));
       }
     }
     uint32_t vals[kGatherRun], idxs[kGatherRun];
 #pragma unroll
     for (int e = 0; e < kGatherRun; ++e) {
-      if (from[e] != 0xFFFFFFFFu) {
+      if (e < cnt) {
         vals[e] = __ldg(p.seg_val + from[e]);
         idxs[e] = __ldg(p.seg_idx + from[e]);
       }
     }
 #pragma unroll
     for (int e = 0; e < kGatherRun; ++e) {
-      if (from[e] != 0xFFFFFFFFu) {
-        const unsigned int j = j0 + e * kCta;
+      if (e < cnt) {
         const uint32_t key = vals[e] & 0x7FFFFFFFu;
-        p.list_idx[base + j] = idxs[e];
-        p.list_val[base + j] = vals[e];
+        p.list_idx[base + j0 + e] = idxs[e];
+        p.list_val[base + j0 + e] = vals[e];
         nonfinite |= key >= kInfKey;
         const unsigned int bin = key >> digit_shift(0), rel = bin - first_bin;  // wraps only for a key below lo
         if (rel < (unsigned int)kGatherBins) atomicAdd(&s_hist[rel], 1u);
