@@ -285,8 +285,13 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
   fp.P = P;
   if (!dense) {
     LaunchScope scope(K_GATHER, st);  // segmented list -> contiguous list and the histogram of the first digit
-    const unsigned int ggrid = (unsigned int)((nseg + kGatherSegs - 1) / kGatherSegs);
-    k_gather<<<ggrid, kCta, 0, st>>>(fp);
+    // blocks per group: about 1024 expected candidates (one step of the copy loop) per block, at least two
+    // (candidates crowd into parts of a bucket), at most eight
+    const unsigned long long ngroups = (nseg + kGatherSegs - 1) / kGatherSegs;
+    const double per_group = (double)n * (p_keep + 6.0 * std::sqrt(p_keep * (1.0 - p_keep) / kSamples)) / (double)ngroups;
+    unsigned int split = (unsigned int)(per_group / 1024.0) + 1;
+    split = split < 2 ? 2 : (split > 8 ? 8 : split);
+    k_gather<<<(unsigned int)(ngroups * split), kCta, 0, st>>>(fp, split);
   }
   {
     LaunchScope scope(dense ? K_FINALIZE_DENSE : K_FINALIZE, st);

@@ -296,8 +296,10 @@ constexpr int kGatherSegs = kGroupSegs;  // one group per block: its list positi
 constexpr int kGatherRun = 4;      // consecutive candidates a thread copies per step
 constexpr int kGatherBins = 256;   // first-digit bins a block of the gather counts in shared memory
 
+// `split` blocks share a group (block b takes group b / split and every split-th step of its entries), so
+// that long lists and crowded groups are spread over more blocks.
 __global__ void __launch_bounds__(kCta)
-k_gather(FinalizeParams p) {
+k_gather(FinalizeParams p, unsigned int split) {
   // Every candidate's key is >= the sampled bound lo, and almost all lie within a few octaves above it:
   // the block counts first digits in a window of kGatherBins bins that starts at lo's bin (16 bins per
   // octave); the rare key beyond the window goes to the global histogram directly.
@@ -309,14 +311,15 @@ k_gather(FinalizeParams p) {
   for (int b = threadIdx.x; b < kGatherBins; b += kCta) s_hist[b] = 0;
   const unsigned int first_bin = p.ctl->lo >> digit_shift(0);
   // list position of the block's first candidate
-  const unsigned long long first_group = (unsigned long long)blockIdx.x * (kGatherSegs / kGroupSegs);
+  const unsigned int group = blockIdx.x / split, part = blockIdx.x % split;
+  const unsigned long long first_group = (unsigned long long)group * (kGatherSegs / kGroupSegs);
   unsigned long long before = 0;
   for (unsigned long long g = threadIdx.x; g < first_group; g += kCta) before += p.group_count[g];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xFFFFFFFFu, before, o);
   if (lane == 0) s_red[warp] = before;
   // offsets of the block's segments
-  const unsigned long long seg0 = (unsigned long long)blockIdx.x * kGatherSegs;
+  const unsigned long long seg0 = (unsigned long long)group * kGatherSegs;
   const unsigned long long seg = seg0 + threadIdx.x;
   const unsigned int c = (threadIdx.x < kGatherSegs && seg < p.nseg) ? p.seg_count[seg] : 0u;
   unsigned int incl = c;
@@ -339,7 +342,7 @@ k_gather(FinalizeParams p) {
   if (threadIdx.x == 0) s_off[kGatherSegs] = total;
   __syncthreads();
   bool nonfinite = false;
-  for (unsigned int j0 = threadIdx.x * kGatherRun; j0 < total; j0 += kCta * kGatherRun) {
+  for (unsigned int j0 = (part * kCta + threadIdx.x) * kGatherRun; j0 < total; j0 += split * kCta * kGatherRun) {
     const int cnt = (int)min((unsigned int)kGatherRun, total - j0);
     uint32_t from[kGatherRun];
     {
