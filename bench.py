@@ -9,7 +9,7 @@ compaction, value codec) and the W workers' payloads are decompressed and
 summed into a dense buffer.  The metric is input-gradient bytes per second.
 Prints ONE JSON line (rank 0).
 
-Workloads (value distributions are described in paper_2506_16235_b200/synth.py):
+Workloads (value distributions are described in synth.py):
   resnet50  25.6M fp32 parameters in ResNet-50's tensor shapes, 25 MB buckets,
             ratio sweep {0.5, 0.1, 0.01, 0.001} x {int8, fp16}, W = 1  (default)
   gpt2      124M fp32 parameters in GPT-2-small's shapes, 25M-element buckets,
@@ -243,7 +243,7 @@ class ResnetWorkload(Workload):
     graph_period = 9
 
     def __init__(self, nsml, torch, device, rank, nlanes=2):
-        from paper_2506_16235_b200 import synth
+        import synth
 
         self.nsml, self.torch = nsml, torch
         self.replicas = []
@@ -334,7 +334,7 @@ class Gpt2Workload(Workload):
     W, RATIO, BITS = 4, 0.01, 8
 
     def __init__(self, nsml, torch, device, rank, buckets=None, nlanes=2):
-        from paper_2506_16235_b200 import synth
+        import synth
 
         self.nsml, self.torch = nsml, torch
         shapes = synth.gpt2_small_shapes()
@@ -435,7 +435,7 @@ class DecoderWorkload(Workload):
     graphs_ok = False  # the controller emits a new ratio every step
 
     def __init__(self, nsml, torch, device, rank, nlanes=2):
-        from paper_2506_16235_b200 import synth
+        import synth
 
         self.nsml, self.torch = nsml, torch
         shapes = synth.decoder_1p3b_shapes()
@@ -525,7 +525,7 @@ class AggWorkload(Workload):
     W, N, RATIO = 8, 350_000_000, 0.05
 
     def __init__(self, nsml, torch, device, rank, nlanes=1):
-        from paper_2506_16235_b200 import synth
+        import synth
 
         self.nsml, self.torch = nsml, torch
         self.k = nsml.nsml_k_of(self.N, self.RATIO)
@@ -561,7 +561,7 @@ class AggWorkload(Workload):
 
     def oracle_sample(self):
         import oracle
-        from paper_2506_16235_b200 import synth
+        import synth
 
         n, k = 35_000_000, 1_750_000
         ps = []
@@ -703,11 +703,13 @@ def run_reference(args, rank):
     if rank != 0:
         return
     import oracle
-    from paper_2506_16235_b200 import synth
+    import synth
 
     # bounded sample of the default workload: one 25 MB bucket at one sweep point per step
     buckets = list(synth.resnet50_buckets(seed=1))
     g = buckets[0]
+    if args.reference_elements:
+        g = g[:int(args.reference_elements)]
     n = g.size
 
     def one(i):
@@ -722,7 +724,7 @@ def run_reference(args, rank):
         one(i)
     dt = time.perf_counter() - t0
     value = args.steps * 4.0 * n / dt / 1e9
-    sample = f"one 25 MB bucket ({n} elements) per step, sweep point i mod 8"
+    sample = f"one bucket of {n} fp32 elements per step, sweep point i mod 8"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
@@ -750,6 +752,8 @@ def main():
     ap.add_argument("--no-large-bucket-leg", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (e2e is then null)")
     ap.add_argument("--no-kernel-times", action="store_true", help="skip the event-bracketed per-kernel pass")
+    ap.add_argument("--reference-elements", type=int, default=None,
+                    help="--impl reference only: elements of the bucket the oracle is timed on (default: one 25 MB bucket)")
     ap.add_argument("--agg-elements", type=int, default=None,
                     help="agg workload only: dense elements (default 350M; smaller sizes are for profiler captures)")
     args = ap.parse_args()

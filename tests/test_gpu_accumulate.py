@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import oracle
-from paper_2506_16235_b200 import synth
+import synth
 
 pytestmark = pytest.mark.gpu
 

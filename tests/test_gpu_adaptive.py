@@ -7,7 +7,7 @@ import torch
 
 import oracle
 from conftest import read_golden
-from paper_2506_16235_b200 import synth
+import synth
 
 pytestmark = pytest.mark.gpu
 
