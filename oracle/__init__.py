@@ -10,6 +10,7 @@ product path must never route through it.
 Pins (what each function is checked against, independently of itself):
   select_topk        brute force over all k-subsets, partial-sort special
                      case, worked examples, invariants
+  select_topk_many   the same brute force, for every k of one bucket at once
   quantize_int8      worked half-way examples, invariants, fractions.Fraction
                      exact arithmetic on small blocks
   f32_to_f16_bits    NumPy's float16 cast on finite in-range inputs, worked
@@ -38,11 +39,13 @@ from .compress import (  # noqa: F401
     widen_bf16,
     keys_of,
     select_topk,
+    select_topk_many,
     quantize_int8,
     dequantize_int8,
     f32_to_f16_bits,
     f16_bits_to_f32,
     compress,
+    compress_many,
     decompress_sum,
     Payload,
 )

@@ -111,6 +111,30 @@ def select_topk(values: np.ndarray, k: int) -> np.ndarray:
     return survivors
 
 
+def select_topk_many(values: np.ndarray, ks: Sequence[int]):
+    """select_topk for several k on the same bucket: the same full sort on
+    (key descending, index ascending), taken once; the survivors for each k
+    are the first k entries of that one order.  Returns a list of ascending
+    uint32 index arrays, one per k."""
+    key = keys_of(values)
+    n = key.size
+    if n >= 2**32:
+        raise ValueError("n must be below 2**32")
+    if any(not (1 <= int(k) <= n) for k in ks):
+        raise ValueError("k out of range")
+    if key.size and int(key.max()) >= _INF_BITS:
+        raise NonFiniteGradient("bucket holds NaN or Inf")
+    hi = (np.uint64(0x7FFFFFFF) - key.astype(np.uint64)) << np.uint64(32)
+    packed = hi | np.arange(n, dtype=np.uint64)
+    packed.sort()  # the full sort
+    out = []
+    for k in ks:
+        survivors = (packed[: int(k)] & np.uint64(0xFFFFFFFF)).astype(np.uint32)
+        survivors.sort()  # payload order = ascending index
+        out.append(survivors)
+    return out
+
+
 def quantize_int8(val: np.ndarray):
     """Symmetric int8 codes with one max-abs scale per QBLOCK survivors.
 
@@ -243,6 +267,32 @@ def compress(
     elif bits == 16:
         p.half = f32_to_f16_bits(raw)
     return p
+
+
+def compress_many(
+    grad: np.ndarray,
+    ratios: Sequence[float],
+    bits: int,
+    prune_mask: Optional[np.ndarray] = None,
+):
+    """compress() of one bucket at several ratios (one full sort serves all
+    of them: the survivors at ratio r are the first k_of(r, n) entries of the
+    sorted order).  Returns one Payload per ratio."""
+    if bits not in (8, 16, 32):
+        raise ValueError("bits must be 8 (int8), 16 (fp16) or 32 (float32 as is)")
+    v = _apply_mask(grad, prune_mask)
+    n = v.size
+    ks = [k_of(r, n) for r in ratios]
+    out = []
+    for k, idx in zip(ks, select_topk_many(v, ks)):
+        raw = v[idx]
+        p = Payload(n=n, k=k, bits=bits, idx=idx, raw=raw)
+        if bits == 8:
+            p.codes, p.scales = quantize_int8(raw)
+        elif bits == 16:
+            p.half = f32_to_f16_bits(raw)
+        out.append(p)
+    return out
 
 
 def decompress_sum(

@@ -1,19 +1,18 @@
 """GPU parity at the five configurations' full sizes.  Index sets, int8 codes,
 scales and fp16 bits are compared bit for bit with the oracle; sums within
-1e-6 of the largest magnitude.  Where the oracle's full sort of every bucket
-would take minutes, a fixed subset of buckets is checked (stated per test)."""
+1e-6 of the largest magnitude."""
 import numpy as np
 import pytest
 import torch
 
 import oracle
-from paper_2506_16235_b200 import synth
+import synth
 
 pytestmark = pytest.mark.gpu
 
 if torch.cuda.is_available():
     import paper_2506_16235_b200 as nsml
-    from gpu_util import check_accumulate, check_compress, payload_to_device
+    from gpu_util import assert_payload_equal, check_accumulate, check_compress, payload_to_device, to_device_grad
 
 
 def test_config1_single_vector():
@@ -48,14 +47,18 @@ def test_config3_gpt2_four_workers(bucket):
     check_accumulate(pts, pos, n, zero_first=True)
 
 
-def test_config4_decoder_bf16_controller_ratios():
-    # one 64M-element bf16 bucket inside the layer stack, at the ratios the controller emits on the
-    # 100 -> 10 -> 1 Gbps trace (first, a middle and the last one)
-    bits16 = synth.decoder_bucket_bf16(5, seed=20)
-    assert bits16.size == 1 << 26
+DECODER_ELEMS = 1_315_723_264
+# steps of the 90-step link trace whose ratios are compressed with: the start, the descent and the
+# oscillation on the 100 Gbps plateau, the 10 Gbps plateau, and the floor reached on the 1 Gbps plateau
+CONFIG4_STEPS = (0, 1, 5, 31, 41, 60, 89)
+
+
+def config4_trace():
+    """Ratios the controller emits on the 100 -> 10 -> 1 Gbps step trace (30 steps per plateau), every
+    step compared with the oracle's controller."""
     ctrl = nsml.Controller(ratio_init=0.1, ratio_min=0.001, ratio_max=0.1, startup_max_steps=0)
     ora = oracle.Controller(oracle.ControllerParams(ratio_init=0.1, ratio_min=0.001, ratio_max=0.1, startup_max_steps=0))
-    dense = 2.0 * 1_315_723_264
+    dense = 2.0 * DECODER_ELEMS
     ratios, last = [], (0.0, 0.0)
     for step in range(90):
         r = ctrl.select_ratio(last[0], last[1], dense)
@@ -65,12 +68,27 @@ def test_config4_decoder_bf16_controller_ratios():
         bw = (100e9, 10e9, 1e9)[step // 30] / 8.0
         last = (sent, 1e-3 + sent / bw)
     assert ratios[0] == 0.1 and min(ratios) == 0.001
-    for ratio in (ratios[0], sorted(set(ratios))[len(set(ratios)) // 2], ratios[-1]):
-        check_compress(bits16, ratio, 16)
-    # the last, short bucket of the set (40,654,848 elements)
-    tail = synth.decoder_bucket_bf16(19, seed=20)
-    assert tail.size == 1_315_723_264 - 19 * (1 << 26)
-    check_compress(tail, 0.01, 16)
+    return ratios
+
+
+@pytest.mark.parametrize("bucket", range(20))
+def test_config4_decoder_bf16_every_bucket_at_controller_ratios(bucket):
+    # every 64M-element bf16 bucket of the 1.3B-parameter set (the last one is short), fp16 values, at six
+    # distinct ratios the controller emits across the three plateaus of the link trace
+    ratios = config4_trace()
+    picked = sorted({ratios[s] for s in CONFIG4_STEPS}, reverse=True)
+    assert len(picked) >= 6 and picked[0] == 0.1 and picked[-1] == 0.001
+    bits16 = synth.decoder_bucket_bf16(bucket, seed=20)
+    assert bits16.size == ((1 << 26) if bucket < 19 else DECODER_ELEMS - 19 * (1 << 26))
+    wants = oracle.compress_many(oracle.widen_bf16(bits16), picked, 16)
+    grad = to_device_grad(bits16)
+    n = grad.numel()
+    ws = nsml.alloc_bytes(nsml.nsml_workspace_bytes(n, nsml.NSML_BF16), "cuda")
+    for ratio, want in zip(picked, wants):
+        payload = nsml.nsml_compress(grad, ratio, 16, workspace=ws)
+        status = nsml.nsml_last_status(ws)
+        assert status == 0, nsml.nsml_strerror(status)
+        assert_payload_equal(payload, want)
 
 
 @pytest.mark.parametrize("ratio", [0.001, 0.05])

@@ -51,6 +51,28 @@ def test_brute_force_small(seed):
         assert oracle.select_topk(g, k).tolist() == brute_force_topk(g, k)
 
 
+@pytest.mark.parametrize("seed", range(20))
+def test_brute_force_small_many_k_from_one_sort(seed):
+    rng = np.random.default_rng(100 + seed)
+    n = int(rng.integers(1, 10))
+    pool = np.array([0.0, -0.0, 0.5, -0.5, 1.0, -1.0, 2.0, 1e-40, -1e-40, 3.5], dtype=np.float32)
+    g = pool[rng.integers(0, pool.size, n)]
+    ks = list(range(n, 0, -1))  # not in increasing order on purpose
+    got = oracle.select_topk_many(g, ks)
+    assert [s.tolist() for s in got] == [brute_force_topk(g, k) for k in ks]
+
+
+def test_compress_many_payloads_carry_the_brute_force_sets():
+    g = np.array([0.5, -2.0, 0.0, 2.0, -0.5, 1.0, -0.0, 0.5], dtype=np.float32)  # the worked example
+    ratios = [1.0, 0.3, 0.75, 0.5]
+    for bits in (8, 16, 32):
+        for ratio, p in zip(ratios, oracle.compress_many(g, ratios, bits)):
+            k = oracle.k_of(ratio, g.size)
+            assert (p.n, p.k, p.bits) == (8, k, bits)
+            assert p.idx.tolist() == brute_force_topk(g, k)
+            assert np.array_equal(p.raw.view(np.uint32), g[p.idx].view(np.uint32))
+
+
 def test_distinct_keys_match_partial_sort():
     rng = np.random.default_rng(7)
     mag = rng.permutation(5000).astype(np.float32) * np.float32(0.125) + np.float32(0.125)
