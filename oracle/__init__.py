@@ -29,8 +29,9 @@ Pins (what each function is checked against, independently of itself):
                      multiplicative-decrease / additive-increase recurrences
   Controller (start-up phase)  parity unpinned: the paper gives neither the
                      increment beta_1, the phase length nor the exit test, so
-                     the start-up recurrence is checked only against the
-                     reading stated in this package.
+                     the start-up recurrence and its three exits (excessive
+                     transfer time, step limit, ratio at its cap) are hand
+                     traced only under the reading stated in this package.
 """
 from .compress import (  # noqa: F401
     QBLOCK,

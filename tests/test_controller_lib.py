@@ -52,6 +52,20 @@ def test_matches_oracle_bit_for_bit(overrides, seed):
         assert st.phase == ora_c.phase and st.calls == ora_c.calls
 
 
+def test_golden_startup_cap_exit_through_the_library():
+    gold = read_golden("h7_startup_cap.txt")
+    kv = dict(item.split("=") for item in gold["params"][0])
+    c = nsml.Controller(ratio_init=float(kv["ratio_init"]), beta1=float(kv["beta1"]), ratio_max=float(kv["ratio_max"]),
+                        startup_max_steps=int(kv["startup_max_steps"]))
+    dense = float(kv["next_dense_bytes"])
+    assert c.select_ratio(0, 0, dense) == float(kv["ratio_init"])
+    for row in gold["step"]:
+        got = c.select_ratio(float(row[0]), float(row[1]), dense)
+        st = c.state()
+        assert (st.phase, st.startup_steps) == (int(row[2]), int(row[3]))
+        assert got == float(row[4])
+
+
 def test_golden_trace_through_the_library():
     gold = read_golden("h4_controller.txt")
     kv = dict(item.split("=") for item in gold["params"][0])

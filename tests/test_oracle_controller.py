@@ -97,6 +97,19 @@ def test_startup_ramp_under_stated_reading():
     assert c.phase == Controller.NETSENSE and r == 0.31000000000000005 * 0.5
 
 
+def test_golden_h7_startup_leaves_when_the_ratio_reaches_its_cap():
+    gold = read_golden("h7_startup_cap.txt")
+    kv = dict(item.split("=") for item in gold["params"][0])
+    c = Controller(ControllerParams(ratio_init=float(kv["ratio_init"]), beta1=float(kv["beta1"]),
+                                    ratio_max=float(kv["ratio_max"]), startup_max_steps=int(kv["startup_max_steps"])))
+    dense = float(kv["next_dense_bytes"])
+    assert c.select_ratio(0, 0, dense) == float(kv["ratio_init"]) and c.phase == Controller.STARTUP
+    for row in gold["step"]:
+        got = c.select_ratio(float(row[0]), float(row[1]), dense)
+        assert (c.phase, c.startup_steps) == (int(row[2]), int(row[3]))
+        assert got == float(row[4])
+
+
 def test_startup_ends_after_max_steps():
     c = Controller(ControllerParams(beta1=0.05, startup_max_steps=2))
     c.select_ratio(0, 0, 1.0)
