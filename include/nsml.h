@@ -235,11 +235,23 @@ int nsml_compress_strategy(int64_t n, double ratio);
  * float(half) or taken as they are, and added in float32 in worker order w = 0..W-1, each dense
  * element by one thread: the result is deterministic.  Device-detected:
  * NSML_ERR_PAYLOAD if a header does not match (magic, version, n, bits, k) or
- * an index is >= n; nothing is written out of range.
+ * an index is >= n; nothing is written out of range.  A header is trusted as
+ * to how long the payload is: a caller that receives payloads from other
+ * workers and knows how many bytes arrived should use the _sized variant.
  * ---------------------------------------------------------------------- */
 int nsml_decompress_accumulate(const void* const* payloads, int W, float* dense, int64_t n,
                                int zero_first, void* workspace, size_t workspace_bytes,
                                void* stream);
+
+/* The same sum (Section 4.2 Step 3, AllGather pattern of Section 5.3) for
+ * payloads whose buffer sizes are known: payload_bytes is a HOST array of W
+ * sizes in bytes (each >= 64, else NSML_ERR_ARG).  A payload whose header
+ * describes more bytes than its buffer holds (a truncated transfer, a k field
+ * corrupted upwards) is reported as NSML_ERR_PAYLOAD on the device and none of
+ * its entries is read. */
+int nsml_decompress_accumulate_sized(const void* const* payloads, const size_t* payload_bytes, int W,
+                                     float* dense, int64_t n, int zero_first, void* workspace,
+                                     size_t workspace_bytes, void* stream);
 
 /* ------------------------------------------------------------------------
  * nsml_decompress_accumulate_static -- the same sum as
@@ -254,12 +266,16 @@ int nsml_decompress_accumulate(const void* const* payloads, int W, float* dense,
  * that loads the library holds it until the process exits.  In exchange the
  * call is limited to n <= NSML_STATIC_MAX_N and W <= NSML_STATIC_MAX_WORKERS;
  * larger arguments are refused with NSML_ERR_CAPACITY and nothing is enqueued.
- * The call, and everything it calls, allocates no host or device memory.
+ * The call, and everything it calls, allocates no host or device memory (its
+ * launches are never bracketed by the events of nsml_prof_enable, which would
+ * allocate, so they do not show in nsml_prof_read).
  *
  *   payloads, W, dense, n, zero_first, stream   as for nsml_decompress_accumulate
  *   status_out  host pointer or NULL.  NULL: the call returns after enqueueing.
  *               Non-NULL: the call also synchronises `stream` and stores the
  *               device-detected status (NSML_OK or NSML_ERR_PAYLOAD) there.
+ *               The caller never sees the scratch, so the asynchronous form
+ *               (NULL) cannot report a device-detected error afterwards.
  *
  * The first call on each device looks up the array's device address (once per
  * device, with that device current); make that first call outside any stream
@@ -374,7 +390,11 @@ int nsml_compress_adaptive(const void* grad, int64_t n, int grad_dtype, double r
  * nsml_accumulate_host_scratch_bytes(n, W, total_payload_bytes); the call copies
  * the inputs to the device, runs the operation and copies the result back, all
  * on `stream`, and returns without synchronising.  payload_host / dense_host
- * are valid once the stream has been synchronised. */
+ * are valid once the stream has been synchronised.
+ * nsml_decompress_accumulate_host reads every payload's header on the host
+ * first: one that does not match n, or that describes more than
+ * payload_bytes[w] bytes, makes the call return NSML_ERR_PAYLOAD before
+ * anything is copied or launched. */
 size_t nsml_compress_host_scratch_bytes(int64_t n, int grad_dtype, double ratio, int bits);
 int nsml_compress_host(const void* grad_host, int64_t n, int grad_dtype, double ratio, int bits,
                        const uint32_t* prune_mask_host, void* payload_host,
@@ -389,6 +409,17 @@ int nsml_decompress_accumulate_host(const void* const* payloads_host, const size
  * host-variant `device_scratch`) to *status_out (host pointer): NSML_OK or the
  * first device-detected error of the last call that used it. */
 int nsml_last_status(const void* workspace, void* stream, int* status_out);
+
+/* Self-test of the bounded waits between thread blocks (the cooperative
+ * kernels of Alg. 2 Step 3 meet at barriers in global memory; every such wait
+ * gives up after a fixed number of polls instead of hanging).  Enqueues a
+ * two-block kernel whose barrier target can never be reached, with a wait
+ * limit of max_polls polls (1 .. 65536; a fraction of a millisecond to a few
+ * milliseconds): each block gives up, the kernel returns by itself and the
+ * status word of `workspace` (device pointer, 256-byte aligned, >= 256 bytes;
+ * any compress workspace will do) reads NSML_ERR_TIMEOUT afterwards.  The
+ * workspace stays usable: every call clears its control block first. */
+int nsml_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int max_polls, void* stream);
 
 /* Static, NUL-terminated description of a status code. */
 const char* nsml_strerror(int status);

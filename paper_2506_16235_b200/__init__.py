@@ -97,6 +97,7 @@ def _load() -> ctypes.CDLL:
         "nsml_accumulate_workspace_bytes": (sz, [i64, ci]),
         "nsml_compress": (ci, [vp, i64, ci, dbl, ci, vp, vp, sz, vp, sz, vp]),
         "nsml_decompress_accumulate": (ci, [ctypes.POINTER(vp), ci, vp, i64, ci, vp, sz, vp]),
+        "nsml_decompress_accumulate_sized": (ci, [ctypes.POINTER(vp), ctypes.POINTER(sz), ci, vp, i64, ci, vp, sz, vp]),
         "nsml_decompress_accumulate_static": (ci, [ctypes.POINTER(vp), ci, vp, i64, ci, vp, ctypes.POINTER(ci)]),
         "nsml_compress_host_scratch_bytes": (sz, [i64, ci, dbl, ci]),
         "nsml_compress_host": (ci, [vp, i64, ci, dbl, ci, vp, vp, sz, vp, sz, vp]),
@@ -113,6 +114,7 @@ def _load() -> ctypes.CDLL:
         "nsml_adaptive_workspace_bytes": (sz, [i64, ci]),
         "nsml_compress_adaptive": (ci, [vp, i64, ci, dbl, dbl, dbl, ci, vp, vp, vp, sz, vp, sz, vp,
                                         ctypes.POINTER(dbl), ctypes.POINTER(ci), ctypes.POINTER(dbl)]),
+        "nsml_selftest_bounded_wait": (ci, [vp, sz, ci, vp]),
         "nsml_last_status": (ci, [vp, vp, ctypes.POINTER(ci)]),
         "nsml_strerror": (ctypes.c_char_p, [ci]),
         "nsml_kernel_count": (ci, []),
@@ -284,8 +286,11 @@ def nsml_compress(grad, ratio: float, bits: int = NSML_BITS_INT8, prune_mask=Non
     return payload[:need]
 
 
-def nsml_decompress_accumulate(payloads: Sequence, dense, zero_first: bool = True, workspace=None, stream=None):
-    """dense (float32 CUDA tensor, n elements) = (0 or dense) + sum of the payloads."""
+def nsml_decompress_accumulate(payloads: Sequence, dense, zero_first: bool = True, workspace=None, stream=None,
+                               sized: bool = False):
+    """dense (float32 CUDA tensor, n elements) = (0 or dense) + sum of the payloads.
+    sized=True passes each payload tensor's size in bytes along, so that a
+    truncated payload is refused on the device."""
     W = len(payloads)
     if not (dense.is_cuda and dense.is_contiguous() and dense.dim() == 1):
         raise ValueError("dense must be a contiguous 1-D CUDA float32 tensor")
@@ -296,8 +301,13 @@ def nsml_decompress_accumulate(payloads: Sequence, dense, zero_first: bool = Tru
     if workspace is None:
         workspace = alloc_bytes(nsml_accumulate_workspace_bytes(n, max(1, min(W, NSML_MAX_WORKERS))), dense.device)
     ptrs = (ctypes.c_void_p * max(W, 1))(*[p.data_ptr() for p in payloads])
-    rc = lib.nsml_decompress_accumulate(ptrs, W, dense.data_ptr(), n, 1 if zero_first else 0,
-                                        workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    if sized:
+        sizes = (ctypes.c_size_t * max(W, 1))(*[p.numel() * p.element_size() for p in payloads])
+        rc = lib.nsml_decompress_accumulate_sized(ptrs, sizes, W, dense.data_ptr(), n, 1 if zero_first else 0,
+                                                  workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
+    else:
+        rc = lib.nsml_decompress_accumulate(ptrs, W, dense.data_ptr(), n, 1 if zero_first else 0,
+                                            workspace.data_ptr(), workspace.numel(), _stream_ptr(stream))
     _check(rc, "nsml_decompress_accumulate")
     return dense
 

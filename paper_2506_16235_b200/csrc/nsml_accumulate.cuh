@@ -19,6 +19,7 @@ constexpr int kDenseTile = 8192;  // dense elements per block iteration (32 KB o
 
 struct PayloadTable {
   const unsigned char* p[NSML_MAX_WORKERS];
+  unsigned long long bytes[NSML_MAX_WORKERS];  // size of the buffer behind p[w]; 0 = not known
 };
 
 struct AccumulateLayout {
@@ -34,18 +35,27 @@ inline AccumulateLayout accumulate_layout(int64_t n, int W) {
   return L;
 }
 
-__device__ inline bool header_ok(const nsml_payload_header* h, unsigned long long n) {
+// A header is accepted when its fields describe a payload for this n in the layout nsml_compress writes
+// and, where the size of the buffer is known (bytes != 0), that layout fits the buffer: a truncated
+// payload, or one whose k field was corrupted upwards, is then refused before anything behind the header
+// is read.
+__host__ __device__ inline bool header_ok(const nsml_payload_header* h, unsigned long long n, unsigned long long bytes = 0) {
   if (h->magic != NSML_PAYLOAD_MAGIC || h->version != NSML_PAYLOAD_VERSION) return false;
   if (h->n != n || h->k < 1 || h->k > n || h->qblock != NSML_QBLOCK) return false;
   if (h->bits != NSML_BITS_INT8 && h->bits != NSML_BITS_FP16 && h->bits != NSML_BITS_FP32) return false;
   const unsigned long long k = h->k;
   const unsigned long long val_off = 64 + (k * 4 + 15) / 16 * 16;
   if (h->idx_off != 64 || h->val_off != val_off) return false;
+  unsigned long long total;
   if (h->bits == NSML_BITS_INT8) {
-    if (h->nblocks != (k + NSML_QBLOCK - 1) / NSML_QBLOCK) return false;
+    const unsigned long long nblocks = (k + NSML_QBLOCK - 1) / NSML_QBLOCK;
+    if (h->nblocks != nblocks) return false;
     if (h->scale_off != val_off + (k + 15) / 16 * 16) return false;
+    total = h->scale_off + (nblocks * 4 + 15) / 16 * 16;
+  } else {
+    total = val_off + (k * (h->bits == NSML_BITS_FP32 ? 4 : 2) + 15) / 16 * 16;
   }
-  return true;
+  return bytes == 0 || total <= bytes;
 }
 
 // offsets[w][b] = first payload entry of worker w whose index is >= b*kDenseTile.
@@ -66,7 +76,7 @@ k_partition(PayloadTable table, int W, unsigned long long n, unsigned int tiles,
   const int w = (int)(g / per);
   const unsigned long long b = g % per;
   const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(table.p[w]);
-  if (!header_ok(h, n)) {
+  if (!header_ok(h, n, table.bytes[w])) {
     if (lane == 0) offsets[g] = 0;
     return;
   }
@@ -100,7 +110,7 @@ k_partition_wide(PayloadTable table, int W, unsigned long long n, unsigned int t
   const int w = (int)(g / per);
   const unsigned long long b = g % per;
   const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(table.p[w]);
-  if (!header_ok(h, n)) {
+  if (!header_ok(h, n, table.bytes[w])) {
     offsets[g] = 0;
     return;
   }
@@ -138,7 +148,7 @@ k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long
     const unsigned char* pbase = table.p[threadIdx.x];
     const nsml_payload_header* h = reinterpret_cast<const nsml_payload_header*>(pbase);
     WorkerView v = {nullptr, nullptr, nullptr, 0};
-    if (header_ok(h, n)) {
+    if (header_ok(h, n, table.bytes[threadIdx.x])) {
       v.idx = reinterpret_cast<const uint32_t*>(pbase + h->idx_off);
       v.val = pbase + h->val_off;
       v.scale = reinterpret_cast<const float*>(pbase + h->scale_off);

@@ -35,7 +35,7 @@ struct ProfRecord {
   cudaEvent_t start, stop;
 };
 static std::mutex g_prof_mutex;
-static bool g_prof_on = false;
+static std::atomic<bool> g_prof_on{false};
 static std::vector<ProfRecord> g_prof_records;
 static double g_prof_ms[K_COUNT];
 static int64_t g_prof_launches[K_COUNT];
@@ -57,8 +57,9 @@ struct LaunchScope {  // brackets one kernel launch
   int id;
   cudaStream_t stream;
   cudaEvent_t start = nullptr, stop = nullptr;
-  LaunchScope(int id_, cudaStream_t s) : id(id_), stream(s) {
-    if (g_prof_on) {
+  // timed = false: never bracket this launch with events (creating events allocates)
+  LaunchScope(int id_, cudaStream_t s, bool timed = true) : id(id_), stream(s) {
+    if (timed && g_prof_on.load(std::memory_order_relaxed)) {
       cudaEventCreate(&start);
       cudaEventCreate(&stop);
       cudaEventRecord(start, stream);
@@ -202,7 +203,7 @@ static bool use_dense(int64_t n, int64_t k, const DeviceInfo& dev) {
 template <int DTYPE, int FDTYPE>
 static int launch_compress(const void* grad, float* residual, const uint32_t* mask, int64_t n, int64_t k, int bits,
                            unsigned char* ws, unsigned char* payload, const CompressLayout& L, const PayloadLayout& P,
-                           const DeviceInfo& dev, cudaStream_t st) {
+                           const DeviceInfo& dev, cudaStream_t st, bool keep_status = false) {
   Ctl* ctl = reinterpret_cast<Ctl*>(ws);
   uint32_t* seg_idx = reinterpret_cast<uint32_t*>(ws + L.seg_idx);
   uint32_t* seg_val = reinterpret_cast<uint32_t*>(ws + L.seg_val);
@@ -224,13 +225,13 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
     if (want > nseg) want = nseg;
     fgrid = (unsigned int)(want < cap ? want : cap);
     LaunchScope scope(K_CLEAR, st);
-    k_clear<<<4, kCta, 0, st>>>(reinterpret_cast<uint4*>(ws), (unsigned int)(L.group_count / 16));
+    k_clear<<<4, kCta, 0, st>>>(reinterpret_cast<uint4*>(ws), (unsigned int)(L.group_count / 16), keep_status ? 1 : 0);
   } else {
     {
       LaunchScope scope(K_SAMPLE, st);  // one cluster of kSampleBlocks blocks
       k_sample<DTYPE><<<kSampleBlocks, kSampleThreads, 0, st>>>(src, residual, (unsigned long long)n, sample_rank(n, k), ctl,
                                                                 reinterpret_cast<uint4*>(ws),
-                                                                (unsigned int)(L.zero_bytes / 16));
+                                                                (unsigned int)(L.zero_bytes / 16), keep_status ? 1 : 0);
     }
     {
       // bucket pass: a block takes 8 segments per step; at most 4 resident blocks per SM
@@ -327,7 +328,7 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
 
 static int compress_impl(const void* grad, int64_t n, int grad_dtype, double ratio, int bits,
                          const uint32_t* prune_mask, void* payload, size_t payload_capacity, void* workspace,
-                         size_t workspace_bytes, cudaStream_t st) {
+                         size_t workspace_bytes, cudaStream_t st, bool keep_status = false) {
   if (grad == nullptr || payload == nullptr || workspace == nullptr) return NSML_ERR_ARG;
   if (grad_dtype != NSML_F32 && grad_dtype != NSML_BF16) return NSML_ERR_ARG;
   if (!valid_bits(bits)) return NSML_ERR_ARG;
@@ -343,15 +344,17 @@ static int compress_impl(const void* grad, int64_t n, int grad_dtype, double rat
   if (rc != NSML_OK) return rc;
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   unsigned char* pl = static_cast<unsigned char*>(payload);
-  if (grad_dtype == NSML_F32) rc = launch_compress<NSML_F32, NSML_F32>(grad, nullptr, prune_mask, n, k, bits, ws, pl, L, P, *dev, st);
-  else rc = launch_compress<NSML_BF16, NSML_BF16>(grad, nullptr, prune_mask, n, k, bits, ws, pl, L, P, *dev, st);
+  if (grad_dtype == NSML_F32) rc = launch_compress<NSML_F32, NSML_F32>(grad, nullptr, prune_mask, n, k, bits, ws, pl, L, P, *dev, st, keep_status);
+  else rc = launch_compress<NSML_BF16, NSML_BF16>(grad, nullptr, prune_mask, n, k, bits, ws, pl, L, P, *dev, st, keep_status);
   if (rc != NSML_OK) return rc;
   if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
   return NSML_OK;
 }
 
-static int accumulate_impl(const void* const* payloads, int W, float* dense, int64_t n, int zero_first,
-                           void* workspace, size_t workspace_bytes, cudaStream_t st) {
+// payload_bytes: sizes of the buffers behind the payload pointers, or nullptr when the caller does not
+// know them.  timed: whether the launches may be bracketed by profiling events.
+static int accumulate_impl(const void* const* payloads, const size_t* payload_bytes, int W, float* dense, int64_t n,
+                           int zero_first, void* workspace, size_t workspace_bytes, cudaStream_t st, bool timed = true) {
   if (payloads == nullptr || dense == nullptr || workspace == nullptr) return NSML_ERR_ARG;
   if (W < 1 || W > NSML_MAX_WORKERS || n < 1 || n > NSML_MAX_N) return NSML_ERR_ARG;
   if (!aligned(dense, 16) || !aligned(workspace, 256)) return NSML_ERR_ARG;
@@ -360,6 +363,10 @@ static int accumulate_impl(const void* const* payloads, int W, float* dense, int
   for (int w = 0; w < W; ++w) {
     if (payloads[w] == nullptr || !aligned(payloads[w], 16)) return NSML_ERR_ARG;
     table.p[w] = static_cast<const unsigned char*>(payloads[w]);
+    if (payload_bytes != nullptr) {
+      if (payload_bytes[w] < sizeof(nsml_payload_header)) return NSML_ERR_ARG;
+      table.bytes[w] = payload_bytes[w];
+    }
   }
   const AccumulateLayout L = accumulate_layout(n, W);
   if (workspace_bytes < L.total) return NSML_ERR_CAPACITY;
@@ -372,7 +379,7 @@ static int accumulate_impl(const void* const* payloads, int W, float* dense, int
   unsigned int* offsets = reinterpret_cast<unsigned int*>(ws + L.offsets);
   const unsigned int tiles = (unsigned int)((n + kDenseTile - 1) / kDenseTile);
   {
-    LaunchScope scope(K_PARTITION, st);  // also clears the status word
+    LaunchScope scope(K_PARTITION, st, timed);  // also clears the status word
     const unsigned long long offsets_needed = (unsigned long long)W * (tiles + 1ull);
     if (offsets_needed <= 32768) {  // few offsets: a warp each, few round trips
       unsigned int grid = (unsigned int)((offsets_needed * 32 + kCta - 1) / kCta);
@@ -383,7 +390,7 @@ static int accumulate_impl(const void* const* payloads, int W, float* dense, int
     }
   }
   {
-    LaunchScope scope(K_MERGE, st);
+    LaunchScope scope(K_MERGE, st, timed);
     unsigned int grid = grid_for(tiles, 1, dev->sms * dev->merge);
     k_merge<<<grid, kCta, 0, st>>>(table, W, dense, (unsigned long long)n, zero_first, tiles, offsets, status);
   }
@@ -630,7 +637,14 @@ int nsml_compress(const void* grad, int64_t n, int grad_dtype, double ratio, int
 
 int nsml_decompress_accumulate(const void* const* payloads, int W, float* dense, int64_t n, int zero_first,
                                void* workspace, size_t workspace_bytes, void* stream) {
-  return accumulate_impl(payloads, W, dense, n, zero_first, workspace, workspace_bytes,
+  return accumulate_impl(payloads, nullptr, W, dense, n, zero_first, workspace, workspace_bytes,
+                         static_cast<cudaStream_t>(stream));
+}
+
+int nsml_decompress_accumulate_sized(const void* const* payloads, const size_t* payload_bytes, int W, float* dense,
+                                     int64_t n, int zero_first, void* workspace, size_t workspace_bytes, void* stream) {
+  if (payload_bytes == nullptr) return NSML_ERR_ARG;
+  return accumulate_impl(payloads, payload_bytes, W, dense, n, zero_first, workspace, workspace_bytes,
                          static_cast<cudaStream_t>(stream));
 }
 
@@ -643,7 +657,7 @@ int nsml_decompress_accumulate_static(const void* const* payloads, int W, float*
   int rc = static_scratch(&scratch);
   if (rc != NSML_OK) return rc;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
-  rc = accumulate_impl(payloads, W, dense, n, zero_first, scratch, NSML_STATIC_SCRATCH_BYTES, st);
+  rc = accumulate_impl(payloads, nullptr, W, dense, n, zero_first, scratch, NSML_STATIC_SCRATCH_BYTES, st, /*timed=*/false);
   if (rc != NSML_OK || status_out == nullptr) return rc;
   int value = 0;
   if (cudaMemcpyAsync(&value, scratch, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return NSML_ERR_CUDA;
@@ -746,9 +760,10 @@ int nsml_compress_adaptive(const void* grad, int64_t n, int grad_dtype, double r
     const int rc = prune_impl(weights, n, use_ratio, prune_mask, workspace, workspace_bytes, st);
     if (rc != NSML_OK) return rc;
   }
-  // Step 3
+  // Step 3.  The mask build shares the workspace and its status word with this step: when it ran, the
+  // word is kept instead of cleared, so that non-finite weights found in Step 2 are still reported.
   return compress_impl(grad, n, grad_dtype, use_ratio, use_bits, prune_mask, payload, payload_capacity, workspace,
-                       workspace_bytes, st);
+                       workspace_bytes, st, /*keep_status=*/weights != nullptr);
 }
 
 // ---- host-buffer variants --------------------------------------------------
@@ -802,9 +817,15 @@ int nsml_decompress_accumulate_host(const void* const* payloads_host, const size
   if (payloads_host == nullptr || payload_bytes == nullptr || dense_host == nullptr || device_scratch == nullptr)
     return NSML_ERR_ARG;
   if (W < 1 || W > NSML_MAX_WORKERS || !aligned(device_scratch, 256)) return NSML_ERR_ARG;
+  if (n < 1 || n > NSML_MAX_N) return NSML_ERR_ARG;
   size_t total = 0;
   for (int w = 0; w < W; ++w) {
     if (payloads_host[w] == nullptr || payload_bytes[w] < sizeof(nsml_payload_header)) return NSML_ERR_ARG;
+    // the header is in host memory here: a payload that does not describe this n, or whose layout is
+    // larger than the bytes handed over (truncated, or a corrupted k), is refused before any copy or launch
+    nsml_payload_header h;
+    std::memcpy(&h, payloads_host[w], sizeof(h));
+    if (!header_ok(&h, (unsigned long long)n, payload_bytes[w])) return NSML_ERR_PAYLOAD;
     total += payload_bytes[w];
   }
   const size_t need = nsml_accumulate_host_scratch_bytes(n, W, total);
@@ -825,7 +846,7 @@ int nsml_decompress_accumulate_host(const void* const* payloads_host, const size
   if (!zero_first &&
       cudaMemcpyAsync(d_dense, dense_host, (size_t)n * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
     return NSML_ERR_CUDA;
-  int rc = accumulate_impl(d_payloads, W, d_dense, n, zero_first, base, ws, st);
+  int rc = accumulate_impl(d_payloads, payload_bytes, W, d_dense, n, zero_first, base, ws, st);
   if (rc != NSML_OK) return rc;
   if (cudaMemcpyAsync(dense_host, d_dense, (size_t)n * 4, cudaMemcpyDeviceToHost, st) != cudaSuccess)
     return NSML_ERR_CUDA;
@@ -839,6 +860,16 @@ int nsml_last_status(const void* workspace, void* stream, int* status_out) {
   if (cudaMemcpyAsync(&value, workspace, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return NSML_ERR_CUDA;
   if (cudaStreamSynchronize(st) != cudaSuccess) return NSML_ERR_CUDA;
   *status_out = value;
+  return NSML_OK;
+}
+
+int nsml_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int max_polls, void* stream) {
+  if (workspace == nullptr || !aligned(workspace, 256) || max_polls < 1 || max_polls > (1 << 16)) return NSML_ERR_ARG;
+  if (workspace_bytes < 256) return NSML_ERR_CAPACITY;
+  cudaStream_t st = static_cast<cudaStream_t>(stream);
+  if (cudaMemsetAsync(workspace, 0, 256, st) != cudaSuccess) return NSML_ERR_CUDA;
+  k_barrier_probe<<<2, 32, 0, st>>>(static_cast<Ctl*>(workspace), max_polls);
+  if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
   return NSML_OK;
 }
 
@@ -874,7 +905,7 @@ int nsml_prof_enable(int on) {
     }
     g_prof_records.clear();
   }
-  g_prof_on = (on != 0);
+  g_prof_on.store(on != 0, std::memory_order_relaxed);
   return NSML_OK;
 }
 

@@ -142,8 +142,9 @@ __device__ __forceinline__ unsigned int block_excl_scan(unsigned int v, unsigned
 // All blocks arrive, then all leave.  `target` = barrier ordinal * gridDim.x.
 // CLUSTER: the grid is one thread-block cluster and the barrier is the hardware's (release / acquire at
 // cluster scope, which orders the blocks' global-memory traffic as well); it cannot time out.
-template <bool CLUSTER = false, int THREADS, bool D>
-__device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, FinalizeShared<THREADS, D>& sh) {
+// SH: any shared-memory struct with an int member `ok`.  max_polls: polls after which the wait gives up.
+template <bool CLUSTER = false, class SH>
+__device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, SH& sh, int max_polls = kMaxPolls) {
   if (CLUSTER) {
     cooperative_groups::this_cluster().sync();
     return true;
@@ -158,7 +159,7 @@ __device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, Fina
       unsigned int seen;
       asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(seen) : "l"(&ctl->barrier) : "memory");
       if (seen >= target) break;
-      if (++polls > kMaxPolls) { ok = 0; break; }
+      if (++polls > max_polls) { ok = 0; break; }
       if (polls > 256) __nanosleep(64);
     }
     if (!ok) set_status(&ctl->status, NSML_ERR_TIMEOUT);
@@ -166,6 +167,15 @@ __device__ __forceinline__ bool grid_barrier(Ctl* ctl, unsigned int target, Fina
   }
   __syncthreads();
   return sh.ok != 0;
+}
+
+// Self-test of the bounded wait: every block arrives once at a barrier whose target is one arrival more
+// than the grid can deliver, so each wait runs out after max_polls polls, the status word becomes
+// NSML_ERR_TIMEOUT and the kernel returns by itself.
+struct BarrierProbeShared { int ok; };
+__global__ void __launch_bounds__(32) k_barrier_probe(Ctl* ctl, int max_polls) {
+  __shared__ BarrierProbeShared sh;
+  grid_barrier(ctl, gridDim.x + 1u, sh, max_polls);
 }
 
 // Adds the block's shared histogram into the global one (non-empty bins only).
@@ -194,9 +204,9 @@ __device__ __forceinline__ void resolve_digit(const unsigned int* ghist, unsigne
 
 // Clears the control block and the histograms of a workspace (what the sample
 // kernel does on the list path) ahead of a dense-mode finalize.
-__global__ void __launch_bounds__(kCta) k_clear(uint4* __restrict__ region, unsigned int count16) {
+__global__ void __launch_bounds__(kCta) k_clear(uint4* __restrict__ region, unsigned int count16, int keep_status) {
   for (unsigned int i = blockIdx.x * kCta + threadIdx.x; i < count16; i += gridDim.x * kCta)
-    region[i] = make_uint4(0u, 0u, 0u, 0u);
+    region[i] = make_uint4((i == 0 && keep_status) ? reinterpret_cast<const unsigned int*>(region)[0] : 0u, 0u, 0u, 0u);
 }
 
 // Phase 5 of both finalize kernels: quantises the k survivors left in raw_val (int8 per block of 1024

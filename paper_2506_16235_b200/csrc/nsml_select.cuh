@@ -75,7 +75,7 @@ __device__ __forceinline__ void find_digit_from_top(const unsigned int (&own)[PE
 template <int DTYPE>
 __global__ void __cluster_dims__(kSampleBlocks, 1, 1) __launch_bounds__(kSampleThreads)
 k_sample(BucketSrc<DTYPE> src, const float* __restrict__ addend, unsigned long long n, unsigned int rank_from_top,
-         Ctl* ctl, uint4* zero_base, unsigned int zero_vec16) {
+         Ctl* ctl, uint4* zero_base, unsigned int zero_vec16, int keep_status) {
   namespace cg = cooperative_groups;
   __shared__ unsigned int s_keys[kSamples];  // block 0: the sample keys, then (first 4096 words) the histogram
   unsigned int* s_hist = s_keys;
@@ -96,8 +96,9 @@ k_sample(BucketSrc<DTYPE> src, const float* __restrict__ addend, unsigned long l
     unsigned int* remote = cluster.map_shared_rank(s_keys, 0);
     remote[stratum] = key;
   }
+  // keep_status: an error an earlier step of the same call left in the status word stays visible
   for (unsigned int i = rank * kSampleThreads + threadIdx.x; i < zero_vec16; i += kSamples)
-    zero_base[i] = make_uint4(0, 0, 0, 0);
+    zero_base[i] = make_uint4((i == 0 && keep_status) ? (unsigned int)ctl->status : 0u, 0, 0, 0);
   cluster.sync();  // release/acquire at cluster scope: keys have landed in block 0, the control region is cleared
   if (rank != 0) return;
 

@@ -112,9 +112,34 @@ def test_corrupt_payloads_are_reported():
     bad[64:68] = torch.tensor([0xFF, 0xFF, 0xFF, 0x7F], dtype=torch.uint8, device="cuda")  # idx[0] far out of range
     canary = torch.zeros(n + 64, device="cuda")
     nsml.nsml_decompress_accumulate([bad], canary[:n], zero_first=True, workspace=ws)
-    assert nsml.nsml_last_status(ws) in (0, nsml.NSML_ERR_PAYLOAD)  # never written out of range
+    assert nsml.nsml_last_status(ws) == nsml.NSML_ERR_PAYLOAD  # reported, and never written out of range
     assert not canary[n:].any()
     assert run(payload) == 0  # workspace stays usable
+
+
+def test_truncated_payload_is_refused_when_sizes_are_passed():
+    n = 50000
+    gs = worker_grads(n, 2, 9)
+    p0, w0 = check_compress(gs[0], 0.05, 8)
+    p1, w1 = check_compress(gs[1], 0.05, 16)
+    ws = nsml.alloc_bytes(nsml.nsml_accumulate_workspace_bytes(n, 2), "cuda")
+    dense = torch.full((n,), 5.0, device="cuda")
+    # whole payloads with their sizes: the same sum as without sizes
+    nsml.nsml_decompress_accumulate([p0, p1], dense, zero_first=True, workspace=ws, sized=True)
+    assert nsml.nsml_last_status(ws) == 0
+    assert np.array_equal(dense.cpu().numpy(), oracle.decompress_sum([w0, w1], n))
+    # a buffer that ends before the payload its header describes: reported, its entries are not read
+    cut = p0[: p0.numel() - 32].clone()
+    nsml.nsml_decompress_accumulate([cut, p1], dense, zero_first=True, workspace=ws, sized=True)
+    assert nsml.nsml_last_status(ws) == nsml.NSML_ERR_PAYLOAD
+    assert np.array_equal(dense.cpu().numpy(), oracle.decompress_sum([w1], n))  # the intact worker's sum only
+    # k corrupted upwards inside a buffer of the right size
+    grown = p0.clone()
+    grown[16:24] = torch.from_numpy(np.array([w0.k * 4], np.uint64).view(np.uint8)).cuda()
+    nsml.nsml_decompress_accumulate([grown], dense, zero_first=True, workspace=ws, sized=True)
+    assert nsml.nsml_last_status(ws) == nsml.NSML_ERR_PAYLOAD
+    nsml.nsml_decompress_accumulate([p0, p1], dense, zero_first=True, workspace=ws, sized=True)
+    assert nsml.nsml_last_status(ws) == 0
 
 
 def test_host_buffer_variants():

@@ -135,6 +135,27 @@ def test_prune_mask_reports_nonfinite():
     assert status == nsml.NSML_ERR_NONFINITE
 
 
+@pytest.mark.parametrize("ratio", [0.01, 0.5])  # list strategy and dense strategy of Step 3
+def test_whole_algorithm_keeps_the_mask_build_error_visible(ratio):
+    # Steps 2 and 3 share one workspace: non-finite weights found while the mask is built (Step 2) must
+    # still be reported after Step 3 has run on the same workspace
+    n = 100_000
+    rng = np.random.default_rng(17)
+    g = rng.standard_normal(n).astype(np.float32)
+    w = rng.standard_normal(n).astype(np.float32)
+    w[4321] = np.inf
+    ws = nsml.alloc_bytes(int(nsml.lib.nsml_adaptive_workspace_bytes(n, nsml.NSML_F32)), "cuda")
+    nsml.nsml_compress_adaptive(to_device_grad(g), ratio, 0.0, 0.0, plain_bits=8, weights=torch.from_numpy(w).cuda(),
+                                workspace=ws)
+    assert nsml.nsml_last_status(ws) == nsml.NSML_ERR_NONFINITE
+    # and the same workspace reports a clean run afterwards
+    w[4321] = 0.25
+    payload, _, _, _, mask = nsml.nsml_compress_adaptive(to_device_grad(g), ratio, 0.0, 0.0, plain_bits=8,
+                                                         weights=torch.from_numpy(w).cuda(), workspace=ws)
+    assert nsml.nsml_last_status(ws) == 0
+    assert_payload_equal(payload, oracle.compress(g, ratio, 8, prune_mask=oracle.prune_mask(w, ratio)))
+
+
 def test_mask_feeds_compress():
     rng = np.random.default_rng(6)
     n = 200_003

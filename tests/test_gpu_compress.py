@@ -256,3 +256,21 @@ def test_buckets_on_concurrent_streams_and_replayed_from_a_graph():
         graph.replay()
         torch.cuda.synchronize()
         assert_payload_equal(payload[:nsml.nsml_payload_bytes(g.size, ratio, bits)], oracle_compress(fresh, ratio, bits))
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    # a barrier that can never complete: the kernel gives up after the poll limit, returns by itself and
+    # leaves NSML_ERR_TIMEOUT in the status word; the workspace then serves an ordinary call
+    g = synth.config1_bucket(n=1 << 18, seed=3)
+    n = g.size
+    ws = nsml.alloc_bytes(nsml.nsml_workspace_bytes(n), "cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    for polls in (1, 2000):
+        assert nsml.lib.nsml_selftest_bounded_wait(ws.data_ptr(), ws.numel(), polls, stream) == 0
+        assert nsml.nsml_last_status(ws) == nsml.NSML_ERR_TIMEOUT
+    assert nsml.lib.nsml_selftest_bounded_wait(ws.data_ptr(), ws.numel(), 0, stream) == nsml.NSML_ERR_ARG
+    assert nsml.lib.nsml_selftest_bounded_wait(ws.data_ptr(), ws.numel(), 1 << 20, stream) == nsml.NSML_ERR_ARG
+    assert "wait" in nsml.nsml_strerror(nsml.NSML_ERR_TIMEOUT)
+    payload = nsml.nsml_compress(torch.from_numpy(g).cuda(), 0.01, 8, workspace=ws)
+    assert nsml.nsml_last_status(ws) == 0
+    assert_payload_equal(payload, oracle.compress(g, 0.01, 8))

@@ -2,12 +2,15 @@
 allocate device memory (its scratch is an array inside the library image).
 Checked through the C ABI against nsml_decompress_accumulate on the same
 payloads, twice in a row, because the array is shared by every call and keeps
-the previous call's contents.  Collected last on purpose."""
+the previous call's contents; against the CPU sum of CPU-built payloads; and
+for leaving the device's free memory untouched.  Collected last on purpose."""
 import ctypes
 
 import numpy as np
 import pytest
 import torch
+
+import oracle
 
 pytestmark = pytest.mark.gpu
 
@@ -15,12 +18,15 @@ if torch.cuda.is_available():
     import paper_2506_16235_b200 as nsml
 
 
-def make_payloads(n, W, seed, ratio=0.03):
+def make_grads(n, W, seed):
     rng = np.random.default_rng(seed)
+    return [(rng.standard_normal(n) * 10.0 ** rng.uniform(-3, -1, n)).astype(np.float32) for _ in range(W)]
+
+
+def make_payloads(n, W, seed, ratio=0.03):
     ws = nsml.alloc_bytes(nsml.nsml_workspace_bytes(n), "cuda")
     out, max_abs = [], 0.0
-    for w in range(W):
-        g = (rng.standard_normal(n) * 10.0 ** rng.uniform(-3, -1, n)).astype(np.float32)
+    for w, g in enumerate(make_grads(n, W, seed)):
         max_abs = max(max_abs, float(np.abs(g).max()))
         bits = 8 if w % 2 == 0 else 16
         out.append(nsml.nsml_compress(torch.from_numpy(g).cuda(), ratio, bits, workspace=ws).clone())
@@ -59,6 +65,36 @@ def test_static_scratch_matches_workspace_variant_twice_in_a_row():
             err = (got.double() - want.double()).abs().max().item()
             assert err <= 1e-6 * max_abs  # the tolerance of the other accumulate tests
             assert torch.equal(got, want)  # and in fact bit-identical: same kernels, same order
+
+
+def test_static_scratch_against_the_cpu_sum_and_without_allocating():
+    # the payloads come from the CPU restatement of the compression, the expected sum from its plain
+    # float64 sum: nothing of the CUDA path is on the expected side
+    n, W, ratio = 300_007, 3, 0.02
+    grads = make_grads(n, W, 21)
+    wants = [oracle.compress(g, ratio, 8 if w % 2 == 0 else 16) for w, g in enumerate(grads)]
+    payloads = [torch.from_numpy(nsml.pack_payload(p.n, p.bits, p.idx, codes=p.codes, scales=p.scales, half=p.half)).cuda()
+                for p in wants]
+    init = np.random.default_rng(5).standard_normal(n).astype(np.float32)
+    tol = 1e-6 * max(float(np.abs(g).max()) for g in grads)
+    got = torch.from_numpy(init.copy()).cuda()
+    assert call_static(payloads, got, True) == (0, 0)  # also the set-up call: the array's address is known from here on
+    err = np.abs(got.cpu().numpy().astype(np.float64) - oracle.decompress_sum(wants, n).astype(np.float64)).max()
+    assert err <= tol
+    # further calls leave the device's free memory as it is, also while per-kernel timing is switched on
+    # (the static path never creates the events that timing uses)
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    nsml.nsml_prof_enable(True)
+    try:
+        for zero_first in (False, True):  # accumulate on top of the first sum, then overwrite again
+            assert call_static(payloads, got, zero_first) == (0, 0)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
+    finally:
+        nsml.nsml_prof_enable(False)
+    want = oracle.decompress_sum(wants, n)  # the last call overwrote
+    assert np.abs(got.cpu().numpy().astype(np.float64) - want.astype(np.float64)).max() <= tol
 
 
 def test_static_scratch_limits_and_status():
