@@ -183,8 +183,12 @@ class Workload:
         self.account(acc, "k_sample", esize * 32768)
         # bucket pass: the bucket read once, one bit per element written
         self.account(acc, "k_mark", esize * n + n // 8)
-        # list stage: the bitmap read, the survivors' values read again from the bucket, index + value written
-        self.account(acc, "k_pick", n // 8 + esize * k + 4 * k + vb * k + s)
+        # list stage: the bitmap read, the survivors' values read again from the bucket and kept with their
+        # indices (8 bytes each, written and read back), then index + value written to the payload
+        self.account(acc, "k_pick_a", n // 8 + esize * k + 4 * k)
+        self.account(acc, "k_pick_settle", 24 * ((n + 8191) // 8192))
+        self.account(acc, "k_pick_b", n // 8 + 4 * k + 4 * k + vb * k + s)
+        self.account(acc, "k_finalize_dense", 0)  # enqueued as the fallback; leaves at once
 
     def merge_bytes(self, acc, n, ks_bits, zero_first=True):
         total = 4 * n if zero_first else 0

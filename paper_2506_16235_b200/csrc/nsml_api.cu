@@ -19,14 +19,14 @@
 namespace nsml {
 
 enum KernelId {
-  K_SAMPLE = 0, K_MARK, K_PICK, K_PARTITION, K_MERGE, K_CLEAR, K_FINALIZE_DENSE,
-  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_PRUNE_WRITE_RANKED, K_COUNT
+  K_SAMPLE = 0, K_MARK, K_PICK_A, K_PARTITION, K_MERGE, K_CLEAR, K_FINALIZE_DENSE,
+  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_PRUNE_WRITE_RANKED, K_PICK_B, K_PICK_SETTLE, K_COUNT
 };
 
-static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_mark", "k_pick", "k_partition", "k_merge",
+static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_mark", "k_pick_a", "k_partition", "k_merge",
                                                   "k_clear", "k_finalize_dense", "k_sumsq", "k_feedback_add",
                                                   "k_feedback_subtract", "k_prune_hist", "k_prune_ties", "k_prune_write",
-                                                  "k_prune_write_ranked"};
+                                                  "k_prune_write_ranked", "k_pick_b", "k_pick_settle"};
 
 static std::atomic<int64_t> g_launches{0};
 
@@ -86,10 +86,6 @@ struct DeviceInfo {
 static DeviceInfo g_dev[64];
 static std::mutex g_dev_mutex;
 
-// Candidates a block of the list stage can hold, by shape (the kernel is the same; only the dynamic
-// shared memory differs, and with it how many other blocks fit beside it on an SM).
-static const unsigned int kPickCaps[3] = {4096, 8192, 20480};
-
 static int device_info(const DeviceInfo** out) {
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return NSML_ERR_CUDA;
@@ -108,9 +104,8 @@ static int device_info(const DeviceInfo** out) {
     prepare(k_finalize_dense<NSML_BF16, kFinSmallThreads>, kFinSmallThreads, finalize_dyn_smem(kFinSmallCache), &d.finalize_small);
     prepare(k_finalize_dense<NSML_F32, kFinLargeThreads>, kFinLargeThreads, finalize_dyn_smem(kFinDenseLargeCache), &d.finalize_large);
     prepare(k_finalize_dense<NSML_BF16, kFinLargeThreads>, kFinLargeThreads, finalize_dyn_smem(kFinDenseLargeCache), &d.finalize_large);
-    int pick = 0;  // the largest shape of the list stage must fit an SM
-    prepare(k_pick<NSML_F32>, kPickThreads, pick_dyn_smem(kPickCaps[2]), &pick);
-    prepare(k_pick<NSML_BF16>, kPickThreads, pick_dyn_smem(kPickCaps[2]), &pick);
+    int pick = 0;
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&pick, k_pick_a<NSML_F32>, kPickThreads, 0);
     int sample = 0;
     prepare(k_sample<NSML_F32>, kSampleThreads, kSampleSmem, &sample);
     prepare(k_sample<NSML_BF16>, kSampleThreads, kSampleSmem, &sample);
@@ -187,12 +182,6 @@ static SampleRanks sample_ranks(int64_t n, int64_t k) {
   return r;
 }
 
-// Candidates the bucket pass is expected to mark (k plus the sampling margin).
-static double expected_candidates(int64_t n, int64_t k) {
-  const double p = (double)k / (double)n;
-  return (double)n * (p + 6.0 * std::sqrt(p * (1.0 - p) / kSamples)) + 64.0;
-}
-
 // Kept fraction from which the select runs over the bucket itself.
 constexpr double kDenseRatio = 0.25;
 
@@ -229,36 +218,26 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
   fp.raw_val = reinterpret_cast<float*>(ws + L.raw_val);
   fp.payload = payload;
   fp.P = P;
-  fp.fine = reinterpret_cast<const unsigned int*>(ws + L.fine);
-  fp.group_count = reinterpret_cast<const unsigned int*>(ws + L.group_count);
-  fp.ngroups = (unsigned int)(((unsigned long long)n + kGroupElems - 1) / kGroupElems);
   fp.bitmap = reinterpret_cast<const uint32_t*>(ws + L.bitmap);
   fp.und = reinterpret_cast<uint2*>(ws + L.und);
   fp.qcount = reinterpret_cast<unsigned int*>(ws + L.qcount);
-  fp.cap = 0;
+  fp.pick_blocks = (unsigned int)(((unsigned long long)n + kPickElems - 1) / kPickElems);
+  fp.per_block = reinterpret_cast<unsigned int*>(ws + L.per_block);
+  fp.stash_val = reinterpret_cast<uint32_t*>(ws + L.stash);
   fp.dense_cache = 0;
-  {
-    // The raw-value area holds k floats on the list strategy (k < n / 4); what lies behind them serves as
-    // the spill area for shares of the candidates that do not fit a block's shared memory.
-    const size_t n_floats = (L.total - L.raw_val) / 4, used = align_up((size_t)k, 1024);
-    const size_t spare = n_floats > used ? n_floats - used : 0;
-    fp.spill_entries = spare / 2;
-    fp.spill_idx = reinterpret_cast<uint32_t*>(fp.raw_val + used);
-    fp.spill_val = fp.spill_idx + fp.spill_entries;
-  }
+  fp.only_on_fallback = 0;
   void* args[] = {&fsrc, &fp};
 
-  if (use_dense(n, k, dev)) {
-    const bool small_shape = (unsigned long long)n <= (unsigned long long)dev.sms * kFinSmallCache;
+  // the select over the bucket itself: the whole job on the dense strategy, the fallback of the list strategy
+  // (as the fallback it takes the small shape whatever the bucket's size: it almost always leaves at once, and
+  // a small grid of small blocks is the cheapest thing to launch for that)
+  auto launch_dense = [&]() -> int {
+    const bool small_shape = fp.only_on_fallback || (unsigned long long)n <= (unsigned long long)dev.sms * kFinSmallCache;
     unsigned long long cap = small_shape ? (unsigned long long)dev.sms : finalize_large_blocks(dev);
     if (cap > (unsigned long long)kMaxFinalizeBlocks) cap = kMaxFinalizeBlocks;
     unsigned long long want = (unsigned long long)n / 4096 + 1;  // at least about 4096 elements per block
     if (want > nseg) want = nseg;
     const unsigned int fgrid = (unsigned int)(want < cap ? want : cap);
-    {
-      LaunchScope scope(K_CLEAR, st);
-      k_clear<<<4, kCta, 0, st>>>(reinterpret_cast<uint4*>(ws), (unsigned int)(L.fine / 16), keep_status ? 1 : 0);
-    }
     LaunchScope scope(K_FINALIZE_DENSE, st);
     cudaError_t le;
     if (small_shape) {
@@ -271,6 +250,14 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
                                        dim3(kFinLargeThreads), args, finalize_dyn_smem(kFinDenseLargeCache), st);
     }
     return le == cudaSuccess ? NSML_OK : NSML_ERR_CUDA;
+  };
+
+  if (use_dense(n, k, dev)) {
+    {
+      LaunchScope scope(K_CLEAR, st);
+      k_clear<<<4, kCta, 0, st>>>(reinterpret_cast<uint4*>(ws), (unsigned int)(L.fine / 16), keep_status ? 1 : 0);
+    }
+    return launch_dense();
   }
 
   const SampleRanks ranks = sample_ranks(n, k);
@@ -280,43 +267,38 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
     const size_t clear_bytes = L.qcount + align_up(((size_t)k / NSML_QBLOCK + 2) * 4, 16);
     const int keys16 = (DTYPE == NSML_BF16 && residual == nullptr) ? 1 : 0;
     k_sample<DTYPE><<<kSampleBlocks, kSampleThreads, kSampleSmem, st>>>(src, residual, (unsigned long long)n, ranks.lo, ranks.hi, keys16,
-                                                              ctl, reinterpret_cast<uint4*>(ws),
-                                                              (unsigned int)(clear_bytes / 16), keep_status ? 1 : 0);
+                                                                        ctl, reinterpret_cast<uint4*>(ws),
+                                                                        (unsigned int)(clear_bytes / 16), keep_status ? 1 : 0);
   }
   {
-    // bucket pass: one wave of resident blocks
+    // bucket pass; at most four blocks per SM: enough loads in flight for the memory system, and half of an
+    // SM's threads stay free for kernels of other streams
     LaunchScope scope(K_MARK, st);
     const int resident = residual != nullptr ? dev.mark_feedback : dev.mark;
-    // at most four blocks per SM: enough loads in flight for the memory system, and half of an SM's threads
-    // stay free for kernels of other streams
     const unsigned int grid = grid_for(((unsigned long long)n + kStreamTile - 1) / kStreamTile, 1, dev.sms * (resident < 4 ? resident : 4));
     uint32_t* bitmap = reinterpret_cast<uint32_t*>(ws + L.bitmap);
     unsigned int* group_count = reinterpret_cast<unsigned int*>(ws + L.group_count);
     unsigned int* fine = reinterpret_cast<unsigned int*>(ws + L.fine);
-    if (residual != nullptr) k_mark<DTYPE, true><<<grid, kCta, 0, st>>>(src, residual, (unsigned long long)n, ctl, bitmap, group_count, fine);
-    else k_mark<DTYPE, false><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, ctl, bitmap, group_count, fine);
+    if (residual != nullptr)
+      k_mark<DTYPE, true><<<grid, kCta, 0, st>>>(src, residual, (unsigned long long)n, (unsigned long long)k, ctl, bitmap, group_count, fine);
+    else
+      k_mark<DTYPE, false><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, (unsigned long long)k, ctl, bitmap, group_count, fine);
   }
   {
-    // list stage: cooperative, every block co-resident; about 1500 expected candidates and at least 32
-    // groups of bitmap per block, no more blocks than SMs
-    LaunchScope scope(K_PICK, st);
-    const double expected = expected_candidates(n, k);
-    unsigned long long want = (unsigned long long)(expected / 1536.0) + 1;
-    const unsigned long long by_groups = (fp.ngroups + 31ull) / 32;
-    if (by_groups > want) want = by_groups;
-    unsigned int fgrid = (unsigned int)(want < (unsigned long long)dev.sms ? want : (unsigned long long)dev.sms);
-    if ((unsigned long long)fgrid > nseg) fgrid = (unsigned int)nseg;
-    if (fgrid > (unsigned int)kMaxFinalizeBlocks) fgrid = kMaxFinalizeBlocks;
-    // room for an average share and a quarter on top; larger shares (candidates crowd into a few tensors)
-    // live in the spill area, and so does everything when not even the largest shape would do
-    const double room = expected / fgrid * 1.25;
-    fp.cap = room <= kPickCaps[0] ? kPickCaps[0] : (room <= kPickCaps[1] ? kPickCaps[1] : (room <= kPickCaps[2] ? kPickCaps[2] : kPickCaps[0]));
-    const size_t smem = pick_dyn_smem(fp.cap);
-    fp.dense_cache = (unsigned int)(smem / 4 / 128 * 128);  // what a fallback to the select over the bucket may use
-    if (cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_pick<FDTYPE>), dim3(fgrid), dim3(kPickThreads), args, smem, st) != cudaSuccess)
-      return NSML_ERR_CUDA;
+    LaunchScope scope(K_PICK_A, st);
+    k_pick_a<FDTYPE><<<fp.pick_blocks, kPickThreads, 0, st>>>(fsrc, fp);
   }
-  return NSML_OK;
+  {
+    LaunchScope scope(K_PICK_SETTLE, st);
+    k_pick_settle<<<1, kPickThreads, 0, st>>>(fp);
+  }
+  {
+    LaunchScope scope(K_PICK_B, st);
+    k_pick_b<<<fp.pick_blocks, kPickThreads, 0, st>>>(fp);
+  }
+  // the fallback: leaves at once unless the list stage raised ctl->fallback
+  fp.only_on_fallback = 1;
+  return launch_dense();
 }
 
 static int compress_impl(const void* grad, int64_t n, int grad_dtype, double ratio, int bits,

@@ -29,12 +29,19 @@ constexpr int kMaxPolls = 1 << 22;
 struct Ctl {
   int status;                 // first device-detected error (NSML_ERR_*), 0 = ok
   unsigned int lo;            // sampled lower bound of the threshold key: candidates are the keys >= max(lo, 1)
-  unsigned int barrier;       // arrivals at the grid barriers of the cooperative kernels
+  unsigned int barrier;       // arrivals at the grid barriers of the cooperative kernel
   unsigned int shift;         // fine histogram: bin = min((key - lo) >> shift, kFineBins - 1)
   unsigned int exact;         // every fine bin below the last holds one representable key value
   unsigned int und_count;     // entries appended to the list of undecided candidates
   unsigned int fallback;      // the list stage gave up (too few candidates, a full table): select over the bucket
-  unsigned int pad;
+  unsigned int mark_done;     // blocks of the bucket pass that have finished
+  unsigned int pick_done;     // blocks of the first list kernel that have finished
+  unsigned int Tbin;          // fine bin that holds the k-th largest key
+  unsigned int rem;           // rank of that key inside its bin, from the top
+  unsigned int by_bin;        // the bin itself decides: above it = above T, in it = equal to T (exact && Tbin not the last)
+  unsigned int T;             // listed case: the threshold key ...
+  unsigned int limit;         // ... and the index up to which ties at T survive
+  unsigned int ties_kept;     // by-bin case: keys equal to T that survive, lowest index first
 };
 static_assert(sizeof(Ctl) <= 256, "control block must fit its 256-byte slot");
 
@@ -43,6 +50,9 @@ constexpr int kMaxFinalizeBlocks = 1024;  // upper bound on blocks of the cooper
 constexpr int kFineBins = 2048;           // bins of the candidates' key histogram built by the bucket pass
 constexpr int kFineStride = 32;            // words between two bins' counters: neighbouring bins, which are hot together, sit in different 128-byte lines
 constexpr int kGroupElems = 4096;         // bucket elements per group; the bucket pass keeps a candidate count per group
+constexpr int kPickGroups = 8;            // groups (32768 elements) a block of the list stage owns
+constexpr int kPickElems = kPickGroups * kGroupElems;
+constexpr int kStashPerBlock = kPickElems;      // values of one block's candidates the stash holds: room for every element
 constexpr int kRoundElems = 128;          // bucket elements per round: 4 words (16 bytes) of the candidate bitmap
 constexpr unsigned int kUndCap = 2048;    // undecided candidates (those in the threshold's fine bin) that can be listed
 
@@ -52,10 +62,13 @@ struct CompressLayout {  // byte offsets inside a compress workspace
   size_t group_count;   // u32[ceil(n / kGroupElems)]: candidates per group
   size_t qcount;        // u32[n / 4096 + 2]: survivors delivered so far per block of 1024 payload entries
   size_t zero_bytes;    // everything before this offset is cleared per call
-  size_t block_counts;  // u64[4][kMaxFinalizeBlocks]: per-block counts exchanged at barriers
+  size_t block_counts;  // u64[4][kMaxFinalizeBlocks]: per-block counts exchanged at barriers (dense select)
   size_t und;           // uint2[kUndCap]: (value bits, index) of the undecided candidates
+  size_t per_block;     // u32[6][ceil(n / kPickElems)]: list stage, per block: candidates, above the bin, in the bin,
+                        //   listed survivors, survivors before the block, in-bin entries before the block
   size_t bitmap;        // u32[4 * ceil(n / kRoundElems)]: bit (i & 31) of word i >> 5 set = element i is a candidate
-  size_t raw_val;       // f32[n]: survivor values before quantisation
+  size_t raw_val;       // f32[n]: survivor values before quantisation (list strategy: at most n / 4 of them) ...
+  size_t stash;         // ... list strategy: u32[ceil(n / kPickElems) * kPickElems]: values of each block's candidates
   size_t total;
 };
 
@@ -65,6 +78,7 @@ inline CompressLayout compress_layout(int64_t n) {
   CompressLayout L;
   const size_t groups = ((size_t)n + kGroupElems - 1) / kGroupElems;
   const size_t rounds = ((size_t)n + kRoundElems - 1) / kRoundElems;
+  const size_t pick_blocks = ((size_t)n + kPickElems - 1) / kPickElems;
   L.hist = 256;
   L.fine = L.hist + 4 * kMaxBins * sizeof(unsigned int);
   L.group_count = L.fine + (size_t)kFineBins * kFineStride * sizeof(unsigned int);
@@ -72,9 +86,13 @@ inline CompressLayout compress_layout(int64_t n) {
   L.zero_bytes = L.qcount + align_up(((size_t)n / 4096 + 2) * 4, 256);
   L.block_counts = L.zero_bytes;
   L.und = L.block_counts + 4 * kMaxFinalizeBlocks * 8;
-  L.bitmap = L.und + (size_t)kUndCap * 8;
+  L.per_block = L.und + (size_t)kUndCap * 8;
+  L.bitmap = L.per_block + align_up(6 * pick_blocks * 4, 256);
   L.raw_val = L.bitmap + align_up(rounds * 16, 256);
-  L.total = L.raw_val + align_up((size_t)n * 4, 256);
+  // the dense select keeps up to n raw values; the list strategy n / 4 raw values and the stash behind them
+  L.stash = L.raw_val + align_up(((size_t)n / 4 + 1024) * 4, 256);
+  L.total = L.stash + pick_blocks * (size_t)kStashPerBlock * 4;
+  if (L.total < L.raw_val + align_up((size_t)n * 4, 256)) L.total = L.raw_val + align_up((size_t)n * 4, 256);
   return L;
 }
 

@@ -1,5 +1,5 @@
 // Bucket -> payload by a radix select over the bucket itself, in one cooperative launch
-// (a kernel of its own, and the fallback inside the list stage's kernel).
+// (the strategy for high kept fractions, and the fallback of the list stage).
 //
 // For calls that keep a large fraction of the bucket (or whose bucket is too
 // small to sample) a candidate list would be about as large as the bucket, so
@@ -30,8 +30,7 @@
 
 namespace nsml {
 
-// The whole select as a device function, so that the list stage can fall back to it inside its own
-// cooperative launch.  s_cache: p.dense_cache words of shared memory (a multiple of 128: a warp step of 32
+// The whole select as a device function.  s_cache: p.dense_cache words of shared memory (a multiple of 128: a warp step of 32
 // words is cached as a whole or not at all); `barriers`: grid barriers this launch has already passed.
 template <int DTYPE, int THREADS>
 __device__ __forceinline__ void dense_select(const BucketSrc<DTYPE>& src, const FinalizeParams& p, FinalizeShared<THREADS>& sh,
@@ -409,6 +408,8 @@ __global__ void __launch_bounds__(THREADS, 1024 / THREADS)  // at most 64 regist
 k_finalize_dense(BucketSrc<DTYPE> src, FinalizeParams p) {
   __shared__ FinalizeShared<THREADS> sh;
   extern __shared__ __align__(16) uint32_t s_dense_cache[];
+  // enqueued behind the list stage as its fallback: nothing to do unless the list stage asked for it
+  if (p.only_on_fallback && __ldcg(&p.ctl->fallback) == 0) return;
   dense_select<DTYPE, THREADS>(src, p, sh, s_dense_cache, 0u);
 }
 

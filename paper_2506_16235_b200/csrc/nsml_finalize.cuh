@@ -35,16 +35,13 @@ struct FinalizeParams {
   PayloadLayout P;
   unsigned int dense_cache;          // values a block of the dense select keeps in shared memory (a multiple of 128)
   // list stage only
-  const unsigned int* fine;          // [kFineBins]
-  const unsigned int* group_count;   // [ngroups]
-  unsigned int ngroups;
   const uint32_t* bitmap;
   uint2* und;                        // [kUndCap]
   unsigned int* qcount;
-  unsigned int cap;                  // candidates a block can hold in shared memory
-  uint32_t* spill_idx;               // [spill_entries] indices, [spill_entries] values: shares larger than cap
-  uint32_t* spill_val;
-  unsigned long long spill_entries;
+  unsigned int pick_blocks;          // blocks of the list kernels: ceil(n / kPickElems)
+  unsigned int* per_block;           // [6][pick_blocks], see CompressLayout
+  uint32_t* stash_val;               // [pick_blocks * kStashPerBlock]
+  int only_on_fallback;              // dense select: leave at once unless the list stage asked for it
 };
 
 constexpr int kUndWarpCap = 192;  // undecided entries a warp of the dense select can list
@@ -189,9 +186,9 @@ __device__ __forceinline__ void write_header(const FinalizeParams& p) {
 // 1024 survivors qb from raw_val into the payload (int8 with a max-abs scale, fp16, or float32 as is);
 // live = false: this group has no block this round.  Called by every thread of the thread block (it
 // holds block barriers).
-template <int THREADS>
-__device__ __forceinline__ void quantize_block(const FinalizeParams& p, FinalizeShared<THREADS>& sh,
-                                               unsigned long long qb, bool live) {
+// SH: any shared-memory struct with a float array qmax of one entry per warp.
+template <class SH>
+__device__ __forceinline__ void quantize_block(const FinalizeParams& p, SH& sh, unsigned long long qb, bool live) {
   const int lane = threadIdx.x & 31;
   const int group = threadIdx.x >> 8, gtid = threadIdx.x & 255;
   const unsigned long long j0 = qb * NSML_QBLOCK + gtid * 4;

@@ -20,6 +20,7 @@
 #pragma once
 
 #include "nsml_common.cuh"
+#include "nsml_select.cuh"
 
 namespace nsml {
 
@@ -38,7 +39,7 @@ __device__ __forceinline__ unsigned int keep_flags(const uint32_t (&bits)[4], fl
 // zeroes a key, not the stored sum.
 template <int DTYPE, bool FEEDBACK>
 __global__ void __launch_bounds__(kCta)
-k_mark(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned long long n, const Ctl* __restrict__ ctl,
+k_mark(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned long long n, unsigned long long k, Ctl* ctl,
        uint32_t* __restrict__ bitmap, unsigned int* __restrict__ group_count, unsigned int* __restrict__ fine) {
   static_assert(kGroupElems % kStreamTile == 0, "a tile lies inside one group");
   // When every bin holds one key value (bfloat16 keys, massive ties) the candidates fall into a few dozen
@@ -53,7 +54,7 @@ k_mark(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned long long n,
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   // Zeros are never candidates; if they are needed (fewer than k non-zero keys) the candidates come out
   // short and the list stage falls back to the select over the bucket itself.
-  const unsigned int lo = max(ctl->lo, 1u), shift = ctl->shift;
+  const unsigned int lo = max(ctl->lo, 1u), shift = ctl->shift;  // (written by the sample kernel)
   const float t = __uint_as_float(lo);
   const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
   const unsigned long long nwords = ((n + kRoundElems - 1) / kRoundElems) * 4;  // whole rounds
@@ -151,6 +152,42 @@ k_mark(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned long long n,
       const unsigned int c = s_fine[b];
       if (c != 0) atomicAdd(fine + b * kFineStride, c);
     }
+  }
+
+  // The block that finishes last resolves the fine bin that holds the k-th largest key, once for everybody:
+  // the list stage starts from it.  (Every thread's adds are ordered before its block's ticket.)
+  __shared__ unsigned int s_tot[kCta / 32], s_out[2], s_last;
+  __shared__ unsigned long long s_sum[kCta / 32];
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) s_last = atomicAdd(&ctl->mark_done, 1u) == gridDim.x - 1;
+  __syncthreads();
+  if (!s_last) return;
+  __threadfence();
+  constexpr int PER = kFineBins / kCta;
+  unsigned int own[PER];
+  unsigned long long mine = 0;
+#pragma unroll
+  for (int b = 0; b < PER; ++b) {
+    own[b] = __ldcg(fine + (size_t)(threadIdx.x * PER + b) * kFineStride);
+    mine += own[b];
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, o);
+  if (lane == 0) s_sum[warp] = mine;
+  __syncthreads();
+  unsigned long long total = 0;
+#pragma unroll
+  for (int w = 0; w < kCta / 32; ++w) total += s_sum[w];
+  if (total < k) {  // fewer candidates than survivors: the select runs over the bucket itself
+    if (threadIdx.x == 0) ctl->fallback = 1u;
+    return;
+  }
+  find_digit_from_top<PER, kCta>(own, (unsigned int)k, s_tot, s_out);
+  if (threadIdx.x == 0) {
+    ctl->Tbin = s_out[0];
+    ctl->rem = s_out[1];
+    ctl->by_bin = ctl->exact != 0 && s_out[0] + 1 < (unsigned int)kFineBins;
   }
 }
 

@@ -1,343 +1,276 @@
-// Marked candidates -> payload, in one cooperative kernel with ONE grid barrier.
+// Marked candidates -> payload, in three plain kernels (many small blocks, one
+// block, many small blocks): no cooperative launch, no waiting between blocks.
 //
 // The bucket pass (nsml_mark.cuh) leaves a bitmap of the candidates (every key
-// >= lo), their number per group of kGroupElems elements and their histogram
-// over kFineBins key bins.  This kernel finds the exact threshold key T and the
-// tie budget r (Alg. 2 Step 3 read as: keep the k largest |g|, ties by lower
-// index), writes the k survivors in index order and quantises them (Alg. 2
+// >= lo), their histogram over kFineBins key bins, and - resolved by its last
+// block - the fine bin Tbin that holds the k-th largest key with the rank `rem`
+// of that key inside the bin.  The kernels here find the exact threshold key T
+// and the tie budget (Alg. 2 Step 3 read as: keep the k largest |g|, ties by
+// lower index), write the k survivors in index order and quantise them (Alg. 2
 // Step 1 "quantize" for fp16; int8 per block of 1024 survivors).
 //
-// Before the barrier, every block for itself:
-//   - resolves the fine bin that holds the k-th largest key (the histogram is
-//     complete: it was built by the previous kernel);
-//   - scans the group counts, which gives it an equal share of the candidates
-//     as a run of whole groups (block order = index order, and the work is
-//     balanced however the candidates crowd into a few tensors);
-//   - expands its groups' bitmap words into a list of indices in shared
-//     memory and reads those elements again from the bucket (scattered loads,
-//     all in flight at once), keeping the values in shared memory too (a share
-//     that does not fit shared memory is kept in a spill area in global memory);
-//   - sorts each candidate into "above the threshold's bin" (a survivor whatever
-//     T turns out to be), "in the bin" or "below" (dropped).
-//   If a bin holds a single key value (bfloat16 keys, or bins one key wide) T is
-//   the bin's key and only ties remain: the block publishes its counts of keys
-//   > T and == T.  Otherwise it appends its in-bin candidates (value, index) to
-//   a short global list and publishes its count of keys above the bin.
-// After the barrier, every block for itself:
-//   - sums the other blocks' counts (survivors before its own first one);
-//   - in the second case reads the whole list of in-bin candidates (at most
-//     kUndCap, typically a few hundred), radix-selects T among them, finds the
-//     index up to which ties at T survive, and counts the list's survivors
-//     that lie before its own index range;
-//   - writes its survivors' indices and values at their final payload
-//     positions (fp16 and float32 values directly; int8 values go through
-//     raw_val, and whichever block delivers the last survivor of a block of
-//     1024 payload entries quantises that block - no waiting, no third phase).
+// Block b of k_pick_a and k_pick_b owns the kPickElems elements from
+// b * kPickElems on, so block order is index order, nothing has to be balanced
+// or agreed on, and the hardware schedules the blocks as SMs become free.
+//
+// A thread of these two kernels owns one bitmap round (four words, 128
+// elements) of its block's range; a block-wide scan of the rounds' popcounts
+// gives every thread the position of its candidates among the block's.  Every
+// access to global memory costs about a microsecond of latency however little
+// it moves, so each kernel issues whatever it needs in as few rounds as it can
+// (control words, per-block counts and bitmap together; candidates eight at a
+// time) and the grids are small enough to be resident at once.
+//
+// k_pick_a, per block: reads the marked elements again from the bucket
+// (scattered loads, eight in flight per thread), keeps the values, in index order, in its stretch of a stash in global memory,
+// and sorts each candidate into "above the threshold's bin" (a survivor
+// whatever T turns out to be), "in the bin" or "below" (dropped).  If a bin holds a single
+// key value (bfloat16 keys, or bins one key wide) T is the bin's key and only
+// ties remain; otherwise the block appends its in-bin candidates (value, index)
+// to a short global list.  It publishes its counts.
+//
+// k_pick_settle, one block: reads the whole list of in-bin candidates (at most
+// kUndCap, typically a few hundred), finds T as the list's rem-th largest key
+// and the index up to which ties at T survive, and writes for every block of
+// the other two kernels the number of survivors before it.
+//
+// k_pick_b, per block: reads its candidates' values back from the stash, counts
+// its survivors per word, scans the counts and writes the survivors' indices
+// and values at their final payload positions (fp16 and float32 values
+// directly; int8 values go through raw_val, and whichever block delivers the
+// last survivor of a block of 1024 payload entries quantises that block - no
+// waiting, no further kernel).
 //
 // Whatever this scheme cannot handle - fewer candidates than k (too few
-// non-zero keys, or a misleading sample), a table that does not fit shared
-// memory, more in-bin candidates or ties than can be listed - is
-// detected by every block alike, and the launch then runs the select over the
-// bucket itself (nsml_dense.cuh) instead: the result is exact in every case.
+// non-zero keys, or a misleading sample), more in-bin candidates or ties than
+// can be listed - raises ctl->fallback; the kernels then leave at once and the
+// select over the bucket itself (nsml_dense.cuh), which is enqueued behind them
+// in any case and otherwise leaves at once itself, produces the payload: the
+// result is exact in every case.
+//
+// Every global index these kernels compute is checked against its array's
+// bound; a violation (which would be a bug) is recorded as NSML_ERR_INTERNAL
+// and the access is skipped.
 #pragma once
 
-#include "nsml_dense.cuh"
 #include "nsml_finalize.cuh"
 
 namespace nsml {
 
-constexpr int kPickThreads = 256;
-constexpr int kPickGroupCap = 1024;   // groups a block can own
+constexpr int kPickThreads = kPickElems / kRoundElems;  // 256: one bitmap round (128 elements) per thread
 constexpr int kPickTieCap = 1024;     // ties at the threshold whose rank by index is worked out from the list
 constexpr int kPickRankCap = 768;     // listed candidates up to which the threshold is found by counting ranks
-constexpr int kPickInbinCap = 16;     // in-bin candidates a warp remembers (more: it walks its run again)
-constexpr int kPickQCap = 64;         // blocks of 1024 payload entries a block can complete
-constexpr int kGroupRounds = kGroupElems / kRoundElems;  // 64
-// shared memory of the list stage for a block that holds `cap` candidates: indices, values, the undecided list
-constexpr size_t pick_dyn_smem(unsigned int cap) { return (size_t)cap * 8 + (size_t)kUndCap * 8; }
+constexpr int kPickQCap = 40;         // blocks of 1024 payload entries a block can complete (kPickElems / 1024 + 2 at most)
+constexpr int kPickFlight = 8;        // candidates a thread fetches at a time
+static_assert(kPickThreads == 256, "the quantisation takes 256 threads per block of 1024 entries");
+static_assert(kPickElems <= 32768 && kPickElems / NSML_QBLOCK + 2 <= kPickQCap, "a block's survivors span at most kPickQCap payload blocks");
+
+// rows of FinalizeParams::per_block
+enum { PB_CANDS = 0, PB_ABOVE, PB_INBIN, PB_LISTED, PB_BEFORE, PB_INBIN_BEFORE };
+
+__device__ __forceinline__ unsigned int fine_bin(uint32_t key, unsigned int lo, unsigned int shift) {
+  return min((key - lo) >> shift, (unsigned int)(kFineBins - 1));
+}
+
+// Exclusive prefix over the block (kPickThreads threads) in thread order; `total` = sum over the block.
+// s_warp: one word per warp.
+__device__ __forceinline__ unsigned int pick_scan(unsigned int v, unsigned int& total, unsigned int* s_warp) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  unsigned int incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= o) incl += up;
+  }
+  __syncthreads();  // s_warp may still be read from an earlier call
+  if (lane == 31) s_warp[warp] = incl;
+  __syncthreads();
+  unsigned int before = 0, all = 0;
+#pragma unroll
+  for (int w = 0; w < kPickThreads / 32; ++w) {
+    const unsigned int c = s_warp[w];
+    if (w < warp) before += c;
+    all += c;
+  }
+  total = all;
+  return before + incl - v;
+}
+
+// This thread's bitmap round as two 64-bit masks: bit e of half h = element round_base + 64 h + e of the
+// bucket is a candidate.  (No other memory access of the kernel depends on anything: issue it first.)
+struct PickRound {
+  unsigned long long half[2];
+  unsigned long long base;  // index of the round's first element
+  __device__ __forceinline__ unsigned int count() const { return __popcll(half[0]) + __popcll(half[1]); }
+};
+__device__ __forceinline__ PickRound pick_round(const FinalizeParams& p) {
+  const unsigned long long round_id = (unsigned long long)blockIdx.x * kPickThreads + threadIdx.x;
+  const unsigned long long rounds_all = (p.n + kRoundElems - 1) / kRoundElems;
+  uint4 m = make_uint4(0u, 0u, 0u, 0u);
+  if (round_id < rounds_all) m = __ldcg(reinterpret_cast<const uint4*>(p.bitmap) + round_id);
+  PickRound r;
+  r.half[0] = ((unsigned long long)m.y << 32) | m.x;
+  r.half[1] = ((unsigned long long)m.w << 32) | m.z;
+  r.base = round_id * kRoundElems;
+  return r;
+}
+
+// Calls f(value, index) for the round's candidates in index order; their values are fetched kPickFlight at a
+// time with load(position among the round's candidates, index).
+template <class L, class F>
+__device__ __forceinline__ void for_round_candidates(PickRound r, L&& load, F&& f) {
+  unsigned int done = 0;
+  while ((r.half[0] | r.half[1]) != 0) {
+    uint32_t idx[kPickFlight], v[kPickFlight];
+    int cnt = 0;
+#pragma unroll
+    for (int u = 0; u < kPickFlight; ++u) {
+      idx[u] = 0;
+      if (r.half[0] != 0) {
+        idx[u] = (uint32_t)r.base + (__ffsll((long long)r.half[0]) - 1);
+        r.half[0] &= r.half[0] - 1;
+        cnt = u + 1;
+      } else if (r.half[1] != 0) {
+        idx[u] = (uint32_t)r.base + 64 + (__ffsll((long long)r.half[1]) - 1);
+        r.half[1] &= r.half[1] - 1;
+        cnt = u + 1;
+      }
+    }
+#pragma unroll
+    for (int u = 0; u < kPickFlight; ++u) v[u] = u < cnt ? load(done + u, idx[u]) : 0u;
+#pragma unroll
+    for (int u = 0; u < kPickFlight; ++u)
+      if (u < cnt) f(v[u], idx[u]);
+    done += cnt;
+  }
+}
 
 template <int DTYPE>
-__global__ void __launch_bounds__(kPickThreads, 4)  // at most 64 registers per thread: a quarter of an SM's register file
-k_pick(BucketSrc<DTYPE> src, FinalizeParams p) {
+__global__ void __launch_bounds__(kPickThreads)
+k_pick_a(BucketSrc<DTYPE> src, FinalizeParams p) {
+  __shared__ unsigned int s_warp[kPickThreads / 32];
+  __shared__ unsigned long long s_red[kPickThreads / 32];
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const unsigned int blk = blockIdx.x, B = p.pick_blocks;
+  Ctl* ctl = p.ctl;
+  const PickRound round = pick_round(p);
+  const unsigned int fallback = __ldcg(&ctl->fallback);
+  const unsigned int lo = max(__ldcg(&ctl->lo), 1u), shift = __ldcg(&ctl->shift);
+  const unsigned int Tbin = __ldcg(&ctl->Tbin);
+  const bool by_bin = __ldcg(&ctl->by_bin) != 0;
+  if (fallback != 0) return;  // the bucket pass found fewer candidates than k
+  uint32_t* my_val = p.stash_val + (size_t)blk * kStashPerBlock;
+
+  unsigned int E;
+  const unsigned int first = pick_scan(round.count(), E, s_warp);  // position of this round's first candidate among the block's
+  unsigned int at = first, above = 0, inbin = 0;
+  bool nonfinite = false, bad = false;
+  for_round_candidates(
+      round,
+      [&](unsigned int, uint32_t idx) { return idx < p.n ? src.raw1(idx) : 0u; },  // a candidate is never a pruned element
+      [&](uint32_t v, uint32_t idx) {
+        // the value goes to the stash, the key is compared with the threshold's bin
+        if (at < (unsigned int)kStashPerBlock) my_val[at] = v; else bad = true;
+        ++at;
+        const uint32_t key = v & 0x7FFFFFFFu;
+        nonfinite |= key >= kInfKey;
+        if (key < lo) return;  // cannot happen: the bucket pass marked it
+        const unsigned int bin = fine_bin(key, lo, shift);
+        above += bin > Tbin;
+        if (bin == Tbin) {
+          ++inbin;
+          if (!by_bin) {  // rare: a few hundred entries in the whole bucket
+            const unsigned int slot = atomicAdd(&ctl->und_count, 1u);
+            if (slot < kUndCap) p.und[slot] = make_uint2(v, idx);
+          }
+        }
+      });
+  if (nonfinite) set_status(&ctl->status, NSML_ERR_NONFINITE);
+  if (bad) set_status(&ctl->status, NSML_ERR_INTERNAL);
+  unsigned long long both = ((unsigned long long)above << 32) | inbin;
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) both += __shfl_xor_sync(0xFFFFFFFFu, both, o);
+  if (lane == 0) s_red[warp] = both;
+  __syncthreads();
+  if (threadIdx.x == 0 && blk < B) {
+    both = 0;
+    for (int w = 0; w < kPickThreads / 32; ++w) both += s_red[w];
+    p.per_block[PB_CANDS * B + blk] = E;
+    p.per_block[PB_ABOVE * B + blk] = (unsigned int)(both >> 32);
+    p.per_block[PB_INBIN * B + blk] = (unsigned int)(both & 0xFFFFFFFFull);
+  }
+}
+
+// One block: the exact threshold, and every block's payload position.
+__global__ void __launch_bounds__(kPickThreads)
+k_pick_settle(FinalizeParams p) {
   constexpr int THREADS = kPickThreads;
   constexpr int NW = THREADS / 32;
   constexpr unsigned int FULL = 0xFFFFFFFFu;
   __shared__ FinalizeShared<THREADS> sh;
-  __shared__ unsigned int s_groups[kPickGroupCap];
-  __shared__ unsigned int s_q[kPickQCap];
-  __shared__ unsigned int s_nq, s_limit, s_T;
-  __shared__ unsigned int s_inbin[kPickThreads / 32][kPickInbinCap];  // positions of a warp's candidates in the threshold's bin
-  extern __shared__ __align__(16) uint32_t s_dyn[];
-  uint32_t* c_idx = s_dyn;
-  uint32_t* c_val = s_dyn + p.cap;
-  uint2* s_u = reinterpret_cast<uint2*>(s_dyn + 2 * (size_t)p.cap);
+  __shared__ uint2 s_u[kUndCap];  // the listed candidates
+  __shared__ unsigned int s_T, s_limit;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const unsigned int lt = (1u << lane) - 1u;
-  const unsigned int G = gridDim.x, blk = blockIdx.x;
-  const unsigned int lo = max(p.ctl->lo, 1u), shift = p.ctl->shift;
-  bool give_up = false;  // block-uniform
-  bool in_shared = true;  // the block's candidates are held in shared memory (else in the spill area)
-
-  // ---------------- the threshold's fine bin; this block's share: a run of whole groups ----------------
-  // The histogram and the group counts are both complete (the previous kernel built them): their loads are
-  // issued together.  The group counts are staged in the shared memory that will hold the candidates.
-  unsigned int Tbin = 0, rem = 0;  // rem: rank of the threshold inside its bin, from the top
-  unsigned long long total;
-  unsigned int E = 0;              // candidates this block owns
-  unsigned int owned_all = 0;      // groups this block owns
-  {
-    constexpr int PER = kFineBins / THREADS;
-    unsigned int own[PER], mine = 0;
+  const unsigned int B = p.pick_blocks;
+  Ctl* ctl = p.ctl;
+  // everything this block reads was written by the kernel before it: one round of loads
+  const unsigned int fallback = __ldcg(&ctl->fallback), rem = __ldcg(&ctl->rem);
+  const bool by_bin = __ldcg(&ctl->by_bin) != 0;
+  const unsigned int und_all = __ldcg(&ctl->und_count);
+  constexpr int kHeld = 8;  // blocks per thread whose counts are held in registers
+  const unsigned int per_thread = (B + THREADS - 1) / THREADS;
+  const unsigned int b_begin = min(B, threadIdx.x * per_thread), b_end = min(B, b_begin + per_thread);
+  unsigned int held_above[kHeld], held_inbin[kHeld];
 #pragma unroll
-    for (int b = 0; b < PER; ++b) own[b] = __ldcg(p.fine + (size_t)(threadIdx.x * PER + b) * kFineStride);
-    uint32_t* staged = s_dyn;  // group counts, when they fit
-    const bool stage = p.ngroups <= 2 * p.cap;
-    if (stage)
-      for (unsigned int g = threadIdx.x; g < p.ngroups; g += THREADS) staged[g] = __ldcg(p.group_count + g);
-#pragma unroll
-    for (int b = 0; b < PER; ++b) mine += own[b];
-    total = block_sum((unsigned long long)mine, sh);  // (its barriers also complete the staging)
-    if (total < p.k) {
-      give_up = true;  // fewer candidates than survivors
-    } else {
-      find_digit_from_top<PER, THREADS>(own, (unsigned int)p.k, sh.tot, sh.out);
-      Tbin = sh.out[0];
-      rem = sh.out[1];
-    }
-    if (!give_up) {
-      auto count_of = [&](unsigned int g) { return stage ? staged[g] : __ldcg(p.group_count + g); };
-      // A block's work is its candidates plus the bitmap rounds of its groups, so the groups are dealt out
-      // by weight: candidates + kGroupRounds for a group that has any, nothing for an empty one.
-      auto weight_of = [&](unsigned int c) { return c != 0 ? c + (unsigned int)kGroupRounds : 0u; };
-      const unsigned int per_thread = (p.ngroups + THREADS - 1) / THREADS;
-      const unsigned int g_begin = min(p.ngroups, threadIdx.x * per_thread);
-      const unsigned int g_end = min(p.ngroups, g_begin + per_thread);
-      unsigned int thread_sum = 0;
-      for (unsigned int g = g_begin; g < g_end; ++g) thread_sum += weight_of(count_of(g));
-      unsigned int all;
-      const unsigned int thread_pos = block_excl_scan(thread_sum, all, sh);  // weight before this thread's groups
-      // a group belongs to the block into whose share [w_lo, w_hi) of the weight its start falls
-      const unsigned long long w_lo = (unsigned long long)blk * all / G, w_hi = (unsigned long long)(blk + 1) * all / G;
-      unsigned int owned = 0, owned_cands = 0, earlier_cands = 0, pos = thread_pos;
-      for (unsigned int g = g_begin; g < g_end; ++g) {
-        const unsigned int c = count_of(g);
-        if (c != 0 && pos >= w_lo && pos < w_hi) {
-          ++owned;
-          owned_cands += c;
-        }
-        if (pos < w_lo) earlier_cands += c;
-        pos += weight_of(c);
-      }
-      unsigned int slot = block_excl_scan(owned, owned_all, sh);
-      const unsigned long long both = block_sum(((unsigned long long)earlier_cands << 32) | owned_cands, sh);
-      E = (unsigned int)(both & 0xFFFFFFFFull);
-      const unsigned long long cands_before = both >> 32;  // candidates of the blocks before this one
-      if (E > p.cap) {
-        // a share too large for shared memory lives in the spill area (its own stretch of it: blocks are in
-        // index order, so the candidates before this block's say where)
-        in_shared = false;
-        c_idx = p.spill_idx + cands_before;
-        c_val = p.spill_val + cands_before;
-      }
-      if (owned_all > (unsigned int)kPickGroupCap || (!in_shared && cands_before + E > p.spill_entries)) {
-        give_up = true;
-      } else {
-        pos = thread_pos;
-        for (unsigned int g = g_begin; g < g_end; ++g) {
-          const unsigned int c = count_of(g);
-          if (c != 0 && pos >= w_lo && pos < w_hi) s_groups[slot++] = g;
-          pos += weight_of(c);
-        }
-      }
-      __syncthreads();  // the list of groups is complete, and the staged counts have been read for the last time
-    }
+  for (int i = 0; i < kHeld; ++i) {
+    const unsigned int b = b_begin + i;
+    held_above[i] = b < b_end ? __ldcg(p.per_block + (size_t)PB_ABOVE * B + b) : 0u;
+    held_inbin[i] = b < b_end ? __ldcg(p.per_block + (size_t)PB_INBIN * B + b) : 0u;
   }
-  // a bin below the last holds exactly one key value when the sample kernel said so
-  // (then the bin itself decides: above it = above T, in it = equal to T)
-  const bool exact = p.ctl->exact != 0 && Tbin + 1 < (unsigned int)kFineBins;
-  {
-    // ---------------- bitmap -> indices, in index order ----------------
-    if (!give_up) {
-      const unsigned long long rounds_all = (p.n + kRoundElems - 1) / kRoundElems;
-      const unsigned int nrounds = owned_all * kGroupRounds;
-      const uint4* bitmap4 = reinterpret_cast<const uint4*>(p.bitmap);
-      unsigned int filled = 0;
-      // A thread takes `rpt` consecutive rounds per pass: one when the block's groups are few (they are then
-      // crowded with candidates, and writing out a round's indices is the long part), up to RP when the
-      // block owns many sparse groups (so that one pass, with its one block-wide scan, usually does).
-      constexpr int RP = 8;
-      const unsigned int rpt = min((unsigned int)RP, (nrounds + THREADS - 1) / THREADS);
-      for (unsigned int r0 = 0; r0 < nrounds; r0 += THREADS * rpt) {
-        uint4 m[RP];
-        unsigned long long round_id[RP];
-        unsigned int cnt = 0;
-#pragma unroll
-        for (int u = 0; u < RP; ++u) {
-          const unsigned int r = r0 + threadIdx.x * rpt + u;
-          m[u] = make_uint4(0u, 0u, 0u, 0u);
-          round_id[u] = 0;
-          if ((unsigned int)u < rpt && r < nrounds) {
-            round_id[u] = (unsigned long long)s_groups[r / kGroupRounds] * kGroupRounds + r % kGroupRounds;
-            if (round_id[u] < rounds_all) m[u] = __ldcg(bitmap4 + round_id[u]);
-          }
-        }
-#pragma unroll
-        for (int u = 0; u < RP; ++u) cnt += __popc(m[u].x) + __popc(m[u].y) + __popc(m[u].z) + __popc(m[u].w);
-        unsigned int step_total;
-        unsigned int at = filled + block_excl_scan(cnt, step_total, sh);
-#pragma unroll
-        for (int u = 0; u < RP; ++u) {
-          const uint32_t first = (uint32_t)(round_id[u] * kRoundElems);
-          const unsigned int words[4] = {m[u].x, m[u].y, m[u].z, m[u].w};
-#pragma unroll
-          for (int w = 0; w < 4; ++w) {
-            unsigned int bits = words[w];
-            while (bits != 0) {
-              const int b = __ffs(bits) - 1;
-              bits &= bits - 1;
-              if (at < E) c_idx[at] = first + w * 32 + b;
-              ++at;
-            }
-          }
-        }
-        filled += step_total;
-      }
-      if (filled != E) give_up = true;  // bitmap and counts disagree - cannot happen
-    }
-  }
-  __syncthreads();
-
-  // ---------------- values of the candidates; where each stands against the threshold's bin ----------------
-  // Each warp owns one contiguous run of the block's candidates, so that warp order and lane order are
-  // index order.  A run's counts stay in shared memory for the write phase.
-  const unsigned int per_run = ((E + NW - 1) / NW + 31) / 32 * 32;
-  const unsigned int run_lo = min(E, warp * per_run), run_hi = min(E, run_lo + per_run);
-  unsigned int n_inbin = 0;  // this warp's candidates in the threshold's bin (listed case; warp-uniform)
-  unsigned int above_run = 0;  // this warp's candidates above the bin
-  if (!give_up) {
-    bool nonfinite = false;
-    for (unsigned int j0 = threadIdx.x; j0 < E; j0 += THREADS * 4) {  // four scattered loads in flight per thread
-      uint32_t v[4];
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const unsigned int j = j0 + u * THREADS;
-        v[u] = (j < E) ? src.raw1(c_idx[j]) : 0u;  // a candidate is never a pruned element
-      }
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const unsigned int j = j0 + u * THREADS;
-        if (j < E) c_val[j] = v[u];
-        nonfinite |= (v[u] & 0x7FFFFFFFu) >= kInfKey;
-      }
-    }
-    if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
-    __syncthreads();
-    unsigned int wa = 0, wc = 0;
-    for (unsigned int j0 = run_lo; j0 < run_hi; j0 += 32) {
-      const unsigned int j = j0 + lane;
-      const bool live = j < run_hi;
-      const uint32_t bits = live ? c_val[j] : 0u;
-      const uint32_t key = bits & 0x7FFFFFFFu;
-      const unsigned int bin = (live && key >= lo) ? min((key - lo) >> shift, (unsigned int)(kFineBins - 1)) : 0u;
-      const bool above = live && key >= lo && bin > Tbin;
-      const bool inbin = live && key >= lo && bin == Tbin;
-      wa += __popc(__ballot_sync(FULL, above));
-      const unsigned int bi = __ballot_sync(FULL, inbin);
-      if (exact) {
-        wc += __popc(bi);  // in the bin = equal to T
-      } else if (bi != 0) {
-        unsigned int base = 0;
-        if (lane == 0) base = atomicAdd(&p.ctl->und_count, (unsigned int)__popc(bi));
-        base = __shfl_sync(FULL, base, 0);
-        const unsigned int at = base + __popc(bi & lt);
-        if (inbin && at < kUndCap) p.und[at] = make_uint2(bits, c_idx[j]);
-        const unsigned int mine = n_inbin + __popc(bi & lt);
-        if (inbin && mine < (unsigned int)kPickInbinCap) s_inbin[warp][mine] = j;
-        n_inbin += __popc(bi);
-      }
-    }
-    above_run = wa;
-    if (lane == 0) sh.run[warp] = ((unsigned long long)wa << 32) | wc;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-      unsigned long long block_a = 0, block_c = 0;
-      for (int w = 0; w < NW; ++w) {
-        block_a += sh.run[w] >> 32;
-        block_c += sh.run[w] & 0xFFFFFFFFull;
-      }
-      p.block_counts[blk] = (block_a << 32) | block_c;
-    }
-  }
-  if (give_up && threadIdx.x == 0) atomicOr(&p.ctl->fallback, 1u);
-  if (!grid_barrier(p.ctl, G, sh)) return;
-
-  // =============================== after the barrier ===============================
-  const unsigned int und_count = __ldcg(&p.ctl->und_count);
-  bool fallback = __ldcg(&p.ctl->fallback) != 0 || und_count > kUndCap;  // the same in every block
-  unsigned long long a_before = 0, c_before = 0, a_all = 0, c_all = 0;
-  if (!fallback) {
-    for (unsigned int b = threadIdx.x; b < G; b += THREADS) {
-      const unsigned long long w = __ldcg(p.block_counts + b);
-      a_all += w >> 32;
-      c_all += w & 0xFFFFFFFFull;
-      if (b < blk) {
-        a_before += w >> 32;
-        c_before += w & 0xFFFFFFFFull;
-      }
-    }
-    a_before = block_sum(a_before, sh);
-    c_before = block_sum(c_before, sh);
-    a_all = block_sum(a_all, sh);
-    c_all = block_sum(c_all, sh);
-  }
-
-  // ---------------- the exact threshold ----------------
-  uint32_t T = 0;               // listed candidates: the threshold key
-  unsigned long long r = 0;     // exact bins: ties (key == T) to keep, lowest index first
-  bool limited = false;         // listed candidates: ties at T survive only up to index `limit`
-  uint32_t limit = 0;
-  unsigned long long u_before = 0;  // listed candidates that survive and lie before this block's index range
-  if (!fallback && exact) {
-    r = p.k - a_all;
-    if (a_all > p.k || c_all < r) {  // cannot happen: the histogram put the k-th largest key into this bin
-      if (threadIdx.x == 0) set_status(&p.ctl->status, NSML_ERR_INTERNAL);
+  for (unsigned int i = threadIdx.x; i < min(und_all, kUndCap); i += THREADS) s_u[i] = __ldcg(p.und + i);
+  if (fallback != 0) return;
+  uint32_t T = 0, limit = 0;
+  unsigned int ties_kept = 0;
+  if (!by_bin) {
+    const unsigned int und_count = und_all;
+    if (und_count > kUndCap) {
+      if (threadIdx.x == 0) ctl->fallback = 1u;
       return;
     }
-  } else if (!fallback) {
-    // every block reads the whole list and selects the rem-th largest key in it: 12 + 12 + 7 bits
-    for (unsigned int i = threadIdx.x; i < und_count; i += THREADS) s_u[i] = __ldcg(p.und + i);
-    if (a_all + und_count < p.k || a_all >= p.k || p.k - a_all != rem) {  // cannot happen
-      if (threadIdx.x == 0) set_status(&p.ctl->status, NSML_ERR_INTERNAL);
+    if (und_count < rem || rem == 0) {  // cannot happen: the bin holds at least rem keys
+      if (threadIdx.x == 0) set_status(&ctl->status, NSML_ERR_INTERNAL);
       return;
     }
-    __syncthreads();  // the list is in place
+    // T is the rem-th largest key of the listed candidates; under (key descending, index ascending) its
+    // entry has rank rem - 1.
+    __syncthreads();  // the list is in shared memory
     if (und_count <= (unsigned int)kPickRankCap) {
-      // short list: every entry's rank under (key descending, index ascending) by counting; the entry of
-      // rank rem - 1 is the last survivor: its key is T, its index the limit for ties at T
-      for (unsigned int i = warp; i < und_count; i += NW) {  // a warp per entry, the lanes share the comparisons
-        const uint32_t key = s_u[i].x & 0x7FFFFFFFu, idx = s_u[i].y;
+      // short list: every entry's rank by counting, a warp per entry, the lanes share the comparisons
+      for (unsigned int i = warp; i < und_count; i += NW) {
+        const uint2 me = s_u[i];
+        const uint32_t key = me.x & 0x7FFFFFFFu;
         unsigned int before = 0;
         for (unsigned int q = lane; q < und_count; q += 32) {
           const uint2 e = s_u[q];
           const uint32_t kq = e.x & 0x7FFFFFFFu;
-          before += kq > key || (kq == key && e.y < idx);
+          before += kq > key || (kq == key && e.y < me.y);
         }
         before = __reduce_add_sync(FULL, before);
         if (lane == 0 && before == rem - 1) {  // ranks are distinct: exactly one entry
           s_T = key;
-          s_limit = idx;
+          s_limit = me.y;
         }
       }
       __syncthreads();
       T = s_T;
       limit = s_limit;
-      limited = true;
     } else {
+      // long list: radix select, 12 + 12 + 7 bits, then the rank by index among the ties at T
       unsigned int prefix = 0, left = rem;
 #pragma unroll
       for (int level = 0; level < 3; ++level) {
         const int nb = 1 << digit_bits(level);
-        __syncthreads();  // the list is in place; the previous level's bins have been read
+        __syncthreads();  // the previous level's bins have been read
         for (int b = threadIdx.x; b < nb; b += THREADS) sh.hist[b] = 0;
         __syncthreads();
         for (unsigned int i = threadIdx.x; i < und_count; i += THREADS) {
@@ -358,121 +291,190 @@ k_pick(BucketSrc<DTYPE> src, FinalizeParams p) {
         left = sh.out[1];
       }
       T = prefix;
-      const unsigned int keep_ties = left;          // ties at T that survive, lowest index first
+      const unsigned int keep = left;                // ties at T that survive, lowest index first
       const unsigned int ties = sh.hist[T & 0x7Fu];  // keys equal to T in the list
-      limited = keep_ties < ties;
-      if (limited && ties > (unsigned int)kPickTieCap) {
-        fallback = true;  // the same decision in every block: they all hold the same list
-      } else if (limited) {
-        // the keep_ties-th smallest index among the ties: the one with keep_ties - 1 tied indices below it
+      if (keep >= ties) {
+        limit = 0xFFFFFFFFu;  // every tie survives
+      } else if (ties > (unsigned int)kPickTieCap) {
+        if (threadIdx.x == 0) ctl->fallback = 1u;
+        return;
+      } else {
+        // the keep-th smallest index among the ties: the one with keep - 1 tied indices below it
         for (unsigned int i = threadIdx.x; i < und_count; i += THREADS) {
-          if ((s_u[i].x & 0x7FFFFFFFu) != T) continue;
-          const uint32_t mine = s_u[i].y;
+          const uint2 me = s_u[i];
+          if ((me.x & 0x7FFFFFFFu) != T) continue;
           unsigned int below = 0;
-          for (unsigned int q = 0; q < und_count; ++q) below += (s_u[q].x & 0x7FFFFFFFu) == T && s_u[q].y < mine;
-          if (below == keep_ties - 1) s_limit = mine;  // indices are distinct: exactly one thread
+          for (unsigned int q = 0; q < und_count; ++q) {
+            const uint2 e = s_u[q];
+            below += (e.x & 0x7FFFFFFFu) == T && e.y < me.y;
+          }
+          if (below == keep - 1) s_limit = me.y;  // indices are distinct: exactly one thread
         }
         __syncthreads();
         limit = s_limit;
       }
     }
-    if (!fallback) {
-      const uint32_t my_first = E != 0 ? c_idx[0] : 0xFFFFFFFFu;
-      unsigned int before = 0;
-      for (unsigned int i = threadIdx.x; i < und_count; i += THREADS) {
-        const uint32_t key = s_u[i].x & 0x7FFFFFFFu;
-        const bool survives = key > T || (key == T && (!limited || s_u[i].y <= limit));
-        before += survives && s_u[i].y < my_first;
-      }
-      u_before = block_sum((unsigned long long)before, sh);
+    // listed survivors per block
+    unsigned int* listed = p.per_block + (size_t)PB_LISTED * B;
+    for (unsigned int b = threadIdx.x; b < B; b += THREADS) listed[b] = 0;
+    __syncthreads();
+    for (unsigned int i = threadIdx.x; i < und_count; i += THREADS) {
+      const uint2 e = s_u[i];
+      const uint32_t key = e.x & 0x7FFFFFFFu;
+      const unsigned int owner = e.y / (unsigned int)kPickElems;
+      if ((key > T || (key == T && e.y <= limit)) && owner < B) atomicAdd(listed + owner, 1u);
     }
-  }
-
-  if (fallback) {
-    // select over the bucket itself; the shared memory of the list stage becomes its value cache
-    dense_select<DTYPE, THREADS>(src, p, sh, s_dyn, 1u);
-    return;
-  }
-
-  // ---------------- write the survivors in index order ----------------
-  if (blk == 0 && threadIdx.x == 0) write_header(p);
-  auto survives_listed = [&](uint32_t key, uint32_t idx) {  // a candidate in the threshold's bin, listed case
-    return key > T || (key == T && (!limited || idx <= limit));
-  };
-  if (!exact) {
-    // survivors per run, now that T is known: those above the bin plus the in-bin ones that pass
-    unsigned int wa = above_run;
-    if (n_inbin <= (unsigned int)kPickInbinCap) {
-      bool s = false;
-      if ((unsigned int)lane < n_inbin) {
-        const unsigned int j = s_inbin[warp][lane];
-        s = survives_listed(c_val[j] & 0x7FFFFFFFu, c_idx[j]);
-      }
-      wa += __popc(__ballot_sync(FULL, s));
-    } else {
-      wa = 0;
-      for (unsigned int j0 = run_lo; j0 < run_hi; j0 += 32) {
-        const unsigned int j = j0 + lane;
-        bool s = false;
-        if (j < run_hi) {
-          const uint32_t key = c_val[j] & 0x7FFFFFFFu;
-          const unsigned int bin = key >= lo ? min((key - lo) >> shift, (unsigned int)(kFineBins - 1)) : 0u;
-          s = key >= lo && (bin > Tbin || (bin == Tbin && survives_listed(key, c_idx[j])));
-        }
-        wa += __popc(__ballot_sync(FULL, s));
-      }
-    }
-    __syncthreads();  // sh.run of the first phase has been read by thread 0
-    if (lane == 0) sh.run[warp] = (unsigned long long)wa << 32;
     __syncthreads();
   }
-  unsigned long long a_here = a_before + u_before, c_here = c_before, block_a = 0, block_c = 0;
-  for (int w = 0; w < NW; ++w) {
-    const unsigned long long rw = sh.run[w];
-    if (w < warp) {
-      a_here += rw >> 32;
-      c_here += rw & 0xFFFFFFFFull;
-    }
-    block_a += rw >> 32;
-    block_c += rw & 0xFFFFFFFFull;
+  // Exclusive prefix over the blocks of (sure survivors [+ listed survivors], in-bin entries): every thread
+  // takes a contiguous range of blocks, sums it (independent loads), the sums are scanned over the block,
+  // and a second walk writes the prefixes.
+  auto value_of = [&](unsigned int b) {  // blocks beyond the held ones
+    unsigned int s = __ldcg(p.per_block + (size_t)PB_ABOVE * B + b);
+    if (!by_bin) s += __ldcg(p.per_block + (size_t)PB_LISTED * B + b);
+    return ((unsigned long long)s << 32) | __ldcg(p.per_block + (size_t)PB_INBIN * B + b);
+  };
+  unsigned long long held[kHeld];
+#pragma unroll
+  for (int i = 0; i < kHeld; ++i) {
+    const unsigned int b = b_begin + i;
+    unsigned int s = held_above[i];
+    if (!by_bin && b < b_end) s += __ldcg(p.per_block + (size_t)PB_LISTED * B + b);  // written by this block, above
+    held[i] = ((unsigned long long)s << 32) | held_inbin[i];
   }
-  // payload positions [p0, p1) of this block's survivors
-  const unsigned long long p0 = a_before + u_before + min(c_before, r);
-  const unsigned long long p1 = a_before + u_before + block_a + min(c_before + block_c, r);
-  if (blk == G - 1 && p1 != p.k) {  // cannot happen
-    if (threadIdx.x == 0) set_status(&p.ctl->status, NSML_ERR_INTERNAL);
+  unsigned long long mine = 0;
+#pragma unroll
+  for (int i = 0; i < kHeld; ++i) mine += held[i];
+  for (unsigned int b = b_begin + kHeld; b < b_end; ++b) mine += value_of(b);
+  unsigned long long incl = mine;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const unsigned long long up = __shfl_up_sync(FULL, incl, o);
+    if (lane >= o) incl += up;
+  }
+  __syncthreads();
+  if (lane == 31) sh.red[warp] = incl;
+  __syncthreads();
+  unsigned long long run = incl - mine, carry = 0;
+#pragma unroll
+  for (int w = 0; w < NW; ++w) {
+    const unsigned long long c = sh.red[w];
+    if (w < warp) run += c;
+    carry += c;
+  }
+#pragma unroll
+  for (int i = 0; i < kHeld; ++i) {
+    const unsigned int b = b_begin + i;
+    if (b < b_end) {
+      p.per_block[PB_BEFORE * B + b] = (unsigned int)(run >> 32);
+      p.per_block[PB_INBIN_BEFORE * B + b] = (unsigned int)(run & 0xFFFFFFFFull);
+    }
+    run += held[i];
+  }
+  for (unsigned int b = b_begin + kHeld; b < b_end; ++b) {
+    p.per_block[PB_BEFORE * B + b] = (unsigned int)(run >> 32);
+    p.per_block[PB_INBIN_BEFORE * B + b] = (unsigned int)(run & 0xFFFFFFFFull);
+    run += value_of(b);
+  }
+  const unsigned long long sure = carry >> 32, in_all = carry & 0xFFFFFFFFull;
+  if (by_bin) {
+    // every in-bin key equals T: the first k - sure of them in index order survive
+    if (sure > p.k || in_all < p.k - sure) {  // cannot happen: the histogram put the k-th largest key into this bin
+      if (threadIdx.x == 0) set_status(&ctl->status, NSML_ERR_INTERNAL);
+      return;
+    }
+    ties_kept = (unsigned int)(p.k - sure);
+  } else if (sure != p.k) {  // cannot happen
+    if (threadIdx.x == 0) set_status(&ctl->status, NSML_ERR_INTERNAL);
     return;
   }
+  if (threadIdx.x == 0) {
+    ctl->T = T;
+    ctl->limit = limit;
+    ctl->ties_kept = ties_kept;
+  }
+}
+
+__global__ void __launch_bounds__(kPickThreads)
+k_pick_b(FinalizeParams p) {
+  constexpr int THREADS = kPickThreads;
+  constexpr int NW = THREADS / 32;
+  struct Scratch {
+    float qmax[NW];  // the quantisation's scratch
+  };
+  __shared__ Scratch sh;
+  __shared__ unsigned int s_warp[NW];
+  __shared__ unsigned int s_q[kPickQCap];
+  __shared__ unsigned int s_nq;
+  const unsigned int blk = blockIdx.x, B = p.pick_blocks;
+  const Ctl* ctl = p.ctl;
+  // everything this block reads first was written by the kernels before it: one round of loads
+  const PickRound round = pick_round(p);
+  const unsigned int fallback = __ldcg(&ctl->fallback);
+  const int status = __ldcg(&ctl->status);
+  const unsigned int lo = max(__ldcg(&ctl->lo), 1u), shift = __ldcg(&ctl->shift), Tbin = __ldcg(&ctl->Tbin);
+  const bool by_bin = __ldcg(&ctl->by_bin) != 0;
+  const uint32_t T = __ldcg(&ctl->T), limit = __ldcg(&ctl->limit);
+  const unsigned long long r = __ldcg(&ctl->ties_kept);  // by-bin case: ties (key == T) to keep, lowest index first
+  const unsigned long long a_before = __ldcg(p.per_block + (size_t)PB_BEFORE * B + blk);
+  const unsigned long long c_before_all = __ldcg(p.per_block + (size_t)PB_INBIN_BEFORE * B + blk);
+  if (fallback != 0 || status == NSML_ERR_INTERNAL) return;
+  const unsigned long long c_before = by_bin ? c_before_all : 0ull;
+  if (blk == 0 && threadIdx.x == 0) write_header(p);
+  const uint32_t* my_val = p.stash_val + (size_t)blk * kStashPerBlock;
   uint32_t* out_idx = reinterpret_cast<uint32_t*>(p.payload + p.P.idx_off);
-  for (unsigned int j0 = run_lo; j0 < run_hi; j0 += 32) {
-    const unsigned int j = j0 + lane;
-    const bool live = j < run_hi;
-    const uint32_t bits = live ? c_val[j] : 0u;
-    const uint32_t idx = live ? c_idx[j] : 0u;
-    const uint32_t key = bits & 0x7FFFFFFFu;
-    const unsigned int bin = (live && key >= lo) ? min((key - lo) >> shift, (unsigned int)(kFineBins - 1)) : 0u;
-    const bool cand = live && key >= lo;
-    bool a, c;
-    if (exact) {
+
+  unsigned int E;
+  const unsigned int first = pick_scan(round.count(), E, s_warp);  // this round's first candidate in the stash
+  // a: survives whatever the ties' ranks; c: a tie at T in the by-bin case (survives while the budget lasts)
+  auto classify = [&](uint32_t v, uint32_t idx, bool& a, bool& c) {
+    const uint32_t key = v & 0x7FFFFFFFu;
+    const bool cand = key >= lo;
+    const unsigned int bin = cand ? fine_bin(key, lo, shift) : 0u;
+    if (by_bin) {
       a = cand && bin > Tbin;
       c = cand && bin == Tbin;
     } else {
-      a = cand && (bin > Tbin || (bin == Tbin && survives_listed(key, idx)));
+      a = cand && (bin > Tbin || (bin == Tbin && (key > T || (key == T && idx <= limit))));
       c = false;
     }
-    const unsigned int ba = __ballot_sync(FULL, a), bc = __ballot_sync(FULL, c);
-    const unsigned long long a_mine = a_here + __popc(ba & lt), c_mine = c_here + __popc(bc & lt);
+  };
+  auto from_stash = [&](unsigned int j, uint32_t) {
+    return first + j < (unsigned int)kStashPerBlock ? __ldcg(my_val + first + j) : 0u;
+  };
+  unsigned int my_a = 0, my_c = 0;  // at most 128 each
+  for_round_candidates(round, from_stash, [&](uint32_t v, uint32_t idx) {
+    bool a, c;
+    classify(v, idx, a, c);
+    my_a += a;
+    my_c += c;
+  });
+  unsigned int packed_all;
+  const unsigned int packed_before = pick_scan(my_a | (my_c << 16), packed_all, s_warp);  // at most kPickElems each: 16 bits do
+  unsigned long long a_mine = a_before + (packed_before & 0xFFFFu), c_mine = c_before + (packed_before >> 16);
+  bool bad = false;
+  for_round_candidates(round, from_stash, [&](uint32_t v, uint32_t idx) {
+    bool a, c;
+    classify(v, idx, a, c);
     if (a || (c && c_mine < r)) {
       const unsigned long long pos = a_mine + min(c_mine, r);
-      out_idx[pos] = idx;
-      if (p.bits == NSML_BITS_FP32) reinterpret_cast<uint32_t*>(p.payload + p.P.val_off)[pos] = bits;
-      else if (p.bits == NSML_BITS_FP16) reinterpret_cast<uint16_t*>(p.payload + p.P.val_off)[pos] = encode_f16(__uint_as_float(bits));
-      else p.raw_val[pos] = __uint_as_float(bits);
+      if (pos < p.k) {
+        out_idx[pos] = idx;
+        if (p.bits == NSML_BITS_FP32) reinterpret_cast<uint32_t*>(p.payload + p.P.val_off)[pos] = v;
+        else if (p.bits == NSML_BITS_FP16) reinterpret_cast<uint16_t*>(p.payload + p.P.val_off)[pos] = encode_f16(__uint_as_float(v));
+        else p.raw_val[pos] = __uint_as_float(v);
+      } else {
+        bad = true;
+      }
     }
-    a_here += __popc(ba);
-    c_here += __popc(bc);
-  }
-  if (p.bits != NSML_BITS_INT8 || p1 == p0) return;  // block-uniform
+    a_mine += a;
+    c_mine += c;
+  });
+  if (bad) set_status(&p.ctl->status, NSML_ERR_INTERNAL);
+  // payload positions [p0, p1) of this block's survivors
+  const unsigned long long p0 = a_before + min(c_before, r);
+  const unsigned long long p1 = a_before + (packed_all & 0xFFFFu) + min(c_before + (packed_all >> 16), r);
+  if (p.bits != NSML_BITS_INT8 || p1 <= p0 || p1 > p.k) return;  // block-uniform
 
   // ---------------- int8: whoever completes a block of 1024 payload entries quantises it ----------------
   __threadfence();  // this thread's raw values are visible device-wide before the block reports them
@@ -483,16 +485,15 @@ k_pick(BucketSrc<DTYPE> src, FinalizeParams p) {
     const unsigned long long q_lo = q * NSML_QBLOCK, q_hi = min(q_lo + NSML_QBLOCK, p.k);
     const unsigned int part = (unsigned int)(min(p1, q_hi) - max(p0, q_lo));
     const unsigned int seen = atomicAdd(p.qcount + q, part);
-    if (seen + part == (unsigned int)(q_hi - q_lo)) s_q[atomicAdd(&s_nq, 1u)] = (unsigned int)q;  // at most kPickQCap: cap / 1024 + 2
+    if (seen + part == (unsigned int)(q_hi - q_lo)) {
+      const unsigned int slot = atomicAdd(&s_nq, 1u);
+      if (slot < (unsigned int)kPickQCap) s_q[slot] = (unsigned int)q;
+    }
   }
   __syncthreads();
   __threadfence();  // the other blocks' raw values, reported before ours, are visible to the loads below
-  const unsigned int nq = s_nq;
-  constexpr int kQGroups = THREADS / 256;
-  for (unsigned int i0 = 0; i0 < nq; i0 += kQGroups) {
-    const unsigned int i = i0 + (threadIdx.x >> 8);
-    quantize_block(p, sh, i < nq ? s_q[i] : 0ull, i < nq);
-  }
+  const unsigned int nq = min(s_nq, (unsigned int)kPickQCap);
+  for (unsigned int i = 0; i < nq; ++i) quantize_block(p, sh, s_q[i], true);  // 256 threads: one group
 }
 
 }  // namespace nsml
