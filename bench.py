@@ -44,7 +44,8 @@ SWEEP = [(r, b) for r in (0.5, 0.1, 0.01, 0.001) for b in (8, 16)]
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
 # profiles/compress_kernels_gpt2_25M_ncu_full.md: 25M-element fp32 buckets, ratio 0.01, int8, W = 4.  Only valid
 # for that workload and for the kernels as they were when the capture was taken.
-NCU_TRAFFIC_25M = {}
+NCU_TRAFFIC_25M = {"k_sample": 1.06e6, "k_compact_bucket": 103.6e6, "k_gather": 4.5e6, "k_finalize": 3.7e6,
+                   "k_partition": 3.9e6, "k_merge": 53.0e6}
 
 
 def measured_peak_gbs():
@@ -180,15 +181,12 @@ class Workload:
             self.account(acc, "k_clear", 256 + 4 * 4 * 4096)
             self.account(acc, "k_finalize_dense", esize * n + 8 * k + 4 * k + vb * k + s)
             return
-        self.account(acc, "k_sample", esize * 32768)
-        # bucket pass: the bucket read once, one bit per element written
-        self.account(acc, "k_mark", esize * n + n // 8)
-        # list stage: the bitmap read, the survivors' values read again from the bucket and kept with their
-        # indices (8 bytes each, written and read back), then index + value written to the payload
-        self.account(acc, "k_pick_a", n // 8 + esize * k + 4 * k)
-        self.account(acc, "k_pick_settle", 24 * ((n + 8191) // 8192))
-        self.account(acc, "k_pick_b", n // 8 + 4 * k + 4 * k + vb * k + s)
-        self.account(acc, "k_finalize_dense", 0)  # enqueued as the fallback; leaves at once
+        self.account(acc, "k_sample", 4 * 8192)
+        self.account(acc, "k_compact_bucket", esize * n + 8 * k)
+        # gather: candidates (index + value) read from the segmented list and written contiguously
+        self.account(acc, "k_gather", 16 * k)
+        # list stage: candidate values read once per phase (4 x 4k keys), indices once, survivors written and re-read
+        self.account(acc, "k_finalize", 16 * k + 4 * k + 8 * k + 4 * k + vb * k + s)
 
     def merge_bytes(self, acc, n, ks_bits, zero_first=True):
         total = 4 * n if zero_first else 0
@@ -634,7 +632,7 @@ class Alg2Workload(Workload):
                     self.account(acc, "k_feedback_subtract", 13 * k)
                     self.compress_bytes(acc, n, 4, self.RATIO, self.BITS)
                     # the bucket pass also reads the mask and the residual and writes gradient + residual back
-                    self.account(acc, "k_mark", n // 8 + 8 * n)
+                    self.account(acc, "k_compact_bucket", n // 8 + 8 * n)
                     self.merge_bytes(acc, n, [(k, self.BITS)])
 
             yield ((i * self.STATE + b) % self.GRADS, b), nsml.nsml_payload_bytes(n, self.RATIO, self.BITS), enqueue

@@ -207,13 +207,11 @@ int nsml_compress(const void* grad, int64_t n, int grad_dtype, double ratio, int
 /* Which of its two internal strategies nsml_compress takes for (n, ratio) on
  * the current device.  Both give the same payload; this is information for
  * byte accounting (the paper prescribes no strategy).
- *   NSML_STRATEGY_LIST   a stratified sample brackets the threshold, one
- *                        streaming pass marks the candidates above the lower
- *                        bound (one bit each) and counts them by key, the
- *                        exact threshold is found among the marked elements
+ *   NSML_STRATEGY_LIST   a stratified sample bounds the threshold from below,
+ *                        one streaming pass keeps the candidates above the
+ *                        bound, an exact radix select runs on that list
  *   NSML_STRATEGY_DENSE  the radix select runs over the bucket itself (high
- *                        kept fractions, buckets too small to sample, and the
- *                        fallback of the list strategy when its sample misled)
+ *                        kept fractions, and buckets too small to sample)
  * Returns the strategy, or NSML_ERR_ARG / NSML_ERR_CUDA. */
 #define NSML_STRATEGY_LIST 0
 #define NSML_STRATEGY_DENSE 1

@@ -17,6 +17,9 @@
 
 namespace nsml {
 
+constexpr int kStreamLoads = 4;  // 16-byte loads a thread keeps in flight
+constexpr int kStreamTile = kCta * 4 * kStreamLoads;  // elements a block takes per step
+
 // ------------------------------------------------------------------------
 // Step 1: sum of squares in float64.  Every square is exact in float64 (a
 // float32 has 24 significant bits), the adds follow a fixed order for a given

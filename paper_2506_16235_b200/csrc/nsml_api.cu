@@ -10,23 +10,22 @@
 #include "nsml_adaptive.cuh"
 #include "nsml_codec.cuh"
 #include "nsml_common.cuh"
-#include "nsml_dense.cuh"
+#include "nsml_compact.cuh"
 #include "nsml_finalize.cuh"
-#include "nsml_mark.cuh"
-#include "nsml_pick.cuh"
+#include "nsml_dense.cuh"
 #include "nsml_select.cuh"
 
 namespace nsml {
 
 enum KernelId {
-  K_SAMPLE = 0, K_MARK, K_PICK_A, K_PARTITION, K_MERGE, K_CLEAR, K_FINALIZE_DENSE,
-  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_PRUNE_WRITE_RANKED, K_PICK_B, K_PICK_SETTLE, K_COUNT
+  K_SAMPLE = 0, K_COMPACT_BUCKET, K_FINALIZE, K_PARTITION, K_MERGE, K_CLEAR, K_FINALIZE_DENSE,
+  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_PRUNE_WRITE_RANKED, K_GATHER, K_COUNT
 };
 
-static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_mark", "k_pick_a", "k_partition", "k_merge",
+static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_compact_bucket", "k_finalize", "k_partition", "k_merge",
                                                   "k_clear", "k_finalize_dense", "k_sumsq", "k_feedback_add",
                                                   "k_feedback_subtract", "k_prune_hist", "k_prune_ties", "k_prune_write",
-                                                  "k_prune_write_ranked", "k_pick_b", "k_pick_settle"};
+                                                  "k_prune_write_ranked", "k_gather"};
 
 static std::atomic<int64_t> g_launches{0};
 
@@ -80,8 +79,9 @@ struct LaunchScope {  // brackets one kernel launch
 struct DeviceInfo {
   bool ready = false;
   int sms = 0;
-  int mark = 0, mark_feedback = 0, finalize_small = 0, finalize_large = 0, merge = 0;  // resident blocks per SM
+  int compact_bucket = 0, compact_feedback = 0, finalize_small = 0, finalize_large = 0, merge = 0;  // resident blocks per SM
   int sumsq = 0, feedback_add = 0, prune_hist = 0, prune_write = 0, prune_write_ranked = 0;  // the same, streaming kernels
+  bool finalize_cluster = false;  // the one-cluster shape of the list stage fits an SM
 };
 static DeviceInfo g_dev[64];
 static std::mutex g_dev_mutex;
@@ -94,21 +94,28 @@ static int device_info(const DeviceInfo** out) {
   if (!d.ready) {
     if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return NSML_ERR_CUDA;
     cudaError_t e = cudaSuccess;
-    auto prepare = [&](auto kernel, int threads, size_t smem, int* resident) {
-      if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_bucket, k_compact_bucket<NSML_F32, false>, kCta, 0);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_compact_bucket<NSML_F32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCompactFeedbackSmem);
+    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_compact_bucket<NSML_BF16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCompactFeedbackSmem);
+    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_feedback, k_compact_bucket<NSML_F32, true>, kCta, kCompactFeedbackSmem);
+    auto prepare = [&](auto kernel, int threads, int cache, int* resident) {
+      if (e == cudaSuccess) e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)finalize_dyn_smem(cache));
       int r = 0;
-      if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, kernel, threads, smem);
+      if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, kernel, threads, finalize_dyn_smem(cache));
       if (*resident == 0 || r < *resident) *resident = r;
     };
-    prepare(k_finalize_dense<NSML_F32, kFinSmallThreads>, kFinSmallThreads, finalize_dyn_smem(kFinSmallCache), &d.finalize_small);
-    prepare(k_finalize_dense<NSML_BF16, kFinSmallThreads>, kFinSmallThreads, finalize_dyn_smem(kFinSmallCache), &d.finalize_small);
-    prepare(k_finalize_dense<NSML_F32, kFinLargeThreads>, kFinLargeThreads, finalize_dyn_smem(kFinDenseLargeCache), &d.finalize_large);
-    prepare(k_finalize_dense<NSML_BF16, kFinLargeThreads>, kFinLargeThreads, finalize_dyn_smem(kFinDenseLargeCache), &d.finalize_large);
-    int pick = 0;
-    if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&pick, k_pick_a<NSML_F32>, kPickThreads, 0);
-    int sample = 0;
-    prepare(k_sample<NSML_F32>, kSampleThreads, kSampleSmem, &sample);
-    prepare(k_sample<NSML_BF16>, kSampleThreads, kSampleSmem, &sample);
+    prepare(k_finalize<NSML_F32, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
+    prepare(k_finalize<NSML_BF16, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
+    prepare(k_finalize_dense<NSML_F32, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
+    prepare(k_finalize_dense<NSML_BF16, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache, &d.finalize_small);
+    int cluster_shape = 0;
+    prepare(k_finalize<NSML_F32, kFinClusterThreads, kFinClusterCache, true>, kFinClusterThreads, kFinClusterCache, &cluster_shape);
+    prepare(k_finalize<NSML_BF16, kFinClusterThreads, kFinClusterCache, true>, kFinClusterThreads, kFinClusterCache, &cluster_shape);
+    d.finalize_cluster = cluster_shape >= 1;
+    prepare(k_finalize<NSML_F32, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache, &d.finalize_large);
+    prepare(k_finalize<NSML_BF16, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache, &d.finalize_large);
+    prepare(k_finalize_dense<NSML_F32, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache, &d.finalize_large);
+    prepare(k_finalize_dense<NSML_BF16, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache, &d.finalize_large);
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.merge, k_merge, kCta, 0);
     // The streaming kernels run as one wave of resident blocks (a second, partial wave would read
     // with a fraction of the SMs' loads in flight).
@@ -117,10 +124,6 @@ static int device_info(const DeviceInfo** out) {
       if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, kernel, kCta, 0);
       if (*out == 0 || r < *out) *out = r;
     };
-    resident(k_mark<NSML_F32, false>, &d.mark);
-    resident(k_mark<NSML_BF16, false>, &d.mark);
-    resident(k_mark<NSML_F32, true>, &d.mark_feedback);
-    resident(k_mark<NSML_BF16, true>, &d.mark_feedback);
     resident(k_sumsq<NSML_F32>, &d.sumsq);
     resident(k_sumsq<NSML_BF16>, &d.sumsq);
     resident(k_feedback_add<NSML_F32>, &d.feedback_add);
@@ -134,7 +137,7 @@ static int device_info(const DeviceInfo** out) {
     if (e == cudaSuccess && (d.sumsq < 1 || d.feedback_add < 1 || d.prune_hist < 1 || d.prune_write < 1 || d.prune_write_ranked < 1)) e = cudaErrorUnknown;
     int coop = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    if (e != cudaSuccess || d.mark < 1 || d.mark_feedback < 1 || d.finalize_small < 1 || d.finalize_large < 1 || pick < 1 || sample < 1 || d.merge < 1 || !coop) {
+    if (e != cudaSuccess || d.compact_bucket < 1 || d.compact_feedback < 1 || d.finalize_small < 1 || d.finalize_large < 1 || d.merge < 1 || !coop) {
       cudaGetLastError();
       return NSML_ERR_CUDA;
     }
@@ -163,37 +166,35 @@ static int64_t k_of(int64_t n, double ratio) {
   return k;
 }
 
-// Ranks (from the top, 1-based) of the two sample keys that bracket the threshold: the expected rank of the
-// k-th largest among kSamples draws plus and minus six standard deviations (the upper one is at least the
-// largest sample key).  lo == 0: do not sample (small bucket, or nearly everything is kept).
-struct SampleRanks {
-  unsigned int lo, hi;
-};
-static SampleRanks sample_ranks(int64_t n, int64_t k) {
-  SampleRanks r = {0u, 0u};
-  if (n < 2 * (int64_t)kSamples) return r;
+// Rank (from the top, 1-based) of the sample key that becomes the bracket's
+// lower bound: the expected rank of the k-th largest among kSamples draws plus
+// six standard deviations.  0 = do not sample (small bucket, or nearly
+// everything is kept): the bracket then starts at key 0.
+static unsigned int sample_rank(int64_t n, int64_t k) {
+  if (n < 2 * (int64_t)kSamples) return 0;
   const double p = (double)k / (double)n;
-  const double mean = kSamples * p, six = 6.0 * std::sqrt(kSamples * p * (1.0 - p));
-  const double j = std::ceil(mean + six) + 1.0;
-  if (j >= (double)kSamples) return r;
-  r.lo = (unsigned int)j;
-  const double h = std::floor(mean - six);
-  r.hi = h >= 1.0 ? (unsigned int)h : 1u;  // at least the largest sample key
-  return r;
+  const double j = std::ceil(kSamples * p + 6.0 * std::sqrt(kSamples * p * (1.0 - p))) + 1.0;
+  if (j >= (double)kSamples) return 0;
+  return (unsigned int)j;
 }
 
-// Kept fraction from which the select runs over the bucket itself.
-constexpr double kDenseRatio = 0.25;
+// Kept fractions from which the dense mode of the finalize kernel is used: for any bucket, and for a bucket
+// that fits the shared-memory caches of one co-resident grid.
+constexpr double kDenseRatioAny = 0.25;
+constexpr double kDenseRatioOnChip = 0.25;
 
 static unsigned long long finalize_large_blocks(const DeviceInfo& dev) {
   return (unsigned long long)dev.sms * (dev.finalize_large < 2 ? dev.finalize_large : 2);
 }
 
-// Dense strategy: the cooperative kernel selects over the bucket itself, with no sample and no bucket pass.
-// Taken when the bucket cannot be sampled and when a large fraction is kept.
-static bool use_dense(int64_t n, int64_t k, const DeviceInfo&) {
+// Dense mode: the finalize kernel selects over the bucket itself, with no sample and no bucket pass.
+// Taken when the bucket cannot be sampled, when the candidate list (8 bytes per entry) would be about
+// as large as the bucket, and for moderate kept fractions when the whole bucket fits the shared-memory
+// caches of one co-resident grid (it is then read from memory once).
+static bool use_dense(int64_t n, int64_t k, const DeviceInfo& dev) {
   const double p_keep = (double)k / (double)n;
-  return sample_ranks(n, k).lo == 0 || p_keep >= kDenseRatio;
+  const bool fits_on_chip = (unsigned long long)n <= finalize_large_blocks(dev) * (unsigned long long)kFinDenseLargeCache;
+  return sample_rank(n, k) == 0 || p_keep >= kDenseRatioAny || (fits_on_chip && p_keep >= kDenseRatioOnChip);
 }
 
 // DTYPE: element type of `grad` (what the sample and the bucket pass read).  FDTYPE: element type of the
@@ -204,9 +205,68 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
                            unsigned char* ws, unsigned char* payload, const CompressLayout& L, const PayloadLayout& P,
                            const DeviceInfo& dev, cudaStream_t st, bool keep_status = false) {
   Ctl* ctl = reinterpret_cast<Ctl*>(ws);
+  uint32_t* seg_idx = reinterpret_cast<uint32_t*>(ws + L.seg_idx);
+  uint32_t* seg_val = reinterpret_cast<uint32_t*>(ws + L.seg_val);
+  unsigned short* seg_count = reinterpret_cast<unsigned short*>(ws + L.seg_count);
   const unsigned long long nseg = ((unsigned long long)n + kSegElems - 1) / kSegElems;
   BucketSrc<DTYPE> src{grad, mask};
   BucketSrc<FDTYPE> fsrc{residual != nullptr ? static_cast<const void*>(residual) : grad, mask};
+  const double p_keep = (double)k / (double)n;
+  const unsigned long long large_cap_blocks = finalize_large_blocks(dev);
+  const bool dense = use_dense(n, k, dev);
+  unsigned int fgrid;
+  bool small_shape;
+  bool cluster_shape = false;
+  if (dense) {
+    small_shape = (unsigned long long)n <= (unsigned long long)dev.sms * kFinSmallCache;
+    unsigned long long cap = small_shape ? (unsigned long long)dev.sms : large_cap_blocks;
+    if (cap > (unsigned long long)kMaxFinalizeBlocks) cap = kMaxFinalizeBlocks;
+    unsigned long long want = (unsigned long long)n / 4096 + 1;  // at least about 4096 elements per block
+    if (want > nseg) want = nseg;
+    fgrid = (unsigned int)(want < cap ? want : cap);
+    LaunchScope scope(K_CLEAR, st);
+    k_clear<<<4, kCta, 0, st>>>(reinterpret_cast<uint4*>(ws), (unsigned int)(L.group_count / 16), keep_status ? 1 : 0);
+  } else {
+    {
+      LaunchScope scope(K_SAMPLE, st);  // one cluster of kSampleBlocks blocks
+      k_sample<DTYPE><<<kSampleBlocks, kSampleThreads, 0, st>>>(src, residual, (unsigned long long)n, sample_rank(n, k), ctl,
+                                                                reinterpret_cast<uint4*>(ws),
+                                                                (unsigned int)(L.zero_bytes / 16), keep_status ? 1 : 0);
+    }
+    {
+      // bucket pass: a block takes 8 segments per step; at most 4 resident blocks per SM
+      LaunchScope scope(K_COMPACT_BUCKET, st);
+      const int resident = residual != nullptr ? dev.compact_feedback : dev.compact_bucket;
+      const int per_sm = resident < 4 ? resident : 4;
+      const unsigned int grid = grid_for(nseg, kCta / 32, dev.sms * per_sm);
+      unsigned int* group_count = reinterpret_cast<unsigned int*>(ws + L.group_count);
+      if (residual != nullptr)
+        k_compact_bucket<DTYPE, true><<<grid, kCta, kCompactFeedbackSmem, st>>>(src, residual, (unsigned long long)n, ctl, seg_idx,
+                                                                                seg_val, seg_count, group_count);
+      else
+        k_compact_bucket<DTYPE, false><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, ctl, seg_idx, seg_val,
+                                                              seg_count, group_count);
+    }
+    // list stage: cooperative, every block co-resident.  The small shape when a block's share of the
+    // expected candidates (k plus the sampling margin) fits its shared-memory cache.
+    fgrid = (unsigned int)dev.sms;
+    if ((unsigned long long)fgrid > nseg) fgrid = (unsigned int)nseg;
+    if (fgrid > (unsigned int)kMaxFinalizeBlocks) fgrid = kMaxFinalizeBlocks;
+    const double expected = (double)n * (p_keep + 6.0 * std::sqrt(p_keep * (1.0 - p_keep) / kSamples)) + 64.0;
+    small_shape = expected / fgrid <= (double)kFinSmallCache;
+    cluster_shape = dev.finalize_cluster && expected <= kFinClusterMaxCandidates && nseg >= (unsigned long long)kFinClusterBlocks;
+    if (cluster_shape) {
+      fgrid = kFinClusterBlocks;
+    } else if (small_shape) {  // short lists: no more blocks than about 4096 candidates each (cheaper barriers, one block = none)
+      unsigned int want = (unsigned int)(expected / 4096.0) + 1;
+      if (want < fgrid) fgrid = want;
+    } else {  // long lists: as many blocks as stay co-resident (two per SM)
+      unsigned long long cap = large_cap_blocks;
+      if (cap > nseg) cap = nseg;
+      if (cap > (unsigned long long)kMaxFinalizeBlocks) cap = kMaxFinalizeBlocks;
+      if (cap > fgrid) fgrid = (unsigned int)cap;
+    }
+  }
   FinalizeParams fp;
   fp.n = (unsigned long long)n;
   fp.k = (unsigned long long)k;
@@ -215,90 +275,55 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
   fp.ctl = ctl;
   fp.hist = reinterpret_cast<unsigned int*>(ws + L.hist);
   fp.block_counts = reinterpret_cast<unsigned long long*>(ws + L.block_counts);
+  fp.seg_count = seg_count;
+  fp.group_count = reinterpret_cast<const unsigned int*>(ws + L.group_count);
+  fp.seg_idx = seg_idx;
+  fp.seg_val = seg_val;
+  fp.list_idx = reinterpret_cast<uint32_t*>(ws + L.list_idx);
+  fp.list_val = reinterpret_cast<uint32_t*>(ws + L.list_val);
   fp.raw_val = reinterpret_cast<float*>(ws + L.raw_val);
   fp.payload = payload;
   fp.P = P;
-  fp.bitmap = reinterpret_cast<const uint32_t*>(ws + L.bitmap);
-  fp.und = reinterpret_cast<uint2*>(ws + L.und);
-  fp.qcount = reinterpret_cast<unsigned int*>(ws + L.qcount);
-  fp.pick_blocks = (unsigned int)(((unsigned long long)n + kPickElems - 1) / kPickElems);
-  fp.per_block = reinterpret_cast<unsigned int*>(ws + L.per_block);
-  fp.stash_val = reinterpret_cast<uint32_t*>(ws + L.stash);
-  fp.dense_cache = 0;
-  fp.only_on_fallback = 0;
-  void* args[] = {&fsrc, &fp};
-
-  // the select over the bucket itself: the whole job on the dense strategy, the fallback of the list strategy
-  // (as the fallback it takes the small shape whatever the bucket's size: it almost always leaves at once, and
-  // a small grid of small blocks is the cheapest thing to launch for that)
-  auto launch_dense = [&]() -> int {
-    const bool small_shape = fp.only_on_fallback || (unsigned long long)n <= (unsigned long long)dev.sms * kFinSmallCache;
-    unsigned long long cap = small_shape ? (unsigned long long)dev.sms : finalize_large_blocks(dev);
-    if (cap > (unsigned long long)kMaxFinalizeBlocks) cap = kMaxFinalizeBlocks;
-    unsigned long long want = (unsigned long long)n / 4096 + 1;  // at least about 4096 elements per block
-    if (want > nseg) want = nseg;
-    const unsigned int fgrid = (unsigned int)(want < cap ? want : cap);
-    LaunchScope scope(K_FINALIZE_DENSE, st);
+  if (!dense) {
+    LaunchScope scope(K_GATHER, st);  // segmented list -> contiguous list and the histogram of the first digit
+    // blocks per group: about 1024 expected candidates (one step of the copy loop) per block, at least two
+    // (candidates crowd into parts of a bucket), at most eight
+    const unsigned long long ngroups = (nseg + kGatherSegs - 1) / kGatherSegs;
+    const double per_group = (double)n * (p_keep + 6.0 * std::sqrt(p_keep * (1.0 - p_keep) / kSamples)) / (double)ngroups;
+    unsigned int split = (unsigned int)(per_group / 1024.0) + 1;
+    split = split < 2 ? 2 : (split > 8 ? 8 : split);
+    k_gather<<<(unsigned int)(ngroups * split), kCta, 0, st>>>(fp, split);
+  }
+  {
+    LaunchScope scope(dense ? K_FINALIZE_DENSE : K_FINALIZE, st);
+    void* args[] = {&fsrc, &fp};
     cudaError_t le;
-    if (small_shape) {
-      fp.dense_cache = kFinSmallCache;
-      le = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_finalize_dense<FDTYPE, kFinSmallThreads>), dim3(fgrid),
-                                       dim3(kFinSmallThreads), args, finalize_dyn_smem(kFinSmallCache), st);
-    } else {
-      fp.dense_cache = kFinDenseLargeCache;
-      le = cudaLaunchCooperativeKernel(reinterpret_cast<void*>(k_finalize_dense<FDTYPE, kFinLargeThreads>), dim3(fgrid),
-                                       dim3(kFinLargeThreads), args, finalize_dyn_smem(kFinDenseLargeCache), st);
-    }
-    return le == cudaSuccess ? NSML_OK : NSML_ERR_CUDA;
-  };
-
-  if (use_dense(n, k, dev)) {
-    {
-      LaunchScope scope(K_CLEAR, st);
-      k_clear<<<4, kCta, 0, st>>>(reinterpret_cast<uint4*>(ws), (unsigned int)(L.fine / 16), keep_status ? 1 : 0);
-    }
-    return launch_dense();
+    auto launch = [&](auto kernel, int threads, int cache) {
+      return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(fgrid), dim3(threads), args,
+                                         finalize_dyn_smem(cache), st);
+    };
+    if (cluster_shape) {
+      // one cluster; the blocks of a cluster are co-scheduled by the hardware, so no cooperative launch is needed
+      cudaLaunchConfig_t cfg = {};
+      cfg.gridDim = dim3(kFinClusterBlocks);
+      cfg.blockDim = dim3(kFinClusterThreads);
+      cfg.dynamicSmemBytes = finalize_dyn_smem(kFinClusterCache);
+      cfg.stream = st;
+      cudaLaunchAttribute attr[1];
+      attr[0].id = cudaLaunchAttributeClusterDimension;
+      attr[0].val.clusterDim.x = kFinClusterBlocks;
+      attr[0].val.clusterDim.y = 1;
+      attr[0].val.clusterDim.z = 1;
+      cfg.attrs = attr;
+      cfg.numAttrs = 1;
+      le = cudaLaunchKernelEx(&cfg, k_finalize<FDTYPE, kFinClusterThreads, kFinClusterCache, true>, fsrc, fp);
+    } else if (small_shape && dense) le = launch(k_finalize_dense<FDTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
+    else if (small_shape) le = launch(k_finalize<FDTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
+    else if (dense) le = launch(k_finalize_dense<FDTYPE, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache);
+    else le = launch(k_finalize<FDTYPE, kFinLargeThreads, kFinLargeCache>, kFinLargeThreads, kFinLargeCache);
+    if (le != cudaSuccess) return NSML_ERR_CUDA;
   }
-
-  const SampleRanks ranks = sample_ranks(n, k);
-  {
-    LaunchScope scope(K_SAMPLE, st);  // one cluster of kSampleBlocks blocks; also clears the per-call counters
-    // the counters of the payload's 1024-entry blocks are cleared only as far as this call's k reaches
-    const size_t clear_bytes = L.qcount + align_up(((size_t)k / NSML_QBLOCK + 2) * 4, 16);
-    const int keys16 = (DTYPE == NSML_BF16 && residual == nullptr) ? 1 : 0;
-    k_sample<DTYPE><<<kSampleBlocks, kSampleThreads, kSampleSmem, st>>>(src, residual, (unsigned long long)n, ranks.lo, ranks.hi, keys16,
-                                                                        ctl, reinterpret_cast<uint4*>(ws),
-                                                                        (unsigned int)(clear_bytes / 16), keep_status ? 1 : 0);
-  }
-  {
-    // bucket pass; at most four blocks per SM: enough loads in flight for the memory system, and half of an
-    // SM's threads stay free for kernels of other streams
-    LaunchScope scope(K_MARK, st);
-    const int resident = residual != nullptr ? dev.mark_feedback : dev.mark;
-    const unsigned int grid = grid_for(((unsigned long long)n + kStreamTile - 1) / kStreamTile, 1, dev.sms * (resident < 4 ? resident : 4));
-    uint32_t* bitmap = reinterpret_cast<uint32_t*>(ws + L.bitmap);
-    unsigned int* group_count = reinterpret_cast<unsigned int*>(ws + L.group_count);
-    unsigned int* fine = reinterpret_cast<unsigned int*>(ws + L.fine);
-    if (residual != nullptr)
-      k_mark<DTYPE, true><<<grid, kCta, 0, st>>>(src, residual, (unsigned long long)n, (unsigned long long)k, ctl, bitmap, group_count, fine);
-    else
-      k_mark<DTYPE, false><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, (unsigned long long)k, ctl, bitmap, group_count, fine);
-  }
-  {
-    LaunchScope scope(K_PICK_A, st);
-    k_pick_a<FDTYPE><<<fp.pick_blocks, kPickThreads, 0, st>>>(fsrc, fp);
-  }
-  {
-    LaunchScope scope(K_PICK_SETTLE, st);
-    k_pick_settle<<<1, kPickThreads, 0, st>>>(fp);
-  }
-  {
-    LaunchScope scope(K_PICK_B, st);
-    k_pick_b<<<fp.pick_blocks, kPickThreads, 0, st>>>(fp);
-  }
-  // the fallback: leaves at once unless the list stage raised ctl->fallback
-  fp.only_on_fallback = 1;
-  return launch_dense();
+  return NSML_OK;
 }
 
 static int compress_impl(const void* grad, int64_t n, int grad_dtype, double ratio, int bits,
@@ -847,7 +872,6 @@ int nsml_selftest_bounded_wait(void* workspace, size_t workspace_bytes, int max_
   if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
   return NSML_OK;
 }
-
 
 const char* nsml_strerror(int status) {
   switch (status) {

@@ -17,58 +17,36 @@ constexpr int kMaxBins = 4096;
 
 constexpr int kCta = 256;          // threads per block in every streaming kernel
 constexpr uint32_t kInfKey = 0x7F800000u;
-constexpr int kStreamLoads = 4;                       // 16-byte loads a thread of a streaming kernel keeps in flight
-constexpr int kStreamTile = kCta * 4 * kStreamLoads;  // elements a block of a streaming kernel takes per step
 
 // Polls before a wait at a grid barrier gives up (each poll sleeps a little,
 // so this is on the order of a second).
 constexpr int kMaxPolls = 1 << 22;
 
 // Control block at the start of a compress workspace.  Cleared (together with
-// the histograms and counters that follow it) at the start of every call.
+// the histograms that follow it) at the start of every call.
 struct Ctl {
   int status;                 // first device-detected error (NSML_ERR_*), 0 = ok
-  unsigned int lo;            // sampled lower bound of the threshold key: candidates are the keys >= max(lo, 1)
-  unsigned int barrier;       // arrivals at the grid barriers of the cooperative kernel
-  unsigned int shift;         // fine histogram: bin = min((key - lo) >> shift, kFineBins - 1)
-  unsigned int exact;         // every fine bin below the last holds one representable key value
-  unsigned int und_count;     // entries appended to the list of undecided candidates
-  unsigned int fallback;      // the list stage gave up (too few candidates, a full table): select over the bucket
-  unsigned int mark_done;     // blocks of the bucket pass that have finished
-  unsigned int pick_done;     // blocks of the first list kernel that have finished
-  unsigned int Tbin;          // fine bin that holds the k-th largest key
-  unsigned int rem;           // rank of that key inside its bin, from the top
-  unsigned int by_bin;        // the bin itself decides: above it = above T, in it = equal to T (exact && Tbin not the last)
-  unsigned int T;             // listed case: the threshold key ...
-  unsigned int limit;         // ... and the index up to which ties at T survive
-  unsigned int ties_kept;     // by-bin case: keys equal to T that survive, lowest index first
+  unsigned int lo;            // sampled lower bound of the threshold key
+  unsigned int barrier;       // arrivals at the finalize kernel's grid barriers
+  unsigned int pad;
 };
 static_assert(sizeof(Ctl) <= 256, "control block must fit its 256-byte slot");
 
-constexpr int kSegElems = 512;            // bucket elements per ownership unit of the dense select
-constexpr int kMaxFinalizeBlocks = 1024;  // upper bound on blocks of the cooperative kernels
-constexpr int kFineBins = 2048;           // bins of the candidates' key histogram built by the bucket pass
-constexpr int kFineStride = 32;            // words between two bins' counters: neighbouring bins, which are hot together, sit in different 128-byte lines
-constexpr int kGroupElems = 4096;         // bucket elements per group; the bucket pass keeps a candidate count per group
-constexpr int kPickGroups = 8;            // groups (32768 elements) a block of the list stage owns
-constexpr int kPickElems = kPickGroups * kGroupElems;
-constexpr int kStashPerBlock = kPickElems;      // values of one block's candidates the stash holds: room for every element
-constexpr int kRoundElems = 128;          // bucket elements per round: 4 words (16 bytes) of the candidate bitmap
-constexpr unsigned int kUndCap = 2048;    // undecided candidates (those in the threshold's fine bin) that can be listed
+constexpr int kSegElems = 512;            // bucket elements per candidate-list segment (4 rounds of 128)
+constexpr int kGroupSegs = 64;            // segments per group; the bucket pass keeps a candidate count per group
+constexpr int kMaxFinalizeBlocks = 1024;  // upper bound on blocks of the finalize kernel
 
 struct CompressLayout {  // byte offsets inside a compress workspace
-  size_t hist;          // u32[4][kMaxBins]: digit histograms of the dense select
-  size_t fine;          // u32[kFineBins * kFineStride]: candidates per fine key bin (one counter per 128-byte line)
-  size_t group_count;   // u32[ceil(n / kGroupElems)]: candidates per group
-  size_t qcount;        // u32[n / 4096 + 2]: survivors delivered so far per block of 1024 payload entries
+  size_t hist;          // u32[4][kMaxBins]: digit histograms (levels 0..2, level 0 again after a rebuild)
+  size_t group_count;   // u32[ceil(segments / kGroupSegs)]: candidates per group of segments
   size_t zero_bytes;    // everything before this offset is cleared per call
-  size_t block_counts;  // u64[4][kMaxFinalizeBlocks]: per-block counts exchanged at barriers (dense select)
-  size_t und;           // uint2[kUndCap]: (value bits, index) of the undecided candidates
-  size_t per_block;     // u32[6][ceil(n / kPickElems)]: list stage, per block: candidates, above the bin, in the bin,
-                        //   listed survivors, survivors before the block, in-bin entries before the block
-  size_t bitmap;        // u32[4 * ceil(n / kRoundElems)]: bit (i & 31) of word i >> 5 set = element i is a candidate
-  size_t raw_val;       // f32[n]: survivor values before quantisation (list strategy: at most n / 4 of them) ...
-  size_t stash;         // ... list strategy: u32[ceil(n / kPickElems) * kPickElems]: values of each block's candidates
+  size_t block_counts;  // u64[4][kMaxFinalizeBlocks]: per-block counts exchanged at barriers
+  size_t seg_count;     // u16[ceil(n / kSegElems)]: entries per segment
+  size_t seg_idx;       // u32[n]: segmented candidate list (bucket pass output); segment s starts at s * kSegElems
+  size_t seg_val;       // u32[n] (float32 bit patterns)
+  size_t list_idx;      // u32[n]: the same candidates, contiguous per finalize block
+  size_t list_val;      // u32[n]
+  size_t raw_val;       // f32[n]: survivor values before quantisation
   size_t total;
 };
 
@@ -76,23 +54,19 @@ __host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a -
 
 inline CompressLayout compress_layout(int64_t n) {
   CompressLayout L;
-  const size_t groups = ((size_t)n + kGroupElems - 1) / kGroupElems;
-  const size_t rounds = ((size_t)n + kRoundElems - 1) / kRoundElems;
-  const size_t pick_blocks = ((size_t)n + kPickElems - 1) / kPickElems;
+  const size_t npad = align_up((size_t)n, kSegElems);
+  const size_t segs = npad / kSegElems;
   L.hist = 256;
-  L.fine = L.hist + 4 * kMaxBins * sizeof(unsigned int);
-  L.group_count = L.fine + (size_t)kFineBins * kFineStride * sizeof(unsigned int);
-  L.qcount = L.group_count + align_up(groups * 4, 256);
-  L.zero_bytes = L.qcount + align_up(((size_t)n / 4096 + 2) * 4, 256);
+  L.group_count = L.hist + 4 * kMaxBins * sizeof(unsigned int);
+  L.zero_bytes = L.group_count + align_up(((segs + kGroupSegs - 1) / kGroupSegs) * 4, 256);
   L.block_counts = L.zero_bytes;
-  L.und = L.block_counts + 4 * kMaxFinalizeBlocks * 8;
-  L.per_block = L.und + (size_t)kUndCap * 8;
-  L.bitmap = L.per_block + align_up(6 * pick_blocks * 4, 256);
-  L.raw_val = L.bitmap + align_up(rounds * 16, 256);
-  // the dense select keeps up to n raw values; the list strategy n / 4 raw values and the stash behind them
-  L.stash = L.raw_val + align_up(((size_t)n / 4 + 1024) * 4, 256);
-  L.total = L.stash + pick_blocks * (size_t)kStashPerBlock * 4;
-  if (L.total < L.raw_val + align_up((size_t)n * 4, 256)) L.total = L.raw_val + align_up((size_t)n * 4, 256);
+  L.seg_count = L.block_counts + 4 * kMaxFinalizeBlocks * 8;
+  L.seg_idx = L.seg_count + align_up(segs * 2, 256);
+  L.seg_val = L.seg_idx + npad * 4;
+  L.list_idx = L.seg_val + npad * 4;
+  L.list_val = L.list_idx + npad * 4;
+  L.raw_val = L.list_val + npad * 4;
+  L.total = L.raw_val + npad * 4;
   return L;
 }
 
@@ -178,21 +152,6 @@ struct BucketSrc {
       for (int e = 0; e < 4; ++e)
         if (m & (1u << e)) bits[e] = 0;
     }
-  }
-
-  // elements i0..i0+3 as stored (all exist; no pruning mask applied), and the mask's four flags for them
-  __device__ __forceinline__ void load_raw4(unsigned long long i0, uint32_t (&bits)[4]) const {
-    if (DTYPE == NSML_F32) {
-      const uint4 v = __ldcs(reinterpret_cast<const uint4*>(static_cast<const uint32_t*>(grad) + i0));
-      bits[0] = v.x; bits[1] = v.y; bits[2] = v.z; bits[3] = v.w;
-    } else {
-      const uint2 v = __ldcs(reinterpret_cast<const uint2*>(static_cast<const uint16_t*>(grad) + i0));
-      bits[0] = v.x << 16; bits[1] = v.x & 0xFFFF0000u;
-      bits[2] = v.y << 16; bits[3] = v.y & 0xFFFF0000u;
-    }
-  }
-  __device__ __forceinline__ unsigned int pruned4(unsigned long long i0) const {
-    return mask != nullptr ? (mask[i0 >> 5] >> (unsigned)(i0 & 31)) & 0xFu : 0u;
   }
 
   // element i as stored (no pruning mask applied), and whether the mask prunes it

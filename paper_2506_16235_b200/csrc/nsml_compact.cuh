@@ -1,0 +1,211 @@
+// Bucket -> segmented candidate list: the one full pass over the bucket
+// (Alg. 2 Steps 2-3: pruned gradients read as zero; everything whose magnitude
+// is below the sampled lower bound is dropped here, in one streaming read).
+//
+// The bucket is cut into segments of kSegElems elements.  A warp takes one
+// segment at a time and appends what it keeps (every key >= lo, lo >= 1) to
+// the segment's own slots of the list, [s * kSegElems, s * kSegElems + count),
+// so nothing can overflow, nothing is allocated and no warp ever waits for
+// another: there is no block or grid synchronisation in this kernel.
+// Segments in increasing order are in index order.
+//
+// Blocks walk the bucket block-cyclically (block b takes segments 8b..8b+7,
+// then 8(b+G).., ...), so at any moment the whole grid reads one compact
+// window of the bucket, which is what DRAM row buffers like.  Every lane
+// keeps its part of the warp's next segment in flight with asynchronous
+// copies into a private shared-memory slot: a lane reads back only what it
+// copied itself, so the double buffer needs no synchronisation either.
+#pragma once
+
+#include "nsml_common.cuh"
+
+namespace nsml {
+
+constexpr int kRound = 128;                       // elements a warp handles per step (32 lanes x 4)
+constexpr int kSegRounds = kSegElems / kRound;    // 4
+// dynamic shared memory of the bucket pass with local accumulation: the residual's double buffers
+constexpr size_t kCompactFeedbackSmem = (size_t)(kCta / 32) * 2 * kSegRounds * 32 * 16;
+
+// Appends the kept elements of one round.  `f` holds this lane's four keep
+// flags (bit e = element lane*4+e of the round).  Returns the round's total.
+__device__ __forceinline__ unsigned int append_round(unsigned int f, const uint32_t (&bits)[4], uint32_t first_index,
+                                                     unsigned long long out_base, uint32_t* __restrict__ seg_idx,
+                                                     uint32_t* __restrict__ seg_val) {
+  const int lane = threadIdx.x & 31;
+  const unsigned int lt = (1u << lane) - 1u;
+  const unsigned int any = __ballot_sync(0xFFFFFFFFu, f != 0);
+  const unsigned int multi = __ballot_sync(0xFFFFFFFFu, (f & (f - 1)) != 0);
+  unsigned int before, total;
+  if (multi == 0) {  // usual case: no lane keeps more than one element
+    before = __popc(any & lt);
+    total = __popc(any);
+  } else {
+    const unsigned int mine = __popc(f);
+    unsigned int incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned int up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+      if (lane >= o) incl += up;
+    }
+    before = incl - mine;
+    total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+  }
+  if (f != 0) {
+    unsigned long long pos = out_base + before;
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+      if (f & (1u << e)) {
+        seg_idx[pos] = first_index + lane * 4 + e;
+        seg_val[pos] = bits[e];
+        ++pos;
+      }
+    }
+  }
+  return total;
+}
+
+// ---- per-lane asynchronous copies (global -> shared) ----
+template <int BYTES>
+__device__ __forceinline__ void cp_async_lane(void* smem_dst, const void* gsrc) {
+  const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+  if (BYTES == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(gsrc) : "memory");
+  else asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(d), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int PENDING>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(PENDING) : "memory"); }
+
+// |v| >= t on floats equals key >= lo for finite v; written as !(|v| < t) so
+// that NaN is kept too (the finalize kernel reports non-finite candidates).
+__device__ __forceinline__ unsigned int keep_flags(const uint32_t (&bits)[4], float t) {
+  unsigned int f = 0;
+#pragma unroll
+  for (int e = 0; e < 4; ++e) f |= (unsigned)(!(fabsf(__uint_as_float(bits[e])) < t)) << e;
+  return f;
+}
+
+// FEEDBACK: the bucket that is compressed is gradient + residual (Section 4.2 Step 3, local accumulation of
+// the filtered gradients).  The residual is streamed beside the gradient, the sum (one float32 add per
+// element) is written back over the residual and is what the candidates are taken from; the pruning mask
+// zeroes a key, not the stored sum.
+template <int DTYPE, bool FEEDBACK = false>
+__global__ void __launch_bounds__(kCta)
+k_compact_bucket(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned long long n, Ctl* ctl,
+                 uint32_t* __restrict__ seg_idx, uint32_t* __restrict__ seg_val, unsigned short* __restrict__ seg_count,
+                 unsigned int* __restrict__ group_count) {
+  constexpr int ESIZE = (DTYPE == NSML_F32) ? 4 : 2;
+  constexpr int LANE_BYTES = 4 * ESIZE;
+  constexpr int BUF_BYTES = kSegRounds * 32 * LANE_BYTES;  // one segment of one warp
+  constexpr int RBUF_BYTES = FEEDBACK ? kSegRounds * 32 * 16 : 0;  // the same segment of the residual
+  __shared__ __align__(16) unsigned char s_fifo[(kCta / 32) * 2 * BUF_BYTES];
+  extern __shared__ __align__(16) unsigned char s_rfifo[];  // FEEDBACK only: (kCta / 32) * 2 * RBUF_BYTES bytes
+  const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  unsigned char* fifo = s_fifo + (size_t)w * 2 * BUF_BYTES + lane * LANE_BYTES;  // round r of buffer b at + (b*kSegRounds + r)*32*LANE_BYTES
+  unsigned char* rfifo = s_rfifo + (size_t)w * 2 * RBUF_BYTES + lane * 16;       // the same for the residual: + (b*kSegRounds + r)*32*16
+
+  const unsigned long long nseg = (n + kSegElems - 1) / kSegElems;
+  const unsigned long long nseg_full = n / kSegElems;  // segments that need no bounds checks
+  const unsigned long long step = (unsigned long long)gridDim.x * (kCta / 32);
+  const unsigned char* g = static_cast<const unsigned char*>(src.grad) + (size_t)lane * 4 * ESIZE;
+
+  unsigned long long seg = (unsigned long long)blockIdx.x * (kCta / 32) + w;
+  if (seg < nseg_full) {
+#pragma unroll
+    for (int r = 0; r < kSegRounds; ++r) {
+      cp_async_lane<LANE_BYTES>(fifo + r * 32 * LANE_BYTES, g + (seg * kSegElems + r * kRound) * ESIZE);
+      if (FEEDBACK) cp_async_lane<16>(rfifo + r * 32 * 16, residual + seg * kSegElems + r * kRound + lane * 4);
+    }
+  }
+  cp_async_commit();
+  // The segment's 16 words of the pruning mask (64 bytes) are fetched by lanes 0-15 one segment ahead, like
+  // the data, and handed to the lanes by shuffle.
+  constexpr int kSegMaskWords = kSegElems / 32;
+  uint32_t mask_words = 0, mask_words_next = 0;
+  if (src.mask != nullptr && seg < nseg_full && lane < kSegMaskWords) mask_words = __ldg(src.mask + seg * kSegMaskWords + lane);
+  // Zeros are never candidates here; if they are needed (fewer than k non-zero
+  // keys) the list comes out short and the finalize kernel's slow path adds them.
+  const float t = __uint_as_float(max(ctl->lo, 1u));
+  int buf = 0;
+
+  while (seg < nseg) {
+    const unsigned long long next = seg + step;
+    if (next < nseg_full) {
+#pragma unroll
+      for (int r = 0; r < kSegRounds; ++r) {
+        cp_async_lane<LANE_BYTES>(fifo + ((buf ^ 1) * kSegRounds + r) * 32 * LANE_BYTES,
+                                  g + (next * kSegElems + r * kRound) * ESIZE);
+        if (FEEDBACK)
+          cp_async_lane<16>(rfifo + ((buf ^ 1) * kSegRounds + r) * 32 * 16, residual + next * kSegElems + r * kRound + lane * 4);
+      }
+    }
+    if (src.mask != nullptr && next < nseg_full && lane < kSegMaskWords)
+      mask_words_next = __ldg(src.mask + next * kSegMaskWords + lane);
+    cp_async_commit();
+    cp_async_wait<1>();  // this segment's copies have landed; the next segment's stay in flight
+
+    const unsigned long long seg_base = seg * kSegElems;
+    unsigned int kept = 0;
+#pragma unroll
+    for (int r = 0; r < kSegRounds; ++r) {
+      uint32_t bits[4];
+      if (seg < nseg_full) {
+        const unsigned char* slot = fifo + (buf * kSegRounds + r) * 32 * LANE_BYTES;
+        if (DTYPE == NSML_F32) {
+          const uint4 v = *reinterpret_cast<const uint4*>(slot);
+          bits[0] = v.x; bits[1] = v.y; bits[2] = v.z; bits[3] = v.w;
+        } else {
+          const uint2 v = *reinterpret_cast<const uint2*>(slot);
+          bits[0] = v.x << 16; bits[1] = v.x & 0xFFFF0000u;
+          bits[2] = v.y << 16; bits[3] = v.y & 0xFFFF0000u;
+        }
+        if (FEEDBACK) {
+          const float4 rv = *reinterpret_cast<const float4*>(rfifo + (buf * kSegRounds + r) * 32 * 16);
+          float4 acc;
+          acc.x = __fadd_rn(__uint_as_float(bits[0]), rv.x);
+          acc.y = __fadd_rn(__uint_as_float(bits[1]), rv.y);
+          acc.z = __fadd_rn(__uint_as_float(bits[2]), rv.z);
+          acc.w = __fadd_rn(__uint_as_float(bits[3]), rv.w);
+          *reinterpret_cast<float4*>(residual + seg_base + r * kRound + lane * 4) = acc;
+          bits[0] = __float_as_uint(acc.x); bits[1] = __float_as_uint(acc.y);
+          bits[2] = __float_as_uint(acc.z); bits[3] = __float_as_uint(acc.w);
+        }
+        if (src.mask != nullptr) {
+          const uint32_t word = __shfl_sync(0xFFFFFFFFu, mask_words, r * (kRound / 32) + (lane >> 3));
+          const uint32_t m = (word >> (unsigned)((lane & 7) * 4)) & 0xFu;
+#pragma unroll
+          for (int e = 0; e < 4; ++e)
+            if (m & (1u << e)) bits[e] = 0;
+        }
+      } else {
+        // the bucket's ragged last segment: plain loads, missing elements read as 0 and are never kept
+        if (FEEDBACK) {
+#pragma unroll
+          for (int e = 0; e < 4; ++e) {
+            const unsigned long long i = seg_base + r * kRound + lane * 4 + e;
+            bits[e] = 0;
+            if (i < n) {
+              const float acc = __fadd_rn(__uint_as_float(src.raw1(i)), residual[i]);
+              residual[i] = acc;
+              bits[e] = src.pruned(i) ? 0u : __float_as_uint(acc);
+            }
+          }
+        } else {
+          src.load_vals4(seg_base + r * kRound + lane * 4, n, bits);
+        }
+      }
+      const unsigned int f = keep_flags(bits, t);
+      if (!__any_sync(0xFFFFFFFFu, f != 0)) continue;
+      kept += append_round(f, bits, (uint32_t)(seg_base + r * kRound), seg_base + kept, seg_idx, seg_val);
+    }
+    if (lane == 0) {
+      seg_count[seg] = (unsigned short)kept;
+      if (kept) atomicAdd(group_count + seg / kGroupSegs, kept);  // result unused: a fire-and-forget reduction
+    }
+    seg = next;
+    buf ^= 1;
+    mask_words = mask_words_next;
+  }
+  cp_async_wait<0>();
+}
+
+}  // namespace nsml

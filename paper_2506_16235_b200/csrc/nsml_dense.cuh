@@ -1,5 +1,4 @@
-// Bucket -> payload by a radix select over the bucket itself, in one cooperative launch
-// (the strategy for high kept fractions, and the fallback of the list stage).
+// Bucket -> payload without a candidate list, in one cooperative kernel.
 //
 // For calls that keep a large fraction of the bucket (or whose bucket is too
 // small to sample) a candidate list would be about as large as the bucket, so
@@ -10,35 +9,35 @@
 // (they carry key 0 and take part in the selection like any other key).
 //
 // The range is read from memory once: phase 0 copies it into shared memory as
-// far as it fits (as a kernel of its own: two blocks per SM hold 2 x 23040
-// values, so a 25 MB float32 bucket stays on chip entirely); what does not fit is read again from the
+// far as it fits (two blocks per SM hold 2 x 23040 values, so a 25 MB float32
+// bucket stays on chip entirely); what does not fit is read again from the
 // bucket in every phase.  All later passes take the range four entries per
 // lane at a time ("words"), each warp walking its own contiguous slice of the
 // cached words and its own slice of the uncached ones, so that block order,
 // warp order and lane order together are index order.
 //
-// Phases, separated by grid barriers (bounded waits, see nsml_finalize.cuh):
+// Phases, separated by grid barriers (same protocol and bounds as k_finalize):
 //   0  load the range, keep the shared-memory copy, histogram of digit 0   | barrier
 //   1  resolve digit 0; histogram of digit 1                               | barrier
 //   2  resolve digit 1; histogram of digit 2                               | barrier
 //   3  resolve digit 2 -> T, r; per-warp counts of keys > T and == T       | barrier
 //   4  prefix over blocks and warps; write survivors in index order        | barrier
-//   5  quantise
+//   5  quantise (shared with k_finalize)
 #pragma once
 
 #include "nsml_finalize.cuh"
 
 namespace nsml {
 
-// The whole select as a device function.  s_cache: p.dense_cache words of shared memory (a multiple of 128: a warp step of 32
-// words is cached as a whole or not at all); `barriers`: grid barriers this launch has already passed.
-template <int DTYPE, int THREADS>
-__device__ __forceinline__ void dense_select(const BucketSrc<DTYPE>& src, const FinalizeParams& p, FinalizeShared<THREADS>& sh,
-                                             uint32_t* s_cache, unsigned int barriers) {
+template <int DTYPE, int THREADS, int CACHE>
+__global__ void __launch_bounds__(THREADS, 1024 / THREADS)  // at most 64 registers per thread
+k_finalize_dense(BucketSrc<DTYPE> src, FinalizeParams p) {
+  static_assert(CACHE % 128 == 0, "a warp step (32 words) is cached as a whole or not at all");
+  __shared__ FinalizeShared<THREADS, true> sh;
+  extern __shared__ __align__(16) uint32_t s_cache[];
   uint4* cache4 = reinterpret_cast<uint4*>(s_cache);
   constexpr int NW = THREADS / 32;
-  const unsigned int CACHE = p.dense_cache;
-  const unsigned int CW = CACHE / 4;  // cached words
+  constexpr unsigned int CW = CACHE / 4;  // cached words
   constexpr unsigned int FULL = 0xFFFFFFFFu;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   const unsigned int G = gridDim.x, blk = blockIdx.x;
@@ -46,6 +45,7 @@ __device__ __forceinline__ void dense_select(const BucketSrc<DTYPE>& src, const 
   const unsigned long long range_hi = min(((unsigned long long)(blk + 1) * p.nseg / G) * kSegElems, p.n);
   const unsigned int E = (unsigned int)(range_hi - range_lo);  // >= 1: the grid has at most nseg blocks
   const unsigned int W = (E + 3) / 4;
+  unsigned int barriers = 0;
 
   // This warp's slices, in words: q = 0 cached, q = 1 not cached.  Slice lengths are multiples of 32.
   const unsigned int cached_w = min(W, CW);
@@ -157,7 +157,7 @@ __device__ __forceinline__ void dense_select(const BucketSrc<DTYPE>& src, const 
   unsigned int above[2] = {0, 0};           // this lane's keys above bin d0, per slice
   unsigned int und_len = 0, und_len0 = 0;   // listed so far (warp-uniform); of those, from slice 0
   bool und_ok = E <= 65536u;                // warp-uniform
-  unsigned short* und = sh.und[warp];
+  unsigned short* und = sh.g.und[warp];
   const unsigned int lt = (1u << lane) - 1u;
   {
     unsigned int zeros = 0;
@@ -192,7 +192,7 @@ __device__ __forceinline__ void dense_select(const BucketSrc<DTYPE>& src, const 
           before = incl - mine;
           total = __shfl_sync(FULL, incl, 31);
         }
-        if (und_ok && und_len + total <= (unsigned int)kUndWarpCap) {
+        if (und_ok && und_len + total <= (unsigned int)kUndCap) {
           unsigned int pos = und_len + before;
 #pragma unroll
           for (int e = 0; e < 4; ++e)
@@ -216,7 +216,7 @@ __device__ __forceinline__ void dense_select(const BucketSrc<DTYPE>& src, const 
   auto for_listed = [&](auto&& f) {
     for (unsigned int i = lane; i < und_len; i += 32) {
       const unsigned int j = und[i];
-      const uint32_t bits = j < CACHE ? s_cache[j] : src.load1(range_lo + j);
+      const uint32_t bits = j < (unsigned int)CACHE ? s_cache[j] : src.load1(range_lo + j);
       f(i < und_len0 ? 0 : 1, bits & 0x7FFFFFFFu);
     }
   };
@@ -401,16 +401,6 @@ __device__ __forceinline__ void dense_select(const BucketSrc<DTYPE>& src, const 
 
   // ---------------- phase 5: quantise, write the header ----------------
   quantize_phase(p, sh);
-}
-
-template <int DTYPE, int THREADS>
-__global__ void __launch_bounds__(THREADS, 1024 / THREADS)  // at most 64 registers per thread
-k_finalize_dense(BucketSrc<DTYPE> src, FinalizeParams p) {
-  __shared__ FinalizeShared<THREADS> sh;
-  extern __shared__ __align__(16) uint32_t s_dense_cache[];
-  // enqueued behind the list stage as its fallback: nothing to do unless the list stage asked for it
-  if (p.only_on_fallback && __ldcg(&p.ctl->fallback) == 0) return;
-  dense_select<DTYPE, THREADS>(src, p, sh, s_dense_cache, 0u);
 }
 
 }  // namespace nsml

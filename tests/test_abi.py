@@ -50,8 +50,7 @@ def test_k_rule_and_sizes(nsml):
     assert nsml.nsml_payload_bytes(1 << 20, 0.01, 8) == 64 + idx + (k + 15) // 16 * 16 + (11 * 4 + 15) // 16 * 16
     assert nsml.nsml_payload_bytes(1 << 20, 0.01, 16) == 64 + idx + (2 * k + 15) // 16 * 16
     assert nsml.nsml_payload_bytes(1 << 20, 0.01, 4) == 0
-    assert 4 * (1 << 20) <= nsml.nsml_workspace_bytes(1 << 20, 0) <= 6 * (1 << 20)
-    assert 4 * (1 << 26) <= nsml.nsml_workspace_bytes(1 << 26, 1) <= 6 * (1 << 26)
+    assert nsml.nsml_workspace_bytes(1 << 20, 0) >= 12 * (1 << 20)
     assert nsml.nsml_workspace_bytes(1 << 20, 7) == 0
     assert nsml.nsml_accumulate_workspace_bytes(1 << 20, 4) > 0
     assert nsml.nsml_accumulate_workspace_bytes(1 << 20, 65) == 0

@@ -111,23 +111,22 @@ def sampled_positions(n, strata=8192):
     hashed offset inside it), restated from its description so that a test can
     build a bucket on which the sample is misleading."""
     s = np.arange(strata, dtype=np.uint64)
-    width = np.uint64(n // strata)  # the last stratum's remainder is never sampled
-    if width < 2:
-        return np.zeros(0, dtype=np.int64)  # buckets this small are not sampled at all
+    begin = s * np.uint64(n) // np.uint64(strata)
+    end = (s + np.uint64(1)) * np.uint64(n) // np.uint64(strata)
     x = (s * np.uint64(0x9E3779B1) + np.uint64(0x85EBCA6B)) & np.uint64(0xFFFFFFFF)
     x ^= x >> np.uint64(16)
     x = (x * np.uint64(0x7FEB352D)) & np.uint64(0xFFFFFFFF)
     x ^= x >> np.uint64(15)
     x = (x * np.uint64(0x846CA68B)) & np.uint64(0xFFFFFFFF)
     x ^= x >> np.uint64(16)
-    return (s * width + ((x * width) >> np.uint64(32))).astype(np.int64)
+    return (begin + x % (end - begin)).astype(np.int64)
 
 
 @pytest.mark.parametrize("n", [20000, 200000, 1 << 20])
 def test_misleading_sample_still_gives_the_exact_result(n):
     # large magnitudes exactly where the sampler looks, small ones elsewhere:
-    # the sampled bracket then keeps far fewer than k elements and the list stage
-    # has to fall back to the select over the bucket itself
+    # the sampled bracket then keeps far fewer than k elements and the repeat
+    # pass has to produce the list
     rng = np.random.default_rng(n)
     g = (rng.standard_normal(n) * 1e-3).astype(np.float32)
     pos = sampled_positions(n)
