@@ -10,10 +10,11 @@ summed into a dense buffer.  The metric is input-gradient bytes per second.
 Prints ONE JSON line (rank 0).
 
 Workloads (value distributions are described in synth.py):
-  resnet50  25.6M fp32 parameters in ResNet-50's tensor shapes, 25 MB buckets,
-            ratio sweep {0.5, 0.1, 0.01, 0.001} x {int8, fp16}, W = 1  (default)
   gpt2      124M fp32 parameters in GPT-2-small's shapes, 25M-element buckets,
-            ratio 0.01, int8, W = 4 workers summed into one dense buffer
+            ratio 0.01, int8, W = 4 workers summed into one dense buffer  (default:
+            the configuration with buckets of the size the bandwidth target is stated for)
+  resnet50  25.6M fp32 parameters in ResNet-50's tensor shapes, 25 MB buckets,
+            ratio sweep {0.5, 0.1, 0.01, 0.001} x {int8, fp16}, W = 1
   decoder   1.3B bf16 parameters, 64M-element buckets, fp16 values, ratio chosen
             every step by the controller from a synthetic 100/10/1 Gbps link trace
   agg       8 workers x int8 payloads for a 350M-element bucket (ratio 0.05),
@@ -21,6 +22,11 @@ Workloads (value distributions are described in synth.py):
   alg2      the whole of Alg. 2 on 25M-element fp32 buckets: L2 norm, pruning mask
             built from synthetic weights, compress of gradient + residual (ratio
             0.01, int8), sum, W = 1
+
+With --gpus N > 1 (started by torchrun, or by this script itself when it is run
+plainly) every rank runs the workload on its own GPU and the ranks' times are
+reduced with MAX; an extra leg times the data-parallel exchange: compress,
+all-gather of the payloads over NCCL, sum of the N payloads.
 """
 from __future__ import annotations
 
@@ -41,11 +47,20 @@ METRIC = "compress+decompress input-gradient GB/s per bucket; % of B200 HBM roof
 UNIT = "GB/s"
 SWEEP = [(r, b) for r in (0.5, 0.1, 0.01, 0.001) for b in (8, 16)]
 
-# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from the ncu capture summarised in
-# profiles/compress_kernels_gpt2_25M_ncu_full.md: 25M-element fp32 buckets, ratio 0.01, int8, W = 4.  Only valid
-# for that workload and for the kernels as they were when the capture was taken.
-NCU_TRAFFIC_25M = {"k_sample": 1.06e6, "k_compact_bucket": 103.6e6, "k_gather": 4.5e6, "k_finalize": 3.7e6,
-                   "k_partition": 3.9e6, "k_merge": 53.0e6}
+def ncu_traffic(workload_key):
+    """DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the kernels of one workload, from
+    the text summary of its ncu capture: lines 'traffic <workload> <kernel> <bytes>'.  Missing file or
+    workload: no figures (the bench then reports traffic as null)."""
+    out = {}
+    try:
+        with open(os.path.join(ROOT, "profiles", "dram_traffic_per_launch.txt")) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) == 4 and parts[0] == "traffic" and parts[1] == workload_key:
+                    out[parts[2]] = float(parts[3])
+    except OSError:
+        pass
+    return out
 
 
 def measured_peak_gbs():
@@ -333,10 +348,16 @@ class Gpt2Workload(Workload):
     name = "gpt2-small: 124M fp32 params, 25M-element buckets, ratio 0.01, int8, W=4 workers summed"
     W, RATIO, BITS = 4, 0.01, 8
 
-    def __init__(self, nsml, torch, device, rank, buckets=None, nlanes=2):
+    def __init__(self, nsml, torch, device, rank, buckets=None, nlanes=2, ratio=None, bits=None, workers=None):
         import synth
 
         self.nsml, self.torch = nsml, torch
+        if ratio is not None:
+            self.RATIO = ratio
+        if bits is not None:
+            self.BITS = bits
+        if workers is not None:
+            self.W = workers
         shapes = synth.gpt2_small_shapes()
         total = synth.total_elements(shapes)
         ranges = synth.bucket_ranges(total, 25_000_000)
@@ -418,15 +439,21 @@ class Gpt2Workload(Workload):
         return self.W * (4 * n + pb), self.W * pb + 4 * n
 
     def oracle_sample(self):
-        import oracle
+        return self.oracle_sample_static()
 
-        n = 4_000_000
-        gs = [self.workers[w][-1][:n].cpu().numpy() for w in range(self.W)]
+    @staticmethod
+    def oracle_sample_static():
+        """The oracle on a bounded sample of this workload: about 10-20 s of one host core."""
+        import oracle
+        import synth
+
+        n, W = 8_000_000, Gpt2Workload.W
+        gs = [synth.gpt2_bucket(2, seed=10 + w)[:n] for w in range(W)]
         t0 = time.perf_counter()
-        ps = [oracle.compress(g, self.RATIO, self.BITS) for g in gs]
+        ps = [oracle.compress(g, Gpt2Workload.RATIO, Gpt2Workload.BITS) for g in gs]
         oracle.decompress_sum(ps, n)
         dt = time.perf_counter() - t0
-        return self.W * 4.0 * n, dt, f"first {n} elements of the last bucket, {self.W} workers compressed and summed"
+        return W * 4.0 * n, dt, f"first {n} elements of bucket 2, {W} workers compressed (ratio 0.01, int8) and summed"
 
 
 class DecoderWorkload(Workload):
@@ -518,6 +545,48 @@ class DecoderWorkload(Workload):
         oracle.decompress_sum([p], n)
         dt = time.perf_counter() - t0
         return 2.0 * n, dt, f"first {n} bf16 elements of bucket 5 at ratio 0.01, fp16 values"
+
+
+class Bf16BucketWorkload(Workload):
+    """Buckets of the largest configuration's size and type, at one fixed ratio: where a pass over a bucket is
+    long enough for the memory system to reach its steady state."""
+
+    name = "decoder-1.3B shapes: three 64M-element bf16 buckets, ratio 0.01, fp16 values, W=1"
+    dtype = "bf16"
+    RATIO, BITS, N, BUCKETS = 0.01, 16, 1 << 26, 3
+    has_host = False
+
+    def __init__(self, nsml, torch, device, rank, nlanes=2):
+        self.nsml, self.torch = nsml, torch
+        gen = torch.Generator(device=device)
+        gen.manual_seed(700 + rank)
+        rs = np.random.default_rng([700, rank])
+        self.buckets = []
+        for _ in range(self.BUCKETS):  # four tensors of 16M elements each, per-tensor sigma log-uniform [1e-6, 1e-2]
+            g = torch.empty(self.N, dtype=torch.bfloat16, device=device)
+            for t in range(4):
+                g[t * (self.N // 4):(t + 1) * (self.N // 4)].normal_(0.0, 10.0 ** rs.uniform(-6.0, -2.0), generator=gen)
+            self.buckets.append(g)
+        n = self.N
+        self.lanes = Lanes(torch, nsml, device, nlanes, nsml.nsml_workspace_bytes(n, nsml.NSML_BF16),
+                           nsml.nsml_accumulate_workspace_bytes(n, 1), nsml.nsml_payload_bytes(n, self.RATIO, self.BITS), 1, n)
+        self.dense = self.lanes.all[0].dense
+        self.sizes = [n] * self.BUCKETS
+        self.input_bytes_per_step = 2.0 * n * self.BUCKETS
+        self.config = {"workload": self.name, "buckets": self.BUCKETS, "bucket_elems": n, "ratio": self.RATIO,
+                       "bits": self.BITS, "W": 1, "streams": nlanes, "l2": "inputs are 384 MB per step"}
+
+    def jobs(self, i):
+        nsml, n = self.nsml, self.N
+        for b, g in enumerate(self.buckets):
+            def enqueue(lane, acc, g=g):
+                p = nsml.nsml_compress(g, self.RATIO, self.BITS, payload=lane.payloads[0], workspace=lane.ws, stream=lane.stream)
+                nsml.nsml_decompress_accumulate([p], lane.dense, zero_first=True, workspace=lane.aws, stream=lane.stream)
+                if acc is not None:
+                    self.compress_bytes(acc, n, 2, self.RATIO, self.BITS)
+                    self.merge_bytes(acc, n, [(nsml.nsml_k_of(n, self.RATIO), self.BITS)])
+
+            yield (b,), nsml.nsml_payload_bytes(n, self.RATIO, self.BITS), enqueue
 
 
 class AggWorkload(Workload):
@@ -658,11 +727,49 @@ WORKLOADS = {"resnet50": ResnetWorkload, "gpt2": Gpt2Workload, "decoder": Decode
 
 
 # --------------------------------------------------------------------------
-# reference arm: the CPU oracle, timed as it stands
+# measurement helpers
 # --------------------------------------------------------------------------
+def per_kernel_table(nsml, torch, wl, peak, steps, first_step=0, traffic=None):
+    """Per-kernel device time of `steps` steps with every launch bracketed by CUDA events on its stream
+    (one stream, eager), beside the algorithmic bytes the workload's accounting gives each kernel.  Event
+    brackets add a few microseconds to a launch, so the fractions are lower bounds."""
+    acc = {}
+    nsml.nsml_prof_reset()
+    nsml.nsml_prof_enable(True)
+    active = wl.lanes.active
+    wl.lanes.active = 1  # one stream: a kernel's events then bracket that kernel alone
+    for i in range(steps):
+        wl.step(first_step + i, acc)
+    torch.cuda.synchronize()
+    wl.lanes.active = active
+    prof = nsml.nsml_prof_read()
+    nsml.nsml_prof_enable(False)
+    table = {}
+    for name, (ms, cnt) in prof.items():
+        if cnt:
+            nbytes = acc.get(name, 0) / cnt
+            gbs = nbytes / (1e-3 * ms / cnt) / 1e9 if ms > 0 else 0.0
+            table[name] = {"launches_per_step": cnt / steps, "us_per_launch": 1e3 * ms / cnt, "ms_per_step": ms / steps,
+                           "algorithmic_bytes_per_launch": nbytes, "algorithmic_GBps": gbs, "frac_of_measured": gbs / peak,
+                           "frac_of_nominal_8TBps": gbs / 8000.0, "traffic": (traffic or {}).get(name)}
+    return table
+
+
+def timed_steps(torch, wl, steps, first_step):
+    """Device time in ms of `steps` steps (all streams forked from and joined to the current one)."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    wl.lanes.fork()
+    for i in range(steps):
+        wl.step(first_step + i)
+    wl.lanes.join()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1)
+
+
 def run_leg(nsml, torch, wl, peak, use_graphs, traffic=None, steps=10):
-    """A second workload measured inside the default run: device time of `steps` steps, then per-kernel
-    device time with every launch bracketed by CUDA events (one stream, eager)."""
+    """A further workload measured inside the default run: device time of `steps` steps, then the per-kernel table."""
     wl.init_graphs(use_graphs)
     warm = max(3, wl.graph_period if wl.use_graphs else 3)
     wl.lanes.fork()
@@ -670,52 +777,101 @@ def run_leg(nsml, torch, wl, peak, use_graphs, traffic=None, steps=10):
         wl.step(i)
     wl.lanes.join()
     torch.cuda.synchronize()
-    b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    b0.record()
-    wl.lanes.fork()
-    for i in range(steps):
-        wl.step(warm + i)
-    wl.lanes.join()
-    b1.record()
-    torch.cuda.synchronize()
-    ms = b0.elapsed_time(b1) / steps
-    acc = {}
-    nsml.nsml_prof_reset()
-    nsml.nsml_prof_enable(True)
-    wl.lanes.active = 1
-    for i in range(5):
-        wl.step(i, acc)
-    torch.cuda.synchronize()
-    prof = nsml.nsml_prof_read()
-    nsml.nsml_prof_enable(False)
-    per = {}
-    for name, (t, cnt) in prof.items():
-        if cnt:
-            gbs = acc.get(name, 0) / (t * 1e-3) / 1e9
-            per[name] = {"launches_per_step": cnt / 5, "us_per_launch": 1e3 * t / cnt, "algorithmic_GBps": gbs,
-                         "frac_of_peak": gbs / peak, "frac_of_nominal_8TBps": gbs / 8000.0,
-                         "traffic": (traffic or {}).get(name)}
-    return {"workload": wl.name, "value": wl.input_bytes_per_step / (ms * 1e-3) / 1e9, "unit": UNIT,
-            "ms_per_step": ms, "kernels": per}
+    ms = timed_steps(torch, wl, steps, warm) / steps
+    return {"workload": wl.name, "value": wl.input_bytes_per_step / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
+            "per_kernel": per_kernel_table(nsml, torch, wl, peak, 5, traffic=traffic)}
 
 
+def serial_compress(nsml, torch, grad, ratio, bits, ws, payload, esize, peak, reps=30):
+    """One nsml_compress at a time on one stream, back to back: what a caller that compresses a single bucket (the
+    last bucket of a backward pass, say) gets.  The algorithmic bytes of the call are one read of the bucket plus
+    the payload written."""
+    n = grad.numel()
+    for _ in range(5):
+        nsml.nsml_compress(grad, ratio, bits, payload=payload, workspace=ws)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(reps):
+        nsml.nsml_compress(grad, ratio, bits, payload=payload, workspace=ws)
+    e1.record()
+    torch.cuda.synchronize()
+    us = 1e3 * e0.elapsed_time(e1) / reps
+    nbytes = esize * n + nsml.nsml_payload_bytes(n, ratio, bits)
+    gbs = nbytes / (us * 1e-6) / 1e9
+    return {"us_per_call": us, "algorithmic_bytes": nbytes, "algorithmic_GBps": gbs, "frac_of_measured": gbs / peak,
+            "frac_of_nominal_8TBps": gbs / 8000.0, "n": n, "ratio": ratio, "bits": bits,
+            "note": "one call at a time on one stream, eager launches; the same bucket every time, so a bucket that "
+                    "fits the 126 MB L2 is partly served from it"}
+
+
+def exchange_leg(nsml, torch, dist, device, rank, world, steps, warm=3):
+    """The data-parallel exchange of one 25M-element bucket per rank (Section 5.3: top-k payloads travel by
+    AllGather; Alg. 1 is fed the measured transfer): every rank compresses its bucket at the ratio rank 0's
+    controller picked, the payloads are all-gathered (NCCL copies the peers' payloads into local memory; no
+    kernel of this library reads a peer's memory), every rank sums the `world` payloads.  Times are device
+    times per phase, MAX over ranks."""
+    from paper_2506_16235_b200 import dp
+
+    n, bits = 25_000_000, 8
+    gen = torch.Generator(device=device)
+    gen.manual_seed(900 + rank)
+    grads = []
+    for r in range(3):  # three buckets rotate: 300 MB > L2
+        g = torch.empty(n, dtype=torch.float32, device=device)
+        rs = np.random.default_rng([900, rank, r])
+        for t in range(50):
+            g[t * (n // 50):(t + 1) * (n // 50)].normal_(0.0, 10.0 ** rs.uniform(-4.0, -2.0), generator=gen)
+        grads.append(g)
+    # a fixed ratio keeps every step's payload the same size; the controller still runs and is fed the measured
+    # all-gather, and its ratio is reported
+    ratio = 0.01
+    ctrl = nsml.Controller()
+    ws = nsml.alloc_bytes(nsml.nsml_workspace_bytes(n), device)
+    aws = nsml.alloc_bytes(nsml.nsml_accumulate_workspace_bytes(n, world), device)
+    payload = nsml.alloc_bytes(nsml.nsml_payload_bytes(n, ratio, bits), device)
+    dense = torch.empty(n, dtype=torch.float32, device=device)
+    sums = [0.0, 0.0, 0.0]
+    last = (0.0, 0.0)
+    ctrl_ratio = None
+    for i in range(warm + steps):
+        ctrl_ratio, phases, last = dp.exchange_round(
+            ctrl, last, 4.0 * n * world,
+            lambda _r, i=i: nsml.nsml_compress(grads[i % 3], ratio, bits, payload=payload, workspace=ws),
+            lambda views: nsml.nsml_decompress_accumulate(views, dense, zero_first=True, workspace=aws, sized=True),
+            on_cuda=True)
+        if i >= warm:
+            for j in range(3):
+                sums[j] += phases[j]
+    status = nsml.nsml_last_status(aws)
+    ms = [x / steps for x in sums]
+    total = sum(ms)
+    return {"workload": f"exchange: one 25M-element fp32 bucket per rank, ratio {ratio}, int8, all-gather of {world} payloads, sum",
+            "value": world * 4.0 * n / (total * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": total,
+            "ms_compress": ms[0], "ms_all_gather": ms[1], "ms_sum": ms[2], "payload_bytes": int(nsml.nsml_payload_bytes(n, ratio, bits)),
+            "all_gather_GBps_per_rank": (world - 1) * nsml.nsml_payload_bytes(n, ratio, bits) / (ms[1] * 1e-3) / 1e9 if world > 1 else None,
+            "controller_ratio_after": ctrl_ratio, "status": status}
+
+
+# --------------------------------------------------------------------------
+# reference arm: the CPU oracle, timed as it stands
+# --------------------------------------------------------------------------
 def run_reference(args, rank):
+    """The oracle as it stands on the host cores, on a bounded sample of the default workload per step: the
+    first `--reference-elements` elements of one 25M-element bucket of the GPT-2-shaped gradient set, compressed
+    for each of the 4 workers (ratio 0.01, int8) and summed."""
     if rank != 0:
         return
     import oracle
     import synth
 
-    # bounded sample of the default workload: one 25 MB bucket at one sweep point per step
-    buckets = list(synth.resnet50_buckets(seed=1))
-    g = buckets[0]
-    if args.reference_elements:
-        g = g[:int(args.reference_elements)]
-    n = g.size
+    n = int(args.reference_elements or 2_000_000)
+    W, ratio, bits = Gpt2Workload.W, Gpt2Workload.RATIO, Gpt2Workload.BITS
+    gs = [synth.gpt2_bucket(2, seed=10 + w)[:n] for w in range(W)]
 
     def one(i):
-        ratio, bits = SWEEP[i % len(SWEEP)]
-        p = oracle.compress(g, ratio, bits)
-        oracle.decompress_sum([p], n)
+        ps = [oracle.compress(g, ratio, bits) for g in gs]
+        oracle.decompress_sum(ps, n)
 
     for i in range(args.warmup):
         one(i)
@@ -723,13 +879,13 @@ def run_reference(args, rank):
     for i in range(args.steps):
         one(i)
     dt = time.perf_counter() - t0
-    value = args.steps * 4.0 * n / dt / 1e9
-    sample = f"one bucket of {n} fp32 elements per step, sweep point i mod 8"
+    value = args.steps * W * 4.0 * n / dt / 1e9
+    sample = f"first {n} elements of bucket 2, {W} workers compressed (ratio {ratio}, int8) and summed, per step"
     print(json.dumps({
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": ResnetWorkload.name, "sample": sample},
+        "config": {"workload": Gpt2Workload.name, "sample": sample},
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
@@ -739,23 +895,38 @@ def run_reference(args, rank):
 # --------------------------------------------------------------------------
 # main arm
 # --------------------------------------------------------------------------
+def spawn_ranks(args):
+    """`python bench.py --gpus N` with N > 1, not started by torchrun: start the N ranks here."""
+    import socket
+    import subprocess
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
-    ap.add_argument("--workload", default="resnet50", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="gpt2", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="nsml", choices=["nsml", "reference"])
     ap.add_argument("--streams", type=int, default=8, help="CUDA streams that independent buckets alternate between")
     ap.add_argument("--no-graphs", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-large-bucket-leg", action="store_true")
+    ap.add_argument("--no-legs", action="store_true", help="skip the further workloads measured inside the default run")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (e2e is then null)")
     ap.add_argument("--no-kernel-times", action="store_true", help="skip the event-bracketed per-kernel pass")
     ap.add_argument("--reference-elements", type=int, default=None,
-                    help="--impl reference only: elements of the bucket the oracle is timed on (default: one 25 MB bucket)")
+                    help="--impl reference only: elements of the bucket the oracle is timed on per step (default 2M)")
     ap.add_argument("--agg-elements", type=int, default=None,
                     help="agg workload only: dense elements (default 350M; smaller sizes are for profiler captures)")
+    ap.add_argument("--buckets", type=int, default=None,
+                    help="gpt2 workload only: use the first this many buckets (smaller sets are for profiler captures)")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -767,6 +938,10 @@ def main():
         args.warmup = 1 if args.warmup is None else args.warmup
         run_reference(args, rank)
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        spawn_ranks(args)
+    if world != args.gpus:
+        raise SystemExit(f"bench.py: --gpus {args.gpus} but {world} rank(s) were started")
 
     import torch
 
@@ -774,9 +949,12 @@ def main():
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    defaults = {"resnet50": (100, 5), "gpt2": (20, 3), "decoder": (90, 3), "agg": (50, 3), "alg2": (20, 8)}[args.workload]
+    if torch.cuda.device_count() <= local_rank:
+        raise SystemExit(f"bench.py: rank {rank} needs GPU {local_rank} but only {torch.cuda.device_count()} are visible")
+    defaults = {"resnet50": (100, 5), "gpt2": (50, 5), "decoder": (90, 3), "agg": (50, 3), "alg2": (20, 8)}[args.workload]
     steps = args.steps or defaults[0]
-    warmup = max(3, defaults[1] if args.warmup is None else args.warmup)
+    warmup_requested = defaults[1] if args.warmup is None else args.warmup
+    warmup = max(3, warmup_requested)
 
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
@@ -789,7 +967,10 @@ def main():
 
     if args.workload == "agg" and args.agg_elements:
         AggWorkload.N = int(args.agg_elements)
-    wl = WORKLOADS[args.workload](nsml, torch, device, rank, nlanes=max(1, args.streams))
+    kwargs = {}
+    if args.workload == "gpt2" and args.buckets:
+        kwargs["buckets"] = list(range(args.buckets))
+    wl = WORKLOADS[args.workload](nsml, torch, device, rank, nlanes=max(1, args.streams), **kwargs)
     wl.init_graphs(not args.no_graphs)
     if wl.use_graphs:
         warmup = max(warmup, wl.graph_period)  # every job has been captured before the timed region starts
@@ -807,16 +988,8 @@ def main():
     wl.lanes.join()
     barrier()
     launches0, replayed0 = nsml.nsml_launch_count(), wl.replayed_launches
-    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     with ClockSampler(local_rank) as clocks:
-        ev0.record()
-        wl.lanes.fork()
-        for i in range(steps):
-            wl.step(warmup + i)
-        wl.lanes.join()
-        ev1.record()
-        torch.cuda.synchronize()
-    elapsed_ms = ev0.elapsed_time(ev1)
+        elapsed_ms = timed_steps(torch, wl, steps, warmup)
     launches = nsml.nsml_launch_count() - launches0 + wl.replayed_launches - replayed0
     barrier()
     if dist is not None:
@@ -825,33 +998,26 @@ def main():
         elapsed_ms = float(t.item())
     value = world * steps * wl.input_bytes_per_step / (elapsed_ms * 1e-3) / 1e9
 
-    # ---- per-kernel device time (same steps again, every launch bracketed by CUDA events) ----
+    # ---- per-kernel device time (further steps, every launch bracketed by CUDA events) ----
     peak, peak_kind = measured_peak_gbs()
     kernels, roofline = {}, None
+    traffic_key = {"gpt2": "gpt2_25M", "agg": "agg_350M"}.get(args.workload)
     if not args.no_kernel_times:
-        acc = {}
-        nsml.nsml_prof_reset()
-        nsml.nsml_prof_enable(True)
-        prof_steps = max(1, min(steps, 10))
-        wl.lanes.active = 1  # one stream: a kernel's events then bracket that kernel alone
-        for i in range(prof_steps):
-            wl.step(warmup + steps + i, acc)
-        torch.cuda.synchronize()
-        wl.lanes.active = len(wl.lanes.all)
-        prof = nsml.nsml_prof_read()
-        nsml.nsml_prof_enable(False)
-        for name, (ms, cnt) in prof.items():
-            if cnt:
-                gbs = acc.get(name, 0) / (ms * 1e-3) / 1e9 if ms > 0 else 0.0
-                kernels[name] = {"launches_per_step": cnt / prof_steps, "us_per_launch": 1e3 * ms / cnt,
-                                 "ms_per_step": ms / prof_steps, "algorithmic_GBps": gbs, "frac_of_peak": gbs / peak}
+        kernels = per_kernel_table(nsml, torch, wl, peak, max(1, min(steps, 10)), warmup + steps,
+                                   traffic=ncu_traffic(traffic_key) if traffic_key else None)
         dominant = max(kernels, key=lambda k: kernels[k]["ms_per_step"])
         d = kernels[dominant]
         roofline = {"bound": "hbm", "kernel": dominant, "achieved": d["algorithmic_GBps"], "peak": peak,
                     "peak_kind": f"of {peak_kind}", "unit": "GB/s", "frac": d["algorithmic_GBps"] / peak,
-                    "frac_of_nominal_8TBps": d["algorithmic_GBps"] / 8000.0,
-                    "traffic": NCU_TRAFFIC_25M.get(dominant) if args.workload == "gpt2" else None,
-                    "us_per_launch": d["us_per_launch"]}
+                    "frac_of_nominal_8TBps": d["algorithmic_GBps"] / 8000.0, "traffic": d["traffic"],
+                    "us_per_launch": d["us_per_launch"], "algorithmic_bytes_per_launch": d["algorithmic_bytes_per_launch"],
+                    "how": "achieved = algorithmic_bytes_per_launch / us_per_launch (CUDA events around every launch, one "
+                           "stream); the dominant kernel is the one with the most device time per step",
+                    "per_kernel": kernels}
+        if rank == 0 and args.workload == "gpt2":
+            g = wl.workers[0][-2] if len(wl.workers[0]) > 1 else wl.workers[0][0]
+            roofline["one_compress_call"] = serial_compress(nsml, torch, g, wl.RATIO, wl.BITS, wl.lanes.all[0].ws,
+                                                            wl.lanes.all[0].payloads[0], 4, peak)
 
     # ---- end to end through the host-buffer entry points ----
     e2e = None
@@ -881,25 +1047,39 @@ def main():
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-        "ms_per_step": elapsed_ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": wl.dtype, "data": "synthetic", "config": wl.config, "clocks": clocks.summary(), "e2e": e2e,
-        "gpu_launches": int(launches), "roofline": roofline, "kernels": kernels,
+        "warmup_requested": warmup_requested, "ms_per_step": elapsed_ms / steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic", "config": wl.config,
+        "clocks": clocks.summary(), "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline,
     }
 
-    # ---- a 25M-element bucket, where the 60 %-of-HBM target applies ----
-    if rank == 0 and args.workload == "resnet50" and not args.no_large_bucket_leg:
-        big = Gpt2Workload(nsml, torch, device, rank, buckets=[2, 3, 2, 3], nlanes=max(1, args.streams))
-        big.name = "four 25M-element fp32 buckets, ratio 0.01, int8, W=4 workers each"
-        out["bucket_25M"] = run_leg(nsml, torch, big, peak, not args.no_graphs, NCU_TRAFFIC_25M)
-        del big
+    # ---- the exchange between ranks (N > 1; at N = 1 the same code path with one payload) ----
+    if world > 1:
+        out["exchange"] = exchange_leg(nsml, torch, dist, device, rank, world, steps=10)
+
+    # ---- further workloads (one GPU, default workload only) ----
+    if rank == 0 and world == 1 and args.workload == "gpt2" and not args.no_legs:
+        legs = {}
+        nl, graphs = max(1, args.streams), not args.no_graphs
+        del wl
         torch.cuda.empty_cache()
-        # the other steps of Alg. 2 (L2 norm, mask from weights, local accumulation) on buckets of that size
-        alg2 = Alg2Workload(nsml, torch, device, rank, nlanes=max(1, args.streams))
-        out["alg2_25M"] = run_leg(nsml, torch, alg2, peak, not args.no_graphs)
-        del alg2
+        for key, make in (
+            ("ratio_0.1_25M", lambda: Gpt2Workload(nsml, torch, device, rank, buckets=[2, 3], nlanes=nl, ratio=0.1, workers=2)),
+            ("ratio_0.001_25M", lambda: Gpt2Workload(nsml, torch, device, rank, buckets=[2, 3], nlanes=nl, ratio=0.001, workers=2)),
+            ("bf16_64M", lambda: Bf16BucketWorkload(nsml, torch, device, rank, nlanes=nl)),
+            ("alg2_25M", lambda: Alg2Workload(nsml, torch, device, rank, nlanes=nl)),
+            ("resnet50_sweep", lambda: ResnetWorkload(nsml, torch, device, rank, nlanes=nl)),
+        ):
+            leg_wl = make()
+            if key.startswith("ratio_"):
+                leg_wl.name = f"two 25M-element fp32 buckets, ratio {leg_wl.RATIO}, int8, W=2 workers each"
+            legs[key] = run_leg(nsml, torch, leg_wl, peak, graphs)
+            del leg_wl
+            torch.cuda.empty_cache()
+        out["legs"] = legs
+        wl = None
 
     if rank == 0 and not args.no_cpu_baseline:
-        nbytes, dt, sample = wl.oracle_sample()
+        nbytes, dt, sample = Gpt2Workload.oracle_sample_static() if wl is None else wl.oracle_sample()
         out["cpu_baseline"] = {"value": nbytes / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                                "sample": sample, "seconds": dt, "host_cores": os.cpu_count()}
     if rank == 0:

@@ -391,10 +391,11 @@ int nsml_compress_adaptive(const void* grad, int64_t n, int grad_dtype, double r
  * the inputs to the device, runs the operation and copies the result back, all
  * on `stream`, and returns without synchronising.  payload_host / dense_host
  * are valid once the stream has been synchronised.
- * nsml_decompress_accumulate_host reads every payload's header on the host
- * first: one that does not match n, or that describes more than
- * payload_bytes[w] bytes, makes the call return NSML_ERR_PAYLOAD before
- * anything is copied or launched. */
+ * The payloads handed to nsml_decompress_accumulate_host may themselves be the
+ * output of an earlier asynchronous call on the same stream, so their headers
+ * are checked on the device, against payload_bytes[w]: a payload that does not
+ * match n, or that describes more bytes than were handed over, is reported as
+ * NSML_ERR_PAYLOAD in the status word and none of its entries is read. */
 size_t nsml_compress_host_scratch_bytes(int64_t n, int grad_dtype, double ratio, int bits);
 int nsml_compress_host(const void* grad_host, int64_t n, int grad_dtype, double ratio, int bits,
                        const uint32_t* prune_mask_host, void* payload_host,

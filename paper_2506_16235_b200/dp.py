@@ -67,6 +67,56 @@ def exchange_payloads(payload: torch.Tensor, group=None):
     return buf, [buf[a:b] for a, b in slots]
 
 
+class _HostClock:
+    def __init__(self):
+        import time
+
+        self._now, self._marks = time.perf_counter, []
+
+    def mark(self):
+        self._marks.append(self._now())
+
+    def phases_ms(self):
+        return [1e3 * (b - a) for a, b in zip(self._marks, self._marks[1:])]
+
+
+class _CudaClock:
+    def __init__(self):
+        self._marks = []
+
+    def mark(self):
+        ev = torch.cuda.Event(enable_timing=True)
+        ev.record()
+        self._marks.append(ev)
+
+    def phases_ms(self):
+        self._marks[-1].synchronize()
+        return [a.elapsed_time(b) for a, b in zip(self._marks, self._marks[1:])]
+
+
+def exchange_round(ctrl, last, dense_bytes_all_ranks: float, compress, accumulate, on_cuda: bool, group=None):
+    """One step of the data-parallel exchange (Fig. 1, Alg. 1 Step 2 and Section 5.3 put together).
+
+    ctrl      this rank's controller (only rank 0's decision is used: ranks must compress at one ratio so that
+              the payloads have one size)
+    last      (bytes, seconds) of the previous step's transfer as this function returned it; (0, 0) at first
+    compress(ratio) -> this rank's payload (uint8 tensor); accumulate(views) sums the gathered payloads
+    Returns (agreed ratio, [compress, all-gather, sum] times in ms each MAX-reduced over the ranks, new `last`):
+    the transfer the controller sees next is all ranks' payload bytes and the slowest rank's all-gather time."""
+    world = dist.get_world_size(group) if dist.is_initialized() else 1
+    ratio = agree_ratio(ctrl.select_ratio(last[0], last[1], dense_bytes_all_ranks), group)
+    clock = _CudaClock() if on_cuda else _HostClock()
+    clock.mark()
+    payload = compress(ratio)
+    clock.mark()
+    _, views = exchange_payloads(payload, group)
+    clock.mark()
+    accumulate(views)
+    clock.mark()
+    phases = [max_over_ranks(ms, group) for ms in clock.phases_ms()]
+    return ratio, phases, (float(world * payload.numel()), max(phases[1] * 1e-3, 1e-9))
+
+
 class GradientExchange:
     """One bucket's data-parallel gradient exchange, every step (Fig. 1 and Alg. 1-2 of the paper put
     together): rank 0's controller picks the ratio from the last measured transfer, every rank compresses
@@ -90,15 +140,9 @@ class GradientExchange:
     def step(self, grad: torch.Tensor, dense: torch.Tensor) -> float:
         """dense <- sum over ranks of their compressed `grad`; returns the ratio used."""
         nsml = self.nsml
-        mine = self.ctrl.select_ratio(self.last[0], self.last[1], 4.0 * self.n * self.world)
-        self.ratio = agree_ratio(mine, self.group)
-        payload = nsml.nsml_compress(grad, self.ratio, self.bits, workspace=self.ws)
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev0.record()
-        _, views = exchange_payloads(payload, self.group)
-        ev1.record()
-        nsml.nsml_decompress_accumulate(views, dense, zero_first=True, workspace=self.aws)
-        ev1.synchronize()
-        seconds = max_over_ranks(ev0.elapsed_time(ev1) * 1e-3, self.group)
-        self.last = (float(self.world * payload.numel()), max(seconds, 1e-9))
+        self.ratio, self.phases_ms, self.last = exchange_round(
+            self.ctrl, self.last, 4.0 * self.n * self.world,
+            lambda ratio: nsml.nsml_compress(grad, ratio, self.bits, workspace=self.ws),
+            lambda views: nsml.nsml_decompress_accumulate(views, dense, zero_first=True, workspace=self.aws, sized=True),
+            on_cuda=True, group=self.group)
         return self.ratio

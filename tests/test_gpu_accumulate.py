@@ -159,3 +159,21 @@ def test_host_buffer_variants():
     nsml.nsml_decompress_accumulate_host([payload_h, payload_h], dense_h, True, scratch2)
     assert nsml.nsml_last_status(scratch2) == 0
     assert np.array_equal(dense_h.numpy(), oracle.decompress_sum([want, want], n))
+
+
+def test_host_variant_reports_a_truncated_payload():
+    # the host-buffer variant passes the sizes it was given to the device check
+    n = 40000
+    g = worker_grads(n, 1, 33)[0]
+    want = oracle.compress(g, 0.05, 8)
+    raw = nsml.pack_payload(want.n, 8, want.idx, codes=want.codes, scales=want.scales)
+    whole = torch.from_numpy(raw).pin_memory()
+    cut = torch.from_numpy(raw[: raw.size - 48].copy()).pin_memory()
+    dense_h = torch.zeros(n).pin_memory()
+    scratch = nsml.alloc_bytes(nsml.lib.nsml_accumulate_host_scratch_bytes(n, 1, raw.size), "cuda")
+    nsml.nsml_decompress_accumulate_host([cut], dense_h, True, scratch)
+    assert nsml.nsml_last_status(scratch) == nsml.NSML_ERR_PAYLOAD
+    assert not dense_h.numpy().any()  # nothing of the cut payload was added
+    nsml.nsml_decompress_accumulate_host([whole], dense_h, True, scratch)
+    assert nsml.nsml_last_status(scratch) == 0
+    assert np.array_equal(dense_h.numpy(), oracle.decompress_sum([want], n))

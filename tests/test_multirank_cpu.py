@@ -68,6 +68,56 @@ def test_two_ranks_agree_and_sum():
     assert a0 == 0 and b0 % 16 == 0 and b0 >= a1 and res[0]["total"] >= b1
 
 
+def _exchange_worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import paper_2506_16235_b200 as nsml
+    from paper_2506_16235_b200 import dp
+
+    # the loop the benchmark's exchange leg runs, with the CPU restatement standing in for the CUDA calls:
+    # controller -> agreed ratio -> compress -> all-gather -> sum, the measured transfer fed back
+    n, bits, steps = 30_000, 8, 5
+    ctrl = nsml.Controller(startup_max_steps=0, ratio_init=0.04 if rank == 0 else 0.5)  # rank 1's own choice must not matter
+    rng = np.random.default_rng(7 + rank)
+    last, ratios, sent, sums = (0.0, 0.0), [], [], []
+    for step in range(steps):
+        g = rng.standard_normal(n).astype(np.float32)
+        dense = {}
+
+        def compress(ratio, g=g):
+            p = oracle.compress(g, ratio, bits)
+            return torch.from_numpy(nsml.pack_payload(n, bits, p.idx, codes=p.codes, scales=p.scales))
+
+        def accumulate(views, dense=dense):
+            parts = [nsml.unpack_payload(v) for v in views]
+            ps = [oracle.Payload(n=n, k=q["k"], bits=bits, idx=q["idx"], raw=np.zeros(0, np.float32), codes=q["codes"],
+                                 scales=q["scales"]) for q in parts]
+            dense["sum"] = oracle.decompress_sum(ps, n)
+
+        ratio, phases, last = dp.exchange_round(ctrl, last, 4.0 * n * world, compress, accumulate, on_cuda=False)
+        assert len(phases) == 3 and all(ms >= 0.0 for ms in phases)
+        assert last[0] == world * nsml.nsml_payload_bytes(n, ratio, bits) and last[1] == max(phases[1] * 1e-3, 1e-9)
+        ratios.append(ratio)
+        sent.append(last)
+        sums.append(float(np.abs(dense["sum"].astype(np.float64)).sum()))
+    out[rank] = dict(ratios=ratios, sent=sent, sums=sums, calls=ctrl.state().calls)
+    dist.destroy_process_group()
+
+
+def test_exchange_rounds_feed_the_controller_with_the_measured_transfer():
+    world, port = 2, _free_port()
+    with mp.Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_exchange_worker, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    assert res[0]["ratios"] == res[1]["ratios"]          # every step both ranks compress at rank 0's ratio
+    assert res[0]["ratios"][0] == 0.04                   # rank 0's initial ratio, not rank 1's 0.5
+    assert len(set(res[0]["ratios"])) > 1                # and the controller moved it as transfers were measured
+    assert res[0]["sent"] == res[1]["sent"]              # MAX-reduced times: both ranks feed the same measurement
+    assert res[0]["sums"] == res[1]["sums"]              # both ranks reconstruct the same dense sums
+    assert res[0]["calls"] == res[1]["calls"] == 5
+
+
 def test_whole_job_value_is_the_aggregate():
     from paper_2506_16235_b200 import dp
 
