@@ -417,6 +417,8 @@ class Gpt2Workload(Workload):
 
             yield (b,), self.W * nsml.nsml_payload_bytes(n, self.RATIO, self.BITS), enqueue
 
+    HOST_LANES = 3  # streams (each with its own device scratch) the workers' host-buffer calls alternate between
+
     def setup_host(self):
         torch, nsml = self.torch, self.nsml
         n = self.sizes[0]
@@ -425,16 +427,32 @@ class Gpt2Workload(Workload):
         self.h_payloads = [torch.empty(pb, dtype=torch.uint8).pin_memory() for _ in range(self.W)]
         self.h_dense = torch.empty(n, dtype=torch.float32).pin_memory()
         dev = self.dense.device
-        self.h_scratch_c = nsml.alloc_bytes(nsml.lib.nsml_compress_host_scratch_bytes(n, 0, self.RATIO, self.BITS), dev)
+        # The calls are asynchronous on their stream, so a caller overlaps them by giving independent calls
+        # their own streams and scratch: while one worker's kernels run, the next worker's gradient is on
+        # its way to the device and the previous worker's payload on its way back.
+        self.h_lanes = [(torch.cuda.Stream(dev),
+                         nsml.alloc_bytes(nsml.lib.nsml_compress_host_scratch_bytes(n, 0, self.RATIO, self.BITS), dev))
+                        for _ in range(self.HOST_LANES)]
         self.h_scratch_a = nsml.alloc_bytes(nsml.lib.nsml_accumulate_host_scratch_bytes(n, self.W, self.W * pb), dev)
         self.host_input_bytes = self.W * 4.0 * n  # one bucket per host step
+        self.config["e2e_streams"] = self.HOST_LANES
 
     def step_host(self, i):
-        nsml = self.nsml
+        torch, nsml = self.torch, self.nsml
         n = self.sizes[0]
         pb = 0
+        cur = torch.cuda.current_stream()
+        start = torch.cuda.Event()
+        start.record(cur)
+        for stream, _ in self.h_lanes:
+            stream.wait_event(start)
         for w in range(self.W):
-            pb = nsml.nsml_compress_host(self.h_grads[w], self.RATIO, self.BITS, self.h_payloads[w], self.h_scratch_c)
+            stream, scratch = self.h_lanes[w % len(self.h_lanes)]
+            pb = nsml.nsml_compress_host(self.h_grads[w], self.RATIO, self.BITS, self.h_payloads[w], scratch, stream=stream)
+        for stream, _ in self.h_lanes:  # the sum needs every worker's payload back in host memory
+            done = torch.cuda.Event()
+            done.record(stream)
+            cur.wait_event(done)
         nsml.nsml_decompress_accumulate_host(self.h_payloads, self.h_dense, True, self.h_scratch_a)
         return self.W * (4 * n + pb), self.W * pb + 4 * n
 

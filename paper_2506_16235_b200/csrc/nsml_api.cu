@@ -178,23 +178,19 @@ static unsigned int sample_rank(int64_t n, int64_t k) {
   return (unsigned int)j;
 }
 
-// Kept fractions from which the dense mode of the finalize kernel is used: for any bucket, and for a bucket
-// that fits the shared-memory caches of one co-resident grid.
+// Kept fraction from which the select runs over the bucket itself.
 constexpr double kDenseRatioAny = 0.25;
-constexpr double kDenseRatioOnChip = 0.25;
 
 static unsigned long long finalize_large_blocks(const DeviceInfo& dev) {
   return (unsigned long long)dev.sms * (dev.finalize_large < 2 ? dev.finalize_large : 2);
 }
 
 // Dense mode: the finalize kernel selects over the bucket itself, with no sample and no bucket pass.
-// Taken when the bucket cannot be sampled, when the candidate list (8 bytes per entry) would be about
-// as large as the bucket, and for moderate kept fractions when the whole bucket fits the shared-memory
-// caches of one co-resident grid (it is then read from memory once).
-static bool use_dense(int64_t n, int64_t k, const DeviceInfo& dev) {
+// Taken when the bucket cannot be sampled and when the candidate list (8 bytes per entry) would be about
+// as large as the bucket.
+static bool use_dense(int64_t n, int64_t k, const DeviceInfo&) {
   const double p_keep = (double)k / (double)n;
-  const bool fits_on_chip = (unsigned long long)n <= finalize_large_blocks(dev) * (unsigned long long)kFinDenseLargeCache;
-  return sample_rank(n, k) == 0 || p_keep >= kDenseRatioAny || (fits_on_chip && p_keep >= kDenseRatioOnChip);
+  return sample_rank(n, k) == 0 || p_keep >= kDenseRatioAny;
 }
 
 // DTYPE: element type of `grad` (what the sample and the bucket pass read).  FDTYPE: element type of the

@@ -39,7 +39,7 @@ constexpr int kMaxFinalizeBlocks = 1024;  // upper bound on blocks of the finali
 struct CompressLayout {  // byte offsets inside a compress workspace
   size_t hist;          // u32[4][kMaxBins]: digit histograms (levels 0..2, level 0 again after a rebuild)
   size_t group_count;   // u32[ceil(segments / kGroupSegs)]: candidates per group of segments
-  size_t zero_bytes;    // everything before this offset is cleared per call
+  size_t zero_bytes;    // everything before this offset is cleared per call 
   size_t block_counts;  // u64[4][kMaxFinalizeBlocks]: per-block counts exchanged at barriers
   size_t seg_count;     // u16[ceil(n / kSegElems)]: entries per segment
   size_t seg_idx;       // u32[n]: segmented candidate list (bucket pass output); segment s starts at s * kSegElems

@@ -21,14 +21,14 @@
 
 namespace nsml {
 
-constexpr int kRound = 128;                       // elements a warp handles per step (32 lanes x 4)
-constexpr int kSegRounds = kSegElems / kRound;    // 4
 // dynamic shared memory of the bucket pass with local accumulation: the residual's double buffers
-constexpr size_t kCompactFeedbackSmem = (size_t)(kCta / 32) * 2 * kSegRounds * 32 * 16;
+// (a warp's segment of the residual: kSegElems float32, two of them per warp)
+constexpr size_t kCompactFeedbackSmem = (size_t)(kCta / 32) * 2 * kSegElems * 4;
 
-// Appends the kept elements of one round.  `f` holds this lane's four keep
-// flags (bit e = element lane*4+e of the round).  Returns the round's total.
-__device__ __forceinline__ unsigned int append_round(unsigned int f, const uint32_t (&bits)[4], uint32_t first_index,
+// Appends the kept elements of one round of 32 * EPL elements.  `f` holds this lane's keep flags (bit e =
+// element lane*EPL+e of the round).  Returns the round's total.
+template <int EPL>
+__device__ __forceinline__ unsigned int append_round(unsigned int f, const uint32_t (&bits)[EPL], uint32_t first_index,
                                                      unsigned long long out_base, uint32_t* __restrict__ seg_idx,
                                                      uint32_t* __restrict__ seg_val) {
   const int lane = threadIdx.x & 31;
@@ -53,9 +53,9 @@ __device__ __forceinline__ unsigned int append_round(unsigned int f, const uint3
   if (f != 0) {
     unsigned long long pos = out_base + before;
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
+    for (int e = 0; e < EPL; ++e) {
       if (f & (1u << e)) {
-        seg_idx[pos] = first_index + lane * 4 + e;
+        seg_idx[pos] = first_index + lane * EPL + e;
         seg_val[pos] = bits[e];
         ++pos;
       }
@@ -77,10 +77,11 @@ __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_gr
 
 // |v| >= t on floats equals key >= lo for finite v; written as !(|v| < t) so
 // that NaN is kept too (the finalize kernel reports non-finite candidates).
-__device__ __forceinline__ unsigned int keep_flags(const uint32_t (&bits)[4], float t) {
+template <int EPL>
+__device__ __forceinline__ unsigned int keep_flags(const uint32_t (&bits)[EPL], float t) {
   unsigned int f = 0;
 #pragma unroll
-  for (int e = 0; e < 4; ++e) f |= (unsigned)(!(fabsf(__uint_as_float(bits[e])) < t)) << e;
+  for (int e = 0; e < EPL; ++e) f |= (unsigned)(!(fabsf(__uint_as_float(bits[e])) < t)) << e;
   return f;
 }
 
@@ -94,29 +95,41 @@ k_compact_bucket(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned lo
                  uint32_t* __restrict__ seg_idx, uint32_t* __restrict__ seg_val, unsigned short* __restrict__ seg_count,
                  unsigned int* __restrict__ group_count) {
   constexpr int ESIZE = (DTYPE == NSML_F32) ? 4 : 2;
-  constexpr int LANE_BYTES = 4 * ESIZE;
-  constexpr int BUF_BYTES = kSegRounds * 32 * LANE_BYTES;  // one segment of one warp
-  constexpr int RBUF_BYTES = FEEDBACK ? kSegRounds * 32 * 16 : 0;  // the same segment of the residual
+  // Elements a lane takes per round: 16 bytes' worth of the gradient (4 float32, 8 bfloat16), so that both
+  // types cost the same number of instructions per byte; with a residual beside it (float32, 16 bytes per
+  // 4 elements) a lane stays at 4 elements.
+  constexpr int EPL = (DTYPE == NSML_BF16 && !FEEDBACK) ? 8 : 4;
+  constexpr int ROUND = 32 * EPL;                 // elements a warp handles per step
+  constexpr int ROUNDS = kSegElems / ROUND;       // steps per segment: 4 or 2
+  constexpr int LANE_BYTES = EPL * ESIZE;         // 16, or 8 (bfloat16 beside a residual)
+  constexpr int BUF_BYTES = kSegElems * ESIZE;    // one segment of one warp
+  constexpr int RBUF_BYTES = FEEDBACK ? kSegElems * 4 : 0;  // the same segment of the residual
   __shared__ __align__(16) unsigned char s_fifo[(kCta / 32) * 2 * BUF_BYTES];
   extern __shared__ __align__(16) unsigned char s_rfifo[];  // FEEDBACK only: (kCta / 32) * 2 * RBUF_BYTES bytes
   const int lane = threadIdx.x & 31, w = threadIdx.x >> 5;
-  unsigned char* fifo = s_fifo + (size_t)w * 2 * BUF_BYTES + lane * LANE_BYTES;  // round r of buffer b at + (b*kSegRounds + r)*32*LANE_BYTES
-  unsigned char* rfifo = s_rfifo + (size_t)w * 2 * RBUF_BYTES + lane * 16;       // the same for the residual: + (b*kSegRounds + r)*32*16
+  unsigned char* fifo = s_fifo + (size_t)w * 2 * BUF_BYTES + lane * LANE_BYTES;  // round r of buffer b at + (b*ROUNDS + r)*32*LANE_BYTES
+  unsigned char* rfifo = s_rfifo + (size_t)w * 2 * RBUF_BYTES + lane * 16;       // the same for the residual: + (b*ROUNDS + r)*32*16
 
   const unsigned long long nseg = (n + kSegElems - 1) / kSegElems;
   const unsigned long long nseg_full = n / kSegElems;  // segments that need no bounds checks
   const unsigned long long step = (unsigned long long)gridDim.x * (kCta / 32);
-  const unsigned char* g = static_cast<const unsigned char*>(src.grad) + (size_t)lane * 4 * ESIZE;
+  const unsigned char* g = static_cast<const unsigned char*>(src.grad) + (size_t)lane * LANE_BYTES;
+
+  // asynchronous copies of one whole segment into buffer b (nothing for the ragged last segment, which is
+  // read with plain loads); one commit group per segment, empty or not
+  auto fetch = [&](unsigned long long s, int b) {
+    if (s < nseg_full) {
+#pragma unroll
+      for (int r = 0; r < ROUNDS; ++r) {
+        cp_async_lane<LANE_BYTES>(fifo + (b * ROUNDS + r) * 32 * LANE_BYTES, g + (s * kSegElems + r * ROUND) * ESIZE);
+        if (FEEDBACK) cp_async_lane<16>(rfifo + (b * ROUNDS + r) * 32 * 16, residual + s * kSegElems + r * ROUND + lane * 4);
+      }
+    }
+    cp_async_commit();
+  };
 
   unsigned long long seg = (unsigned long long)blockIdx.x * (kCta / 32) + w;
-  if (seg < nseg_full) {
-#pragma unroll
-    for (int r = 0; r < kSegRounds; ++r) {
-      cp_async_lane<LANE_BYTES>(fifo + r * 32 * LANE_BYTES, g + (seg * kSegElems + r * kRound) * ESIZE);
-      if (FEEDBACK) cp_async_lane<16>(rfifo + r * 32 * 16, residual + seg * kSegElems + r * kRound + lane * 4);
-    }
-  }
-  cp_async_commit();
+  fetch(seg, 0);
   // The segment's 16 words of the pruning mask (64 bytes) are fetched by lanes 0-15 one segment ahead, like
   // the data, and handed to the lanes by shuffle.
   constexpr int kSegMaskWords = kSegElems / 32;
@@ -129,59 +142,57 @@ k_compact_bucket(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned lo
 
   while (seg < nseg) {
     const unsigned long long next = seg + step;
-    if (next < nseg_full) {
-#pragma unroll
-      for (int r = 0; r < kSegRounds; ++r) {
-        cp_async_lane<LANE_BYTES>(fifo + ((buf ^ 1) * kSegRounds + r) * 32 * LANE_BYTES,
-                                  g + (next * kSegElems + r * kRound) * ESIZE);
-        if (FEEDBACK)
-          cp_async_lane<16>(rfifo + ((buf ^ 1) * kSegRounds + r) * 32 * 16, residual + next * kSegElems + r * kRound + lane * 4);
-      }
-    }
+    fetch(next, buf ^ 1);
     if (src.mask != nullptr && next < nseg_full && lane < kSegMaskWords)
       mask_words_next = __ldg(src.mask + next * kSegMaskWords + lane);
-    cp_async_commit();
     cp_async_wait<1>();  // this segment's copies have landed; the next segment's stay in flight
 
     const unsigned long long seg_base = seg * kSegElems;
     unsigned int kept = 0;
 #pragma unroll
-    for (int r = 0; r < kSegRounds; ++r) {
-      uint32_t bits[4];
+    for (int r = 0; r < ROUNDS; ++r) {
+      uint32_t bits[EPL];
       if (seg < nseg_full) {
-        const unsigned char* slot = fifo + (buf * kSegRounds + r) * 32 * LANE_BYTES;
+        const unsigned char* slot = fifo + (buf * ROUNDS + r) * 32 * LANE_BYTES;
         if (DTYPE == NSML_F32) {
           const uint4 v = *reinterpret_cast<const uint4*>(slot);
           bits[0] = v.x; bits[1] = v.y; bits[2] = v.z; bits[3] = v.w;
+        } else if (EPL == 8) {
+          const uint4 v = *reinterpret_cast<const uint4*>(slot);
+          bits[0] = v.x << 16; bits[1] = v.x & 0xFFFF0000u;
+          bits[2] = v.y << 16; bits[3] = v.y & 0xFFFF0000u;
+          bits[4 % EPL] = v.z << 16; bits[5 % EPL] = v.z & 0xFFFF0000u;
+          bits[6 % EPL] = v.w << 16; bits[7 % EPL] = v.w & 0xFFFF0000u;
         } else {
           const uint2 v = *reinterpret_cast<const uint2*>(slot);
           bits[0] = v.x << 16; bits[1] = v.x & 0xFFFF0000u;
           bits[2] = v.y << 16; bits[3] = v.y & 0xFFFF0000u;
         }
         if (FEEDBACK) {
-          const float4 rv = *reinterpret_cast<const float4*>(rfifo + (buf * kSegRounds + r) * 32 * 16);
+          const float4 rv = *reinterpret_cast<const float4*>(rfifo + (buf * ROUNDS + r) * 32 * 16);
           float4 acc;
           acc.x = __fadd_rn(__uint_as_float(bits[0]), rv.x);
           acc.y = __fadd_rn(__uint_as_float(bits[1]), rv.y);
           acc.z = __fadd_rn(__uint_as_float(bits[2]), rv.z);
           acc.w = __fadd_rn(__uint_as_float(bits[3]), rv.w);
-          *reinterpret_cast<float4*>(residual + seg_base + r * kRound + lane * 4) = acc;
+          *reinterpret_cast<float4*>(residual + seg_base + r * ROUND + lane * 4) = acc;
           bits[0] = __float_as_uint(acc.x); bits[1] = __float_as_uint(acc.y);
           bits[2] = __float_as_uint(acc.z); bits[3] = __float_as_uint(acc.w);
         }
         if (src.mask != nullptr) {
-          const uint32_t word = __shfl_sync(0xFFFFFFFFu, mask_words, r * (kRound / 32) + (lane >> 3));
-          const uint32_t m = (word >> (unsigned)((lane & 7) * 4)) & 0xFu;
+          // this lane's EPL mask bits inside the round's ROUND / 32 words
+          const uint32_t word = __shfl_sync(0xFFFFFFFFu, mask_words, r * (ROUND / 32) + lane * EPL / 32);
+          const uint32_t m = (word >> (unsigned)((lane * EPL) & 31)) & ((1u << EPL) - 1u);
 #pragma unroll
-          for (int e = 0; e < 4; ++e)
+          for (int e = 0; e < EPL; ++e)
             if (m & (1u << e)) bits[e] = 0;
         }
       } else {
         // the bucket's ragged last segment: plain loads, missing elements read as 0 and are never kept
         if (FEEDBACK) {
 #pragma unroll
-          for (int e = 0; e < 4; ++e) {
-            const unsigned long long i = seg_base + r * kRound + lane * 4 + e;
+          for (int e = 0; e < EPL; ++e) {
+            const unsigned long long i = seg_base + r * ROUND + lane * EPL + e;
             bits[e] = 0;
             if (i < n) {
               const float acc = __fadd_rn(__uint_as_float(src.raw1(i)), residual[i]);
@@ -190,12 +201,18 @@ k_compact_bucket(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned lo
             }
           }
         } else {
-          src.load_vals4(seg_base + r * kRound + lane * 4, n, bits);
+#pragma unroll
+          for (int q = 0; q < EPL / 4; ++q) {
+            uint32_t four[4];
+            src.load_vals4(seg_base + r * ROUND + lane * EPL + q * 4, n, four);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) bits[q * 4 + e] = four[e];
+          }
         }
       }
-      const unsigned int f = keep_flags(bits, t);
+      const unsigned int f = keep_flags<EPL>(bits, t);
       if (!__any_sync(0xFFFFFFFFu, f != 0)) continue;
-      kept += append_round(f, bits, (uint32_t)(seg_base + r * kRound), seg_base + kept, seg_idx, seg_val);
+      kept += append_round<EPL>(f, bits, (uint32_t)(seg_base + r * ROUND), seg_base + kept, seg_idx, seg_val);
     }
     if (lane == 0) {
       seg_count[seg] = (unsigned short)kept;

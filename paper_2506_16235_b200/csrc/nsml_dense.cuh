@@ -21,8 +21,9 @@
 //   1  resolve digit 0; histogram of digit 1                               | barrier
 //   2  resolve digit 1; histogram of digit 2                               | barrier
 //   3  resolve digit 2 -> T, r; per-warp counts of keys > T and == T       | barrier
-//   4  prefix over blocks and warps; write survivors in index order        | barrier
-//   5  quantise (shared with k_finalize)
+//   4  prefix over blocks and warps; write survivors in index order
+//      (float32 and fp16 values straight into the payload)
+//   5  int8 only, behind one more barrier: quantise (shared with k_finalize)
 #pragma once
 
 #include "nsml_finalize.cuh"
@@ -389,7 +390,7 @@ k_finalize_dense(BucketSrc<DTYPE> src, FinalizeParams p) {
         __syncwarp();
         for (unsigned int i = lane; i < ta + tc; i += 32) {
           out_idx[step_base + i] = stage_idx[i];
-          p.raw_val[step_base + i] = __uint_as_float(stage_val[i]);
+          put_value(p, step_base + i, stage_val[i]);
         }
         __syncwarp();  // the staging area is read before the next step overwrites it
       }
@@ -397,10 +398,11 @@ k_finalize_dense(BucketSrc<DTYPE> src, FinalizeParams p) {
       c_here += total >> 16;
     }
   }
+  // ---------------- phase 5: the header; int8: quantise ----------------
+  if (blk == 0 && threadIdx.x == 0) write_header(p);
+  if (p.bits != NSML_BITS_INT8) return;  // float32 and fp16 values are in the payload already
   if (!grid_barrier(p.ctl, ++barriers * G, sh)) return;
-
-  // ---------------- phase 5: quantise, write the header ----------------
-  quantize_phase(p, sh);
+  quantize_all(p, sh);
 }
 
 }  // namespace nsml

@@ -7,19 +7,22 @@
 // survivors in index order and quantises them (Alg. 2 Step 1 "quantize" for
 // fp16; int8 per block of 1024 survivors).
 //
-// One block per SM, all co-resident (cooperative launch).  The bucket pass
-// also leaves a candidate count per group of 64 segments; every block scans
-// those, which gives it the list position of every group without a barrier,
-// and takes an equal share of the candidates in list order (so "index order"
-// is block order, and the blocks' work is balanced however the candidates
-// crowd).  Phases, separated by grid barriers:
-//   0  gather the share into one contiguous array (global, plus a copy in
-//      shared memory when it fits), histogram of key digit 0               | barrier
-//   1  every block resolves digit 0; histogram of digit 1                  | barrier
+// All blocks are co-resident (cooperative launch).  k_gather (below) first
+// makes the segmented list contiguous and counts the candidates' first key
+// digit.  The bucket pass also leaves a candidate count per group of 64
+// segments; every block of k_finalize scans those, which gives it the total,
+// and takes an equal share of the contiguous list (so "index order" is block
+// order, and the blocks' work is balanced however the candidates crowd).
+// Phases, separated by grid barriers:
+//   0  copy the share's values into shared memory as far as they fit
+//   1  every block resolves digit 0 (from the gather's histogram);
+//      histogram of digit 1                                                | barrier
 //   2  resolve digit 1; histogram of digit 2                               | barrier
 //   3  resolve digit 2 -> T, r; count own keys > T and == T                | barrier
-//   4  prefix over blocks; write survivors (index, raw value) in order     | barrier
-//   5  quantise blocks of 1024 survivors, write the header
+//   4  prefix over blocks; write survivors in order: index, and the value
+//      as float32 / fp16 directly or, for int8, parked in raw_val
+//   5  block 0 writes the header; int8 only, behind one more barrier: quantise
+//      blocks of 1024 survivors
 // If the list holds fewer than k candidates (fewer than k non-zero keys, or a
 // misleading sample) phase 0 is replaced by a slow path in which block b owns
 // an index range and rebuilds its array from the bucket: every non-zero key
@@ -77,10 +80,7 @@ struct FinalizeParams {
 };
 
 template <int THREADS, bool DENSE>
-struct GatherScratch {
-  unsigned int off[THREADS];  // exclusive offset of each thread's 8 segments within the chunk
-  uint4 cnt8[THREADS];        // the 8 segment counts of each thread (16 bits each)
-};
+struct GatherScratch {};  // the list kernel needs none: k_gather has made its list contiguous
 constexpr int kUndCap = 192;  // undecided entries a warp of the dense kernel can list
 template <int THREADS>
 struct GatherScratch<THREADS, true> {  // the dense kernel gathers nothing; it lists undecided entries per warp
@@ -96,7 +96,6 @@ struct FinalizeShared {
   unsigned int scan[(THREADS / 32)];
   unsigned int tot[(THREADS / 32)];
   unsigned int out[2];
-  unsigned long long start[2];  // gather: first group of this block's share, list position where that group starts
   float qmax[(THREADS / 32)];
   int ok;
 };
@@ -209,89 +208,87 @@ __global__ void __launch_bounds__(kCta) k_clear(uint4* __restrict__ region, unsi
     region[i] = make_uint4((i == 0 && keep_status) ? reinterpret_cast<const unsigned int*>(region)[0] : 0u, 0u, 0u, 0u);
 }
 
-// Phase 5 of both finalize kernels: quantises the k survivors left in raw_val (int8 per block of 1024
-// with a max-abs scale, or fp16) into the payload and writes the payload header.
+__device__ __forceinline__ void write_header(const FinalizeParams& p) {
+  nsml_payload_header h;
+  h.magic = NSML_PAYLOAD_MAGIC;
+  h.version = NSML_PAYLOAD_VERSION;
+  h.n = p.n;
+  h.k = p.k;
+  h.bits = (uint32_t)p.bits;
+  h.qblock = NSML_QBLOCK;
+  h.nblocks = p.P.nblocks;
+  h.idx_off = p.P.idx_off;
+  h.val_off = p.P.val_off;
+  h.scale_off = p.P.scale_off;
+  *reinterpret_cast<nsml_payload_header*>(p.payload) = h;
+}
+
+// A survivor's value on its way out: float32 and fp16 values go straight to their payload position (Alg. 2
+// Step 1 "quantize" for fp16); int8 values are parked in raw_val until their block of 1024 is complete.
+__device__ __forceinline__ void put_value(const FinalizeParams& p, unsigned long long pos, uint32_t bits) {
+  if (p.bits == NSML_BITS_FP32) reinterpret_cast<uint32_t*>(p.payload + p.P.val_off)[pos] = bits;
+  else if (p.bits == NSML_BITS_FP16) reinterpret_cast<uint16_t*>(p.payload + p.P.val_off)[pos] = encode_f16(__uint_as_float(bits));
+  else p.raw_val[pos] = __uint_as_float(bits);
+}
+
+// int8: thread group `threadIdx.x >> 8` (256 threads) converts the block of 1024 survivors qb from raw_val
+// into codes and a max-abs scale; live = false: this group has no block this round.  Called by every thread
+// of the thread block (it holds block barriers).
 template <int THREADS, bool D>
-__device__ __forceinline__ void quantize_phase(const FinalizeParams& p, FinalizeShared<THREADS, D>& sh) {
-  const unsigned int G = gridDim.x, blk = blockIdx.x;
+__device__ __forceinline__ void quantize_block(const FinalizeParams& p, FinalizeShared<THREADS, D>& sh, unsigned long long qb,
+                                               bool live) {
   const int lane = threadIdx.x & 31;
-  if (blk == 0 && threadIdx.x == 0) {
-    nsml_payload_header h;
-    h.magic = NSML_PAYLOAD_MAGIC;
-    h.version = NSML_PAYLOAD_VERSION;
-    h.n = p.n;
-    h.k = p.k;
-    h.bits = (uint32_t)p.bits;
-    h.qblock = NSML_QBLOCK;
-    h.nblocks = p.P.nblocks;
-    h.idx_off = p.P.idx_off;
-    h.val_off = p.P.val_off;
-    h.scale_off = p.P.scale_off;
-    *reinterpret_cast<nsml_payload_header*>(p.payload) = h;
+  const int group = threadIdx.x >> 8, gtid = threadIdx.x & 255;
+  const unsigned long long j0 = qb * NSML_QBLOCK + gtid * 4;
+  float v[4] = {0.f, 0.f, 0.f, 0.f};
+  int cnt = 0;
+  if (live) {
+    if (j0 + 4 <= p.k) {
+      const float4 f = __ldcg(reinterpret_cast<const float4*>(p.raw_val + j0));
+      v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
+      cnt = 4;
+    } else if (j0 < p.k) {
+      cnt = (int)(p.k - j0);
+      for (int e = 0; e < cnt; ++e) v[e] = __ldcg(p.raw_val + j0 + e);
+    }
   }
-  // a group of 256 threads (8 warps) quantises one block of 1024 survivors at a time
+  // max-abs of the 1024 survivors: warp shuffles, then one value per warp through shared memory
+  float m = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
+  __syncthreads();  // qmax of the previous round has been read
+  if (lane == 0) sh.qmax[threadIdx.x >> 5] = m;
+  __syncthreads();
+  m = sh.qmax[group * 8];
+#pragma unroll
+  for (int w = 1; w < 8; ++w) m = fmaxf(m, sh.qmax[group * 8 + w]);
+  const float scale = __fdiv_rn(m, 127.0f);
+  if (live) {
+    if (gtid == 0) reinterpret_cast<float*>(p.payload + p.P.scale_off)[qb] = scale;
+    signed char* out = reinterpret_cast<signed char*>(p.payload + p.P.val_off);
+    if (cnt == 4) {
+      uint32_t w = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) w |= ((uint32_t)encode_i8(v[e], scale) & 0xFFu) << (8 * e);
+      *reinterpret_cast<uint32_t*>(out + j0) = w;
+    } else {
+      for (int e = 0; e < cnt; ++e) out[j0 + e] = (signed char)encode_i8(v[e], scale);
+    }
+  }
+}
+
+// int8 only, after a grid barrier behind the write phase: every block of 1024 survivors parked in raw_val
+// becomes codes and a scale, a group of 256 threads per block.  (Measured against letting whichever thread
+// block delivers a payload block's last survivor quantise it, with no barrier: the atomic, the fences and the
+// read-back cost that variant as much as the barrier costs this one, 34.9 against 33.2 us for the list stage
+// of a 25M-element bucket.)
+template <int THREADS, bool D>
+__device__ __forceinline__ void quantize_all(const FinalizeParams& p, FinalizeShared<THREADS, D>& sh) {
   const unsigned long long qblocks = (p.k + NSML_QBLOCK - 1) / NSML_QBLOCK;
   constexpr int kQGroups = THREADS / 256;
-  const int group = threadIdx.x >> 8, gtid = threadIdx.x & 255;
-  for (unsigned long long q0 = (unsigned long long)blk * kQGroups; q0 < qblocks; q0 += (unsigned long long)G * kQGroups) {
-    const unsigned long long qb = q0 + group;
-    const unsigned long long j0 = qb * NSML_QBLOCK + gtid * 4;
-    float v[4] = {0.f, 0.f, 0.f, 0.f};
-    int cnt = 0;
-    if (qb < qblocks) {
-      if (j0 + 4 <= p.k) {
-        const float4 f = __ldcg(reinterpret_cast<const float4*>(p.raw_val + j0));
-        v[0] = f.x; v[1] = f.y; v[2] = f.z; v[3] = f.w;
-        cnt = 4;
-      } else if (j0 < p.k) {
-        cnt = (int)(p.k - j0);
-        for (int e = 0; e < cnt; ++e) v[e] = __ldcg(p.raw_val + j0 + e);
-      }
-    }
-    if (p.bits == NSML_BITS_FP32) {  // values travel as they are (Alg. 2 when Step 1 does not quantise)
-      float* out = reinterpret_cast<float*>(p.payload + p.P.val_off);
-      if (cnt == 4) {
-        *reinterpret_cast<float4*>(out + j0) = make_float4(v[0], v[1], v[2], v[3]);
-      } else {
-        for (int e = 0; e < cnt; ++e) out[j0 + e] = v[e];
-      }
-      continue;
-    }
-    if (p.bits == NSML_BITS_FP16) {
-      uint16_t* out = reinterpret_cast<uint16_t*>(p.payload + p.P.val_off);
-      if (cnt == 4) {
-        uint2 w;
-        w.x = (uint32_t)encode_f16(v[0]) | ((uint32_t)encode_f16(v[1]) << 16);
-        w.y = (uint32_t)encode_f16(v[2]) | ((uint32_t)encode_f16(v[3]) << 16);
-        *reinterpret_cast<uint2*>(out + j0) = w;
-      } else {
-        for (int e = 0; e < cnt; ++e) out[j0 + e] = encode_f16(v[e]);
-      }
-      continue;
-    }
-    // max-abs of the 1024 survivors: warp shuffles, then one value per warp through shared memory
-    float m = fmaxf(fmaxf(fabsf(v[0]), fabsf(v[1])), fmaxf(fabsf(v[2]), fabsf(v[3])));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xFFFFFFFFu, m, o));
-    __syncthreads();  // qmax of the previous round has been read
-    if (lane == 0) sh.qmax[threadIdx.x >> 5] = m;
-    __syncthreads();
-    m = sh.qmax[group * 8];
-#pragma unroll
-    for (int w = 1; w < 8; ++w) m = fmaxf(m, sh.qmax[group * 8 + w]);
-    const float scale = __fdiv_rn(m, 127.0f);
-    if (qb < qblocks) {
-      if (gtid == 0) reinterpret_cast<float*>(p.payload + p.P.scale_off)[qb] = scale;
-      signed char* out = reinterpret_cast<signed char*>(p.payload + p.P.val_off);
-      if (cnt == 4) {
-        uint32_t w = 0;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) w |= ((uint32_t)encode_i8(v[e], scale) & 0xFFu) << (8 * e);
-        *reinterpret_cast<uint32_t*>(out + j0) = w;
-      } else {
-        for (int e = 0; e < cnt; ++e) out[j0 + e] = (signed char)encode_i8(v[e], scale);
-      }
-    }
+  for (unsigned long long q0 = (unsigned long long)blockIdx.x * kQGroups; q0 < qblocks; q0 += (unsigned long long)gridDim.x * kQGroups) {
+    const unsigned long long qb = q0 + (threadIdx.x >> 8);
+    quantize_block(p, sh, qb, qb < qblocks);
   }
 }
 
@@ -705,7 +702,7 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
           if (a || (c && c_mine < r)) {
             const unsigned long long pos = a_mine + min(c_mine, r);
             out_idx[pos] = idx[u];
-            p.raw_val[pos] = __uint_as_float(bits[u]);
+            put_value(p, pos, bits[u]);
           }
           a_here += __popc(ba);
           c_here += __popc(bc);
@@ -713,10 +710,11 @@ k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
       }
     }
   }
+  // ---------------- phase 5: the header; int8: quantise ----------------
+  if (blk == 0 && threadIdx.x == 0) write_header(p);
+  if (p.bits != NSML_BITS_INT8) return;  // float32 and fp16 values are in the payload already
   if (!grid_barrier<CLUSTER>(p.ctl, ++barriers * G, sh)) return;
-
-  // ---------------- phase 5: quantise, write the header ----------------
-  quantize_phase(p, sh);
+  quantize_all(p, sh);
 }
 
 }  // namespace nsml
