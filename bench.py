@@ -713,9 +713,12 @@ class Alg2Workload(Workload):
                 nsml.nsml_decompress_accumulate([p], lane.dense, zero_first=True, workspace=lane.aws, stream=lane.stream)
                 if acc is not None:
                     self.account(acc, "k_sumsq", 4 * n)
-                    self.account(acc, "k_prune_hist", 3 * 4 * n)
-                    self.account(acc, "k_prune_ties", 3 * 4096 * 4)
-                    self.account(acc, "k_prune_write", 4 * n + n // 8)
+                    # mask build in two passes (sampled window); the four-pass kernels behind them leave at once
+                    self.account(acc, "k_prune_sample", 4 * 8192)
+                    self.account(acc, "k_prune_count", 4 * n)
+                    self.account(acc, "k_prune_settle", 4 * 4096)
+                    self.account(acc, "k_prune_mark", 4 * n + n // 8)
+                    self.account(acc, "k_prune_fix", 8 * 1024)
                     self.account(acc, "k_feedback_subtract", 13 * k)
                     self.compress_bytes(acc, n, 4, self.RATIO, self.BITS)
                     # the bucket pass also reads the mask and the residual and writes gradient + residual back

@@ -176,10 +176,19 @@ struct PruneCtl {
   unsigned int list_ok;        // the tie list holds every key that shares the threshold's 24-bit prefix
   unsigned int use_limit;      // ties are decided by index: pruned iff index <= idx_limit
   unsigned int idx_limit;
+  // two-pass path (sampled window)
+  unsigned int win_lo, win_shift;  // window of complemented keys: bin = (key - win_lo) >> win_shift, kPruneFineBins bins
+  unsigned int above;              // keys at or beyond the window's end
+  unsigned int fast_ok;            // the window held the threshold and its bin was short enough to list: mask done in two passes
+  unsigned int fast_bin, fast_rem; // the threshold's bin, rank left inside it
+  unsigned int fast_listed;        // keys of that bin appended by the mask pass
 };
+constexpr int kPruneFineBins = 4096;
+constexpr int kPruneSamples = 8192;
 constexpr unsigned int kTieCap = 1024;  // keys sharing the threshold's 24-bit prefix that the tie list can hold
 
 struct PruneLayout {
+  size_t fine;       // u32[kPruneFineBins]: keys per bin of the sampled window (two-pass path)
   size_t hist;       // u32[3][kMaxBins]
   size_t tie_list;   // uint2[kTieCap]: (index, last key digit) of the keys that share the threshold's 24-bit prefix
   size_t tile_ties;  // u32[tiles]
@@ -189,7 +198,8 @@ struct PruneLayout {
 inline PruneLayout prune_layout(int64_t n) {
   PruneLayout L;
   const size_t tiles = ((size_t)n + kStreamTile - 1) / kStreamTile;
-  L.hist = 256;
+  L.fine = 256;
+  L.hist = L.fine + kPruneFineBins * sizeof(unsigned int);
   L.tie_list = L.hist + 3 * kMaxBins * sizeof(unsigned int);
   L.tile_ties = L.tie_list + kTieCap * sizeof(uint2);
   L.total = L.tile_ties + align_up(tiles * 4, 256);
@@ -235,6 +245,7 @@ k_prune_hist(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int m, Prun
   constexpr int NB = (LEVEL == 2) ? 128 : kMaxBins;
   __shared__ unsigned int s_hist[NB];
   __shared__ unsigned int s_tot[kCta / 32], s_out[2];
+  if (ctl->fast_ok != 0) return;  // the two-pass path has built the mask
   unsigned int prefix = 0;
   bool collect = false;
   // The block's first tile is requested before the previous level is resolved, so that the resolve (a read
@@ -332,6 +343,7 @@ k_prune_ties(BucketSrc<NSML_F32> src, unsigned long long n, PruneCtl* ctl, const
   __shared__ unsigned int s_cnt[kCta / 32];
   __shared__ uint32_t s_tied[kTieCap];
   __shared__ unsigned int s_ntied;
+  if (ctl->fast_ok != 0) return;  // the two-pass path has built the mask
   prune_resolve<128>(hist + 2 * kMaxBins, ctl->rem2, s_tot, s_out);
   const uint32_t T = (ctl->prefix24 << 7) | s_out[0];
   const unsigned int r = s_out[1], cT = hist[2 * kMaxBins + s_out[0]];
@@ -391,6 +403,7 @@ k_prune_ties(BucketSrc<NSML_F32> src, unsigned long long n, PruneCtl* ctl, const
 __global__ void __launch_bounds__(kCta)
 k_prune_write(BucketSrc<NSML_F32> src, unsigned long long n, const PruneCtl* ctl, const unsigned int* __restrict__ tile_ties,
               uint32_t* __restrict__ mask) {
+  if (ctl->fast_ok != 0) return;  // the two-pass path has built the mask
   const uint32_t T = ctl->T;
   const unsigned int r = ctl->r, cT = ctl->cT;
   const bool by_index = ctl->use_limit != 0;  // ties pruned iff their index is <= idx_limit
@@ -472,7 +485,7 @@ k_prune_write_ranked(BucketSrc<NSML_F32> src, unsigned long long n, const PruneC
   __shared__ unsigned long long s_red[kCta / 32];
   const uint32_t T = ctl->T;
   const unsigned int r = ctl->r, cT = ctl->cT;
-  if (r >= cT || ctl->use_limit != 0) return;
+  if (ctl->fast_ok != 0 || r >= cT || ctl->use_limit != 0) return;
   const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   // A block takes a contiguous range of tiles and carries the number of ties seen so far; within a tile a thread
@@ -537,6 +550,237 @@ k_prune_write_ranked(BucketSrc<NSML_F32> src, unsigned long long n, const PruneC
       mask[i0 / 32] = word;
     }
     before += all;
+  }
+}
+
+// ------------------------------------------------------------------------
+// Step 2 in two passes over the weights instead of four.  A stratified sample
+// of the weights brackets the m-th largest complemented key between two sample
+// keys six sigma apart (k_prune_sample); one pass counts the keys beyond the
+// bracket and the keys inside it in kPruneFineBins bins (k_prune_count); one
+// block finds the bin that holds the threshold (k_prune_settle); the mask pass
+// prunes everything beyond that bin and lists the bin's few keys
+// (k_prune_mark); one block ranks the listed keys - larger complemented key
+// first, then lower index - and sets the bits of the first `rem` of them
+// (k_prune_fix).  When the sample misleads (the threshold lies outside the
+// bracket) or the bin holds more keys than can be listed (massive ties),
+// fast_ok stays 0 and the four-pass kernels above, which are enqueued behind
+// these in any case and otherwise leave at once, build the mask: the result is
+// exact either way.
+// ------------------------------------------------------------------------
+__global__ void __launch_bounds__(1024)
+k_prune_sample(BucketSrc<NSML_F32> src, unsigned long long n, unsigned int rank_lo, unsigned int rank_hi, PruneCtl* ctl) {
+  constexpr int THREADS = 1024, PER_THREAD = kPruneSamples / THREADS;  // 8 scattered loads in flight per thread
+  __shared__ __align__(16) unsigned int s_hist_lo[kMaxBins];
+  __shared__ __align__(16) unsigned int s_hist_hi[kMaxBins];
+  __shared__ unsigned int s_tot[THREADS / 32], s_out[2];
+  const int t = threadIdx.x;
+  const unsigned long long width = n / kPruneSamples;  // >= 2
+  uint32_t keys[PER_THREAD];
+#pragma unroll
+  for (int s = 0; s < PER_THREAD; ++s) {
+    const unsigned int stratum = (unsigned int)s * THREADS + t;
+    const unsigned long long pos = (unsigned long long)stratum * width +
+                                   (((unsigned long long)mix32(stratum * 0x9E3779B1u + 0x85EBCA6Bu) * width) >> 32);
+    keys[s] = prune_key(src.raw1(pos));
+  }
+  unsigned int prefix_lo = 0, prefix_hi = 0, rem_lo = rank_lo, rem_hi = rank_hi;
+#pragma unroll
+  for (int level = 0; level < 2; ++level) {  // 12 + 12 bits
+    const int shift = digit_shift(level);
+    __syncthreads();
+    for (int b = t; b < kMaxBins; b += THREADS) {
+      s_hist_lo[b] = 0;
+      s_hist_hi[b] = 0;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int s = 0; s < PER_THREAD; ++s) {
+      const unsigned int bin = (keys[s] >> shift) & (kMaxBins - 1);
+      if (level == 0 || (keys[s] >> 19) == prefix_lo) atomicAdd(&s_hist_lo[bin], 1u);
+      if (level == 1 && (keys[s] >> 19) == prefix_hi) atomicAdd(&s_hist_hi[bin], 1u);
+    }
+    __syncthreads();
+    unsigned int own[4];
+    {
+      const uint4 v = reinterpret_cast<const uint4*>(s_hist_lo)[t];
+      own[0] = v.x; own[1] = v.y; own[2] = v.z; own[3] = v.w;
+    }
+    find_digit_from_top<4, THREADS>(own, rem_lo, s_tot, s_out);
+    prefix_lo = (prefix_lo << 12) | s_out[0];
+    rem_lo = s_out[1];
+    if (level == 1) {
+      const uint4 h = reinterpret_cast<const uint4*>(s_hist_hi)[t];
+      own[0] = h.x; own[1] = h.y; own[2] = h.z; own[3] = h.w;
+    }
+    find_digit_from_top<4, THREADS>(own, rem_hi, s_tot, s_out);
+    prefix_hi = (prefix_hi << 12) | s_out[0];
+    rem_hi = s_out[1];
+  }
+  if (t != 0) return;
+  const unsigned int lo = prefix_lo << 7, hi = (prefix_hi + 1u) << 7;  // hi: first key above hi's 24-bit class
+  const unsigned int span = hi > lo ? hi - lo : 0u;
+  unsigned int shift = 0;
+  while ((span >> shift) >= (unsigned int)(kPruneFineBins * 3 / 4)) ++shift;
+  ctl->win_lo = lo;
+  ctl->win_shift = shift;
+}
+
+// Pass 1: keys beyond the window are counted, keys inside it (about 7 % of them) go into the block's copy of the
+// window's histogram in shared memory, which is added to the global one at the end (a warp's adds go to 32
+// neighbouring counters, one memory transaction; single adds to scattered counters run at a few dozen per ns for
+// the whole GPU and made this pass 85 us).
+__global__ void __launch_bounds__(kCta)
+k_prune_count(BucketSrc<NSML_F32> src, unsigned long long n, PruneCtl* ctl, unsigned int* __restrict__ fine) {
+  __shared__ unsigned int s_hist[kPruneFineBins];
+  __shared__ unsigned int s_above[kCta / 32];
+  const unsigned int lo = ctl->win_lo, shift = ctl->win_shift;
+  for (int b = threadIdx.x; b < kPruneFineBins; b += kCta) s_hist[b] = 0;
+  __syncthreads();
+  const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
+  // The tests run on the weight itself: complemented key >= E  <=>  |w| <= float(0x7FFFFFFF - E) for finite w.
+  const unsigned long long win_end = (unsigned long long)lo + ((unsigned long long)kPruneFineBins << shift);
+  const float t_end = win_end > 0x7FFFFFFFull ? -1.0f : __uint_as_float(min(0x7FFFFFFFu - (unsigned int)win_end, 0x7F7FFFFFu));
+  const float t_lo = __uint_as_float(min(0x7FFFFFFFu - lo, 0x7F7FFFFFu));
+  unsigned int above = 0;
+  bool nonfinite = false;
+  for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    uint32_t bits[kStreamLoads][4];
+    int cnt[kStreamLoads];
+    const bool whole = (tile + 1) * kStreamTile <= n;
+    load_tile(src, tile * kStreamTile, n, bits, cnt);
+#pragma unroll
+    for (int u = 0; u < kStreamLoads; ++u)
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (!whole && e >= cnt[u]) continue;
+        const float a = fabsf(__uint_as_float(bits[u][e]));
+        nonfinite |= !(a <= 3.4028234663852886e38f);  // NaN or an infinity
+        const bool beyond = a <= t_end;
+        above += beyond;
+        if (!beyond && a <= t_lo) atomicAdd(&s_hist[(prune_key(bits[u][e]) - lo) >> shift], 1u);  // about 7 % of the keys
+      }
+  }
+  if (nonfinite) set_status(&ctl->status, NSML_ERR_NONFINITE);
+  above = __reduce_add_sync(0xFFFFFFFFu, above);
+  if ((threadIdx.x & 31) == 0) s_above[threadIdx.x >> 5] = above;
+  __syncthreads();
+  for (int b = threadIdx.x; b < kPruneFineBins; b += kCta) {
+    const unsigned int c = s_hist[b];
+    if (c != 0) atomicAdd(fine + b, c);  // result unused: a reduction
+  }
+  if (threadIdx.x == 0) {
+    unsigned int t = 0;
+#pragma unroll
+    for (int w = 0; w < kCta / 32; ++w) t += s_above[w];
+    if (t != 0) atomicAdd(&ctl->above, t);
+  }
+}
+
+// One block: the window's bin that holds the m-th largest key, if the window holds it at all.
+__global__ void __launch_bounds__(kCta)
+k_prune_settle(unsigned int m, PruneCtl* ctl, const unsigned int* __restrict__ fine) {
+  __shared__ unsigned int s_tot[kCta / 32], s_out[2];
+  __shared__ unsigned long long s_sum[kCta / 32];
+  constexpr int PER = kPruneFineBins / kCta;
+  unsigned int own[PER];
+  unsigned long long mine = 0;
+#pragma unroll
+  for (int b = 0; b < PER; ++b) {
+    own[b] = __ldcg(fine + threadIdx.x * PER + b);
+    mine += own[b];
+  }
+  const unsigned int above = __ldcg(&ctl->above);
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, o);
+  if ((threadIdx.x & 31) == 0) s_sum[threadIdx.x >> 5] = mine;
+  __syncthreads();
+  unsigned long long inside = 0;
+#pragma unroll
+  for (int w = 0; w < kCta / 32; ++w) inside += s_sum[w];
+  if (m <= above || (unsigned long long)m > above + inside) return;  // the threshold lies outside the window
+  find_digit_from_top<PER, kCta>(own, m - above, s_tot, s_out);
+  if (threadIdx.x == 0) {
+    const unsigned int bin = s_out[0];
+    if (__ldcg(fine + bin) <= kTieCap) {  // short enough to list
+      ctl->fast_bin = bin;
+      ctl->fast_rem = s_out[1];
+      ctl->fast_ok = 1u;
+    }
+  }
+}
+
+// Pass 2: prunes every key beyond the threshold's bin, lists the bin's keys (their bits stay 0 for k_prune_fix).
+// The tests run on the weight itself: complemented key >= E  <=>  |w| <= float(0x7FFFFFFF - E) for finite w.
+__global__ void __launch_bounds__(kCta)
+k_prune_mark(BucketSrc<NSML_F32> src, unsigned long long n, PruneCtl* ctl, uint2* __restrict__ tie_list,
+             uint32_t* __restrict__ mask) {
+  if (ctl->fast_ok == 0) return;
+  const unsigned long long bin_lo = (unsigned long long)ctl->win_lo + ((unsigned long long)ctl->fast_bin << ctl->win_shift);
+  const unsigned long long bin_hi = bin_lo + (1ull << ctl->win_shift);  // first key beyond the bin
+  // largest magnitude key that is pruned for sure / that is still in the bin (0x7F7FFFFF: the largest finite)
+  const float t_beyond = bin_hi > 0x7FFFFFFFull ? -1.0f : __uint_as_float(min(0x7FFFFFFFu - (unsigned int)bin_hi, 0x7F7FFFFFu));
+  const float t_bin = __uint_as_float(min(0x7FFFFFFFu - (unsigned int)bin_lo, 0x7F7FFFFFu));
+  const unsigned long long tiles = (n + kStreamTile - 1) / kStreamTile;
+  const unsigned long long nwords = (n + 31) / 32;
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  for (unsigned long long tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
+    const unsigned long long base = tile * kStreamTile;
+    uint32_t bits[kStreamLoads][4];
+    int cnt[kStreamLoads];
+    const bool whole = base + kStreamTile <= n;
+    load_tile(src, base, n, bits, cnt);
+#pragma unroll
+    for (int u = 0; u < kStreamLoads; ++u) {
+      unsigned int f = 0;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (!whole && e >= cnt[u]) continue;
+        const float a = fabsf(__uint_as_float(bits[u][e]));
+        if (a <= t_beyond) {
+          f |= 1u << e;
+        } else if (a <= t_bin) {  // rare: at most kTieCap keys in the whole bucket
+          const unsigned int slot = atomicAdd(&ctl->fast_listed, 1u);
+          const unsigned long long i = base + (unsigned long long)(u * kCta + threadIdx.x) * 4 + e;
+          if (slot < kTieCap) tie_list[slot] = make_uint2((uint32_t)i, prune_key(bits[u][e]));
+        }
+      }
+      // the 4-bit flags of eight neighbouring lanes make one mask word
+      unsigned int x = f << (4 * (lane & 7));
+      x |= __shfl_xor_sync(0xFFFFFFFFu, x, 1);
+      x |= __shfl_xor_sync(0xFFFFFFFFu, x, 2);
+      x |= __shfl_xor_sync(0xFFFFFFFFu, x, 4);
+      const unsigned long long word = base / 32 + warp * 4 + (lane >> 3) + (unsigned long long)u * (kCta / 8);
+      if ((lane & 7) == 0 && word < nwords) mask[word] = x;
+    }
+  }
+}
+
+// The first fast_rem of the listed keys under (complemented key descending, index ascending) are pruned.  Every
+// block holds the whole list and ranks its share of the entries (ranking is quadratic in the list's length).
+constexpr int kPruneFixBlocks = 16;
+__global__ void __launch_bounds__(kCta)
+k_prune_fix(PruneCtl* ctl, const uint2* __restrict__ tie_list, uint32_t* __restrict__ mask) {
+  __shared__ uint2 s_list[kTieCap];
+  if (ctl->fast_ok == 0) return;
+  const unsigned int listed = min(__ldcg(&ctl->fast_listed), kTieCap), rem = ctl->fast_rem;
+  for (unsigned int i = threadIdx.x; i < listed; i += kCta) s_list[i] = __ldcg(tie_list + i);
+  __syncthreads();
+  if (listed < rem) {  // cannot happen: the bin holds at least rem keys
+    if (threadIdx.x == 0) set_status(&ctl->status, NSML_ERR_INTERNAL);
+    return;
+  }
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  // a warp per entry, the lanes share the comparisons
+  for (unsigned int i = blockIdx.x * (kCta / 32) + warp; i < listed; i += gridDim.x * (kCta / 32)) {
+    const uint2 me = s_list[i];
+    unsigned int before = 0;
+    for (unsigned int q = lane; q < listed; q += 32) {
+      const uint2 e = s_list[q];
+      before += e.y > me.y || (e.y == me.y && e.x < me.x);
+    }
+    before = __reduce_add_sync(0xFFFFFFFFu, before);
+    if (lane == 0 && before < rem) atomicOr(mask + (me.x >> 5), 1u << (me.x & 31));
   }
 }
 

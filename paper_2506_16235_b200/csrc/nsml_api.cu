@@ -19,13 +19,14 @@ namespace nsml {
 
 enum KernelId {
   K_SAMPLE = 0, K_COMPACT_BUCKET, K_FINALIZE, K_PARTITION, K_MERGE, K_CLEAR, K_FINALIZE_DENSE,
-  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_PRUNE_WRITE_RANKED, K_GATHER, K_COUNT
+  K_SUMSQ, K_FEEDBACK_ADD, K_FEEDBACK_SUBTRACT, K_PRUNE_HIST, K_PRUNE_TIES, K_PRUNE_WRITE, K_PRUNE_WRITE_RANKED, K_GATHER, K_PRUNE_SAMPLE, K_PRUNE_COUNT, K_PRUNE_SETTLE, K_PRUNE_MARK, K_PRUNE_FIX, K_COUNT
 };
 
 static const char* const kKernelNames[K_COUNT] = {"k_sample", "k_compact_bucket", "k_finalize", "k_partition", "k_merge",
                                                   "k_clear", "k_finalize_dense", "k_sumsq", "k_feedback_add",
                                                   "k_feedback_subtract", "k_prune_hist", "k_prune_ties", "k_prune_write",
-                                                  "k_prune_write_ranked", "k_gather"};
+                                                  "k_prune_write_ranked", "k_gather", "k_prune_sample", "k_prune_count",
+                                                  "k_prune_settle", "k_prune_mark", "k_prune_fix"};
 
 static std::atomic<int64_t> g_launches{0};
 
@@ -486,6 +487,36 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
   const unsigned int grid = stream_grid(n, *dev, dev->prune_hist < 8 ? dev->prune_hist : 8, 1u << 16);
   const unsigned int wgrid = stream_grid(n, *dev, dev->prune_write < 8 ? dev->prune_write : 8, 1u << 16);
   const unsigned long long un = (unsigned long long)n;
+  // Two passes where a sample can bracket the threshold: ranks (from the top, among the complemented keys of
+  // kPruneSamples weights) six standard deviations either side of the expected rank of the m-th largest.
+  if (n >= 2 * (int64_t)kPruneSamples) {
+    const double p = (double)m / (double)n, mean = kPruneSamples * p, six = 6.0 * std::sqrt(kPruneSamples * p * (1.0 - p));
+    const double r_lo = std::ceil(mean + six) + 1.0, r_hi = std::floor(mean - six);
+    if (r_lo < (double)kPruneSamples && r_hi >= 1.0) {
+      unsigned int* fine = reinterpret_cast<unsigned int*>(ws + L.fine);
+      {
+        LaunchScope scope(K_PRUNE_SAMPLE, st);
+        k_prune_sample<<<1, 1024, 0, st>>>(src, un, (unsigned int)r_lo, (unsigned int)r_hi, ctl);
+      }
+      {
+        LaunchScope scope(K_PRUNE_COUNT, st);
+        k_prune_count<<<grid, kCta, 0, st>>>(src, un, ctl, fine);
+      }
+      {
+        LaunchScope scope(K_PRUNE_SETTLE, st);
+        k_prune_settle<<<1, kCta, 0, st>>>((unsigned int)m, ctl, fine);
+      }
+      {
+        LaunchScope scope(K_PRUNE_MARK, st);
+        k_prune_mark<<<wgrid, kCta, 0, st>>>(src, un, ctl, tie_list, mask);
+      }
+      {
+        LaunchScope scope(K_PRUNE_FIX, st);
+        k_prune_fix<<<kPruneFixBlocks, kCta, 0, st>>>(ctl, tie_list, mask);
+      }
+    }
+  }
+  // The four-pass build: every kernel of it leaves at once when the two passes above have built the mask.
   {
     LaunchScope scope(K_PRUNE_HIST, st);
     k_prune_hist<0><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);

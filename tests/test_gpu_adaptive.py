@@ -128,6 +128,45 @@ def test_prune_mask_25m_bucket():
     check_mask(w, 0.01)
 
 
+def prune_sampled_positions(n, strata=8192):
+    """Positions the mask build's stratified sampler reads (one per stratum, a hashed offset inside it),
+    restated from its description so that a test can build weights on which the sample misleads."""
+    s = np.arange(strata, dtype=np.uint64)
+    width = np.uint64(n // strata)
+    x = (s * np.uint64(0x9E3779B1) + np.uint64(0x85EBCA6B)) & np.uint64(0xFFFFFFFF)
+    x ^= x >> np.uint64(16)
+    x = (x * np.uint64(0x7FEB352D)) & np.uint64(0xFFFFFFFF)
+    x ^= x >> np.uint64(15)
+    x = (x * np.uint64(0x846CA68B)) & np.uint64(0xFFFFFFFF)
+    x ^= x >> np.uint64(16)
+    return (s * width + ((x * width) >> np.uint64(32))).astype(np.int64)
+
+
+@pytest.mark.parametrize("n", [70_001, 1 << 20])
+def test_prune_mask_misleading_sample_still_exact(n):
+    # tiny (then huge) magnitudes exactly where the sampler looks: the sampled window misses the threshold and
+    # the four-pass build has to produce the mask
+    rng = np.random.default_rng(n)
+    w = rng.standard_normal(n).astype(np.float32)
+    pos = prune_sampled_positions(n)
+    for fill in (1e-9, 1e9):
+        w2 = w.copy()
+        w2[pos] = (fill * (1.0 + rng.random(pos.size))).astype(np.float32)
+        for ratio in (0.01, 0.5):
+            check_mask(w2, ratio)
+
+
+def test_prune_mask_two_pass_path_with_ties_in_the_threshold_bin():
+    # Gaussian weights rounded to few mantissa bits: every key has many equals, the threshold's bin holds tens
+    # of equal keys and only some of them (lowest indices first) are pruned
+    rng = np.random.default_rng(77)
+    n = 3_000_017
+    w = rng.standard_normal(n).astype(np.float32)
+    w = (w.view(np.uint32) & np.uint32(0xFFFFF000)).view(np.float32)  # 11 mantissa bits left
+    for ratio in (0.2, 0.003):
+        check_mask(w, ratio)
+
+
 def test_prune_mask_reports_nonfinite():
     w = np.ones(5000, dtype=np.float32)
     w[123] = np.nan
