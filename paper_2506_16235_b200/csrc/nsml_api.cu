@@ -487,12 +487,14 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
   const unsigned int grid = stream_grid(n, *dev, dev->prune_hist < 8 ? dev->prune_hist : 8, 1u << 16);
   const unsigned int wgrid = stream_grid(n, *dev, dev->prune_write < 8 ? dev->prune_write : 8, 1u << 16);
   const unsigned long long un = (unsigned long long)n;
+  bool two_pass = false;
   // Two passes where a sample can bracket the threshold: ranks (from the top, among the complemented keys of
   // kPruneSamples weights) six standard deviations either side of the expected rank of the m-th largest.
   if (n >= 2 * (int64_t)kPruneSamples) {
     const double p = (double)m / (double)n, mean = kPruneSamples * p, six = 6.0 * std::sqrt(kPruneSamples * p * (1.0 - p));
     const double r_lo = std::ceil(mean + six) + 1.0, r_hi = std::floor(mean - six);
     if (r_lo < (double)kPruneSamples && r_hi >= 1.0) {
+      two_pass = true;
       unsigned int* fine = reinterpret_cast<unsigned int*>(ws + L.fine);
       {
         LaunchScope scope(K_PRUNE_SAMPLE, st);
@@ -516,30 +518,36 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
       }
     }
   }
-  // The four-pass build: every kernel of it leaves at once when the two passes above have built the mask.
+  // The four-pass build: every kernel of it leaves at once when the two passes above have built the mask.  Behind
+  // the two-pass path it is the rare fallback, so it gets small grids (two blocks per SM): what counts there is
+  // how little the six launches cost when they have nothing to do.
+  const unsigned int small = (unsigned int)dev->sms * 2;
+  const unsigned int fgrid = two_pass && grid > small ? small : grid;
+  const unsigned int fwgrid = two_pass && wgrid > small ? small : wgrid;
   {
     LaunchScope scope(K_PRUNE_HIST, st);
-    k_prune_hist<0><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
+    k_prune_hist<0><<<fgrid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
     LaunchScope scope(K_PRUNE_HIST, st);
-    k_prune_hist<1><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
+    k_prune_hist<1><<<fgrid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
     LaunchScope scope(K_PRUNE_HIST, st);
-    k_prune_hist<2><<<grid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
+    k_prune_hist<2><<<fgrid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
     LaunchScope scope(K_PRUNE_TIES, st);
-    k_prune_ties<<<grid, kCta, 0, st>>>(src, un, ctl, hist, tie_list, tile_ties);
+    k_prune_ties<<<fgrid, kCta, 0, st>>>(src, un, ctl, hist, tie_list, tile_ties);
   }
   {
     LaunchScope scope(K_PRUNE_WRITE, st);
-    k_prune_write<<<wgrid, kCta, 0, st>>>(src, un, ctl, tile_ties, mask);
+    k_prune_write<<<fwgrid, kCta, 0, st>>>(src, un, ctl, tile_ties, mask);
   }
   {
     LaunchScope scope(K_PRUNE_WRITE_RANKED, st);  // returns at once unless ties have to be ranked
-    const unsigned int rgrid = stream_grid(n, *dev, dev->prune_write_ranked < 8 ? dev->prune_write_ranked : 8, 1u << 16);
+    unsigned int rgrid = stream_grid(n, *dev, dev->prune_write_ranked < 8 ? dev->prune_write_ranked : 8, 1u << 16);
+    if (two_pass && rgrid > small) rgrid = small;
     k_prune_write_ranked<<<rgrid, kCta, 0, st>>>(src, un, ctl, tile_ties, mask);
   }
   if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
