@@ -946,6 +946,8 @@ def main():
                     help="--impl reference only: elements of the bucket the oracle is timed on per step (default 2M)")
     ap.add_argument("--agg-elements", type=int, default=None,
                     help="agg workload only: dense elements (default 350M; smaller sizes are for profiler captures)")
+    ap.add_argument("--exchange", action="store_true",
+                    help="time the exchange leg on one GPU as well (one payload: the same code path as with N ranks)")
     ap.add_argument("--buckets", type=int, default=None,
                     help="gpt2 workload only: use the first this many buckets (smaller sets are for profiler captures)")
     args = ap.parse_args()
@@ -1074,7 +1076,7 @@ def main():
     }
 
     # ---- the exchange between ranks (N > 1; at N = 1 the same code path with one payload) ----
-    if world > 1:
+    if world > 1 or args.exchange:
         out["exchange"] = exchange_leg(nsml, torch, dist, device, rank, world, steps=10)
 
     # ---- further workloads (one GPU, default workload only) ----
