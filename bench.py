@@ -32,6 +32,7 @@ from __future__ import annotations
 
 import argparse
 import json
+import math
 import os
 import sys
 import threading
@@ -138,6 +139,8 @@ class Workload:
     name = ""
     dtype = "f32"
 
+    job_turn = 0        # jobs enqueued so far (the lane of a job is its turn modulo the number of lanes)
+    rotate_lanes = False  # keep counting turns from step to step instead of starting every step at lane 0
     use_graphs = False  # replay each job from a CUDA graph captured on its stream
     graph_period = 1    # steps after which the set of distinct jobs repeats (all graphs exist after that many)
     graphs_ok = True    # False where every step brings new jobs (nothing to replay)
@@ -159,7 +162,13 @@ class Workload:
         self.before_step(i)
         sent = 0
         graphs = self.use_graphs and acc is None and self.lanes.active == len(self.lanes.all)
-        for ordinal, (key, nbytes, enqueue) in enumerate(self.jobs(i)):
+        if not self.rotate_lanes:
+            self.job_turn = 0
+        for key, nbytes, enqueue in self.jobs(i):
+            # rotate_lanes: the turn count runs on from step to step, so with fewer jobs per step than lanes the
+            # next step's first jobs start on the idle lanes while this step's last ones finish
+            ordinal = self.job_turn
+            self.job_turn += 1
             lane = self.lanes.all[ordinal % self.lanes.active]
             sent += nbytes
             if not graphs:
@@ -184,6 +193,7 @@ class Workload:
     def init_graphs(self, use_graphs):
         self.use_graphs = use_graphs and self.graphs_ok
         self.graph_cache = {}
+        self.job_turn = 0
         self.replayed_launches = 0
         self.home_stream = self.torch.cuda.current_stream()
 
@@ -219,13 +229,17 @@ class Lanes:
     payload buffers, so that the latency-bound list stage of one bucket
     overlaps the streaming pass of the next."""
 
-    def __init__(self, torch, nsml, device, nlanes, ws_bytes, aws_bytes, payload_bytes, W, dense_elems):
+    def __init__(self, torch, nsml, device, nlanes, ws_bytes, aws_bytes, payload_bytes, W, dense_elems, branches=1):
         self.torch = torch
         self.all = []
         for _ in range(nlanes):
             lane = type("Lane", (), {})()
             lane.stream = torch.cuda.Stream(device)
             lane.ws = nsml.alloc_bytes(ws_bytes, device) if ws_bytes else None
+            # branches > 1: the compress calls of one job are independent of one another; each gets a stream and a
+            # workspace of its own beside the lane's (the job's sum waits for all of them)
+            lane.side = [torch.cuda.Stream(device) for _ in range(branches - 1)]
+            lane.side_ws = [nsml.alloc_bytes(ws_bytes, device) for _ in range(branches - 1)]
             lane.aws = nsml.alloc_bytes(aws_bytes, device)
             lane.payloads = [nsml.alloc_bytes(payload_bytes, device) for _ in range(W)] if payload_bytes else []
             lane.dense = torch.empty(dense_elems, dtype=torch.float32, device=device)
@@ -384,14 +398,17 @@ class Gpt2Workload(Workload):
         nmax = max(self.sizes)
         pb = nsml.nsml_payload_bytes(nmax, self.RATIO, self.BITS)
         self.lanes = Lanes(torch, nsml, device, nlanes, nsml.nsml_workspace_bytes(nmax),
-                           nsml.nsml_accumulate_workspace_bytes(nmax, self.W), pb, self.W, nmax)
+                           nsml.nsml_accumulate_workspace_bytes(nmax, self.W), pb, self.W, nmax, branches=self.W)
         self.dense = self.lanes.all[0].dense
         self.ctrl = nsml.Controller()
         self.dense_bytes = 4.0 * sum(self.sizes)
         self.input_bytes_per_step = self.W * self.dense_bytes
         self.last = (0.0, 0.0)
+        self.rotate_lanes = True
+        self.graph_period = math.lcm(len(self.sizes), nlanes) // len(self.sizes)
         self.config = {"workload": self.name, "buckets": len(self.sizes), "bucket_elems": self.sizes,
                        "ratio": self.RATIO, "bits": self.BITS, "W": self.W, "streams": nlanes,
+                       "streams_per_job": self.W,
                        "l2": "inputs are 2 GB per step, far larger than the 126 MB L2"}
 
     def before_step(self, i):
@@ -404,10 +421,27 @@ class Gpt2Workload(Workload):
         nsml = self.nsml
         for b, n in enumerate(self.sizes):
             def enqueue(lane, acc, b=b, n=n):
-                # the W workers' buckets are compressed one after the other on this job's stream, then summed;
-                # other buckets run on the other streams meanwhile
-                ps = [nsml.nsml_compress(self.workers[w][b], self.RATIO, self.BITS, payload=lane.payloads[w],
-                                         workspace=lane.ws, stream=lane.stream) for w in range(self.W)]
+                # The W workers' buckets are compressed independently of one another (each worker would do it on
+                # its own GPU): worker 0 on the job's stream, the others on the lane's side streams, each with a
+                # workspace of its own; the sum waits for all of them.  Other buckets run on the other lanes
+                # meanwhile.  (The event-bracketed per-kernel pass, acc given, keeps everything on one stream.)
+                torch = self.torch
+                fan = acc is None and len(lane.side) >= self.W - 1 and self.W > 1
+                if fan:
+                    start = torch.cuda.Event()
+                    start.record(lane.stream)
+                ps = []
+                for w in range(self.W):
+                    st = lane.side[w - 1] if fan and w else lane.stream
+                    ws = lane.side_ws[w - 1] if fan and w else lane.ws
+                    if fan and w:
+                        st.wait_event(start)
+                    ps.append(nsml.nsml_compress(self.workers[w][b], self.RATIO, self.BITS, payload=lane.payloads[w],
+                                                 workspace=ws, stream=st))
+                    if fan and w:
+                        done = torch.cuda.Event()
+                        done.record(st)
+                        lane.stream.wait_event(done)
                 nsml.nsml_decompress_accumulate(ps, lane.dense[:n], zero_first=True, workspace=lane.aws, stream=lane.stream)
                 if acc is not None:
                     k = nsml.nsml_k_of(n, self.RATIO)

@@ -95,7 +95,7 @@ static int device_info(const DeviceInfo** out) {
   if (!d.ready) {
     if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return NSML_ERR_CUDA;
     cudaError_t e = cudaSuccess;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_bucket, k_compact_bucket<NSML_F32, false>, kCta, 0);
+    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_bucket, k_compact_bucket<NSML_F32, false, true>, kCta, 0);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_compact_bucket<NSML_F32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCompactFeedbackSmem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_compact_bucket<NSML_BF16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCompactFeedbackSmem);
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_feedback, k_compact_bucket<NSML_F32, true>, kCta, kCompactFeedbackSmem);
@@ -156,6 +156,51 @@ static inline unsigned int grid_for(unsigned long long work_items, unsigned long
   if (blocks < 1) blocks = 1;
   if (blocks > (unsigned long long)cap) blocks = cap;
   return (unsigned int)blocks;
+}
+
+// The short, latency-bound kernels (sample, gather, list stage, partition) are launched at the highest stream
+// priority.  When several buckets are in flight on several streams, every bucket pass that is ready sits in
+// front of the device's block scheduler with thousands of blocks to place; a list-stage kernel that becomes
+// ready later is otherwise placed only after all of them, so the passes of a step ran first, back to back,
+// and the list stages afterwards with nothing to overlap them (measured with a timer in every kernel:
+// 250 us of an 800 us step).  At high priority its few blocks are placed as soon as blocks of the running pass
+// retire, and it runs beside the next pass.
+static int high_priority() {
+  static const int p = [] {
+    int least = 0, greatest = 0;
+    return cudaDeviceGetStreamPriorityRange(&least, &greatest) == cudaSuccess ? greatest : 0;
+  }();
+  return p;
+}
+
+template <class... KArgs, class... Args>
+static cudaError_t launch_prio(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, bool cooperative,
+                               unsigned int cluster_x, bool high, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[3];
+  unsigned int na = 0;
+  attr[na].id = cudaLaunchAttributePriority;
+  attr[na].val.priority = high ? high_priority() : 0;
+  ++na;
+  if (cooperative) {
+    attr[na].id = cudaLaunchAttributeCooperative;
+    attr[na].val.cooperative = 1;
+    ++na;
+  }
+  if (cluster_x) {
+    attr[na].id = cudaLaunchAttributeClusterDimension;
+    attr[na].val.clusterDim.x = cluster_x;
+    attr[na].val.clusterDim.y = 1;
+    attr[na].val.clusterDim.z = 1;
+    ++na;
+  }
+  cfg.attrs = attr;
+  cfg.numAttrs = na;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 static int64_t k_of(int64_t n, double ratio) {
@@ -226,23 +271,29 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
   } else {
     {
       LaunchScope scope(K_SAMPLE, st);  // one cluster of kSampleBlocks blocks
-      k_sample<DTYPE><<<kSampleBlocks, kSampleThreads, 0, st>>>(src, residual, (unsigned long long)n, sample_rank(n, k), ctl,
-                                                                reinterpret_cast<uint4*>(ws),
-                                                                (unsigned int)(L.zero_bytes / 16), keep_status ? 1 : 0);
+      // (the cluster shape is part of the kernel's definition)
+      launch_prio(k_sample<DTYPE>, dim3(kSampleBlocks), dim3(kSampleThreads), 0, st, false, 0, true, src, residual, (unsigned long long)n,
+                  sample_rank(n, k), ctl, reinterpret_cast<uint4*>(ws), (unsigned int)(L.zero_bytes / 16), keep_status ? 1 : 0);
     }
     {
-      // bucket pass: a block takes 8 segments per step; at most 4 resident blocks per SM
+      // bucket pass.  With a residual: persistent blocks, a block takes 8 segments per step, at most 4
+      // resident blocks per SM.  Without: a warp per 2 KB of the bucket, eight warps per block.
       LaunchScope scope(K_COMPACT_BUCKET, st);
-      const int resident = residual != nullptr ? dev.compact_feedback : dev.compact_bucket;
+      const int resident = dev.compact_feedback;
       const int per_sm = resident < 4 ? resident : 4;
-      const unsigned int grid = grid_for(nseg, kCta / 32, dev.sms * per_sm);
+      constexpr unsigned long long kPlainSegs = (kCta / 32) * compact_segs_per_warp<DTYPE>();  // segments per block
+      const unsigned int grid = residual != nullptr ? grid_for(nseg, kCta / 32, dev.sms * per_sm)
+                                                    : (unsigned int)((nseg + kPlainSegs - 1) / kPlainSegs);
       unsigned int* group_count = reinterpret_cast<unsigned int*>(ws + L.group_count);
       if (residual != nullptr)
         k_compact_bucket<DTYPE, true><<<grid, kCta, kCompactFeedbackSmem, st>>>(src, residual, (unsigned long long)n, ctl, seg_idx,
                                                                                 seg_val, seg_count, group_count);
+      else if (mask != nullptr)
+        k_compact_bucket<DTYPE, false, true><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, ctl, seg_idx, seg_val,
+                                                                    seg_count, group_count);
       else
-        k_compact_bucket<DTYPE, false><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, ctl, seg_idx, seg_val,
-                                                              seg_count, group_count);
+        k_compact_bucket<DTYPE, false, false><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, ctl, seg_idx, seg_val,
+                                                                     seg_count, group_count);
     }
     // list stage: cooperative, every block co-resident.  The small shape when a block's share of the
     // expected candidates (k plus the sampling margin) fits its shared-memory cache.
@@ -289,31 +340,18 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
     const double per_group = (double)n * (p_keep + 6.0 * std::sqrt(p_keep * (1.0 - p_keep) / kSamples)) / (double)ngroups;
     unsigned int split = (unsigned int)(per_group / 1024.0) + 1;
     split = split < 2 ? 2 : (split > 8 ? 8 : split);
-    k_gather<<<(unsigned int)(ngroups * split), kCta, 0, st>>>(fp, split);
+    launch_prio(k_gather, dim3((unsigned int)(ngroups * split)), dim3(kGatherThreads), 0, st, false, 0, true, fp, split);
   }
   {
     LaunchScope scope(dense ? K_FINALIZE_DENSE : K_FINALIZE, st);
-    void* args[] = {&fsrc, &fp};
     cudaError_t le;
-    auto launch = [&](auto kernel, int threads, int cache) {
-      return cudaLaunchCooperativeKernel(reinterpret_cast<void*>(kernel), dim3(fgrid), dim3(threads), args,
-                                         finalize_dyn_smem(cache), st);
+    auto launch = [&](auto kernel, int threads, int cache) {  // cooperative: every block co-resident
+      return launch_prio(kernel, dim3(fgrid), dim3(threads), finalize_dyn_smem(cache), st, true, 0, !dense, fsrc, fp);  // (the dense select streams the whole bucket: normal priority)
     };
     if (cluster_shape) {
       // one cluster; the blocks of a cluster are co-scheduled by the hardware, so no cooperative launch is needed
-      cudaLaunchConfig_t cfg = {};
-      cfg.gridDim = dim3(kFinClusterBlocks);
-      cfg.blockDim = dim3(kFinClusterThreads);
-      cfg.dynamicSmemBytes = finalize_dyn_smem(kFinClusterCache);
-      cfg.stream = st;
-      cudaLaunchAttribute attr[1];
-      attr[0].id = cudaLaunchAttributeClusterDimension;
-      attr[0].val.clusterDim.x = kFinClusterBlocks;
-      attr[0].val.clusterDim.y = 1;
-      attr[0].val.clusterDim.z = 1;
-      cfg.attrs = attr;
-      cfg.numAttrs = 1;
-      le = cudaLaunchKernelEx(&cfg, k_finalize<FDTYPE, kFinClusterThreads, kFinClusterCache, true>, fsrc, fp);
+      le = launch_prio(k_finalize<FDTYPE, kFinClusterThreads, kFinClusterCache, true>, dim3(kFinClusterBlocks), dim3(kFinClusterThreads),
+                       finalize_dyn_smem(kFinClusterCache), st, false, kFinClusterBlocks, true, fsrc, fp);
     } else if (small_shape && dense) le = launch(k_finalize_dense<FDTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
     else if (small_shape) le = launch(k_finalize<FDTYPE, kFinSmallThreads, kFinSmallCache>, kFinSmallThreads, kFinSmallCache);
     else if (dense) le = launch(k_finalize_dense<FDTYPE, kFinLargeThreads, kFinDenseLargeCache>, kFinLargeThreads, kFinDenseLargeCache);
@@ -380,10 +418,10 @@ static int accumulate_impl(const void* const* payloads, const size_t* payload_by
     const unsigned long long offsets_needed = (unsigned long long)W * (tiles + 1ull);
     if (offsets_needed <= 32768) {  // few offsets: a warp each, few round trips
       unsigned int grid = (unsigned int)((offsets_needed * 32 + kCta - 1) / kCta);
-      k_partition<<<grid, kCta, 0, st>>>(table, W, (unsigned long long)n, tiles, offsets, status);
+      launch_prio(k_partition, dim3(grid), dim3(kCta), 0, st, false, 0, true, table, W, (unsigned long long)n, tiles, offsets, status);
     } else {  // many offsets: a thread each
       unsigned int grid = (unsigned int)((offsets_needed + kCta - 1) / kCta);
-      k_partition_wide<<<grid, kCta, 0, st>>>(table, W, (unsigned long long)n, tiles, offsets, status);
+      launch_prio(k_partition_wide, dim3(grid), dim3(kCta), 0, st, false, 0, true, table, W, (unsigned long long)n, tiles, offsets, status);
     }
   }
   {

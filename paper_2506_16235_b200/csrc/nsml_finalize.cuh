@@ -302,26 +302,27 @@ __device__ __forceinline__ void quantize_all(const FinalizeParams& p, FinalizeSh
 constexpr int kGatherSegs = kGroupSegs;  // one group per block: its list position is a plain sum of group counts
 constexpr int kGatherRun = 4;      // consecutive candidates a thread copies per step
 constexpr int kGatherBins = 256;   // first-digit bins a block of the gather counts in shared memory
+constexpr int kGatherThreads = 128;  // threads per block (at least kGatherSegs)
 
 // `split` blocks share a group (block b takes group b / split and every split-th step of its entries), so
 // that long lists and crowded groups are spread over more blocks.
-__global__ void __launch_bounds__(kCta)
+__global__ void __launch_bounds__(kGatherThreads)
 k_gather(FinalizeParams p, unsigned int split) {
   // Every candidate's key is >= the sampled bound lo, and almost all lie within a few octaves above it:
   // the block counts first digits in a window of kGatherBins bins that starts at lo's bin (16 bins per
   // octave); the rare key beyond the window goes to the global histogram directly.
   __shared__ unsigned int s_hist[kGatherBins];
   __shared__ unsigned int s_off[kGatherSegs + 1];  // exclusive offsets of the block's segments, total at the end
-  __shared__ unsigned long long s_red[kCta / 32];
-  __shared__ unsigned int s_scan[kCta / 32];
+  __shared__ unsigned long long s_red[kGatherThreads / 32];
+  __shared__ unsigned int s_scan[kGatherThreads / 32];
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (int b = threadIdx.x; b < kGatherBins; b += kCta) s_hist[b] = 0;
+  for (int b = threadIdx.x; b < kGatherBins; b += kGatherThreads) s_hist[b] = 0;
   const unsigned int first_bin = p.ctl->lo >> digit_shift(0);
   // list position of the block's first candidate
   const unsigned int group = blockIdx.x / split, part = blockIdx.x % split;
   const unsigned long long first_group = (unsigned long long)group * (kGatherSegs / kGroupSegs);
   unsigned long long before = 0;
-  for (unsigned long long g = threadIdx.x; g < first_group; g += kCta) before += p.group_count[g];
+  for (unsigned long long g = threadIdx.x; g < first_group; g += kGatherThreads) before += p.group_count[g];
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) before += __shfl_xor_sync(0xFFFFFFFFu, before, o);
   if (lane == 0) s_red[warp] = before;
@@ -340,7 +341,7 @@ k_gather(FinalizeParams p, unsigned int split) {
   unsigned long long base = 0;
   unsigned int warps_before = 0, total = 0;
 #pragma unroll
-  for (int w = 0; w < kCta / 32; ++w) {
+  for (int w = 0; w < kGatherThreads / 32; ++w) {
     base += s_red[w];
     if (w < warp) warps_before += s_scan[w];
     total += s_scan[w];
@@ -349,7 +350,7 @@ k_gather(FinalizeParams p, unsigned int split) {
   if (threadIdx.x == 0) s_off[kGatherSegs] = total;
   __syncthreads();
   bool nonfinite = false;
-  for (unsigned int j0 = (part * kCta + threadIdx.x) * kGatherRun; j0 < total; j0 += split * kCta * kGatherRun) {
+  for (unsigned int j0 = (part * kGatherThreads + threadIdx.x) * kGatherRun; j0 < total; j0 += split * kGatherThreads * kGatherRun) {
     const int cnt = (int)min((unsigned int)kGatherRun, total - j0);
     uint32_t from[kGatherRun];
     {
@@ -394,7 +395,7 @@ k_gather(FinalizeParams p, unsigned int split) {
   }
   if (nonfinite) set_status(&p.ctl->status, NSML_ERR_NONFINITE);
   __syncthreads();
-  for (int b = threadIdx.x; b < kGatherBins; b += kCta) {
+  for (int b = threadIdx.x; b < kGatherBins; b += kGatherThreads) {
     const unsigned int n_b = s_hist[b];
     if (n_b) atomicAdd(&p.hist[first_bin + b], n_b);  // first_bin + b <= 4095: a count here came from a real key
   }
