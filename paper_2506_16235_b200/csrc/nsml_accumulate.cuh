@@ -159,20 +159,38 @@ k_merge(PayloadTable table, int W, float* __restrict__ dense, unsigned long long
     s_view[threadIdx.x] = v;
   }
 
+  // offsets of the block's next tile, fetched by the first warp one tile ahead (two workers per lane), so that a
+  // tile costs one round trip to memory (its entries) instead of two
+  unsigned int ahead_a[2] = {0, 0}, ahead_b[2] = {0, 0};
+  if (threadIdx.x < 32 && blockIdx.x < tiles) {
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+      const int w = threadIdx.x * 2 + h;
+      if (w < W) {
+        ahead_a[h] = offsets[w * per + blockIdx.x];
+        ahead_b[h] = offsets[w * per + blockIdx.x + 1];
+      }
+    }
+  }
   for (unsigned int tile = blockIdx.x; tile < tiles; tile += gridDim.x) {
     const unsigned long long lo = (unsigned long long)tile * kDenseTile;
     const unsigned int len = (unsigned int)min((unsigned long long)kDenseTile, n - lo);
     __syncthreads();  // the previous tile is fully written out (first tile: the views are in place)
     if (threadIdx.x < 32) {
-      // the first warp reads the tile's offsets (two workers per lane) and scans the counts
+      // the first warp hands out the tile's offsets and scans the counts
       unsigned int cnt[2];
 #pragma unroll
       for (int h = 0; h < 2; ++h) {
         const int w = threadIdx.x * 2 + h;
         cnt[h] = 0;
         if (w < W) {
-          unsigned int a = offsets[w * per + tile];
-          unsigned int b = offsets[w * per + tile + 1];
+          unsigned int a = ahead_a[h];
+          unsigned int b = ahead_b[h];
+          const unsigned long long next = (unsigned long long)tile + gridDim.x;
+          if (next < tiles) {
+            ahead_a[h] = offsets[w * per + next];
+            ahead_b[h] = offsets[w * per + next + 1];
+          }
           if (b < a) b = a;  // only a corrupt (unsorted) payload gets here
           s_from[w] = a;
           s_to[w] = b;
