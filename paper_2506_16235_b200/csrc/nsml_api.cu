@@ -536,7 +536,7 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
       unsigned int* fine = reinterpret_cast<unsigned int*>(ws + L.fine);
       {
         LaunchScope scope(K_PRUNE_SAMPLE, st);
-        k_prune_sample<<<1, 1024, 0, st>>>(src, un, (unsigned int)r_lo, (unsigned int)r_hi, ctl);
+        launch_prio(k_prune_sample, dim3(1), dim3(1024), 0, st, false, 0, true, src, un, (unsigned int)r_lo, (unsigned int)r_hi, ctl);
       }
       {
         LaunchScope scope(K_PRUNE_COUNT, st);
@@ -544,15 +544,17 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
       }
       {
         LaunchScope scope(K_PRUNE_SETTLE, st);
-        k_prune_settle<<<1, kCta, 0, st>>>((unsigned int)m, ctl, fine);
+        launch_prio(k_prune_settle, dim3(1), dim3(kCta), 0, st, false, 0, true, (unsigned int)m, ctl, fine);
       }
       {
         LaunchScope scope(K_PRUNE_MARK, st);
-        k_prune_mark<<<wgrid, kCta, 0, st>>>(src, un, ctl, tie_list, mask);
+        // a block per 16 KB tile: short-lived blocks on one moving window read faster than persistent ones
+        const unsigned long long mark_tiles = (un + kStreamTile - 1) / kStreamTile;
+        k_prune_mark<<<(unsigned int)mark_tiles, kCta, 0, st>>>(src, un, ctl, tie_list, mask);
       }
       {
         LaunchScope scope(K_PRUNE_FIX, st);
-        k_prune_fix<<<kPruneFixBlocks, kCta, 0, st>>>(ctl, tie_list, mask);
+        launch_prio(k_prune_fix, dim3(kPruneFixBlocks), dim3(kCta), 0, st, false, 0, true, ctl, tie_list, mask);
       }
     }
   }
