@@ -274,3 +274,26 @@ def test_bounded_wait_runs_out_and_reports_timeout():
     payload = nsml.nsml_compress(torch.from_numpy(g).cuda(), 0.01, 8, workspace=ws)
     assert nsml.nsml_last_status(ws) == 0
     assert_payload_equal(payload, oracle.compress(g, 0.01, 8))
+
+# The bucket pass gives every warp 2 KB of the bucket (one float32 segment of 512 elements, two bfloat16
+# segments) and every block eight warps: sizes at and around the segment, warp and block boundaries, with the
+# ragged last segment falling to the first, a middle and the last warp of a block, with and without a mask.
+PASS_EDGE_SIZES = [16384, 16385, 16384 + 511, 16384 + 512, 16384 + 513, 16384 + 1024 + 1, 20480 - 1, 20480, 20480 + 1,
+                   24576 + 7 * 512 + 3, 8 * 4096 - 512 + 5, 8 * 4096 + 1]
+
+
+@pytest.mark.parametrize("n", PASS_EDGE_SIZES)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_bucket_pass_tails(n, dtype):
+    rng = np.random.default_rng(n)
+    g = (rng.standard_normal(n) * 10.0 ** rng.uniform(-5, -2, n)).astype(np.float32)
+    g[-3:] = [3.0, -4.0, 5.0]  # the last elements are survivors: a dropped tail shows
+    g[0] = -6.0
+    if dtype == "bf16":
+        g = synth.f32_to_bf16_bits(g)
+    mask = rng.random(n) < 0.3
+    mask[-2] = True
+    for ratio in (0.003, 0.05):  # list strategy
+        assert nsml.nsml_compress_strategy(n, ratio) == 0
+        check_compress(g, ratio, 16)
+        check_compress(g, ratio, 8, mask_bool=mask)
