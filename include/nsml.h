@@ -22,7 +22,12 @@
  *   - "device pointer" = CUDA global memory of the current device, owned by the
  *     caller before and after the call.  "host pointer" = ordinary memory.
  *   - Device work is enqueued on `stream` (a cudaStream_t passed as void*, NULL
- *     = the default stream) and the call returns without synchronising.
+ *     = the default stream) and the call returns without synchronising.  The
+ *     short, latency-bound kernels of a call (sample, gather, list stage,
+ *     partition) are launched at the device's highest stream priority, whatever
+ *     the priority of `stream`: with several buckets in flight on several
+ *     streams they are then placed between the blocks of other buckets'
+ *     streaming passes instead of behind them.  Order within `stream` is kept.
  *   - Argument errors are returned at once and enqueue nothing.  Errors that only
  *     the device can see (non-finite input, corrupt payload, a bounded wait that
  *     ran out) are written to a status word at the start of `workspace`; read it

@@ -80,7 +80,7 @@ struct LaunchScope {  // brackets one kernel launch
 struct DeviceInfo {
   bool ready = false;
   int sms = 0;
-  int compact_bucket = 0, compact_feedback = 0, finalize_small = 0, finalize_large = 0, merge = 0;  // resident blocks per SM
+  int compact_feedback = 0, finalize_small = 0, finalize_large = 0, merge = 0;  // resident blocks per SM
   int sumsq = 0, feedback_add = 0, prune_hist = 0, prune_write = 0, prune_write_ranked = 0;  // the same, streaming kernels
   bool finalize_cluster = false;  // the one-cluster shape of the list stage fits an SM
 };
@@ -95,8 +95,7 @@ static int device_info(const DeviceInfo** out) {
   if (!d.ready) {
     if (cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return NSML_ERR_CUDA;
     cudaError_t e = cudaSuccess;
-    e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_bucket, k_compact_bucket<NSML_F32, false, true>, kCta, 0);
-    if (e == cudaSuccess) e = cudaFuncSetAttribute(k_compact_bucket<NSML_F32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCompactFeedbackSmem);
+    e = cudaFuncSetAttribute(k_compact_bucket<NSML_F32, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCompactFeedbackSmem);
     if (e == cudaSuccess) e = cudaFuncSetAttribute(k_compact_bucket<NSML_BF16, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCompactFeedbackSmem);
     if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.compact_feedback, k_compact_bucket<NSML_F32, true>, kCta, kCompactFeedbackSmem);
     auto prepare = [&](auto kernel, int threads, int cache, int* resident) {
@@ -138,7 +137,7 @@ static int device_info(const DeviceInfo** out) {
     if (e == cudaSuccess && (d.sumsq < 1 || d.feedback_add < 1 || d.prune_hist < 1 || d.prune_write < 1 || d.prune_write_ranked < 1)) e = cudaErrorUnknown;
     int coop = 0;
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev);
-    if (e != cudaSuccess || d.compact_bucket < 1 || d.compact_feedback < 1 || d.finalize_small < 1 || d.finalize_large < 1 || d.merge < 1 || !coop) {
+    if (e != cudaSuccess || d.compact_feedback < 1 || d.finalize_small < 1 || d.finalize_large < 1 || d.merge < 1 || !coop) {
       cudaGetLastError();
       return NSML_ERR_CUDA;
     }
