@@ -207,9 +207,9 @@ class Workload:
             self.account(acc, "k_finalize_dense", esize * n + 8 * k + 4 * k + vb * k + s)
             return
         self.account(acc, "k_sample", 4 * 8192)
-        self.account(acc, "k_compact_bucket", esize * n + 8 * k)
-        # gather: candidates (index + value) read from the segmented list and written contiguously
-        self.account(acc, "k_gather", 16 * k)
+        self.account(acc, "k_compact_bucket", esize * n + 6 * k)  # candidates: 16-bit offset in the segment + value
+        # gather: candidates read from the segmented list (6 bytes) and written contiguously (index + value)
+        self.account(acc, "k_gather", 14 * k)
         # list stage: candidate values read once per phase (4 x 4k keys), indices once, survivors written and re-read
         self.account(acc, "k_finalize", 16 * k + 4 * k + 8 * k + 4 * k + vb * k + s)
 

@@ -246,7 +246,7 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
                            unsigned char* ws, unsigned char* payload, const CompressLayout& L, const PayloadLayout& P,
                            const DeviceInfo& dev, cudaStream_t st, bool keep_status = false) {
   Ctl* ctl = reinterpret_cast<Ctl*>(ws);
-  uint32_t* seg_idx = reinterpret_cast<uint32_t*>(ws + L.seg_idx);
+  unsigned short* seg_off = reinterpret_cast<unsigned short*>(ws + L.seg_off);
   uint32_t* seg_val = reinterpret_cast<uint32_t*>(ws + L.seg_val);
   unsigned short* seg_count = reinterpret_cast<unsigned short*>(ws + L.seg_count);
   const unsigned long long nseg = ((unsigned long long)n + kSegElems - 1) / kSegElems;
@@ -285,13 +285,13 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
                                                     : (unsigned int)((nseg + kPlainSegs - 1) / kPlainSegs);
       unsigned int* group_count = reinterpret_cast<unsigned int*>(ws + L.group_count);
       if (residual != nullptr)
-        k_compact_bucket<DTYPE, true><<<grid, kCta, kCompactFeedbackSmem, st>>>(src, residual, (unsigned long long)n, ctl, seg_idx,
+        k_compact_bucket<DTYPE, true><<<grid, kCta, kCompactFeedbackSmem, st>>>(src, residual, (unsigned long long)n, ctl, seg_off,
                                                                                 seg_val, seg_count, group_count);
       else if (mask != nullptr)
-        k_compact_bucket<DTYPE, false, true><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, ctl, seg_idx, seg_val,
+        k_compact_bucket<DTYPE, false, true><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, ctl, seg_off, seg_val,
                                                                     seg_count, group_count);
       else
-        k_compact_bucket<DTYPE, false, false><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, ctl, seg_idx, seg_val,
+        k_compact_bucket<DTYPE, false, false><<<grid, kCta, 0, st>>>(src, nullptr, (unsigned long long)n, ctl, seg_off, seg_val,
                                                                      seg_count, group_count);
     }
     // list stage: cooperative, every block co-resident.  The small shape when a block's share of the
@@ -324,7 +324,7 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
   fp.block_counts = reinterpret_cast<unsigned long long*>(ws + L.block_counts);
   fp.seg_count = seg_count;
   fp.group_count = reinterpret_cast<const unsigned int*>(ws + L.group_count);
-  fp.seg_idx = seg_idx;
+  fp.seg_off = seg_off;
   fp.seg_val = seg_val;
   fp.list_idx = reinterpret_cast<uint32_t*>(ws + L.list_idx);
   fp.list_val = reinterpret_cast<uint32_t*>(ws + L.list_val);

@@ -42,11 +42,11 @@ struct CompressLayout {  // byte offsets inside a compress workspace
   size_t zero_bytes;    // everything before this offset is cleared per call 
   size_t block_counts;  // u64[4][kMaxFinalizeBlocks]: per-block counts exchanged at barriers
   size_t seg_count;     // u16[ceil(n / kSegElems)]: entries per segment
-  size_t seg_idx;       // u32[n]: segmented candidate list (bucket pass output); segment s starts at s * kSegElems
+  size_t seg_off;       // u16[n]: segmented candidate list (bucket pass output), a candidate's offset inside its segment; segment s starts at s * kSegElems
   size_t seg_val;       // u32[n] (float32 bit patterns)
   size_t list_idx;      // u32[n]: the same candidates, contiguous per finalize block
   size_t list_val;      // u32[n]
-  size_t raw_val;       // f32[n]: survivor values before quantisation
+  size_t raw_val;       // f32[n]: survivor values before quantisation (the same memory as seg_val)
   size_t total;
 };
 
@@ -61,12 +61,14 @@ inline CompressLayout compress_layout(int64_t n) {
   L.zero_bytes = L.group_count + align_up(((segs + kGroupSegs - 1) / kGroupSegs) * 4, 256);
   L.block_counts = L.zero_bytes;
   L.seg_count = L.block_counts + 4 * kMaxFinalizeBlocks * 8;
-  L.seg_idx = L.seg_count + align_up(segs * 2, 256);
-  L.seg_val = L.seg_idx + npad * 4;
+  L.seg_off = L.seg_count + align_up(segs * 2, 256);
+  L.seg_val = L.seg_off + npad * 2;
   L.list_idx = L.seg_val + npad * 4;
   L.list_val = L.list_idx + npad * 4;
-  L.raw_val = L.list_val + npad * 4;
-  L.total = L.raw_val + npad * 4;
+  // raw_val shares the memory of seg_val: the segmented list is dead once k_gather has copied it, the
+  // survivors' raw values are written after that (list strategy), and the dense strategy has no list at all
+  L.raw_val = L.seg_val;
+  L.total = L.list_val + npad * 4;
   return L;
 }
 

@@ -30,8 +30,8 @@ constexpr size_t kCompactFeedbackSmem = (size_t)(kCta / 32) * 2 * kSegElems * 4;
 // Appends the kept elements of one round of 32 * EPL elements.  `f` holds this lane's keep flags (bit e =
 // element lane*EPL+e of the round).  Returns the round's total.
 template <int EPL>
-__device__ __forceinline__ unsigned int append_round(unsigned int f, const uint32_t (&bits)[EPL], uint32_t first_index,
-                                                     unsigned long long out_base, uint32_t* __restrict__ seg_idx,
+__device__ __forceinline__ unsigned int append_round(unsigned int f, const uint32_t (&bits)[EPL], unsigned int first_offset,
+                                                     unsigned long long out_base, unsigned short* __restrict__ seg_off,
                                                      uint32_t* __restrict__ seg_val) {
   const int lane = threadIdx.x & 31;
   const unsigned int lt = (1u << lane) - 1u;
@@ -57,7 +57,7 @@ __device__ __forceinline__ unsigned int append_round(unsigned int f, const uint3
 #pragma unroll
     for (int e = 0; e < EPL; ++e) {
       if (f & (1u << e)) {
-        seg_idx[pos] = first_index + lane * EPL + e;
+        seg_off[pos] = (unsigned short)(first_offset + lane * EPL + e);
         seg_val[pos] = bits[e];
         ++pos;
       }
@@ -115,7 +115,7 @@ __host__ __device__ constexpr int compact_segs_per_warp() { return DTYPE == NSML
 
 template <int DTYPE, bool MASKED>
 __device__ __forceinline__ void compact_plain(const BucketSrc<DTYPE>& src, unsigned long long n, const Ctl* ctl,
-                                              uint32_t* __restrict__ seg_idx, uint32_t* __restrict__ seg_val,
+                                              unsigned short* __restrict__ seg_off, uint32_t* __restrict__ seg_val,
                                               unsigned short* __restrict__ seg_count, unsigned int* __restrict__ group_count) {
   constexpr int ESIZE = (DTYPE == NSML_F32) ? 4 : 2;
   constexpr int EPL = 16 / ESIZE;                 // elements a lane takes per round: 16 bytes' worth
@@ -175,7 +175,7 @@ __device__ __forceinline__ void compact_plain(const BucketSrc<DTYPE>& src, unsig
       }
       const unsigned int f = keep_flags<EPL>(bits, t);
       if (!__any_sync(0xFFFFFFFFu, f != 0)) continue;
-      kept += append_round<EPL>(f, bits, (uint32_t)(seg_base + r * ROUND), seg_base + kept, seg_idx, seg_val);
+      kept += append_round<EPL>(f, bits, (unsigned int)(r * ROUND), seg_base + kept, seg_off, seg_val);
     }
     if (lane == 0) {
       seg_count[seg] = (unsigned short)kept;
@@ -193,10 +193,10 @@ __device__ __forceinline__ void compact_plain(const BucketSrc<DTYPE>& src, unsig
 template <int DTYPE, bool FEEDBACK = false, bool MASKED = true>
 __global__ void __launch_bounds__(kCta)
 k_compact_bucket(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned long long n, Ctl* ctl,
-                 uint32_t* __restrict__ seg_idx, uint32_t* __restrict__ seg_val, unsigned short* __restrict__ seg_count,
+                 unsigned short* __restrict__ seg_off, uint32_t* __restrict__ seg_val, unsigned short* __restrict__ seg_count,
                  unsigned int* __restrict__ group_count) {
   if (!FEEDBACK) {
-    compact_plain<DTYPE, MASKED>(src, n, ctl, seg_idx, seg_val, seg_count, group_count);
+    compact_plain<DTYPE, MASKED>(src, n, ctl, seg_off, seg_val, seg_count, group_count);
     return;
   }
   constexpr int ESIZE = (DTYPE == NSML_F32) ? 4 : 2;
@@ -296,7 +296,7 @@ k_compact_bucket(BucketSrc<DTYPE> src, float* __restrict__ residual, unsigned lo
       }
       const unsigned int f = keep_flags<EPL>(bits, t);
       if (!__any_sync(0xFFFFFFFFu, f != 0)) continue;
-      kept += append_round<EPL>(f, bits, (uint32_t)(seg_base + r * ROUND), seg_base + kept, seg_idx, seg_val);
+      kept += append_round<EPL>(f, bits, (unsigned int)(r * ROUND), seg_base + kept, seg_off, seg_val);
     }
     if (lane == 0) {
       seg_count[seg] = (unsigned short)kept;

@@ -70,7 +70,7 @@ struct FinalizeParams {
   unsigned long long* block_counts;  // [4][kMaxFinalizeBlocks]
   const unsigned short* seg_count;
   const unsigned int* group_count;   // [ceil(nseg / kGroupSegs)]
-  const uint32_t* seg_idx;
+  const unsigned short* seg_off;     // a candidate's offset inside its segment
   const uint32_t* seg_val;
   uint32_t* list_idx;
   uint32_t* list_val;
@@ -377,7 +377,7 @@ k_gather(FinalizeParams p, unsigned int split) {
     for (int e = 0; e < kGatherRun; ++e) {
       if (e < cnt) {
         vals[e] = __ldg(p.seg_val + from[e]);
-        idxs[e] = __ldg(p.seg_idx + from[e]);
+        idxs[e] = (from[e] & ~(uint32_t)(kSegElems - 1)) + __ldg(p.seg_off + from[e]);
       }
     }
 #pragma unroll
