@@ -401,8 +401,12 @@ k_gather(FinalizeParams p, unsigned int split) {
   }
 }
 
+// Registers: at most 64 per thread; the small shape is held to 48 (five blocks per SM by registers, no spills).
+// The kernel waits for memory most of its time, and what it costs other streams' kernels is the registers it
+// holds meanwhile: with 48 instead of 64 the eight-stream step of the default workload went from 0.722 to
+// 0.702 ms at the same time for a lone call (40: 0.704 ms with a few spills, 32: 0.719 ms and 6 us more alone).
 template <int DTYPE, int THREADS, int CACHE, bool CLUSTER = false>
-__global__ void __launch_bounds__(THREADS, 1024 / THREADS)  // at most 64 registers per thread
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 5 : 1024 / THREADS)
 k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   __shared__ FinalizeShared<THREADS, false> sh;
   extern __shared__ __align__(16) uint32_t s_cache[];  // the first CACHE candidate values of this block
