@@ -405,8 +405,10 @@ k_gather(FinalizeParams p, unsigned int split) {
 // The kernel waits for memory most of its time, and what it costs other streams' kernels is the registers it
 // holds meanwhile: with 48 instead of 64 the eight-stream step of the default workload went from 0.722 to
 // 0.702 ms at the same time for a lone call (40: 0.704 ms with a few spills, 32: 0.719 ms and 6 us more alone).
+// The large shape (two 512-thread blocks per SM) is held to 40: at 64 its grid took every register of every SM
+// for the length of the kernel (ratio 0.1 on 25M-element buckets: 884 -> 921 GB/s, the kernel alone 47 -> 49 us).
 template <int DTYPE, int THREADS, int CACHE, bool CLUSTER = false>
-__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 5 : 1024 / THREADS)
+__global__ void __launch_bounds__(THREADS, THREADS == 256 ? 5 : (THREADS == 512 ? 3 : 1))
 k_finalize(BucketSrc<DTYPE> src, FinalizeParams p) {
   __shared__ FinalizeShared<THREADS, false> sh;
   extern __shared__ __align__(16) uint32_t s_cache[];  // the first CACHE candidate values of this block
