@@ -823,6 +823,15 @@ def timed_steps(torch, wl, steps, first_step):
     return e0.elapsed_time(e1)
 
 
+def whole_step(table, ms_per_step, peak):
+    """The step as one unit: the algorithmic bytes of all its launches (per-kernel table) over the device time
+    of the step as it is timed (all streams)."""
+    nbytes = sum(k["algorithmic_bytes_per_launch"] * k["launches_per_step"] for k in table.values())
+    gbs = nbytes / (ms_per_step * 1e-3) / 1e9
+    return {"algorithmic_bytes_per_step": nbytes, "ms_per_step": ms_per_step, "algorithmic_GBps": gbs,
+            "frac_of_measured": gbs / peak, "frac_of_nominal_8TBps": gbs / 8000.0}
+
+
 def run_leg(nsml, torch, wl, peak, use_graphs, traffic=None, steps=10):
     """A further workload measured inside the default run: device time of `steps` steps, then the per-kernel table."""
     wl.init_graphs(use_graphs)
@@ -833,8 +842,9 @@ def run_leg(nsml, torch, wl, peak, use_graphs, traffic=None, steps=10):
     wl.lanes.join()
     torch.cuda.synchronize()
     ms = timed_steps(torch, wl, steps, warm) / steps
+    table = per_kernel_table(nsml, torch, wl, peak, 5, traffic=traffic)
     return {"workload": wl.name, "value": wl.input_bytes_per_step / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
-            "per_kernel": per_kernel_table(nsml, torch, wl, peak, 5, traffic=traffic)}
+            "whole_step": whole_step(table, ms, peak), "per_kernel": table}
 
 
 def serial_compress(nsml, torch, grad, ratio, bits, ws, payload, esize, peak, reps=30):
@@ -1070,6 +1080,7 @@ def main():
                     "us_per_launch": d["us_per_launch"], "algorithmic_bytes_per_launch": d["algorithmic_bytes_per_launch"],
                     "how": "achieved = algorithmic_bytes_per_launch / us_per_launch (CUDA events around every launch, one "
                            "stream); the dominant kernel is the one with the most device time per step",
+                    "whole_step": whole_step(kernels, elapsed_ms / steps, peak),
                     "per_kernel": kernels}
         if rank == 0 and args.workload == "gpt2":
             g = wl.workers[0][-2] if len(wl.workers[0]) > 1 else wl.workers[0][0]
