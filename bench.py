@@ -847,11 +847,12 @@ def run_leg(nsml, torch, wl, peak, use_graphs, traffic=None, steps=10):
             "whole_step": whole_step(table, ms, peak), "per_kernel": table}
 
 
-def serial_compress(nsml, torch, grad, ratio, bits, ws, payload, esize, peak, reps=30):
+def serial_compress(nsml, torch, grad, ratio, bits, ws, payload, esize, peak, reps=30, restore_candidates=4096):
     """One nsml_compress at a time on one stream, back to back: what a caller that compresses a single bucket (the
     last bucket of a backward pass, say) gets.  The algorithmic bytes of the call are one read of the bucket plus
     the payload written."""
     n = grad.numel()
+    nsml.nsml_set_list_block_candidates(4096)  # the library's default: what a lone call should use
     for _ in range(5):
         nsml.nsml_compress(grad, ratio, bits, payload=payload, workspace=ws)
     torch.cuda.synchronize()
@@ -861,11 +862,13 @@ def serial_compress(nsml, torch, grad, ratio, bits, ws, payload, esize, peak, re
         nsml.nsml_compress(grad, ratio, bits, payload=payload, workspace=ws)
     e1.record()
     torch.cuda.synchronize()
+    nsml.nsml_set_list_block_candidates(restore_candidates)
     us = 1e3 * e0.elapsed_time(e1) / reps
     nbytes = esize * n + nsml.nsml_payload_bytes(n, ratio, bits)
     gbs = nbytes / (us * 1e-6) / 1e9
     return {"us_per_call": us, "algorithmic_bytes": nbytes, "algorithmic_GBps": gbs, "frac_of_measured": gbs / peak,
             "frac_of_nominal_8TBps": gbs / 8000.0, "n": n, "ratio": ratio, "bits": bits,
+            "list_block_candidates": 4096,
             "note": "one call at a time on one stream, eager launches; the same bucket every time, so a bucket that "
                     "fits the 126 MB L2 is partly served from it"}
 
@@ -981,6 +984,8 @@ def main():
     ap.add_argument("--workload", default="gpt2", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="nsml", choices=["nsml", "reference"])
     ap.add_argument("--streams", type=int, default=8, help="CUDA streams that independent buckets alternate between")
+    ap.add_argument("--list-block-candidates", type=int, default=8192,
+                    help="nsml_set_list_block_candidates for the multi-stream workloads (library default: 4096)")
     ap.add_argument("--no-graphs", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-legs", action="store_true", help="skip the further workloads measured inside the default run")
@@ -1037,7 +1042,11 @@ def main():
     kwargs = {}
     if args.workload == "gpt2" and args.buckets:
         kwargs["buckets"] = list(range(args.buckets))
+    # several buckets in flight: the list stage takes more candidates per block (fewer SMs held while it waits
+    # for memory); the one-call-at-a-time measurement below goes back to the library's default
+    nsml.nsml_set_list_block_candidates(args.list_block_candidates)
     wl = WORKLOADS[args.workload](nsml, torch, device, rank, nlanes=max(1, args.streams), **kwargs)
+    wl.config["list_block_candidates"] = args.list_block_candidates
     wl.init_graphs(not args.no_graphs)
     if wl.use_graphs:
         warmup = max(warmup, wl.graph_period)  # every job has been captured before the timed region starts
@@ -1085,7 +1094,8 @@ def main():
         if rank == 0 and args.workload == "gpt2":
             g = wl.workers[0][-2] if len(wl.workers[0]) > 1 else wl.workers[0][0]
             roofline["one_compress_call"] = serial_compress(nsml, torch, g, wl.RATIO, wl.BITS, wl.lanes.all[0].ws,
-                                                            wl.lanes.all[0].payloads[0], 4, peak)
+                                                            wl.lanes.all[0].payloads[0], 4, peak,
+                                                            restore_candidates=args.list_block_candidates)
 
     # ---- end to end through the host-buffer entry points ----
     e2e = None
@@ -1130,17 +1140,22 @@ def main():
         nl, graphs = max(1, args.streams), not args.no_graphs
         del wl
         torch.cuda.empty_cache()
-        for key, make in (
-            ("ratio_0.1_25M", lambda: Gpt2Workload(nsml, torch, device, rank, buckets=[2, 3], nlanes=nl, ratio=0.1, workers=2)),
-            ("ratio_0.001_25M", lambda: Gpt2Workload(nsml, torch, device, rank, buckets=[2, 3], nlanes=nl, ratio=0.001, workers=2)),
-            ("bf16_64M", lambda: Bf16BucketWorkload(nsml, torch, device, rank, nlanes=nl)),
-            ("alg2_25M", lambda: Alg2Workload(nsml, torch, device, rank, nlanes=nl)),
-            ("resnet50_sweep", lambda: ResnetWorkload(nsml, torch, device, rank, nlanes=nl)),
+        # (key, workload, candidates per list-stage block: the legs with few calls in flight keep the library's default)
+        for key, make, candidates in (
+            ("ratio_0.1_25M", lambda: Gpt2Workload(nsml, torch, device, rank, buckets=[2, 3], nlanes=nl, ratio=0.1, workers=2),
+             args.list_block_candidates),
+            ("ratio_0.001_25M", lambda: Gpt2Workload(nsml, torch, device, rank, buckets=[2, 3], nlanes=nl, ratio=0.001, workers=2),
+             args.list_block_candidates),
+            ("bf16_64M", lambda: Bf16BucketWorkload(nsml, torch, device, rank, nlanes=nl), args.list_block_candidates),
+            ("alg2_25M", lambda: Alg2Workload(nsml, torch, device, rank, nlanes=nl), 4096),
+            ("resnet50_sweep", lambda: ResnetWorkload(nsml, torch, device, rank, nlanes=nl), 4096),
         ):
+            nsml.nsml_set_list_block_candidates(candidates)
             leg_wl = make()
             if key.startswith("ratio_"):
                 leg_wl.name = f"two 25M-element fp32 buckets, ratio {leg_wl.RATIO}, int8, W=2 workers each"
             legs[key] = run_leg(nsml, torch, leg_wl, peak, graphs)
+            legs[key]["list_block_candidates"] = candidates
             del leg_wl
             torch.cuda.empty_cache()
         out["legs"] = legs

@@ -222,6 +222,20 @@ int nsml_compress(const void* grad, int64_t n, int grad_dtype, double ratio, int
 #define NSML_STRATEGY_DENSE 1
 int nsml_compress_strategy(int64_t n, double ratio);
 
+/* nsml_set_list_block_candidates -- a tuning knob of the list strategy, for the
+ * whole process: about how many candidates one thread block of the list stage
+ * takes when the list is short (up to about a million candidates).  The result
+ * of nsml_compress does not depend on it.  Fewer candidates per block = more
+ * blocks = a shorter list stage for a call that has the GPU to itself; more
+ * candidates per block = fewer SMs held while the stage waits for memory, which
+ * is what counts when several buckets are compressed on several streams at
+ * once (25M-element buckets, ratio 0.01, measured on one B200: 4096 -> a lone
+ * call 69 us, the eight-stream step 0.70 ms; 8192 -> 75 us and 0.67 ms).
+ *   candidates   1024 ... 8192; the default is 4096
+ * Returns NSML_OK, or NSML_ERR_ARG for a value out of range (nothing changes).
+ * Takes effect for calls made after it returns. */
+int nsml_set_list_block_candidates(int candidates);
+
 /* ------------------------------------------------------------------------
  * nsml_decompress_accumulate -- dense += sum over W payloads (plain sum, no
  * averaging), after optionally zeroing dense.

@@ -92,6 +92,7 @@ def _load() -> ctypes.CDLL:
         "nsml_ctrl_load": (ci, [vp, vp, sz]),
         "nsml_k_of": (i64, [i64, dbl]),
         "nsml_compress_strategy": (ci, [i64, dbl]),
+        "nsml_set_list_block_candidates": (ci, [ci]),
         "nsml_payload_bytes": (sz, [i64, dbl, ci]),
         "nsml_workspace_bytes": (sz, [i64, ci]),
         "nsml_accumulate_workspace_bytes": (sz, [i64, ci]),
@@ -200,6 +201,11 @@ def nsml_select_ratio(ctrl: Controller, last_bytes: float, last_seconds: float, 
 # --------------------------------------------------------------------------
 def nsml_k_of(n: int, ratio: float) -> int:
     return int(lib.nsml_k_of(int(n), float(ratio)))
+
+
+def nsml_set_list_block_candidates(candidates: int) -> None:
+    """Tuning knob of the list stage (1024 ... 8192, default 4096); the results do not depend on it."""
+    _check(lib.nsml_set_list_block_candidates(int(candidates)), "nsml_set_list_block_candidates")
 
 
 def nsml_compress_strategy(n: int, ratio: float) -> int:

@@ -223,6 +223,9 @@ static unsigned int sample_rank(int64_t n, int64_t k) {
   return (unsigned int)j;
 }
 
+// Candidates per block of the list stage's small shape (nsml_set_list_block_candidates).
+static std::atomic<int> g_list_block_candidates{4096};
+
 // Kept fraction from which the select runs over the bucket itself.
 constexpr double kDenseRatioAny = 0.25;
 
@@ -305,7 +308,7 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
     if (cluster_shape) {
       fgrid = kFinClusterBlocks;
     } else if (small_shape) {  // short lists: no more blocks than about 4096 candidates each (cheaper barriers, one block = none)
-      unsigned int want = (unsigned int)(expected / 4096.0) + 1;
+      unsigned int want = (unsigned int)(expected / (double)g_list_block_candidates.load(std::memory_order_relaxed)) + 1;
       if (want < fgrid) fgrid = want;
     } else {  // long lists: as many blocks as stay co-resident (two per SM)
       unsigned long long cap = large_cap_blocks;
@@ -684,6 +687,12 @@ int nsml_compress_strategy(int64_t n, double ratio) {
   const int rc = device_info(&dev);
   if (rc != NSML_OK) return rc;
   return use_dense(n, k, *dev) ? NSML_STRATEGY_DENSE : NSML_STRATEGY_LIST;
+}
+
+int nsml_set_list_block_candidates(int candidates) {
+  if (candidates < 1024 || candidates > kFinSmallCache) return NSML_ERR_ARG;
+  g_list_block_candidates.store(candidates, std::memory_order_relaxed);
+  return NSML_OK;
 }
 
 size_t nsml_payload_bytes(int64_t n, double ratio, int bits) {

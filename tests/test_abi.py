@@ -111,3 +111,11 @@ def test_sized_entry_points_check_their_size_arguments_on_the_host(nsml):
                                                     None) == nsml.NSML_ERR_ARG
     assert nsml.lib.nsml_decompress_accumulate_sized(ptrs, None, 1, scratch, n, 1, scratch, 4096, None) == nsml.NSML_ERR_ARG
     assert nsml.lib.nsml_decompress_accumulate_sized(ptrs, too_short, 1, scratch, n, 1, scratch, 4096, None) == nsml.NSML_ERR_ARG
+
+
+def test_list_block_candidates_knob_checks_its_range(nsml):
+    # a plain host-side setting: no GPU needed
+    for bad in (0, 1023, 8193, -5):
+        assert nsml.lib.nsml_set_list_block_candidates(bad) == nsml.NSML_ERR_ARG
+    for good in (1024, 8192, 4096):  # leaves the default in place
+        assert nsml.lib.nsml_set_list_block_candidates(good) == nsml.NSML_OK

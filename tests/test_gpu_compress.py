@@ -297,3 +297,17 @@ def test_bucket_pass_tails(n, dtype):
         assert nsml.nsml_compress_strategy(n, ratio) == 0
         check_compress(g, ratio, 16)
         check_compress(g, ratio, 8, mask_bool=mask)
+
+
+@pytest.mark.parametrize("candidates", [1024, 8192])
+def test_list_block_candidates_knob_does_not_change_the_payload(candidates):
+    rng = np.random.default_rng(77)
+    n = 3_000_001
+    g = (rng.standard_normal(n) * 10.0 ** rng.uniform(-4, -1, n)).astype(np.float32)
+    nsml.nsml_set_list_block_candidates(candidates)
+    try:
+        for ratio in (0.002, 0.02, 0.2):  # cluster shape, small shape, large shape of the list stage
+            check_compress(g, ratio, 8)
+            check_compress(g, ratio, 16)
+    finally:
+        nsml.nsml_set_list_block_candidates(4096)
