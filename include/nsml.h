@@ -229,8 +229,11 @@ int nsml_compress_strategy(int64_t n, double ratio);
  * blocks = a shorter list stage for a call that has the GPU to itself; more
  * candidates per block = fewer SMs held while the stage waits for memory, which
  * is what counts when several buckets are compressed on several streams at
- * once (25M-element buckets, ratio 0.01, measured on one B200: 4096 -> a lone
- * call 69 us, the eight-stream step 0.70 ms; 8192 -> 75 us and 0.67 ms).
+ * once.  Above the default the gather kernel in front of the list stage also
+ * runs as one block per group of segments instead of two.  Measured on one
+ * B200, 25M-element buckets, ratio 0.01: 4096 -> a lone call 69 us, the
+ * eight-stream step of 20 calls and 5 sums 0.70 ms; 8192 -> about 83 us and
+ * 0.65 ms.
  *   candidates   1024 ... 8192; the default is 4096
  * Returns NSML_OK, or NSML_ERR_ARG for a value out of range (nothing changes).
  * Takes effect for calls made after it returns. */

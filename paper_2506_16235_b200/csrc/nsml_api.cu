@@ -341,7 +341,10 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
     const unsigned long long ngroups = (nseg + kGatherSegs - 1) / kGatherSegs;
     const double per_group = (double)n * (p_keep + 6.0 * std::sqrt(p_keep * (1.0 - p_keep) / kSamples)) / (double)ngroups;
     unsigned int split = (unsigned int)(per_group / 1024.0) + 1;
-    split = split < 2 ? 2 : (split > 8 ? 8 : split);
+    // (with more than the default candidates per list-stage block the caller has asked for few, long blocks: one
+    // gather block per group then, 21 instead of 16 us alone, 2-3 % more throughput with eight streams)
+    const unsigned int min_split = g_list_block_candidates.load(std::memory_order_relaxed) > 4096 ? 1u : 2u;
+    split = split < min_split ? min_split : (split > 8 ? 8 : split);
     launch_prio(k_gather, dim3((unsigned int)(ngroups * split)), dim3(kGatherThreads), 0, st, false, 0, true, fp, split);
   }
   {
