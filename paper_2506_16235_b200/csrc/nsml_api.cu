@@ -312,6 +312,9 @@ static int launch_compress(const void* grad, float* residual, const uint32_t* ma
       if (want < fgrid) fgrid = want;
     } else {  // long lists: as many blocks as stay co-resident (two per SM)
       unsigned long long cap = large_cap_blocks;
+      // (a caller that asked for few, long list-stage blocks gets one per SM while a block's share still fits its cache)
+      if (g_list_block_candidates.load(std::memory_order_relaxed) > 4096 && expected / dev.sms <= (double)kFinLargeCache)
+        cap = (unsigned long long)dev.sms;
       if (cap > nseg) cap = nseg;
       if (cap > (unsigned long long)kMaxFinalizeBlocks) cap = kMaxFinalizeBlocks;
       if (cap > fgrid) fgrid = (unsigned int)cap;

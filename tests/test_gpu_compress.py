@@ -306,8 +306,11 @@ def test_list_block_candidates_knob_does_not_change_the_payload(candidates):
     g = (rng.standard_normal(n) * 10.0 ** rng.uniform(-4, -1, n)).astype(np.float32)
     nsml.nsml_set_list_block_candidates(candidates)
     try:
-        for ratio in (0.002, 0.02, 0.2):  # cluster shape, small shape, large shape of the list stage
+        for ratio in (0.002, 0.02, 0.2):  # cluster shape and small shape of the list stage
             check_compress(g, ratio, 8)
             check_compress(g, ratio, 16)
+        # the large shape (more than about 1.2M expected candidates): one block per SM above the default setting
+        big = (rng.standard_normal(8_000_003) * 10.0 ** rng.uniform(-4, -1, 8_000_003)).astype(np.float32)
+        check_compress(big, 0.2, 8)
     finally:
         nsml.nsml_set_list_block_candidates(4096)
