@@ -570,35 +570,36 @@ static int prune_impl(const float* weights, int64_t n, double ratio, uint32_t* m
   }
   // The four-pass build: every kernel of it leaves at once when the two passes above have built the mask.  Behind
   // the two-pass path it is the rare fallback, so it gets small grids (two blocks per SM): what counts there is
-  // how little the six launches cost when they have nothing to do.
+  // how little the six launches cost when they have nothing to do; they are then launched at high priority
+  // like the other short kernels, so that they do not queue behind other streams' passes.
   const unsigned int small = (unsigned int)dev->sms * 2;
   const unsigned int fgrid = two_pass && grid > small ? small : grid;
   const unsigned int fwgrid = two_pass && wgrid > small ? small : wgrid;
   {
     LaunchScope scope(K_PRUNE_HIST, st);
-    k_prune_hist<0><<<fgrid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
+    launch_prio(k_prune_hist<0>, dim3(fgrid), dim3(kCta), 0, st, false, 0, two_pass, src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
     LaunchScope scope(K_PRUNE_HIST, st);
-    k_prune_hist<1><<<fgrid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
+    launch_prio(k_prune_hist<1>, dim3(fgrid), dim3(kCta), 0, st, false, 0, two_pass, src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
     LaunchScope scope(K_PRUNE_HIST, st);
-    k_prune_hist<2><<<fgrid, kCta, 0, st>>>(src, un, (unsigned int)m, ctl, hist, tie_list);
+    launch_prio(k_prune_hist<2>, dim3(fgrid), dim3(kCta), 0, st, false, 0, two_pass, src, un, (unsigned int)m, ctl, hist, tie_list);
   }
   {
     LaunchScope scope(K_PRUNE_TIES, st);
-    k_prune_ties<<<fgrid, kCta, 0, st>>>(src, un, ctl, hist, tie_list, tile_ties);
+    launch_prio(k_prune_ties, dim3(fgrid), dim3(kCta), 0, st, false, 0, two_pass, src, un, ctl, hist, tie_list, tile_ties);
   }
   {
     LaunchScope scope(K_PRUNE_WRITE, st);
-    k_prune_write<<<fwgrid, kCta, 0, st>>>(src, un, ctl, tile_ties, mask);
+    launch_prio(k_prune_write, dim3(fwgrid), dim3(kCta), 0, st, false, 0, two_pass, src, un, ctl, tile_ties, mask);
   }
   {
     LaunchScope scope(K_PRUNE_WRITE_RANKED, st);  // returns at once unless ties have to be ranked
     unsigned int rgrid = stream_grid(n, *dev, dev->prune_write_ranked < 8 ? dev->prune_write_ranked : 8, 1u << 16);
     if (two_pass && rgrid > small) rgrid = small;
-    k_prune_write_ranked<<<rgrid, kCta, 0, st>>>(src, un, ctl, tile_ties, mask);
+    launch_prio(k_prune_write_ranked, dim3(rgrid), dim3(kCta), 0, st, false, 0, two_pass, src, un, ctl, tile_ties, mask);
   }
   if (cudaGetLastError() != cudaSuccess) return NSML_ERR_CUDA;
   return NSML_OK;
