@@ -625,6 +625,8 @@ class Bf16BucketWorkload(Workload):
         self.dense = self.lanes.all[0].dense
         self.sizes = [n] * self.BUCKETS
         self.input_bytes_per_step = 2.0 * n * self.BUCKETS
+        self.rotate_lanes = True  # three independent jobs per step: the next step's start on the idle lanes
+        self.graph_period = math.lcm(self.BUCKETS, nlanes) // self.BUCKETS
         self.config = {"workload": self.name, "buckets": self.BUCKETS, "bucket_elems": n, "ratio": self.RATIO,
                        "bits": self.BITS, "W": 1, "streams": nlanes, "l2": "inputs are 384 MB per step"}
 
