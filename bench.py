@@ -726,6 +726,7 @@ class Alg2Workload(Workload):
         self.lanes = Lanes(torch, nsml, device, nlanes, nsml.nsml_workspace_bytes(n), nsml.nsml_accumulate_workspace_bytes(n, 1),
                            nsml.nsml_payload_bytes(n, self.RATIO, self.BITS), 1, n)
         for lane in self.lanes.all:
+            lane.side = [torch.cuda.Stream(device)]  # the norm runs beside the mask build
             lane.l2ws = nsml.alloc_bytes(nsml.lib.nsml_l2_workspace_bytes(), device)
             lane.pws = nsml.alloc_bytes(nsml.nsml_prune_workspace_bytes(n), device)
             lane.mask = torch.empty((n + 31) // 32, dtype=torch.int32, device=device)
@@ -741,9 +742,21 @@ class Alg2Workload(Workload):
         k = nsml.nsml_k_of(n, self.RATIO)
         for b in range(self.STATE):
             def enqueue(lane, acc, b=b, g=self.grads[(i * self.STATE + b) % self.GRADS]):
-                nsml.nsml_grad_l2(g, workspace=lane.l2ws, stream=lane.stream, sync=False)
+                # Step 1 reads the gradient, Step 2 the weights: they run side by side (the norm on the lane's side
+                # stream), Step 3 waits for both.  (The event-bracketed per-kernel pass keeps one stream.)
+                torch = self.torch
+                fan = acc is None and len(lane.side) >= 1
+                if fan:
+                    start = torch.cuda.Event()
+                    start.record(lane.stream)
+                    lane.side[0].wait_event(start)
+                nsml.nsml_grad_l2(g, workspace=lane.l2ws, stream=lane.side[0] if fan else lane.stream, sync=False)
                 nsml.nsml_prune_mask_build(self.weights[b], self.RATIO, prune_mask=lane.mask, workspace=lane.pws,
                                            stream=lane.stream)
+                if fan:
+                    done = torch.cuda.Event()
+                    done.record(lane.side[0])
+                    lane.stream.wait_event(done)
                 p = nsml.nsml_compress_feedback(g, self.residual[b], self.RATIO, self.BITS, prune_mask=lane.mask,
                                                 payload=lane.payloads[0], workspace=lane.ws, stream=lane.stream)
                 nsml.nsml_decompress_accumulate([p], lane.dense, zero_first=True, workspace=lane.aws, stream=lane.stream)
