@@ -999,8 +999,9 @@ def main():
     ap.add_argument("--workload", default="gpt2", choices=sorted(WORKLOADS))
     ap.add_argument("--impl", default="nsml", choices=["nsml", "reference"])
     ap.add_argument("--streams", type=int, default=8, help="CUDA streams that independent buckets alternate between")
-    ap.add_argument("--list-block-candidates", type=int, default=8192,
-                    help="nsml_set_list_block_candidates for the multi-stream workloads (library default: 4096)")
+    ap.add_argument("--list-block-candidates", type=int, default=None,
+                    help="nsml_set_list_block_candidates (library default: 4096); default here: 8192 for the workloads "
+                         "with many calls in flight (gpt2, decoder), 4096 for the others")
     ap.add_argument("--no-graphs", action="store_true", help="launch every call eagerly instead of replaying CUDA graphs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-legs", action="store_true", help="skip the further workloads measured inside the default run")
@@ -1059,6 +1060,8 @@ def main():
         kwargs["buckets"] = list(range(args.buckets))
     # several buckets in flight: the list stage takes more candidates per block (fewer SMs held while it waits
     # for memory); the one-call-at-a-time measurement below goes back to the library's default
+    if args.list_block_candidates is None:
+        args.list_block_candidates = 8192 if args.workload in ("gpt2", "decoder") else 4096
     nsml.nsml_set_list_block_candidates(args.list_block_candidates)
     wl = WORKLOADS[args.workload](nsml, torch, device, rank, nlanes=max(1, args.streams), **kwargs)
     wl.config["list_block_candidates"] = args.list_block_candidates
