@@ -232,9 +232,9 @@ int nsml_compress_strategy(int64_t n, double ratio);
  * once.  Above the default the gather kernel in front of the list stage also
  * runs as one block per group of segments instead of two, and long lists get
  * one list-stage block per SM instead of two.  Measured on one
- * B200, 25M-element buckets, ratio 0.01: 4096 -> a lone call 69 us, the
- * eight-stream step of 20 calls and 5 sums 0.70 ms; 8192 -> about 83 us and
- * 0.65 ms.
+ * B200, 25M-element buckets, ratio 0.01, int8: 2048 -> a lone call 65 us;
+ * 4096 -> 68 us, the eight-stream step of 20 calls and 5 sums 0.70 ms;
+ * 8192 -> 81 us and 0.63 ms.
  *   candidates   1024 ... 8192; the default is 4096
  * Returns NSML_OK, or NSML_ERR_ARG for a value out of range (nothing changes).
  * Takes effect for calls made after it returns. */
